@@ -1,0 +1,142 @@
+"""ctypes front end of the CPU checker (test infrastructure, never the product path).
+
+Builds `libslo.so` from `sparseloco_oracle.cpp` with g++ on first use and
+exposes the checker's functions on numpy arrays.  Nothing here computes: every
+step of Eq. 2 runs inside the C++ file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import List, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sparseloco_oracle.cpp")
+_LIB = os.path.join(_HERE, "libslo.so")
+_lib = None
+
+FLAG_NONFINITE = 1
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math",
+                               "-fPIC", "-shared", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        vp, u64, u32, i32, f32 = (ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
+                                  ctypes.c_float)
+        L.slo_num_chunks.restype = u64
+        L.slo_num_chunks.argtypes = [vp, u32, i32]
+        L.slo_codes_stride.restype = u64
+        L.slo_codes_stride.argtypes = [i32, i32]
+        L.slo_compress.restype = i32
+        L.slo_compress.argtypes = [vp, vp, vp, vp, u32, f32, i32, i32, i32, vp, vp, vp, vp]
+        L.slo_aggregate.restype = i32
+        L.slo_aggregate.argtypes = [i32, vp, vp, vp, vp, u32, i32, i32, i32, vp]
+        L.slo_outer_apply.restype = i32
+        L.slo_outer_apply.argtypes = [vp, vp, u64, f32]
+        L.slo_quantise.restype = u32
+        L.slo_quantise.argtypes = [f32, f32, i32]
+        L.slo_dequantise.restype = f32
+        L.slo_dequantise.argtypes = [u32, f32, i32]
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def _off(offsets) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(offsets, dtype=np.uint64))
+
+
+def num_chunks(offsets, chunk: int) -> int:
+    off = _off(offsets)
+    return int(lib().slo_num_chunks(_p(off), len(off) - 1, chunk))
+
+
+def codes_stride(k: int, bits: int) -> int:
+    return int(lib().slo_codes_stride(k, bits))
+
+
+def compress(theta_local: np.ndarray, theta_global: np.ndarray, err: np.ndarray, offsets,
+             beta: float, chunk: int, k: int, bits: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, int]:
+    """Eq. 2 lines 1-4 for one replica.  `err` is updated in place.
+    Returns (idx[n_c, k] u16, codes[n_c, stride] u8, scales[n_c] f32, flags)."""
+    off = _off(offsets)
+    for a in (theta_local, theta_global, err):
+        assert a.dtype == np.float32 and a.flags.c_contiguous
+    nc = num_chunks(off, chunk)
+    idx = np.empty((nc, k), dtype=np.uint16)
+    codes = np.empty((nc, codes_stride(k, bits)), dtype=np.uint8)
+    scales = np.empty(nc, dtype=np.float32)
+    flags = np.zeros(1, dtype=np.uint32)
+    rc = lib().slo_compress(_p(theta_local), _p(theta_global), _p(err), _p(off), len(off) - 1,
+                            beta, chunk, k, bits, _p(idx), _p(codes), _p(scales), _p(flags))
+    if rc != 0:
+        raise ValueError(f"slo_compress rejected its arguments ({rc})")
+    return idx, codes, scales, int(flags[0])
+
+
+def aggregate(msgs: Sequence[Tuple[np.ndarray, np.ndarray, np.ndarray]], offsets, chunk: int, k: int,
+              bits: int) -> np.ndarray:
+    """Dense mean update from the messages of the replicas, added in the order
+    given; the divisor is always len(msgs)."""
+    off = _off(offsets)
+    n = len(msgs)
+    keep: List[np.ndarray] = []
+    def arr(i):
+        a = (ctypes.c_void_p * n)()
+        for r, m in enumerate(msgs):
+            c = np.ascontiguousarray(m[i])
+            keep.append(c)
+            a[r] = _p(c)
+        return a
+    pi, pc, ps = arr(0), arr(1), arr(2)
+    update = np.empty(int(off[-1]), dtype=np.float32)
+    rc = lib().slo_aggregate(n, pi, pc, ps, _p(off), len(off) - 1, chunk, k, bits, _p(update))
+    if rc != 0:
+        raise ValueError(f"slo_aggregate rejected its arguments ({rc})")
+    return update
+
+
+def outer_apply(theta_global: np.ndarray, update: np.ndarray, outer_lr: float) -> None:
+    assert theta_global.dtype == np.float32 and update.dtype == np.float32
+    rc = lib().slo_outer_apply(_p(theta_global), _p(update), theta_global.size, outer_lr)
+    if rc != 0:
+        raise ValueError("slo_outer_apply rejected its arguments")
+
+
+def quantise(v: float, s: float, bits: int) -> int:
+    return int(lib().slo_quantise(v, s, bits))
+
+
+def dequantise(code: int, s: float, bits: int) -> float:
+    return float(lib().slo_dequantise(code, s, bits))
+
+
+def outer_round(theta_locals: Sequence[np.ndarray], theta_global: np.ndarray, errs: Sequence[np.ndarray],
+                offsets, beta: float, chunk: int, k: int, bits: int, outer_lr: float):
+    """One whole outer step (all of Eq. 2) for R replicas; theta_global and the
+    error buffers are updated in place.  Returns the R messages and the update."""
+    msgs = []
+    flags = 0
+    for tl, e in zip(theta_locals, errs):
+        i, c, s, f = compress(tl, theta_global, e, offsets, beta, chunk, k, bits)
+        msgs.append((i, c, s))
+        flags |= f
+    upd = aggregate(msgs, offsets, chunk, k, bits)
+    outer_apply(theta_global, upd, outer_lr)
+    return msgs, upd, flags
