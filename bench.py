@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the SparseLoCo outer step (paper §2.1, Eq. 2) on B200.
+
+A step = one whole outer round over one synthetic parameter set: sl_compress_batch for R
+replicas (Eq. 2 lines 1-4) followed by sl_aggregate_apply (line 5).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1b|0p5b|180m|tiny]
+  python bench.py --impl reference ...     # the CPU checker timed on the host cores
+
+Between steps the replicas' parameters are re-drawn around the new theta_global (untimed);
+every step is timed on the device with CUDA events on the launching stream.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2601_02360_b200 import synth
+
+METRIC = "sparseloco_outer_step_params_per_s"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# --------------------------------------------------------------------------- byte counts
+def message_bytes(wl: synth.Workload) -> int:
+    """Bytes of ONE replica's message: idx u16[k] + packed codes + one float scale per chunk."""
+    stride = 4 * wl.k if wl.bits == 32 else (wl.k * wl.bits + 7) // 8
+    return wl.n_chunks() * (2 * wl.k + stride + 4)
+
+
+def compress_bytes(wl: synth.Workload) -> int:
+    """Algorithmic bytes of one sl_compress_batch launch: per replica theta_local read, e read,
+    e written (12 B/element); theta_global read once for all replicas; messages written."""
+    return wl.n_total * (12 * wl.R + 4) + wl.R * message_bytes(wl)
+
+
+def aggregate_apply_bytes(wl: synth.Workload) -> int:
+    """theta_global read and written once, every message read once."""
+    return wl.n_total * 8 + wl.R * message_bytes(wl)
+
+
+def step_bytes_strict(wl: synth.Workload) -> int:
+    """Least traffic of a whole step: N(12R + 8) + messages written once and read once."""
+    return wl.n_total * (12 * wl.R + 8) + 2 * wl.R * message_bytes(wl)
+
+
+# --------------------------------------------------------------------------- distributed plumbing
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), \
+        int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def init_dist(backend: str):
+    import torch.distributed as dist
+    rank, local, world = dist_env()
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29500")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, local, world
+
+
+def barrier(world: int) -> None:
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device="cpu") -> float:
+    """The slowest rank's time: the job is as slow as its slowest shard."""
+    if world <= 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Every rank owns an independent shard of the job (no exchange between shards): its own
+    parameter set drawn from its own seed."""
+    return base_seed + 1000003 * rank
+
+
+def job_value(params_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: parameters all ranks pushed through one outer step per second."""
+    return params_per_rank * world / (ms_per_step * 1e-3)
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="sl_clocks_", suffix=".csv")
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    smax.append(float(f[1]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+# --------------------------------------------------------------------------- the CPU checker, timed
+def cpu_sample_workload(wl: synth.Workload) -> synth.Workload:
+    """Bounded sample of the workload for the CPU timing: the first transformer layer (its
+    seven matrices and two norm vectors) when the set has one, else the whole set."""
+    if len(wl.tensors) > 9:
+        return synth.sub_arena(wl, list(range(9)), wl.name + "_layer0")
+    return wl
+
+
+def oracle_round(slo, tls, tg, errs, off, wl, threads):
+    """One outer step on the CPU checker as it stands; replicas spread over host threads."""
+    def one(r):
+        return slo.compress(tls[r], tg, errs[r], off, wl.beta, wl.chunk, wl.k, wl.bits)
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        res = list(ex.map(one, range(len(tls))))
+    upd = slo.aggregate([(i, c, s) for i, c, s, _ in res], off, wl.chunk, wl.k, wl.bits)
+    slo.outer_apply(tg, upd, wl.outer_lr)
+
+
+def time_oracle(wl_sample: synth.Workload, steps: int, warmup: int, seed: int, inputs=None):
+    """Times `steps` outer steps of the CPU checker on the sample.  Returns (ms list, threads)."""
+    from oracle import slo
+    slo.build()
+    cores = os.cpu_count() or 1
+    threads = max(1, min(cores, wl_sample.R))
+    off = wl_sample.offsets()
+    if inputs is None:
+        tg_t = synth.gen_theta_global(wl_sample, "cpu", seed)
+        rho = synth.row_scales(wl_sample, seed)
+        tg = tg_t.numpy().copy()
+    else:
+        tg = inputs[0].copy()
+    errs = [np.zeros(wl_sample.n_total, np.float32) for _ in range(wl_sample.R)]
+    times = []
+    for t in range(warmup + steps):
+        if inputs is None:
+            tls = [synth.gen_theta_local(wl_sample, torch.from_numpy(tg), t, r, seed, rho=rho).numpy()
+                   for r in range(wl_sample.R)]
+        else:
+            tls = inputs[1]
+        t0 = time.perf_counter()
+        oracle_round(slo, tls, tg, errs, off, wl_sample, threads)
+        dt = (time.perf_counter() - t0) * 1e3
+        if t >= warmup:
+            times.append(dt)
+    return times, threads
+
+
+def run_reference(args) -> None:
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    wl = synth.workload(args.workload)
+    sample = cpu_sample_workload(wl)
+    times, threads = time_oracle(sample, args.steps, args.warmup, args.seed)
+    ms = float(np.mean(times))
+    value = sample.n_total / (ms * 1e-3)
+    desc = (f"{sample.name}: {len(sample.tensors)} tensors, {sample.n_total} params x R={sample.R}, "
+            f"one outer step per timed step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "R": wl.R, "k": wl.k, "bits": wl.bits, "chunk": wl.chunk,
+                   "beta": wl.beta, "outer_lr": wl.outer_lr, "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- the CUDA path, timed
+class DeviceState:
+    def __init__(self, wl: synth.Workload, seed: int, device):
+        from paper_2601_02360_b200 import api
+        self.api = api
+        self.wl = wl
+        self.seed = seed
+        self.dev = device
+        self.layout = api.Layout(wl.offsets())
+        n = wl.n_total
+        self.theta_global = synth.gen_theta_global(wl, device, seed)
+        self.rho = synth.row_scales(wl, seed)
+        self.theta_local = [torch.empty(n, dtype=torch.float32, device=device) for _ in range(wl.R)]
+        self.err = [torch.zeros(n, dtype=torch.float32, device=device) for _ in range(wl.R)]
+        self.idx, self.codes, self.scales = api.alloc_messages(self.layout, wl.chunk, wl.k, wl.bits,
+                                                               wl.R, device)
+        self.flags = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def redraw_locals(self, rnd: int) -> None:
+        for r in range(self.wl.R):
+            synth.gen_theta_local(self.wl, self.theta_global, rnd, r, self.seed,
+                                  out=self.theta_local[r], rho=self.rho)
+
+    def compress(self) -> None:
+        w = self.wl
+        self.api.sl_compress_batch(self.theta_local, self.theta_global, self.err, self.layout, w.beta,
+                                   w.chunk, w.k, w.bits, self.idx, self.codes, self.scales, self.flags)
+
+    def aggregate_apply(self) -> None:
+        w = self.wl
+        self.api.sl_aggregate_apply(self.idx, self.codes, self.scales, self.layout, w.chunk, w.k, w.bits,
+                                    self.theta_global, w.outer_lr, self.flags)
+
+
+def host_memory_available() -> int:
+    try:
+        import psutil
+        avail = psutil.virtual_memory().available
+    except Exception:
+        avail = 8 << 30
+    for p in ("/sys/fs/cgroup/memory.max", "/sys/fs/cgroup/memory/memory.limit_in_bytes"):
+        try:
+            v = open(p).read().strip()
+            if v.isdigit():
+                used = 0
+                try:
+                    used = int(open(os.path.join(os.path.dirname(p), "memory.current")).read())
+                except Exception:
+                    pass
+                avail = min(avail, int(v) - used)
+        except OSError:
+            pass
+    return avail
+
+
+def run_e2e(st: DeviceState, steps: int, world: int):
+    """The same step with HOST inputs and outputs: every step copies the replicas' parameters
+    from pinned host memory to the device, runs the two calls, and reads the messages and the
+    new theta_global back.  Returns (ms per step, h2d bytes, d2h bytes, note)."""
+    wl = st.wl
+    n = wl.n_total
+    need = n * 4
+    budget = int(host_memory_available() * 0.5)
+    pool = max(1, min(wl.R, budget // need - 1))
+    host_tl = [torch.empty(n, dtype=torch.float32).pin_memory() for _ in range(pool)]
+    for p in range(pool):
+        host_tl[p].copy_(st.theta_local[p])
+    host_tg = torch.empty(n, dtype=torch.float32).pin_memory()
+    host_msgs = [[torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in grp]
+                 for grp in (st.idx, st.codes, st.scales)]
+    torch.cuda.synchronize()
+    h2d = wl.R * n * 4
+    d2h = n * 4 + sum(t.numel() * t.element_size() for grp in host_msgs for t in grp)
+    times = []
+    for s in range(steps + 1):
+        barrier(world)
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for r in range(wl.R):
+            st.theta_local[r].copy_(host_tl[r % pool], non_blocking=True)
+        st.compress()
+        for grp_d, grp_h in zip((st.idx, st.codes, st.scales), host_msgs):
+            for d, h in zip(grp_d, grp_h):
+                h.copy_(d, non_blocking=True)
+        st.aggregate_apply()
+        host_tg.copy_(st.theta_global, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize()
+        if s > 0:   # the first pass warms the pinned pages and the copy engines
+            times.append(e0.elapsed_time(e1))
+    note = f"pinned pool of {pool} distinct replica buffers" + ("" if pool == wl.R else f" reused for R={wl.R}")
+    del host_tl, host_tg, host_msgs
+    return float(np.mean(times)), h2d, d2h, note
+
+
+def run_ours(args) -> None:
+    from paper_2601_02360_b200 import api
+    rank, local, world = init_dist("nccl")
+    assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    api.load()
+    wl = synth.workload(args.workload)
+    if args.R:
+        wl = wl.replace(R=args.R)
+    if args.k:
+        wl = wl.replace(k=args.k)
+    st = DeviceState(wl, rank_seed(args.seed, rank), dev)
+    stream = torch.cuda.current_stream()
+
+    sampler = ClockSampler(local)
+    t_step, t_comp, t_agg = [], [], []
+    for s in range(args.warmup + args.steps):
+        st.redraw_locals(s)
+        if s == args.warmup:
+            barrier(world)
+            torch.cuda.synchronize()
+            if rank == 0:
+                sampler.start()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(stream)
+        st.compress()
+        ev[1].record(stream)
+        st.aggregate_apply()
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            t_comp.append(ev[0].elapsed_time(ev[1]))
+            t_agg.append(ev[1].elapsed_time(ev[2]))
+            t_step.append(ev[0].elapsed_time(ev[2]))
+    torch.cuda.synchronize()
+    barrier(world)
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = max_over_ranks(float(np.sum(t_step)), world, dev)
+    ms_per_step = total_ms / args.steps
+    flags = int(st.flags.item())
+
+    e2e = None
+    if not args.no_e2e:
+        e_ms, h2d, d2h, note = run_e2e(st, args.e2e_steps, world)
+        e_ms = max_over_ranks(e_ms, world, dev)
+        e2e = {"value": job_value(wl.n_total, world, e_ms), "unit": UNIT, "ms_per_step": e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "note": note}
+
+    if rank != 0:
+        return
+    peak, peak_src = measured_peak_gbs()
+    comp_ms = float(np.mean(t_comp))
+    agg_ms = float(np.mean(t_agg))
+    achieved = compress_bytes(wl) / (comp_ms * 1e-3) / 1e9
+    traffic = None
+    try:
+        prof = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
+        per_unit = prof.get("compress_dram_bytes_per_replica_element")
+        if per_unit:
+            traffic = per_unit * wl.n_total * wl.R
+    except Exception:
+        pass
+    line = {
+        "metric": METRIC, "value": job_value(wl.n_total, world, ms_per_step), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "params": wl.n_total, "tensors": len(wl.tensors),
+                   "chunks": wl.n_chunks(), "R": wl.R, "k": wl.k, "bits": wl.bits, "chunk": wl.chunk,
+                   "beta": wl.beta, "outer_lr": wl.outer_lr,
+                   "l2": "inputs (GBs per launch) far larger than the 126 MB L2; no flush needed",
+                   "sharding": "none: every rank runs an independent parameter set" if world > 1 else "single GPU",
+                   "step": "sl_compress_batch + sl_aggregate_apply; theta_local re-drawn between steps (untimed)"},
+        "step_hbm": {"bytes_strict": step_bytes_strict(wl),
+                     "gbs_strict": step_bytes_strict(wl) / (np.mean(t_step) * 1e-3) / 1e9,
+                     "frac_of_peak": step_bytes_strict(wl) / (np.mean(t_step) * 1e-3) / 1e9 / peak,
+                     "frac_of_8tbs": step_bytes_strict(wl) / (np.mean(t_step) * 1e-3) / 1e9 / 8000.0},
+        "kernels_ms": {"sl_compress_batch": comp_ms, "sl_aggregate_apply": agg_ms},
+        "roofline": {"kernel": "sl_compress_batch", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "algorithmic_bytes": compress_bytes(wl)},
+        "clocks": clocks, "device_flags": flags,
+        "gpu_launches": 2 * args.steps,
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if not args.no_cpu:
+        sample = cpu_sample_workload(wl)
+        n_s = sample.n_total
+        inputs = (st.theta_global[:n_s].cpu().numpy(), [t[:n_s].cpu().numpy() for t in st.theta_local])
+        times, threads = time_oracle(sample, 1, 0, args.seed, inputs=inputs)
+        cpu_ms = float(np.mean(times))
+        line["cpu_baseline"] = {
+            "value": n_s / (cpu_ms * 1e-3), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "ms": cpu_ms,
+            "sample": f"first {len(sample.tensors)} tensors of the workload ({n_s} params) x R={wl.R}, "
+                      f"one outer step, replicas spread over {threads} host threads"}
+    print(json.dumps(line))
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="1b", choices=["tiny", "180m", "0p5b", "1b"])
+    ap.add_argument("--R", type=int, default=0)
+    ap.add_argument("--k", type=int, default=0)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

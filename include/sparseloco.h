@@ -1,0 +1,132 @@
+/* sparseloco.h — C ABI of the SparseLoCo outer synchronisation step on NVIDIA B200 (sm_100a).
+ *
+ * The step is Eq. 2 of the paper (§2.1, "Background: SparseLoCo"), run every H inner steps:
+ *
+ *   line 1   delta   = theta_global - theta_local                  (pseudo-gradient)
+ *   line 2   e'      = beta * e + delta                            (error feedback)
+ *   line 3   message = Q(Top-k(e'))   k largest magnitudes of every chunk, then quantised
+ *   line 4   e       = e' - message                                (what was sent leaves the buffer)
+ *   line 5   update  = (1/R) * sum_r message_r ;  theta_global -= outer_lr * update
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - Every data pointer is a DEVICE pointer unless it is marked HOST.  The caller owns every
+ *    buffer; the library allocates nothing and keeps no state between calls.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *    and use the current CUDA device.  Host arrays (layout offsets, pointer tables) are read
+ *    before the call returns.
+ *  - Return value: SL_OK or a negative SL_ERR_*; nothing throws, aborts or prints.  All argument
+ *    checks happen on the host before anything is launched.  Conditions met on the device never
+ *    trap: they OR a bit into `*flags`.
+ *  - Arithmetic is IEEE binary32, round-to-nearest-even, denormals kept, each operation rounded
+ *    once; beta*e + delta and theta - outer_lr*update are single fused roundings.
+ *
+ * Arena and chunks
+ * ----------------
+ *  Parameters live in a flat fp32 arena of `n_total` elements holding `n_tensors` tensors back
+ *  to back (row-major).  Chunks are runs of `chunk` consecutive elements of ONE tensor (the
+ *  paper's 64 x 64 = 4096 elements, §3 "Training Configuration", Table 8); the last chunk of a
+ *  tensor may be short and keeps k_eff = min(k, its length).  Chunks are numbered through the
+ *  arena in order: chunk g owns idx[g*k .. g*k+k), codes[g*stride .. (g+1)*stride), scales[g].
+ *
+ * Message of one chunk
+ * --------------------
+ *  idx    uint16[k]  chunk-local positions of the kept elements, ascending; unused slots 0xFFFF.
+ *  scales float      s = largest magnitude of e' in the chunk.
+ *  codes  bits in {2,4,8}: slot j's code sits at bit j*bits of the chunk's `stride` bytes,
+ *         least-significant bits first.  With L = 2^(bits-1): code = sign << (bits-1) | q,
+ *         q = number of thresholds s*(j/L), j = 1..L-1, that |e'| reaches; the value it stands
+ *         for is sign * s * (2q+1)/(2L).  bits = 32: no quantisation (the paper's own runs, §3),
+ *         codes is float[k] per chunk holding e' verbatim.
+ *  Ties in magnitude go to the lower position; +0 and -0 tie; values are ordered by the low 31
+ *  bits of their pattern, so NaN > Inf > finite and nothing is sanitised (SL_FLAG_NONFINITE).
+ */
+#ifndef SPARSELOCO_H_
+#define SPARSELOCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  SL_OK = 0,
+  SL_ERR_INVALID_ARG = -1, /* null pointer, k < 1, k > chunk, bits not in {2,4,8,32}, R out of range,
+                              beta / outer_lr not finite, offsets not ascending or not ending at n_total */
+  SL_ERR_ALIGNMENT = -2,   /* a float pointer not 4-byte aligned or idx not 2-byte aligned */
+  SL_ERR_UNSUPPORTED = -3, /* chunk > SL_MAX_CHUNK, n_tensors > SL_MAX_TENSORS, more than 2^31 chunks */
+  SL_ERR_CUDA = -4         /* a CUDA runtime call or a launch failed (the error is not cleared) */
+};
+
+enum {
+  SL_FLAG_NONFINITE = 1u, /* some chunk's largest magnitude was Inf or NaN */
+  SL_FLAG_BAD_INDEX = 2u  /* sl_aggregate*: a message slot named a position past its chunk; skipped */
+};
+
+#define SL_MAX_CHUNK 8192     /* elements; any chunk size in [1, SL_MAX_CHUNK] is accepted */
+#define SL_MAX_TENSORS 2048   /* tensors per call; split larger arenas into several calls */
+#define SL_MAX_REPLICAS 64    /* replicas per batched / aggregate call */
+
+/* HOST description of an arena.  offset[0] = 0 < ... (non-decreasing) ... offset[n_tensors] =
+ * n_total.  A single tensor is n_tensors = 1, offset = {0, n}.  The tuned kernels need every
+ * offset to be a multiple of 4 elements and every arena pointer 16-byte aligned; otherwise the
+ * calls fall back to a slower kernel with identical results. */
+typedef struct sl_layout {
+  uint64_t n_total;
+  uint32_t n_tensors;
+  const uint64_t* offset; /* HOST, [n_tensors + 1] */
+} sl_layout;
+
+/* Number of chunks of the arena, sum over tensors of ceil(n_t / chunk).  0 on bad arguments. */
+uint64_t sl_num_chunks(const sl_layout* layout, int chunk);
+
+/* Bytes of `codes` ONE chunk owns: ceil(k*bits/8), or 4*k when bits == 32.  0 on bad arguments.
+ * A replica's codes buffer is sl_num_chunks() * sl_codes_stride() bytes. */
+uint64_t sl_codes_stride(int k, int bits);
+
+/* Eq. 2 lines 1-4 for ONE replica: pseudo-gradient, error feedback, chunk-wise Top-k,
+ * quantisation, residual.
+ *   theta_local, theta_global  [n_total] read only
+ *   err     [n_total] read and overwritten in place with the residual (persists across steps)
+ *   idx     [n_c * k], codes [n_c * stride] bytes, scales [n_c]: fully overwritten
+ *   flags   optional device word, sticky OR of SL_FLAG_*; never cleared by the library */
+int sl_compress(const float* theta_local, const float* theta_global, float* err,
+                const sl_layout* layout, float beta, int chunk, int k, int bits,
+                uint16_t* idx, uint8_t* codes, float* scales, uint32_t* flags, void* stream);
+
+/* The same for R replicas that share theta_global, in one launch; results are identical to R
+ * calls of sl_compress.  The pointer tables are HOST arrays of R DEVICE pointers.  theta_global
+ * is fetched from memory once per chunk for all replicas. */
+int sl_compress_batch(int R, const float* const* theta_local, const float* theta_global,
+                      float* const* err, const sl_layout* layout, float beta, int chunk, int k,
+                      int bits, uint16_t* const* idx, uint8_t* const* codes, float* const* scales,
+                      uint32_t* flags, void* stream);
+
+/* Eq. 2 line 5, first half: decompress R messages and average them into a dense update.
+ * Replicas are added in the order 0..R-1 starting from +0 and the sum is divided by R (always
+ * R, however many replicas sent a position).  `update` [n_total] is fully overwritten;
+ * positions nobody sent are +0.  A slot whose position is >= its chunk's length (other than the
+ * 0xFFFF padding) is skipped and raises SL_FLAG_BAD_INDEX. */
+int sl_aggregate(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                 const float* const* scales, const sl_layout* layout, int chunk, int k, int bits,
+                 float* update, uint32_t* flags, void* stream);
+
+/* Eq. 2 line 5, second half: plain SGD outer step (no momentum, Table 8),
+ * theta_global[i] = fma(-outer_lr, update[i], theta_global[i]) for i < n. */
+int sl_outer_apply(float* theta_global, const float* update, uint64_t n, float outer_lr, void* stream);
+
+/* Both halves of line 5 in one pass: the dense update lives in shared memory only and
+ * theta_global is read and written once.  Same result as sl_aggregate + sl_outer_apply. */
+int sl_aggregate_apply(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                       const float* const* scales, const sl_layout* layout, int chunk, int k,
+                       int bits, float* theta_global, float outer_lr, uint32_t* flags, void* stream);
+
+/* Static description of an SL_* return code. */
+const char* sl_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPARSELOCO_H_ */

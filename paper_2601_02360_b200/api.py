@@ -1,0 +1,184 @@
+"""Thin Python binding of the C ABI in include/sparseloco.h (argument marshalling only).
+
+Every function has the name and the meaning of the C entry point it forwards
+to; tensors are torch CUDA tensors whose device pointers are passed through.
+All work happens in the CUDA library `csrc/libsparseloco.so`; there is no
+Python or CPU implementation behind these calls, and a missing or unloadable
+library raises instead of falling back.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+SL_OK, SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_CUDA = 0, -1, -2, -3, -4
+SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX = 1, 2
+SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 2048, 64
+
+EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
+           "sl_outer_apply", "sl_aggregate_apply", "sl_strerror")
+
+
+class SlLayout(ctypes.Structure):
+    _fields_ = [("n_total", ctypes.c_uint64), ("n_tensors", ctypes.c_uint32),
+                ("offset", ctypes.POINTER(ctypes.c_uint64))]
+
+
+class SparseLoCoError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def load(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads the CUDA library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _build.LIB_PATH
+    if not os.path.exists(p):
+        raise RuntimeError(f"{p} is missing: build it with `python -m paper_2601_02360_b200.build` "
+                           "(there is no fallback path)")
+    L = ctypes.CDLL(p)
+    vp, u64, i32, f32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int, ctypes.c_float
+    lp = ctypes.POINTER(SlLayout)
+    L.sl_num_chunks.restype = u64
+    L.sl_num_chunks.argtypes = [lp, i32]
+    L.sl_codes_stride.restype = u64
+    L.sl_codes_stride.argtypes = [i32, i32]
+    L.sl_compress.restype = i32
+    L.sl_compress.argtypes = [vp, vp, vp, lp, f32, i32, i32, i32, vp, vp, vp, vp, vp]
+    L.sl_compress_batch.restype = i32
+    L.sl_compress_batch.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, vp, vp, vp, vp, vp]
+    L.sl_aggregate.restype = i32
+    L.sl_aggregate.argtypes = [i32, vp, vp, vp, lp, i32, i32, i32, vp, vp, vp]
+    L.sl_outer_apply.restype = i32
+    L.sl_outer_apply.argtypes = [vp, vp, u64, f32, vp]
+    L.sl_aggregate_apply.restype = i32
+    L.sl_aggregate_apply.argtypes = [i32, vp, vp, vp, lp, i32, i32, i32, vp, f32, vp, vp]
+    L.sl_strerror.restype = ctypes.c_char_p
+    L.sl_strerror.argtypes = [i32]
+    if path is None:
+        _lib = L
+    return L
+
+
+def strerror(code: int) -> str:
+    return load().sl_strerror(code).decode()
+
+
+class Layout:
+    """Host description of an arena (`sl_layout`): element offsets of its tensors."""
+
+    def __init__(self, offsets: Sequence[int]):
+        self.offsets = np.ascontiguousarray(np.asarray(offsets, dtype=np.uint64))
+        assert self.offsets.ndim == 1 and len(self.offsets) >= 1
+        self.c = SlLayout(int(self.offsets[-1]), len(self.offsets) - 1,
+                          self.offsets.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)))
+
+    @property
+    def n_total(self) -> int:
+        return int(self.offsets[-1])
+
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def _layout(layout) -> Layout:
+    return layout if isinstance(layout, Layout) else Layout(layout)
+
+
+def _ptr(t) -> int:
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _ptr_table(ts: Sequence) -> ctypes.Array:
+    a = (ctypes.c_void_p * len(ts))()
+    for i, t in enumerate(ts):
+        a[i] = _ptr(t)
+    return a
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != SL_OK:
+        raise SparseLoCoError(rc, what)
+
+
+def sl_num_chunks(layout, chunk: int) -> int:
+    return int(load().sl_num_chunks(_layout(layout).ref(), chunk))
+
+
+def sl_codes_stride(k: int, bits: int) -> int:
+    return int(load().sl_codes_stride(k, bits))
+
+
+def sl_compress(theta_local, theta_global, err, layout, beta: float, chunk: int, k: int, bits: int,
+                idx, codes, scales, flags=None, stream=None) -> None:
+    _check(load().sl_compress(_ptr(theta_local), _ptr(theta_global), _ptr(err), _layout(layout).ref(),
+                              beta, chunk, k, bits, _ptr(idx), _ptr(codes), _ptr(scales), _ptr(flags),
+                              _stream(stream)), "sl_compress")
+
+
+def sl_compress_batch(theta_local: Sequence, theta_global, err: Sequence, layout, beta: float, chunk: int,
+                      k: int, bits: int, idx: Sequence, codes: Sequence, scales: Sequence, flags=None,
+                      stream=None) -> None:
+    R = len(theta_local)
+    assert len(err) == len(idx) == len(codes) == len(scales) == R
+    _check(load().sl_compress_batch(R, _ptr_table(theta_local), _ptr(theta_global), _ptr_table(err),
+                                    _layout(layout).ref(), beta, chunk, k, bits, _ptr_table(idx),
+                                    _ptr_table(codes), _ptr_table(scales), _ptr(flags), _stream(stream)),
+           "sl_compress_batch")
+
+
+def sl_aggregate(idx: Sequence, codes: Sequence, scales: Sequence, layout, chunk: int, k: int, bits: int,
+                 update, flags=None, stream=None) -> None:
+    R = len(idx)
+    assert len(codes) == len(scales) == R
+    _check(load().sl_aggregate(R, _ptr_table(idx), _ptr_table(codes), _ptr_table(scales),
+                               _layout(layout).ref(), chunk, k, bits, _ptr(update), _ptr(flags),
+                               _stream(stream)), "sl_aggregate")
+
+
+def sl_outer_apply(theta_global, update, n: int, outer_lr: float, stream=None) -> None:
+    _check(load().sl_outer_apply(_ptr(theta_global), _ptr(update), n, outer_lr, _stream(stream)),
+           "sl_outer_apply")
+
+
+def sl_aggregate_apply(idx: Sequence, codes: Sequence, scales: Sequence, layout, chunk: int, k: int,
+                       bits: int, theta_global, outer_lr: float, flags=None, stream=None) -> None:
+    R = len(idx)
+    assert len(codes) == len(scales) == R
+    _check(load().sl_aggregate_apply(R, _ptr_table(idx), _ptr_table(codes), _ptr_table(scales),
+                                     _layout(layout).ref(), chunk, k, bits, _ptr(theta_global), outer_lr,
+                                     _ptr(flags), _stream(stream)), "sl_aggregate_apply")
+
+
+def alloc_messages(layout, chunk: int, k: int, bits: int, R: int, device="cuda"):
+    """Device buffers for R replicas' messages: lists (idx, codes, scales)."""
+    nc = sl_num_chunks(layout, chunk)
+    st = sl_codes_stride(k, bits)
+    idx = [torch.empty(nc * k, dtype=torch.uint16, device=device) for _ in range(R)]
+    codes = [torch.empty(nc * st, dtype=torch.uint8, device=device) for _ in range(R)]
+    scales = [torch.empty(nc, dtype=torch.float32, device=device) for _ in range(R)]
+    return idx, codes, scales

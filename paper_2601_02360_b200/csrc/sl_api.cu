@@ -1,0 +1,219 @@
+// Host side of the C ABI declared in include/sparseloco.h: argument checks, the by-value
+// arena table, dispatch.  No allocation, no state, no synchronisation.
+#include <cmath>
+#include <memory>
+#include <new>
+
+#include "sl_common.cuh"
+
+namespace {
+
+using namespace sl;
+
+inline bool bits_ok(int bits) { return bits == 2 || bits == 4 || bits == 8 || bits == 32; }
+inline bool aligned(const void* p, uintptr_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+
+inline uint64_t codes_stride(int k, int bits) {
+  return bits == 32 ? (uint64_t)k * 4u : ((uint64_t)k * (uint64_t)bits + 7u) / 8u;
+}
+
+int check_common(const sl_layout* L, int chunk, int k, int bits) {
+  if (!L || !L->offset) return SL_ERR_INVALID_ARG;
+  if (chunk < 1 || k < 1 || k > chunk || !bits_ok(bits)) return SL_ERR_INVALID_ARG;
+  if (chunk > SL_MAX_CHUNK) return SL_ERR_UNSUPPORTED;
+  if (L->n_tensors < 1) return SL_ERR_INVALID_ARG;
+  if (L->n_tensors > SL_MAX_TENSORS) return SL_ERR_UNSUPPORTED;
+  if (L->offset[0] != 0 || L->offset[L->n_tensors] != L->n_total) return SL_ERR_INVALID_ARG;
+  uint64_t nc = 0;
+  for (uint32_t t = 0; t < L->n_tensors; ++t) {
+    if (L->offset[t + 1] < L->offset[t]) return SL_ERR_INVALID_ARG;
+    nc += (L->offset[t + 1] - L->offset[t] + (uint64_t)chunk - 1) / (uint64_t)chunk;
+  }
+  if (nc > 0x7FFFFFFFull) return SL_ERR_UNSUPPORTED;
+  return SL_OK;
+}
+
+template <int T>
+void fill_table(Table<T>& tb, const sl_layout* L, int chunk, bool* offsets_mult4) {
+  tb.n_tensors = L->n_tensors;
+  uint32_t nc = 0;
+  bool m4 = true;
+  for (uint32_t t = 0; t < L->n_tensors; ++t) {
+    tb.first_chunk[t] = nc;
+    tb.offset[t] = L->offset[t];
+    m4 = m4 && (L->offset[t] % 4 == 0);
+    nc += (uint32_t)((L->offset[t + 1] - L->offset[t] + (uint64_t)chunk - 1) / (uint64_t)chunk);
+  }
+  tb.first_chunk[L->n_tensors] = nc;
+  tb.offset[L->n_tensors] = L->n_total;
+  m4 = m4 && (L->n_total % 4 == 0);
+  tb.n_chunks = nc;
+  *offsets_mult4 = m4;
+}
+
+template <int T>
+int compress_impl(int R, const float* const* theta_local, const float* theta_global, float* const* err,
+                  const sl_layout* L, float beta, int chunk, int k, int bits, uint16_t* const* idx,
+                  uint8_t* const* codes, float* const* scales, uint32_t* flags, cudaStream_t st) {
+  std::unique_ptr<CompressArgs<T>> a(new (std::nothrow) CompressArgs<T>);
+  if (!a) return SL_ERR_CUDA;
+  bool m4;
+  fill_table(a->tb, L, chunk, &m4);
+  bool al16 = m4 && aligned(theta_global, 16);
+  for (int r = 0; r < R; ++r) {
+    a->p.theta_local[r] = theta_local[r];
+    a->p.err[r] = err[r];
+    a->p.idx[r] = idx[r];
+    a->p.codes[r] = codes[r];
+    a->p.scales[r] = scales[r];
+    al16 = al16 && aligned(theta_local[r], 16) && aligned(err[r], 16) && aligned(idx[r], 16) &&
+           aligned(codes[r], 16) && aligned(scales[r], 4);
+  }
+  a->theta_global = theta_global;
+  a->flags = flags;
+  a->beta = beta;
+  a->chunk = chunk;
+  a->k = k;
+  a->bits = bits;
+  a->R = R;
+  a->stride = (uint32_t)codes_stride(k, bits);
+  return launch_compress<T>(*a, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+}
+
+int compress_checked(int R, const float* const* theta_local, const float* theta_global,
+                     float* const* err, const sl_layout* L, float beta, int chunk, int k, int bits,
+                     uint16_t* const* idx, uint8_t* const* codes, float* const* scales,
+                     uint32_t* flags, void* stream) {
+  if (R < 1 || R > SL_MAX_REPLICAS) return SL_ERR_INVALID_ARG;
+  if (!theta_local || !theta_global || !err || !idx || !codes || !scales) return SL_ERR_INVALID_ARG;
+  if (!std::isfinite(beta)) return SL_ERR_INVALID_ARG;
+  const int rc = check_common(L, chunk, k, bits);
+  if (rc != SL_OK) return rc;
+  if (!aligned(theta_global, 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
+  for (int r = 0; r < R; ++r) {
+    if (!theta_local[r] || !err[r] || !idx[r] || !codes[r] || !scales[r]) return SL_ERR_INVALID_ARG;
+    if (!aligned(theta_local[r], 4) || !aligned(err[r], 4) || !aligned(scales[r], 4) ||
+        !aligned(idx[r], 2) || (bits == 32 && !aligned(codes[r], 4)))
+      return SL_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  if (L->n_tensors <= 256)
+    return compress_impl<256>(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx, codes,
+                              scales, flags, st);
+  return compress_impl<SL_MAX_TENSORS>(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx,
+                                       codes, scales, flags, st);
+}
+
+template <int T>
+int aggregate_impl(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                   const float* const* scales, const sl_layout* L, int chunk, int k, int bits, float* out,
+                   float outer_lr, bool apply, uint32_t* flags, cudaStream_t st) {
+  std::unique_ptr<AggregateArgs<T>> a(new (std::nothrow) AggregateArgs<T>);
+  if (!a) return SL_ERR_CUDA;
+  bool m4;
+  fill_table(a->tb, L, chunk, &m4);
+  bool al16 = m4 && aligned(out, 16);
+  for (int r = 0; r < R; ++r) {
+    a->m.idx[r] = idx[r];
+    a->m.codes[r] = codes[r];
+    a->m.scales[r] = scales[r];
+    al16 = al16 && aligned(idx[r], 16) && aligned(codes[r], 16);
+  }
+  a->out = out;
+  a->flags = flags;
+  a->outer_lr = outer_lr;
+  a->chunk = chunk;
+  a->k = k;
+  a->bits = bits;
+  a->R = R;
+  a->stride = (uint32_t)codes_stride(k, bits);
+  return launch_aggregate<T>(*a, apply, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+}
+
+int aggregate_checked(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                      const float* const* scales, const sl_layout* L, int chunk, int k, int bits,
+                      float* out, float outer_lr, bool apply, uint32_t* flags, void* stream) {
+  if (R < 1 || R > SL_MAX_REPLICAS) return SL_ERR_INVALID_ARG;
+  if (!idx || !codes || !scales || !out) return SL_ERR_INVALID_ARG;
+  if (!std::isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
+  const int rc = check_common(L, chunk, k, bits);
+  if (rc != SL_OK) return rc;
+  if (!aligned(out, 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
+  for (int r = 0; r < R; ++r) {
+    if (!idx[r] || !codes[r] || !scales[r]) return SL_ERR_INVALID_ARG;
+    if (!aligned(idx[r], 2) || !aligned(scales[r], 4) || (bits == 32 && !aligned(codes[r], 4)))
+      return SL_ERR_ALIGNMENT;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  if (L->n_tensors <= 256)
+    return aggregate_impl<256>(R, idx, codes, scales, L, chunk, k, bits, out, outer_lr, apply, flags, st);
+  return aggregate_impl<SL_MAX_TENSORS>(R, idx, codes, scales, L, chunk, k, bits, out, outer_lr, apply,
+                                        flags, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+uint64_t sl_num_chunks(const sl_layout* L, int chunk) {
+  if (!L || !L->offset || chunk < 1) return 0;
+  uint64_t nc = 0;
+  for (uint32_t t = 0; t < L->n_tensors; ++t) {
+    if (L->offset[t + 1] < L->offset[t]) return 0;
+    nc += (L->offset[t + 1] - L->offset[t] + (uint64_t)chunk - 1) / (uint64_t)chunk;
+  }
+  return nc;
+}
+
+uint64_t sl_codes_stride(int k, int bits) {
+  if (k < 1 || !bits_ok(bits)) return 0;
+  return codes_stride(k, bits);
+}
+
+int sl_compress(const float* theta_local, const float* theta_global, float* err, const sl_layout* L,
+                float beta, int chunk, int k, int bits, uint16_t* idx, uint8_t* codes, float* scales,
+                uint32_t* flags, void* stream) {
+  return compress_checked(1, &theta_local, theta_global, &err, L, beta, chunk, k, bits, &idx, &codes,
+                          &scales, flags, stream);
+}
+
+int sl_compress_batch(int R, const float* const* theta_local, const float* theta_global,
+                      float* const* err, const sl_layout* L, float beta, int chunk, int k, int bits,
+                      uint16_t* const* idx, uint8_t* const* codes, float* const* scales,
+                      uint32_t* flags, void* stream) {
+  return compress_checked(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx, codes, scales,
+                          flags, stream);
+}
+
+int sl_aggregate(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                 const float* const* scales, const sl_layout* L, int chunk, int k, int bits,
+                 float* update, uint32_t* flags, void* stream) {
+  return aggregate_checked(R, idx, codes, scales, L, chunk, k, bits, update, 0.0f, false, flags, stream);
+}
+
+int sl_outer_apply(float* theta_global, const float* update, uint64_t n, float outer_lr, void* stream) {
+  if (!theta_global || !update || !std::isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
+  if (!aligned(theta_global, 4) || !aligned(update, 4)) return SL_ERR_ALIGNMENT;
+  return launch_outer_apply(theta_global, update, n, outer_lr, (cudaStream_t)stream) == cudaSuccess
+             ? SL_OK : SL_ERR_CUDA;
+}
+
+int sl_aggregate_apply(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                       const float* const* scales, const sl_layout* L, int chunk, int k, int bits,
+                       float* theta_global, float outer_lr, uint32_t* flags, void* stream) {
+  return aggregate_checked(R, idx, codes, scales, L, chunk, k, bits, theta_global, outer_lr, true, flags,
+                           stream);
+}
+
+const char* sl_strerror(int code) {
+  switch (code) {
+    case SL_OK: return "ok";
+    case SL_ERR_INVALID_ARG: return "invalid argument";
+    case SL_ERR_ALIGNMENT: return "misaligned pointer";
+    case SL_ERR_UNSUPPORTED: return "size outside what this build supports";
+    case SL_ERR_CUDA: return "CUDA runtime or launch failure";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

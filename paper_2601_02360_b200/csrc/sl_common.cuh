@@ -1,0 +1,122 @@
+// Shared device-side pieces of the SparseLoCo outer-step kernels (paper §2.1, Eq. 2).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sparseloco.h"
+
+namespace sl {
+
+// ---------------------------------------------------------------------------
+// arena description handed to the kernels BY VALUE (kernel parameter space =
+// constant bank), so that the library needs no device-side table and no state.
+// first_chunk[t] = number of chunks owned by tensors before t.
+// ---------------------------------------------------------------------------
+template <int T>
+struct Table {
+  uint32_t n_tensors;
+  uint32_t n_chunks;
+  uint32_t first_chunk[T + 1];
+  uint64_t offset[T + 1];
+};
+
+struct ChunkRef {
+  uint64_t base;  // element offset of the chunk in the arena
+  int len;        // elements in the chunk (1..chunk)
+};
+
+// chunk g -> (base, len): binary search over the tensors' first chunks
+template <int T>
+__device__ __forceinline__ ChunkRef locate(const Table<T>& tb, uint32_t g, int chunk) {
+  uint32_t lo = 0, hi = tb.n_tensors;  // first_chunk[lo] <= g < first_chunk[hi]
+  while (hi - lo > 1) {
+    const uint32_t mid = (lo + hi) >> 1;
+    if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
+  }
+  ChunkRef c;
+  c.base = tb.offset[lo] + (uint64_t)(g - tb.first_chunk[lo]) * (uint64_t)chunk;
+  const uint64_t left = tb.offset[lo + 1] - c.base;
+  c.len = left < (uint64_t)chunk ? (int)left : chunk;
+  return c;
+}
+
+// per-replica pointer tables, by value as well
+struct CompressPtrs {
+  const float* theta_local[SL_MAX_REPLICAS];
+  float* err[SL_MAX_REPLICAS];
+  uint16_t* idx[SL_MAX_REPLICAS];
+  uint8_t* codes[SL_MAX_REPLICAS];
+  float* scales[SL_MAX_REPLICAS];
+};
+
+struct MessagePtrs {
+  const uint16_t* idx[SL_MAX_REPLICAS];
+  const uint8_t* codes[SL_MAX_REPLICAS];
+  const float* scales[SL_MAX_REPLICAS];
+};
+
+template <int T>
+struct CompressArgs {
+  Table<T> tb;
+  CompressPtrs p;
+  const float* theta_global;
+  uint32_t* flags;
+  float beta;
+  int chunk, k, bits, R;
+  uint32_t stride;  // bytes of codes per chunk
+};
+
+template <int T>
+struct AggregateArgs {
+  Table<T> tb;
+  MessagePtrs m;
+  float* out;       // dense update (aggregate) or theta_global (aggregate + apply)
+  uint32_t* flags;
+  float outer_lr;
+  int chunk, k, bits, R;
+  uint32_t stride;
+};
+
+// ---------------------------------------------------------------------------
+// the quantiser Q of Eq. 2 line 3 (paper leaves Q open; this build's reading):
+// scale s = chunk maximum, L = 2^(bits-1) levels, thresholds s*(j/L),
+// reconstruction at the level's midpoint s*(2q+1)/(2L).  Every product is one
+// explicitly rounded multiply so that nothing can be contracted.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t key_of(float v) { return __float_as_uint(v) & 0x7FFFFFFFu; }
+
+// q = number of thresholds t_j = s*(j/L), j = 1..L-1, with |v| >= t_j.  The t_j are
+// non-decreasing in j, so the count is found by bisection on j.
+__device__ __forceinline__ uint32_t quant_level(float v, float s, int bits) {
+  const float a = fabsf(v);
+  if (bits == 2) return (a >= __fmul_rn(s, 0.5f)) ? 1u : 0u;
+  const int L = 1 << (bits - 1);
+  const float invL = 1.0f / (float)L;  // power of two: j * invL is exact
+  int lo = 0, hi = L - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (a >= __fmul_rn(s, (float)mid * invL)) lo = mid; else hi = mid - 1;
+  }
+  return (uint32_t)lo;
+}
+
+__device__ __forceinline__ uint32_t quant_code(float v, float s, int bits) {
+  return ((__float_as_uint(v) >> 31) << (bits - 1)) | quant_level(v, s, bits);
+}
+
+__device__ __forceinline__ float dequant(uint32_t code, float s, int bits) {
+  const int L = 1 << (bits - 1);
+  const uint32_t q = code & (uint32_t)(L - 1);
+  const uint32_t sign = (code >> (bits - 1)) & 1u;
+  const float mag = __fmul_rn(s, (float)(2u * q + 1u) * (0.5f / (float)L));
+  return __uint_as_float(__float_as_uint(mag) | (sign << 31));
+}
+
+// ---------------------------------------------------------------------------
+// launchers implemented in the kernel files (host side, return cudaError_t)
+// ---------------------------------------------------------------------------
+template <int T> cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream_t st);
+template <int T> cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned16, cudaStream_t st);
+cudaError_t launch_outer_apply(float* theta, const float* update, uint64_t n, float lr, cudaStream_t st);
+
+}  // namespace sl

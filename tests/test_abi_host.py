@@ -1,0 +1,98 @@
+"""Host-only checks of the C ABI: the library loads without a GPU, exports every symbol the
+header declares, and rejects bad arguments before anything is launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2601_02360_b200 import api, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "sparseloco.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return api.load()
+
+
+def _declared():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(sl_[a-z_]+)\s*\(", src)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert set(names) == set(api.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    with pytest.raises(RuntimeError, match="no fallback"):
+        api.load(str(tmp_path / "absent.so"))
+
+
+def test_sizes(lib):
+    lay = api.Layout([0, 4096 * 3 + 5, 4096 * 3 + 5, 4096 * 4 + 5 + 100])
+    assert api.sl_num_chunks(lay, 4096) == 4 + 0 + 2
+    assert api.sl_num_chunks(lay, 0) == 0
+    assert api.sl_codes_stride(64, 2) == 16
+    assert api.sl_codes_stride(2, 2) == 1
+    assert api.sl_codes_stride(63, 4) == 32
+    assert api.sl_codes_stride(32, 32) == 128
+    assert api.sl_codes_stride(64, 3) == 0
+    assert api.strerror(api.SL_OK) == "ok" and "align" in api.strerror(api.SL_ERR_ALIGNMENT)
+
+
+def _call_compress(lib, lay, chunk=4096, k=64, bits=2, beta=0.95, ptr=0x1000, idx=0x1000, R=None):
+    if R is None:
+        return lib.sl_compress(ptr, 0x1000, 0x1000, lay.ref(), beta, chunk, k, bits, idx, 0x1000, 0x1000, 0, 0)
+    tab = (ctypes.c_void_p * max(R, 1))(*([0x1000] * max(R, 1)))
+    return lib.sl_compress_batch(R, tab, 0x1000, tab, lay.ref(), beta, chunk, k, bits, tab, tab, tab, 0, 0)
+
+
+def test_bad_arguments_are_rejected_on_the_host(lib):
+    # every call below must return before any CUDA work: the pointers are fake
+    lay = api.Layout([0, 8192])
+    E = api
+    assert _call_compress(lib, lay, k=0) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, chunk=64, k=65) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, bits=3) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, chunk=0) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, beta=float("nan")) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, beta=float("inf")) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, ptr=0) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, chunk=api.SL_MAX_CHUNK + 1) == E.SL_ERR_UNSUPPORTED
+    assert _call_compress(lib, lay, ptr=0x1002) == E.SL_ERR_ALIGNMENT
+    assert _call_compress(lib, lay, idx=0x1001) == E.SL_ERR_ALIGNMENT
+    assert _call_compress(lib, lay, R=0) == E.SL_ERR_INVALID_ARG
+    assert _call_compress(lib, lay, R=api.SL_MAX_REPLICAS + 1) == E.SL_ERR_INVALID_ARG
+    assert lib.sl_compress(0x1000, 0x1000, 0x1000, None, 0.9, 4096, 64, 2, 0x1000, 0x1000, 0x1000, 0, 0) \
+        == E.SL_ERR_INVALID_ARG
+    bad = api.Layout([0, 100, 50, 200])           # offsets go backwards
+    assert _call_compress(lib, bad) == E.SL_ERR_INVALID_ARG
+    wrong_total = api.Layout([0, 100, 200])
+    wrong_total.c.n_total = 150
+    assert _call_compress(lib, wrong_total) == E.SL_ERR_INVALID_ARG
+    many = api.Layout(np.arange(api.SL_MAX_TENSORS + 2) * 4)
+    assert _call_compress(lib, many) == E.SL_ERR_UNSUPPORTED
+    tab = (ctypes.c_void_p * 2)(0x1000, 0x1000)
+    assert lib.sl_aggregate(2, tab, tab, tab, lay.ref(), 4096, 64, 2, 0, 0, 0) == E.SL_ERR_INVALID_ARG
+    assert lib.sl_aggregate(0, tab, tab, tab, lay.ref(), 4096, 64, 2, 0x1000, 0, 0) == E.SL_ERR_INVALID_ARG
+    assert lib.sl_aggregate_apply(2, tab, tab, tab, lay.ref(), 4096, 64, 2, 0x1000, float("nan"), 0, 0) \
+        == E.SL_ERR_INVALID_ARG
+    assert lib.sl_aggregate_apply(2, tab, tab, tab, lay.ref(), 4096, 64, 5, 0x1000, 1.0, 0, 0) \
+        == E.SL_ERR_INVALID_ARG
+    assert lib.sl_outer_apply(0, 0x1000, 10, 1.0, 0) == E.SL_ERR_INVALID_ARG
+    assert lib.sl_outer_apply(0x1001, 0x1000, 10, 1.0, 0) == E.SL_ERR_ALIGNMENT
+    assert lib.sl_outer_apply(0x1000, 0x1000, 10, float("inf"), 0) == E.SL_ERR_INVALID_ARG
+
+
+def test_binding_raises_with_the_library_message(lib):
+    with pytest.raises(api.SparseLoCoError, match="invalid argument"):
+        api.sl_compress(0x1000, 0x1000, 0x1000, [0, 8192], 0.9, 4096, 0, 2, 0x1000, 0x1000, 0x1000, None, 0)

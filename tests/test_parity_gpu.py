@@ -1,0 +1,290 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU checker, element by
+element on the same seeded inputs (bar: see parity_util)."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import slo
+from paper_2601_02360_b200 import api, synth
+from parity_util import (GpuStep, assert_close, assert_exact, compare_messages, oracle_compress_all,
+                         run_and_compare)
+
+pytestmark = pytest.mark.gpu
+f32 = np.float32
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand(n, seed, noise=1e-3, err=5e-4):
+    rng = np.random.default_rng(seed)
+    tg = rng.normal(0, 0.02, n).astype(f32)
+    return tg, rng, noise, err
+
+
+def _case(n, R, seed, noise=1e-3, err=5e-4):
+    tg, rng, _, _ = _rand(n, seed)
+    tls = [(tg + rng.normal(0, noise, n).astype(f32)).astype(f32) for _ in range(R)]
+    errs = [rng.normal(0, err, n).astype(f32) for _ in range(R)]
+    return tg, tls, errs
+
+
+def test_hand_worked_example_on_gpu():
+    g = json.load(open(os.path.join(GOLD, "w1_dyadic.json")))
+    tg = np.array(g["theta_global"], f32)
+    tls = [np.array(r["theta_local"], f32) for r in g["replicas"]]
+    errs = [np.array(r["err_in"], f32) for r in g["replicas"]]
+    gs = GpuStep([0, 8], 2, g["chunk"], g["k"], g["bits"])
+    gs.upload(tg, tls, errs)
+    gs.compress(g["beta"])
+    msgs = gs.messages_host()
+    for r, rep in enumerate(g["replicas"]):
+        assert msgs[r][0].tolist() == [rep["idx"]]
+        assert msgs[r][1].tolist() == [rep["packed"]]
+        assert msgs[r][2].tolist() == [rep["scale"]]
+        assert gs.err[r].cpu().numpy().tolist() == rep["err_out"]
+    gs.aggregate_apply(g["outer_lr"])
+    assert gs.theta_global.cpu().numpy().tolist() == g["theta_global_out"]
+
+
+def test_tiny_config():
+    wl = synth.workload("tiny")
+    tgt = synth.gen_theta_global(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r).numpy() for r in range(wl.R)]
+    errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    what="tiny")
+
+
+def test_tiny_config_three_rounds_carrying_err():
+    wl = synth.workload("tiny")
+    tgt = synth.gen_theta_global(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r).numpy() for r in range(wl.R)]
+    errs = [synth.gen_error(wl, r).numpy() for r in range(wl.R)]
+    nxt = lambda t, tg: [synth.gen_theta_local(wl, torch.from_numpy(tg), t, r).numpy() for r in range(wl.R)]
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    rounds=3, next_locals=nxt, what="tiny x3")
+
+
+@pytest.mark.parametrize("chunk,k,bits", [
+    (4096, 64, 2), (4096, 32, 2), (4096, 16, 2), (4096, 128, 2), (4096, 64, 4), (4096, 64, 8),
+    (4096, 32, 32), (4096, 1, 2), (4096, 4096, 32), (4096, 4096, 2), (8192, 100, 4), (256, 8, 2),
+    (100, 7, 8), (8, 2, 2), (1, 1, 32), (2048, 2048, 8), (4096, 60, 2), (4096, 63, 4),
+])
+def test_ragged_multi_tensor_arena(chunk, k, bits):
+    # several tiles plus ragged tails; tensor sizes that are NOT multiples of 4 elements
+    sizes = [3 * chunk + 5, 1, chunk, 7, 2 * chunk + chunk // 2 + 3, max(1, chunk // 3)]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), 3, seed=chunk * 131 + k * 7 + bits)
+    run_and_compare(off, tg, tls, errs, 0.95, chunk, k, bits, 0.8, what=f"ragged C{chunk} k{k} b{bits}")
+
+
+@pytest.mark.parametrize("k,bits", [(16, 2), (32, 2), (64, 2), (128, 2), (64, 4), (64, 8), (32, 32)])
+def test_aligned_arena_fast_path_shapes(k, bits):
+    # every tensor a multiple of 4 elements (the layout the tuned kernels accept), short tails included
+    sizes = [5 * 4096, 1024, 4096 + 2048, 512, 4, 3 * 4096 + 4092, 4096]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), 4, seed=k * 3 + bits)
+    run_and_compare(off, tg, tls, errs, 0.95, 4096, k, bits, 1.0, what=f"aligned k{k} b{bits}")
+
+
+def _adversarial_chunks(chunk, k):
+    """(name, e' target) chunks; built with theta_global = 0, err = 0, beta = 0 => e' = -theta_local."""
+    rng = np.random.default_rng(99)
+    out = {}
+    out["all_equal"] = np.full(chunk, 0.125, f32)
+    out["all_zero"] = np.zeros(chunk, f32)
+    z = np.zeros(chunk, f32); z[::2] = -0.0
+    out["signed_zeros"] = z
+    s = np.zeros(chunk, f32); s[chunk // 3] = -7.0
+    out["one_spike"] = s
+    t = rng.normal(0, 1, chunk).astype(f32)
+    kth = np.sort(np.abs(t))[-min(k, chunk)]
+    t[np.abs(t) < kth] = 0
+    dup = rng.choice(chunk, size=chunk // 4, replace=False)
+    t[dup] = kth * np.where(rng.random(len(dup)) < 0.5, -1, 1).astype(f32)   # many ties exactly at the k-th key
+    out["ties_at_boundary"] = t
+    out["two_levels"] = np.where(rng.random(chunk) < 0.5, f32(1.0), f32(-0.5)).astype(f32)
+    sub = (rng.integers(-50, 50, chunk) * f32(2.0 ** -149)).astype(f32)
+    out["subnormals"] = sub
+    d = np.round(rng.normal(0, 3, chunk)).astype(f32) * f32(2.0 ** -13)
+    out["dyadic_grid"] = d
+    big = rng.normal(0, 1, chunk).astype(f32) * f32(1e30)
+    out["huge"] = big
+    asc = np.arange(chunk, dtype=f32)
+    out["ascending"] = asc
+    out["descending"] = asc[::-1].copy()
+    return out
+
+
+@pytest.mark.parametrize("chunk,k,bits", [(4096, 64, 2), (4096, 128, 2), (4096, 16, 2), (4096, 64, 8),
+                                          (4096, 64, 32), (512, 64, 2), (4096, 1000, 4)])
+def test_adversarial_chunks(chunk, k, bits):
+    cases = _adversarial_chunks(chunk, k)
+    n = chunk * len(cases)
+    ep = np.concatenate(list(cases.values()))
+    tg = np.zeros(n, f32)
+    tls = [(-ep).astype(f32), np.roll(-ep, chunk).astype(f32)]
+    errs = [np.zeros(n, f32), np.zeros(n, f32)]
+    run_and_compare([0, n], tg, tls, errs, 0.0, chunk, k, bits, 1.0, what=f"adversarial C{chunk} k{k} b{bits}")
+
+
+def test_nonfinite_values_raise_the_flag_without_trapping():
+    chunk, k = 4096, 64
+    n = 3 * chunk
+    tg, tls, errs = _case(n, 2, seed=5)
+    tls[0][17] = np.inf
+    tls[0][chunk + 5] = np.nan
+    tls[1][2 * chunk + 100] = -np.inf
+    gs, _, _ = run_and_compare([0, n], tg, tls, errs, 0.95, chunk, k, 2, 1.0, what="nonfinite")
+    assert int(gs.flags.item()) & api.SL_FLAG_NONFINITE
+
+
+def test_batched_equals_per_replica_calls():
+    wl = synth.workload("tiny").replace(R=3)
+    tgt = synth.gen_theta_global(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r).numpy() for r in range(wl.R)]
+    errs = [synth.gen_error(wl, r).numpy() for r in range(wl.R)]
+    a = GpuStep(wl.offsets(), wl.R, wl.chunk, wl.k, wl.bits)
+    b = GpuStep(wl.offsets(), wl.R, wl.chunk, wl.k, wl.bits)
+    for g, batched in ((a, True), (b, False)):
+        g.upload(tgt.numpy(), tls, errs)
+        g.compress(wl.beta, batched=batched)
+    compare_messages(a.messages_host(), b.messages_host(), "batched vs single")
+    for r in range(wl.R):
+        assert torch.equal(a.err[r], b.err[r])
+
+
+def test_aggregate_then_apply_equals_fused_and_checker():
+    wl = synth.workload("tiny").replace(R=4)
+    off = wl.offsets()
+    tgt = synth.gen_theta_global(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r).numpy() for r in range(wl.R)]
+    errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    gs = GpuStep(off, wl.R, wl.chunk, wl.k, wl.bits)
+    gs.upload(tgt.numpy(), tls, errs)
+    gs.compress(wl.beta)
+    upd = torch.full((wl.n_total,), 7.0, dtype=torch.float32, device="cuda")  # must be fully overwritten
+    api.sl_aggregate(gs.idx, gs.codes, gs.scales, gs.layout, wl.chunk, wl.k, wl.bits, upd, gs.flags)
+    ora = slo.aggregate(gs.messages_host(), off, wl.chunk, wl.k, wl.bits)
+    assert_close(upd.cpu().numpy(), ora, "dense update")
+    th2 = gs.theta_global.clone()
+    api.sl_outer_apply(th2, upd, wl.n_total, 0.8)
+    gs.aggregate_apply(0.8)
+    assert torch.equal(th2, gs.theta_global)
+    want = tgt.numpy().copy()
+    slo.outer_apply(want, ora, 0.8)
+    assert_close(gs.theta_global.cpu().numpy(), want, "theta_global")
+    # a replica that dropped out: its message is left out, the caller passes fewer messages
+    upd3 = torch.empty_like(upd)
+    api.sl_aggregate(gs.idx[:3], gs.codes[:3], gs.scales[:3], gs.layout, wl.chunk, wl.k, wl.bits, upd3)
+    assert_close(upd3.cpu().numpy(), slo.aggregate(gs.messages_host()[:3], off, wl.chunk, wl.k, wl.bits),
+                 "three of four")
+    assert int(gs.flags.item()) == 0
+
+
+def test_aggregate_skips_out_of_range_positions_and_flags_them():
+    chunk, k = 256, 8
+    n = chunk + 40          # second chunk is 40 long
+    tg, tls, errs = _case(n, 1, seed=3)
+    gs = GpuStep([0, n], 1, chunk, k, 2)
+    gs.upload(tg, tls, errs)
+    gs.compress(0.9)
+    torch.cuda.synchronize()
+    idx = gs.idx[0].cpu().numpy().copy()
+    idx[k + 2] = 200        # beyond the short chunk's 40 elements
+    gs.idx[0].copy_(torch.from_numpy(idx))
+    upd = torch.empty(n, dtype=torch.float32, device="cuda")
+    api.sl_aggregate(gs.idx, gs.codes, gs.scales, gs.layout, chunk, k, 2, upd, gs.flags)
+    assert int(gs.flags.item()) & api.SL_FLAG_BAD_INDEX
+    idx[k + 2] = 0xFFFF     # the checker sees the slot as padding: same result
+    msgs = [(idx.reshape(2, k), gs.codes[0].cpu().numpy().reshape(2, -1), gs.scales[0].cpu().numpy())]
+    assert_close(upd.cpu().numpy(), slo.aggregate(msgs, [0, n], chunk, k, 2), "skipped slot")
+
+
+def test_outer_apply_unaligned_and_tail():
+    rng = np.random.default_rng(0)
+    for n, shift in [(1, 0), (5, 1), (1027, 0), (4099, 3), (1 << 20, 0)]:
+        th = rng.normal(0, 1, n + 4).astype(f32)
+        up = rng.normal(0, 1, n + 4).astype(f32)
+        dth = torch.from_numpy(th).cuda()
+        dup = torch.from_numpy(up).cuda()
+        api.sl_outer_apply(dth[shift:], dup[shift:], n, 0.8)
+        want = th.copy()
+        w = want[shift:shift + n]
+        slo.outer_apply(w, up[shift:shift + n].copy(), 0.8)
+        want[shift:shift + n] = w
+        assert_close(dth.cpu().numpy(), want, f"outer_apply n={n} shift={shift}")
+
+
+def test_checkpoint_resume_on_gpu_is_bit_identical():
+    wl = synth.workload("tiny")
+    off = wl.offsets()
+    def run(rounds, state=None):
+        gs = GpuStep(off, wl.R, wl.chunk, wl.k, wl.bits)
+        if state is None:
+            gs.theta_global.copy_(synth.gen_theta_global(wl))
+            t0 = 0
+        else:
+            gs.theta_global.copy_(state[0])
+            for r in range(wl.R):
+                gs.err[r].copy_(state[1][r])
+            t0 = state[2]
+        for t in range(t0, t0 + rounds):
+            for r in range(wl.R):
+                synth.gen_theta_local(wl, gs.theta_global, t, r, out=gs.theta_local[r])
+            gs.compress(wl.beta)
+            gs.aggregate_apply(wl.outer_lr)
+        torch.cuda.synchronize()
+        return gs.theta_global.cpu(), [e.cpu() for e in gs.err], t0 + rounds
+    a = run(4)
+    b = run(2, run(2))
+    assert torch.equal(a[0], b[0]) and all(torch.equal(x, y) for x, y in zip(a[1], b[1]))
+
+
+def test_180m_sub_arena_three_rounds():
+    full = synth.workload("180m")
+    # one whole layer (7 matrices + 2 norm vectors) and the final norm; value law of the full config
+    keep = list(range(9)) + [len(full.tensors) - 1]
+    wl = synth.sub_arena(full, keep)
+    tgt = synth.gen_theta_global(wl)
+    rho = synth.row_scales(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r, rho=rho).numpy() for r in range(wl.R)]
+    errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    nxt = lambda t, tg: [synth.gen_theta_local(wl, torch.from_numpy(tg), t, r, rho=rho).numpy()
+                         for r in range(wl.R)]
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    rounds=3, next_locals=nxt, what="180m sub-arena")
+
+
+@pytest.mark.parametrize("variant", ["ties_literal", "ties_dyadic"])
+def test_tie_heavy_variants(variant):
+    full = synth.workload("1b").replace(variant=variant, R=2)
+    keep = [0, 4, 7, 8]     # q (2048x2048), gate (2048x5632), two norm vectors
+    wl = synth.sub_arena(full, keep)
+    tgt = synth.gen_theta_global(wl)
+    rho = synth.row_scales(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r, rho=rho).numpy() for r in range(wl.R)]
+    errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    nxt = lambda t, tg: [synth.gen_theta_local(wl, torch.from_numpy(tg), t, r, rho=rho).numpy()
+                         for r in range(wl.R)]
+    if variant == "ties_dyadic":
+        # the stress is real only if the k-th and (k+1)-th magnitudes tie in most chunks
+        d = (tgt.numpy() - tls[0])[: 2048 * 2048].reshape(-1, 4096)
+        srt = np.sort(np.abs(d), axis=1)
+        assert (srt[:, -wl.k] == srt[:, -wl.k - 1]).mean() > 0.5
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    rounds=2, next_locals=nxt, what=variant)
+
+
+@pytest.mark.parametrize("k,R", [(16, 2), (32, 8), (128, 2)])
+def test_density_sweep_cells_on_sub_arena(k, R):
+    full = synth.workload("1b").replace(k=k, R=R)
+    wl = synth.sub_arena(full, [0, 6, 7])     # q, down, one norm vector
+    tgt = synth.gen_theta_global(wl)
+    rho = synth.row_scales(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r, rho=rho).numpy() for r in range(wl.R)]
+    errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    what=f"sweep k{k} R{R}")
