@@ -1,5 +1,13 @@
 // Eq. 2 lines 1-4 (paper §2.1): pseudo-gradient, error feedback, chunk-wise Top-k,
-// quantisation, residual.  One CTA owns one (chunk, replica) pair.
+// quantisation, residual.
+//
+// Two kernels with identical results:
+//   compress_generic_kernel  any chunk length / k / code width / alignment; one CTA per
+//                            (chunk, replica); exact 4-pass radix select in shared memory.
+//   compress_c4096_kernel    the tuned path for full 4096-element chunks, k <= 128: one CTA per
+//                            chunk walks all R replicas with theta_global held in registers, a
+//                            cheap lower bound on the k-th magnitude prunes the chunk to a few
+//                            hundred candidates, one warp finishes the exact selection.
 #include "sl_common.cuh"
 
 namespace sl {
@@ -8,6 +16,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
+constexpr uint32_t kFull = 0xFFFFFFFFu;
 
 __device__ __forceinline__ uint32_t lanemask_lt() {
   uint32_t m;
@@ -15,86 +24,50 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
   return m;
 }
 
-// ---------------------------------------------------------------------------
-// Generic exact kernel: any chunk length up to SL_MAX_CHUNK, any k <= chunk,
-// any supported code width, no alignment requirement.
-//
-//  1. e' = fma(beta, e, theta_global - theta_local) into shared memory.
-//  2. the k-th largest 31-bit magnitude key by a 4-pass radix select
-//     (8+8+8+7 bits, shared-memory histogram, suffix scan by one warp).
-//  3. kept set = keys above the k-th key plus the lowest-positioned ties;
-//     emitted in ascending position with warp ballots (each warp walks one
-//     contiguous region of the chunk, regions are stitched by prefix counts).
-//  4. codes packed in shared memory, residual patched in shared memory, then
-//     one coalesced write of e and of the message.
-// ---------------------------------------------------------------------------
-template <int T>
-__global__ void __launch_bounds__(kThreads)
-compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float* ep = reinterpret_cast<float*>(smem_raw);                          // [chunk]
-  uint32_t* hist = reinterpret_cast<uint32_t*>(ep + a.chunk);              // [256]
-  uint32_t* cw = hist + 256;                                               // [ceil(stride/4)] packed codes
-  __shared__ uint32_t s_wmax[kWarps];
-  __shared__ uint32_t s_weq[kWarps], s_wgt[kWarps];
-  __shared__ uint32_t s_digit, s_need;
+// scratch of the block-wide exact selection (shared by both kernels)
+struct SelectScratch {
+  uint32_t hist[256];
+  uint32_t weq[kWarps], wgt[kWarps];
+  uint32_t digit, need;
+};
 
+// ---------------------------------------------------------------------------
+// Block-wide exact selection + emission on a chunk whose e' sits in shared memory.
+//   * k_eff-th largest 31-bit magnitude key by a 4-pass radix select (8+8+8+7 bits);
+//   * kept set = keys above it plus the lowest-positioned ties, emitted in ascending
+//     position with warp ballots (each warp walks one contiguous region, regions are
+//     stitched by prefix counts);
+//   * codes OR-ed into `cw` (zeroed by the caller), residual patched into `ep`.
+// All threads of the CTA must call it; it ends with a barrier.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void block_select_emit(float* ep, int len, int k_eff, int bits, float s,
+                                                  SelectScratch& sc, uint32_t* cw,
+                                                  uint16_t* __restrict__ oidx, uint8_t* __restrict__ ocodes) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t g = blockIdx.x / (uint32_t)a.R;
-  const int r = (int)(blockIdx.x % (uint32_t)a.R);
-  const ChunkRef c = locate(a.tb, g, a.chunk);
-  const int len = c.len;
-  const int k = a.k, bits = a.bits;
-  const int k_eff = k < len ? k : len;
-
-  const float* __restrict__ tl = a.p.theta_local[r] + c.base;
-  const float* __restrict__ tg = a.theta_global + c.base;
-  float* __restrict__ er = a.p.err[r] + c.base;
-
-  // ---- 1. pseudo-gradient and error feedback ------------------------------
-  uint32_t tmax = 0;
-  for (int i = tid; i < len; i += kThreads) {
-    const float d = __fsub_rn(tg[i], tl[i]);
-    const float e = __fmaf_rn(a.beta, er[i], d);
-    ep[i] = e;
-    tmax = max(tmax, key_of(e));
-  }
-  tmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
-  if (lane == 0) s_wmax[warp] = tmax;
-  const uint32_t cwords = (a.stride + 3) >> 2;
-  if (bits != 32)
-    for (uint32_t i = tid; i < cwords; i += kThreads) cw[i] = 0;
-  __syncthreads();
-  uint32_t smax = 0;
-#pragma unroll
-  for (int w = 0; w < kWarps; ++w) smax = max(smax, s_wmax[w]);
-  const float s = __uint_as_float(smax);
-
-  // ---- 2. radix select of the k_eff-th largest key -------------------------
   uint32_t prefix = 0, need = (uint32_t)k_eff;
 #pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = pass == 0 ? 23 : pass == 1 ? 15 : pass == 2 ? 7 : 0;
     const int width = pass == 3 ? 7 : 8;
     const int hs = shift + width;                 // bits above this digit are already fixed
-    hist[tid] = 0;
+    sc.hist[tid] = 0;
     __syncthreads();
     for (int i = tid; i < len; i += kThreads) {
       const uint32_t key = key_of(ep[i]);
-      if ((key >> hs) == (prefix >> hs)) atomicAdd(&hist[(key >> shift) & ((1u << width) - 1u)], 1u);
+      if ((key >> hs) == (prefix >> hs)) atomicAdd(&sc.hist[(key >> shift) & ((1u << width) - 1u)], 1u);
     }
     __syncthreads();
     if (warp == 0) {
       uint32_t h[8], mine = 0;
 #pragma unroll
-      for (int b = 0; b < 8; ++b) { h[b] = hist[lane * 8 + b]; mine += h[b]; }
+      for (int b = 0; b < 8; ++b) { h[b] = sc.hist[lane * 8 + b]; mine += h[b]; }
       uint32_t suf = mine;                        // inclusive suffix sum over lanes >= lane
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, suf, d);
+        const uint32_t o = __shfl_down_sync(kFull, suf, d);
         if (lane + d < 32) suf += o;
       }
-      const uint32_t vote = __ballot_sync(0xFFFFFFFFu, suf >= need);
+      const uint32_t vote = __ballot_sync(kFull, suf >= need);
       const int sel = 31 - __clz(vote);           // highest lane whose suffix still reaches `need`
       if (lane == sel) {
         uint32_t cum = suf - mine, digit = (uint32_t)lane * 8u, left = need;
@@ -106,17 +79,16 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
             else cum += h[bb];
           }
         }
-        s_digit = digit;
-        s_need = left;
+        sc.digit = digit;
+        sc.need = left;
       }
     }
     __syncthreads();
-    prefix |= s_digit << shift;
-    need = s_need;
+    prefix |= sc.digit << shift;
+    need = sc.need;
   }
   const uint32_t kth = prefix;                    // the k_eff-th largest key; `need` ties of it are kept
 
-  // ---- 3. ordered emission --------------------------------------------------
   const int rw = ((len + kThreads - 1) / kThreads) * 32;   // region per warp, multiple of 32
   const int r0 = warp * rw;
   const int r1 = min(len, r0 + rw);
@@ -124,29 +96,27 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   for (int i0 = r0; i0 < r1; i0 += 32) {
     const int i = i0 + lane;
     const uint32_t key = i < r1 ? key_of(ep[i]) : 0u;
-    ceq += __popc(__ballot_sync(0xFFFFFFFFu, i < r1 && key == kth));
-    cgt += __popc(__ballot_sync(0xFFFFFFFFu, i < r1 && key > kth));
+    ceq += __popc(__ballot_sync(kFull, i < r1 && key == kth));
+    cgt += __popc(__ballot_sync(kFull, i < r1 && key > kth));
   }
-  if (lane == 0) { s_weq[warp] = ceq; s_wgt[warp] = cgt; }
+  if (lane == 0) { sc.weq[warp] = ceq; sc.wgt[warp] = cgt; }
   __syncthreads();
   uint32_t eq_base = 0, out_base = 0;
   for (int w = 0; w < warp; ++w) {
-    const uint32_t weq = s_weq[w];
+    const uint32_t weq = sc.weq[w];
     const uint32_t room = need > eq_base ? need - eq_base : 0u;
-    out_base += s_wgt[w] + min(room, weq);
+    out_base += sc.wgt[w] + min(room, weq);
     eq_base += weq;
   }
-  uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
-  uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
   for (int i0 = r0; i0 < r1; i0 += 32) {
     const int i = i0 + lane;
     const bool in = i < r1;
     const float v = in ? ep[i] : 0.0f;
     const uint32_t key = key_of(v);
     const bool eq = in && key == kth;
-    const uint32_t eqm = __ballot_sync(0xFFFFFFFFu, eq);
+    const uint32_t eqm = __ballot_sync(kFull, eq);
     const bool keep = in && (key > kth || (eq && eq_base + __popc(eqm & lanemask_lt()) < need));
-    const uint32_t km = __ballot_sync(0xFFFFFFFFu, keep);
+    const uint32_t km = __ballot_sync(kFull, keep);
     if (keep) {
       const uint32_t slot = out_base + __popc(km & lanemask_lt());
       oidx[slot] = (uint16_t)i;
@@ -165,8 +135,64 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
     out_base += __popc(km);
   }
   __syncthreads();
+}
 
-  // ---- 4. write-back ---------------------------------------------------------
+// ---------------------------------------------------------------------------
+// Generic kernel.  TAILS = false: CTA b handles chunk b / R of replica b % R.
+// TAILS = true: CTA b handles the short last chunk of tensor b / R (if it has one); this is
+// how the tuned path delegates the ragged ends of the tensors.
+// ---------------------------------------------------------------------------
+template <int T, bool TAILS>
+__global__ void __launch_bounds__(kThreads)
+compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* ep = reinterpret_cast<float*>(smem_raw);                          // [chunk]
+  uint32_t* cw = reinterpret_cast<uint32_t*>(ep + a.chunk);                // [ceil(stride/4)] packed codes
+  __shared__ SelectScratch sc;
+  __shared__ uint32_t s_wmax[kWarps];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = (int)(blockIdx.x % (uint32_t)a.R);
+  uint32_t g = blockIdx.x / (uint32_t)a.R;
+  if (TAILS) {
+    const uint32_t t = g;
+    const uint64_t n_t = a.tb.offset[t + 1] - a.tb.offset[t];
+    if (n_t % (uint64_t)a.chunk == 0) return;     // no short chunk in this tensor
+    g = a.tb.first_chunk[t + 1] - 1;
+  }
+  const ChunkRef c = locate(a.tb, g, a.chunk);
+  const int len = c.len;
+  const int k = a.k, bits = a.bits;
+  const int k_eff = k < len ? k : len;
+
+  const float* __restrict__ tl = a.p.theta_local[r] + c.base;
+  const float* __restrict__ tg = a.theta_global + c.base;
+  float* __restrict__ er = a.p.err[r] + c.base;
+
+  // pseudo-gradient and error feedback
+  uint32_t tmax = 0;
+  for (int i = tid; i < len; i += kThreads) {
+    const float d = __fsub_rn(tg[i], tl[i]);
+    const float e = __fmaf_rn(a.beta, er[i], d);
+    ep[i] = e;
+    tmax = max(tmax, key_of(e));
+  }
+  tmax = __reduce_max_sync(kFull, tmax);
+  if (lane == 0) s_wmax[warp] = tmax;
+  const uint32_t cwords = (a.stride + 3) >> 2;
+  if (bits != 32)
+    for (uint32_t i = tid; i < cwords; i += kThreads) cw[i] = 0;
+  __syncthreads();
+  uint32_t smax = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) smax = max(smax, s_wmax[w]);
+  const float s = __uint_as_float(smax);
+
+  uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
+  uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
+  block_select_emit(ep, len, k_eff, bits, s, sc, cw, oidx, ocodes);
+
+  // write-back
   for (int i = tid; i < len; i += kThreads) er[i] = ep[i];
   for (int j = k_eff + tid; j < k; j += kThreads) oidx[j] = 0xFFFFu;
   if (bits != 32) {
@@ -181,21 +207,271 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   }
 }
 
+// ---------------------------------------------------------------------------
+// Tuned kernel: chunk = 4096, k <= 128, (k * bits) % 32 == 0, 16-byte aligned arena.
+//
+// Thread t owns the float4s number t, t+256, t+512, t+768 of the chunk (coalesced 128-bit
+// accesses): element (j, c) of its registers is position 1024 j + 4 t + c.
+//
+// Per replica:
+//  A  e' = fma(beta, e, theta_global - theta_local) in registers and into shared memory;
+//     per-thread maximum key.  The chunk is cut into kp >= k groups of whole threads
+//     (kp = power of two); every group's maximum is >= the smallest group maximum T1, so at
+//     least k keys are >= T1: T1 is a lower bound of the k-th largest key.
+//  B  keys >= T1 (a few hundred) are compacted to a candidate list (order irrelevant).
+//  C  warp 0 bisects the key range [T1, max] for a threshold that leaves exactly k
+//     candidates; if the range collapses first, the k-th key is tied and the lowest
+//     positions among its ties are found by a second bisection over positions.
+//  D  warp 0 marks the kept positions in a 4096-bit map, walks the map in ascending position
+//     (each lane owns 128 positions, slots from a prefix sum of popcounts), writes idx and
+//     codes and patches the residual in shared memory.
+//  E  the error buffer is written back from shared memory, 128 bits per thread and access.
+// If the candidate list overflows (tie-heavy or constant chunks), the block-wide exact
+// selection of the generic kernel takes over for that (chunk, replica).
+// ---------------------------------------------------------------------------
+constexpr int kC = 4096;
+constexpr int kCandMax = 1024;
+constexpr int kMaxCodeWords = 32;   // k * bits / 32 <= 128 * 8 / 32
+
+struct FastSmem {
+  float ep[2][kC];                  // e' of the current / previous replica (double buffered)
+  uint32_t cand_key[kCandMax];
+  uint16_t cand_pos[kCandMax];
+  uint32_t bitmap[kC / 32];
+  uint32_t cw[kMaxCodeWords];
+  uint32_t wmin[2][kWarps], wmax[2][kWarps];
+  uint32_t count;
+  SelectScratch sc;
+};
+
+template <int T>
+__global__ void __launch_bounds__(kThreads, 3)
+compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  FastSmem& sm = *reinterpret_cast<FastSmem*>(smem_raw);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t g = blockIdx.x;
+  const ChunkRef c = locate(a.tb, g, kC);
+  if (c.len != kC) return;                        // short chunks go to the generic tail launch
+  const int k = a.k, bits = a.bits, R = a.R;
+  const float beta = a.beta;
+
+  // group size for the lower bound: kp = max(8, pow2ceil(k)) groups of 256/kp threads
+  int kp = 8;
+  while (kp < k) kp <<= 1;
+  const int group_lanes = kThreads / kp;          // 32, 16, 8, 4 or 2 lanes
+
+  if (tid < kC / 32) sm.bitmap[tid] = 0;
+  if (tid < kMaxCodeWords) sm.cw[tid] = 0;
+  if (tid == 0) sm.count = 0;
+
+  const float4* __restrict__ tg4 = reinterpret_cast<const float4*>(a.theta_global + c.base);
+  float4 G[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) G[j] = __ldg(tg4 + tid + 256 * j);
+
+#pragma unroll 1
+  for (int r = 0; r < R; ++r) {
+    float* ep = sm.ep[r & 1];
+    const float4* __restrict__ tl4 = reinterpret_cast<const float4*>(a.p.theta_local[r] + c.base);
+    float4* __restrict__ er4 = reinterpret_cast<float4*>(a.p.err[r] + c.base);
+
+    // ---- A ----------------------------------------------------------------
+    float4 Lc[4], E[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) Lc[j] = __ldcs(tl4 + tid + 256 * j);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) E[j] = __ldcs(er4 + tid + 256 * j);
+    uint32_t key[16];
+    uint32_t tmax = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float4 v;
+      v.x = __fmaf_rn(beta, E[j].x, __fsub_rn(G[j].x, Lc[j].x));
+      v.y = __fmaf_rn(beta, E[j].y, __fsub_rn(G[j].y, Lc[j].y));
+      v.z = __fmaf_rn(beta, E[j].z, __fsub_rn(G[j].z, Lc[j].z));
+      v.w = __fmaf_rn(beta, E[j].w, __fsub_rn(G[j].w, Lc[j].w));
+      reinterpret_cast<float4*>(ep)[tid + 256 * j] = v;
+      key[4 * j + 0] = key_of(v.x);
+      key[4 * j + 1] = key_of(v.y);
+      key[4 * j + 2] = key_of(v.z);
+      key[4 * j + 3] = key_of(v.w);
+      tmax = max(tmax, max(max(key[4 * j], key[4 * j + 1]), max(key[4 * j + 2], key[4 * j + 3])));
+    }
+    uint32_t gmax = tmax;
+    for (int d = 1; d < group_lanes; d <<= 1) gmax = max(gmax, __shfl_xor_sync(kFull, gmax, d));
+    const uint32_t wmin = __reduce_min_sync(kFull, gmax);
+    const uint32_t wmax = __reduce_max_sync(kFull, tmax);
+    if (lane == 0) { sm.wmin[r & 1][warp] = wmin; sm.wmax[r & 1][warp] = wmax; }
+    __syncthreads();                              // (1)
+    uint32_t T1 = 0xFFFFFFFFu, smax = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { T1 = min(T1, sm.wmin[r & 1][w]); smax = max(smax, sm.wmax[r & 1][w]); }
+
+    // ---- B ----------------------------------------------------------------
+    {
+      uint32_t mask = 0;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) mask |= (key[e] >= T1 ? 1u : 0u) << e;
+      const uint32_t cnt = __popc(mask);
+      uint32_t incl = cnt;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(kFull, incl, d);
+        if (lane >= d) incl += o;
+      }
+      uint32_t base = 0;
+      if (lane == 31) base = atomicAdd(&sm.count, incl);
+      base = __shfl_sync(kFull, base, 31);
+      uint32_t at = base + incl - cnt;
+      while (mask) {
+        const int b = __ffs(mask) - 1;
+        mask &= mask - 1;
+        const int p = ((b >> 2) << 10) + (tid << 2) + (b & 3);
+        if (at < (uint32_t)kCandMax) {
+          sm.cand_key[at] = key_of(ep[p]);
+          sm.cand_pos[at] = (uint16_t)p;
+        }
+        ++at;
+      }
+    }
+    __syncthreads();                              // (2)
+    const uint32_t C = sm.count;
+    const float s = __uint_as_float(smax);
+    uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
+    uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
+    const int cwords = (k * bits) >> 5;
+
+    if (C > (uint32_t)kCandMax) {
+      // ---- overflow: block-wide exact selection on the whole chunk ---------
+      block_select_emit(ep, kC, k, bits, s, sm.sc, sm.cw, oidx, ocodes);
+      if (bits != 32 && tid < cwords) {
+        reinterpret_cast<uint32_t*>(ocodes)[tid] = sm.cw[tid];
+        sm.cw[tid] = 0;
+      }
+      if (tid == 0) sm.count = 0;
+    } else if (warp == 0) {
+      // ---- C: threshold with exactly k candidates at or above it -------------
+      uint32_t lo = T1, hi = smax + 1u, cnt_hi = 0;
+      uint32_t thr_ge = T1;                       // keep key >= thr_ge ...
+      uint32_t thr_eq = 0xFFFFFFFFu, pos_le = 0;  // ... and key == thr_eq with position <= pos_le
+      if (C != (uint32_t)k) {
+        bool exact = false;
+        while (hi - lo > 1u) {
+          const uint32_t mid = lo + ((hi - lo) >> 1);
+          uint32_t cnt = 0;
+          for (uint32_t i = lane; i < C; i += 32) cnt += sm.cand_key[i] >= mid ? 1u : 0u;
+          cnt = __reduce_add_sync(kFull, cnt);
+          if (cnt == (uint32_t)k) { thr_ge = mid; exact = true; break; }
+          if (cnt > (uint32_t)k) lo = mid; else { hi = mid; cnt_hi = cnt; }
+        }
+        if (!exact) {
+          // the k-th key is `lo` and it is tied: keep all keys above it and the
+          // (k - cnt_hi) lowest positions among the ties
+          thr_ge = lo + 1u;
+          thr_eq = lo;
+          const uint32_t need = (uint32_t)k - cnt_hi;
+          uint32_t plo = 0, phi = kC - 1;         // smallest P with #(ties at position <= P) >= need
+          while (plo < phi) {
+            const uint32_t pm = (plo + phi) >> 1;
+            uint32_t cnt = 0;
+            for (uint32_t i = lane; i < C; i += 32)
+              cnt += (sm.cand_key[i] == thr_eq && (uint32_t)sm.cand_pos[i] <= pm) ? 1u : 0u;
+            cnt = __reduce_add_sync(kFull, cnt);
+            if (cnt >= need) phi = pm; else plo = pm + 1;
+          }
+          pos_le = plo;
+        }
+      }
+      // ---- D: mark, walk in ascending position, emit ---------------------------
+      for (uint32_t i = lane; i < C; i += 32) {
+        const uint32_t ck = sm.cand_key[i];
+        const uint32_t cp = sm.cand_pos[i];
+        if (ck >= thr_ge || (ck == thr_eq && cp <= pos_le)) atomicOr(&sm.bitmap[cp >> 5], 1u << (cp & 31u));
+      }
+      __syncwarp();
+      uint4 bm = reinterpret_cast<uint4*>(sm.bitmap)[lane];
+      const uint32_t mine = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
+      uint32_t incl = mine;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(kFull, incl, d);
+        if (lane >= d) incl += o;
+      }
+      uint32_t slot = incl - mine;
+      const uint32_t words[4] = {bm.x, bm.y, bm.z, bm.w};
+#pragma unroll
+      for (int w = 0; w < 4; ++w) {
+        uint32_t m = words[w];
+        while (m) {
+          const int b = __ffs(m) - 1;
+          m &= m - 1;
+          const int p = lane * 128 + w * 32 + b;
+          const float v = ep[p];
+          oidx[slot] = (uint16_t)p;
+          float sent;
+          if (bits == 32) {
+            reinterpret_cast<float*>(ocodes)[slot] = v;
+            sent = v;
+          } else {
+            const uint32_t code = quant_code(v, s, bits);
+            atomicOr(&sm.cw[(slot * (uint32_t)bits) >> 5], code << ((slot * (uint32_t)bits) & 31u));
+            sent = dequant(code, s, bits);
+          }
+          ep[p] = __fsub_rn(v, sent);             // line 4: the residual
+          ++slot;
+        }
+      }
+      reinterpret_cast<uint4*>(sm.bitmap)[lane] = make_uint4(0, 0, 0, 0);
+      __syncwarp();
+      if (bits != 32 && lane < cwords) {
+        reinterpret_cast<uint32_t*>(ocodes)[lane] = sm.cw[lane];
+        sm.cw[lane] = 0;
+      }
+      if (lane == 0) sm.count = 0;
+    }
+    if (tid == 0) {
+      a.p.scales[r][g] = s;
+      if (smax >= 0x7F800000u && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_NONFINITE);
+    }
+    __syncthreads();                              // (3)
+
+    // ---- E: residual back to the error buffer -------------------------------
+#pragma unroll
+    for (int j = 0; j < 4; ++j) __stcs(er4 + tid + 256 * j, reinterpret_cast<const float4*>(ep)[tid + 256 * j]);
+  }
+}
+
 }  // namespace
 
 template <int T>
 cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream_t st) {
-  (void)aligned16;
   if (a.tb.n_chunks == 0) return cudaSuccess;
-  const size_t smem = (size_t)a.chunk * 4 + 256 * 4 + (a.bits == 32 ? 0 : (size_t)((a.stride + 3) / 4) * 4);
-  const uint64_t blocks = (uint64_t)a.tb.n_chunks * (uint64_t)a.R;
-  if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(compress_generic_kernel<T>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t gsmem = (size_t)a.chunk * 4 + (a.bits == 32 ? 0 : (size_t)((a.stride + 3) / 4) * 4);
+  cudaError_t e;
+  if (gsmem > 40 * 1024) {
+    e = cudaFuncSetAttribute(compress_generic_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(compress_generic_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsmem);
     if (e != cudaSuccess) return e;
   }
-  compress_generic_kernel<T><<<(unsigned)blocks, kThreads, smem, st>>>(a);
+  const bool fast = aligned16 && a.chunk == kC && a.k <= 128 && ((a.k * a.bits) % 32) == 0;
+  if (fast) {
+    e = cudaFuncSetAttribute(compress_c4096_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)sizeof(FastSmem));
+    if (e != cudaSuccess) return e;
+    compress_c4096_kernel<T><<<a.tb.n_chunks, kThreads, sizeof(FastSmem), st>>>(a);
+    bool tails = false;
+    for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
+      tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)kC) != 0;
+    if (tails)
+      compress_generic_kernel<T, true><<<a.tb.n_tensors * (unsigned)a.R, kThreads, gsmem, st>>>(a);
+    return cudaPeekAtLastError();
+  }
+  const uint64_t blocks = (uint64_t)a.tb.n_chunks * (uint64_t)a.R;
+  if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
+  compress_generic_kernel<T, false><<<(unsigned)blocks, kThreads, gsmem, st>>>(a);
   return cudaPeekAtLastError();
 }
 
