@@ -341,6 +341,8 @@ def run_ours(args) -> None:
         wl = wl.replace(R=args.R)
     if args.k:
         wl = wl.replace(k=args.k)
+    if args.first_tensors:
+        wl = synth.sub_arena(wl, list(range(args.first_tensors)), f"{wl.name}[:{args.first_tensors}]")
     st = DeviceState(wl, rank_seed(args.seed, rank), dev)
     stream = torch.cuda.current_stream()
 
@@ -439,6 +441,8 @@ def main() -> None:
     ap.add_argument("--workload", default="1b", choices=["tiny", "180m", "0p5b", "1b"])
     ap.add_argument("--R", type=int, default=0)
     ap.add_argument("--k", type=int, default=0)
+    ap.add_argument("--first-tensors", type=int, default=0,
+                    help="keep only the first N tensors of the workload (small cases for profiling)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")

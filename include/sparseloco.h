@@ -62,7 +62,8 @@ enum {
 
 enum {
   SL_FLAG_NONFINITE = 1u, /* some chunk's largest magnitude was Inf or NaN */
-  SL_FLAG_BAD_INDEX = 2u  /* sl_aggregate*: a message slot named a position past its chunk; skipped */
+  SL_FLAG_BAD_INDEX = 2u, /* sl_aggregate*: a message slot named a position past its chunk; skipped */
+  SL_FLAG_TIMEOUT = 4u    /* a bounded wait on an on-chip copy ran out; the outputs are not to be trusted */
 };
 
 #define SL_MAX_CHUNK 8192     /* elements; any chunk size in [1, SL_MAX_CHUNK] is accepted */

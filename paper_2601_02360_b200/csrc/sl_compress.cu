@@ -210,42 +210,229 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 // ---------------------------------------------------------------------------
 // Tuned kernel: chunk = 4096, k <= 128, (k * bits) % 32 == 0, 16-byte aligned arena.
 //
-// Thread t owns the float4s number t, t+256, t+512, t+768 of the chunk (coalesced 128-bit
-// accesses): element (j, c) of its registers is position 1024 j + 4 t + c.
+// One CTA per chunk walks all R replicas; theta_global stays in registers.  The CTA is warp
+// specialised: 8 producer warps (256 threads) and one selector warp.
 //
-// Per replica:
-//  A  e' = fma(beta, e, theta_global - theta_local) in registers and into shared memory;
-//     per-thread maximum key.  The chunk is cut into kp >= k groups of whole threads
-//     (kp = power of two); every group's maximum is >= the smallest group maximum T1, so at
-//     least k keys are >= T1: T1 is a lower bound of the k-th largest key.
-//  B  keys >= T1 (a few hundred) are compacted to a candidate list (order irrelevant).
-//  C  warp 0 bisects the key range [T1, max] for a threshold that leaves exactly k
-//     candidates; if the range collapses first, the k-th key is tied and the lowest
-//     positions among its ties are found by a second bisection over positions.
-//  D  warp 0 marks the kept positions in a 4096-bit map, walks the map in ascending position
-//     (each lane owns 128 positions, slots from a prefix sum of popcounts), writes idx and
-//     codes and patches the residual in shared memory.
-//  E  the error buffer is written back from shared memory, 128 bits per thread and access.
-// If the candidate list overflows (tie-heavy or constant chunks), the block-wide exact
-// selection of the generic kernel takes over for that (chunk, replica).
+//  * theta_local and e of replica r arrive by TMA bulk copies (cp.async.bulk + mbarrier) in a
+//    3-deep ring of 32 KB stages, issued up to three replicas ahead by the selector's lane 0.
+//  * Producers, per replica (thread t owns float4s t, t+256, t+512, t+768 of the chunk):
+//      A  e' = fma(beta, e, theta_global - theta_local), written in place of e in the stage;
+//         per-thread maximum key.  The chunk is cut into kp >= k groups of whole threads
+//         (kp a power of two); at least k keys are >= the smallest group maximum T1, so T1 is
+//         a lower bound of the k-th largest key.
+//      B  the keys >= T1 (a few hundred) are compacted into a candidate list.
+//  * Selector, per replica, concurrently with the producers' next replica:
+//      C  bisects the key range [T1, max] for a threshold that leaves exactly k candidates;
+//         if the range collapses first the k-th key is tied, and the lowest positions among
+//         its ties are found by a second bisection over positions.
+//      D  marks the kept positions in a 4096-bit map, walks it in ascending position (each
+//         lane owns 128 positions, slots from a prefix sum of popcounts), writes idx and
+//         codes, patches the residual into the stage.
+//      E  one TMA bulk store sends the stage's 16 KB of e' to the error buffer; when the
+//         store has read the stage, the loads of replica r+3 are issued into it.
+//  If the candidate list overflows (tie-heavy or constant chunks) the selector runs an exact
+//  warp-wide radix select over the whole chunk instead of C.
+//
+// Hand-offs: named barrier 1 = producers only; 2,3 = candidate list [parity] ready
+// (producers arrive, selector waits); 4,5 = candidate list [parity] free again (selector
+// arrives, producers wait).  Every mbarrier wait is bounded; running out raises
+// SL_FLAG_TIMEOUT and the kernel carries on (no trap, no hang).
 // ---------------------------------------------------------------------------
 constexpr int kC = 4096;
+constexpr int kStages = 3;
 constexpr int kCandMax = 1024;
-constexpr int kMaxCodeWords = 32;   // k * bits / 32 <= 128 * 8 / 32
+constexpr int kCandReg = 12;          // candidates per lane held in registers (C <= 384)
+constexpr int kMaxCodeWords = 32;     // k * bits / 32 <= 128 * 8 / 32
+constexpr int kFastThreads = kThreads + 32;
+constexpr uint32_t kWaitLimit = 1u << 22;
 
-struct FastSmem {
-  float ep[2][kC];                  // e' of the current / previous replica (double buffered)
-  uint32_t cand_key[kCandMax];
-  uint16_t cand_pos[kCandMax];
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// bounded wait on a phase; false = gave up
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_store_1d(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+
+struct alignas(16) FastSmem {
+  float tl[kStages][kC];              // theta_local of replica r in stage r % 3
+  float ee[kStages][kC];              // e, then e' in place, then the source of the bulk store
+  uint32_t cand_key[2][kCandMax];
+  uint16_t cand_pos[2][kCandMax];
   uint32_t bitmap[kC / 32];
+  uint32_t hist[256];
   uint32_t cw[kMaxCodeWords];
-  uint32_t wmin[2][kWarps], wmax[2][kWarps];
-  uint32_t count;
-  SelectScratch sc;
+  uint32_t wmin[kStages][kWarps], wmax[kStages][kWarps];   // ring: producers run up to two replicas ahead
+  uint32_t count[2];
+  uint64_t full[kStages];
 };
 
+// number of candidate keys >= mid; keys either in registers (NREG > 0) or in shared memory
+template <int NREG>
+__device__ __forceinline__ uint32_t count_ge(const uint32_t* ck_reg, const uint32_t* ck_smem, uint32_t C,
+                                             uint32_t mid, int lane) {
+  uint32_t cnt = 0;
+  if (NREG > 0) {
+#pragma unroll
+    for (int i = 0; i < NREG; ++i) cnt += ck_reg[i] >= mid ? 1u : 0u;
+  } else {
+    for (uint32_t i = lane; i < C; i += 32) cnt += ck_smem[i] >= mid ? 1u : 0u;
+  }
+  return __reduce_add_sync(kFull, cnt);
+}
+
+// Phase C + marking: threshold among C candidates, kept positions OR-ed into the bitmap.
+template <int NREG>
+__device__ __forceinline__ void select_candidates(const uint32_t* cand_key, const uint16_t* cand_pos, uint32_t C,
+                                                  uint32_t k, uint32_t T1, uint32_t smax, uint32_t* bitmap,
+                                                  int lane, uint32_t* stats) {
+  uint32_t ck[NREG > 0 ? NREG : 1];
+  if (NREG > 0) {
+#pragma unroll
+    for (int i = 0; i < NREG; ++i) {
+      const uint32_t at = (uint32_t)lane + 32u * (uint32_t)i;
+      ck[i] = at < C ? cand_key[at] : 0u;          // padding 0 is below every probe (probes are > T1 >= 0)
+    }
+  }
+  uint32_t lo = T1, hi = smax + 1u, cnt_hi = 0;
+  uint32_t thr_ge = T1;                            // keep key >= thr_ge ...
+  uint32_t thr_eq = 0xFFFFFFFFu, pos_le = 0;       // ... and key == thr_eq at position <= pos_le
+  if (C != k) {
+    bool exact = false;
+    while (hi - lo > 1u) {
+      const uint32_t mid = lo + ((hi - lo) >> 1);
+      const uint32_t cnt = count_ge<NREG>(ck, cand_key, C, mid, lane);
+#ifdef SL_STATS
+      if (lane == 0) atomicAdd(&stats[1], 1u);
+#endif
+      if (cnt == k) { thr_ge = mid; exact = true; break; }
+      if (cnt > k) lo = mid; else { hi = mid; cnt_hi = cnt; }
+    }
+    if (!exact) {
+      // the k-th key is `lo` and it is tied: keep every key above it and the (k - cnt_hi)
+      // lowest positions among the ties
+      thr_ge = lo + 1u;
+      thr_eq = lo;
+      const uint32_t need = k - cnt_hi;
+      uint32_t plo = 0, phi = kC - 1;              // smallest P with #(ties at position <= P) >= need
+      while (plo < phi) {
+        const uint32_t pm = (plo + phi) >> 1;
+        uint32_t cnt = 0;
+        for (uint32_t i = lane; i < C; i += 32)
+          cnt += (cand_key[i] == thr_eq && (uint32_t)cand_pos[i] <= pm) ? 1u : 0u;
+        cnt = __reduce_add_sync(kFull, cnt);
+        if (cnt >= need) phi = pm; else plo = pm + 1;
+      }
+      pos_le = plo;
+#ifdef SL_STATS
+      if (lane == 0) atomicAdd(&stats[2], 1u);
+#endif
+    }
+  }
+  if (NREG > 0) {
+#pragma unroll
+    for (int i = 0; i < NREG; ++i) {
+      const uint32_t at = (uint32_t)lane + 32u * (uint32_t)i;
+      if (at < C) {
+        const uint32_t cp = cand_pos[at];
+        if (ck[i] >= thr_ge || (ck[i] == thr_eq && cp <= pos_le)) atomicOr(&bitmap[cp >> 5], 1u << (cp & 31u));
+      }
+    }
+  } else {
+    for (uint32_t i = lane; i < C; i += 32) {
+      const uint32_t k_i = cand_key[i];
+      const uint32_t cp = cand_pos[i];
+      if (k_i >= thr_ge || (k_i == thr_eq && cp <= pos_le)) atomicOr(&bitmap[cp >> 5], 1u << (cp & 31u));
+    }
+  }
+}
+
+// Overflow path of the selector: exact radix select over the whole chunk by one warp, kept
+// positions written to the bitmap (one ballot = one bitmap word).
+__device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, uint32_t* hist, uint32_t* bitmap,
+                                                 int lane) {
+  uint32_t prefix = 0, need = k;
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = pass == 0 ? 23 : pass == 1 ? 15 : pass == 2 ? 7 : 0;
+    const int width = pass == 3 ? 7 : 8;
+    const int hs = shift + width;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) hist[lane * 8 + b] = 0;
+    __syncwarp();
+    for (int i = lane; i < kC; i += 32) {
+      const uint32_t key = key_of(ep[i]);
+      if ((key >> hs) == (prefix >> hs)) atomicAdd(&hist[(key >> shift) & ((1u << width) - 1u)], 1u);
+    }
+    __syncwarp();
+    uint32_t h[8], mine = 0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) { h[b] = hist[lane * 8 + b]; mine += h[b]; }
+    uint32_t suf = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_down_sync(kFull, suf, d);
+      if (lane + d < 32) suf += o;
+    }
+    const uint32_t vote = __ballot_sync(kFull, suf >= need);
+    const int sel = 31 - __clz(vote);
+    uint32_t cum = suf - mine, digit = (uint32_t)lane * 8u, left = need;
+    bool found = false;
+#pragma unroll
+    for (int bb = 7; bb >= 0; --bb) {
+      if (!found) {
+        if (cum + h[bb] >= need) { found = true; digit = (uint32_t)(lane * 8 + bb); left = need - cum; }
+        else cum += h[bb];
+      }
+    }
+    digit = __shfl_sync(kFull, digit, sel);
+    need = __shfl_sync(kFull, left, sel);
+    prefix |= digit << shift;
+    __syncwarp();
+  }
+  const uint32_t kth = prefix;
+  uint32_t eq_seen = 0;
+  for (int w = 0; w < kC / 32; ++w) {
+    const uint32_t key = key_of(ep[w * 32 + lane]);
+    const bool eq = key == kth;
+    const uint32_t eqm = __ballot_sync(kFull, eq);
+    const bool keep = key > kth || (eq && eq_seen + __popc(eqm & lanemask_lt()) < need);
+    const uint32_t km = __ballot_sync(kFull, keep);
+    if (lane == 0) bitmap[w] = km;
+    eq_seen += __popc(eqm);
+  }
+}
+
 template <int T>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kFastThreads, 2)
 compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   FastSmem& sm = *reinterpret_cast<FastSmem*>(smem_raw);
@@ -255,62 +442,69 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   const ChunkRef c = locate(a.tb, g, kC);
   if (c.len != kC) return;                        // short chunks go to the generic tail launch
   const int k = a.k, bits = a.bits, R = a.R;
-  const float beta = a.beta;
-
-  // group size for the lower bound: kp = max(8, pow2ceil(k)) groups of 256/kp threads
-  int kp = 8;
-  while (kp < k) kp <<= 1;
-  const int group_lanes = kThreads / kp;          // 32, 16, 8, 4 or 2 lanes
+  constexpr uint32_t kBytes = kC * 4;
 
   if (tid < kC / 32) sm.bitmap[tid] = 0;
   if (tid < kMaxCodeWords) sm.cw[tid] = 0;
-  if (tid == 0) sm.count = 0;
-
-  const float4* __restrict__ tg4 = reinterpret_cast<const float4*>(a.theta_global + c.base);
-  float4 G[4];
+  if (tid == 0) {
+    sm.count[0] = 0;
+    sm.count[1] = 0;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) G[j] = __ldg(tg4 + tid + 256 * j);
+    for (int s = 0; s < kStages; ++s) mbar_init(&sm.full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  __syncthreads();
+  bool timed_out = false;
+
+  if (warp < kWarps) {
+    // ======================= producers =======================================
+    int kp = 8;                                   // kp = max(8, pow2ceil(k)) groups of 256/kp threads
+    while (kp < k) kp <<= 1;
+    const int group_lanes = kThreads / kp;        // 32, 16, 8, 4 or 2 lanes
+    const float beta = a.beta;
+    const float4* __restrict__ tg4 = reinterpret_cast<const float4*>(a.theta_global + c.base);
+    float4 G[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) G[j] = __ldcs(tg4 + tid + 256 * j);
 
 #pragma unroll 1
-  for (int r = 0; r < R; ++r) {
-    float* ep = sm.ep[r & 1];
-    const float4* __restrict__ tl4 = reinterpret_cast<const float4*>(a.p.theta_local[r] + c.base);
-    float4* __restrict__ er4 = reinterpret_cast<float4*>(a.p.err[r] + c.base);
-
-    // ---- A ----------------------------------------------------------------
-    float4 Lc[4], E[4];
+    for (int r = 0; r < R; ++r) {
+      const int s = r % kStages, p = r & 1;
+      if (!mbar_wait(&sm.full[s], (uint32_t)((r / kStages) & 1))) timed_out = true;
+      const float4* tl4 = reinterpret_cast<const float4*>(sm.tl[s]);
+      float4* ee4 = reinterpret_cast<float4*>(sm.ee[s]);
+      // ---- A ----
+      uint32_t key[16];
+      uint32_t tmax = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) Lc[j] = __ldcs(tl4 + tid + 256 * j);
+      for (int j = 0; j < 4; ++j) {
+        const float4 L = tl4[tid + 256 * j];
+        const float4 E = ee4[tid + 256 * j];
+        float4 v;
+        v.x = __fmaf_rn(beta, E.x, __fsub_rn(G[j].x, L.x));
+        v.y = __fmaf_rn(beta, E.y, __fsub_rn(G[j].y, L.y));
+        v.z = __fmaf_rn(beta, E.z, __fsub_rn(G[j].z, L.z));
+        v.w = __fmaf_rn(beta, E.w, __fsub_rn(G[j].w, L.w));
+        ee4[tid + 256 * j] = v;
+        key[4 * j + 0] = key_of(v.x);
+        key[4 * j + 1] = key_of(v.y);
+        key[4 * j + 2] = key_of(v.z);
+        key[4 * j + 3] = key_of(v.w);
+        tmax = max(tmax, max(max(key[4 * j], key[4 * j + 1]), max(key[4 * j + 2], key[4 * j + 3])));
+      }
+      fence_async_smem();                         // e' must be visible to the later bulk store
+      uint32_t gmax = tmax;
+      for (int d = 1; d < group_lanes; d <<= 1) gmax = max(gmax, __shfl_xor_sync(kFull, gmax, d));
+      const uint32_t wmin = __reduce_min_sync(kFull, gmax);
+      const uint32_t wmax = __reduce_max_sync(kFull, tmax);
+      if (lane == 0) { sm.wmin[s][warp] = wmin; sm.wmax[s][warp] = wmax; }
+      named_sync(1, kThreads);
+      uint32_t T1 = 0xFFFFFFFFu;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) E[j] = __ldcs(er4 + tid + 256 * j);
-    uint32_t key[16];
-    uint32_t tmax = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float4 v;
-      v.x = __fmaf_rn(beta, E[j].x, __fsub_rn(G[j].x, Lc[j].x));
-      v.y = __fmaf_rn(beta, E[j].y, __fsub_rn(G[j].y, Lc[j].y));
-      v.z = __fmaf_rn(beta, E[j].z, __fsub_rn(G[j].z, Lc[j].z));
-      v.w = __fmaf_rn(beta, E[j].w, __fsub_rn(G[j].w, Lc[j].w));
-      reinterpret_cast<float4*>(ep)[tid + 256 * j] = v;
-      key[4 * j + 0] = key_of(v.x);
-      key[4 * j + 1] = key_of(v.y);
-      key[4 * j + 2] = key_of(v.z);
-      key[4 * j + 3] = key_of(v.w);
-      tmax = max(tmax, max(max(key[4 * j], key[4 * j + 1]), max(key[4 * j + 2], key[4 * j + 3])));
-    }
-    uint32_t gmax = tmax;
-    for (int d = 1; d < group_lanes; d <<= 1) gmax = max(gmax, __shfl_xor_sync(kFull, gmax, d));
-    const uint32_t wmin = __reduce_min_sync(kFull, gmax);
-    const uint32_t wmax = __reduce_max_sync(kFull, tmax);
-    if (lane == 0) { sm.wmin[r & 1][warp] = wmin; sm.wmax[r & 1][warp] = wmax; }
-    __syncthreads();                              // (1)
-    uint32_t T1 = 0xFFFFFFFFu, smax = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) { T1 = min(T1, sm.wmin[r & 1][w]); smax = max(smax, sm.wmax[r & 1][w]); }
-
-    // ---- B ----------------------------------------------------------------
-    {
+      for (int w = 0; w < kWarps; ++w) T1 = min(T1, sm.wmin[s][w]);
+      // ---- B ----
+      if (r >= 2) named_sync(4 + p, kFastThreads);   // the selector is done with candidate list p
       uint32_t mask = 0;
 #pragma unroll
       for (int e = 0; e < 16; ++e) mask |= (key[e] >= T1 ? 1u : 0u) << e;
@@ -322,75 +516,62 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         if (lane >= d) incl += o;
       }
       uint32_t base = 0;
-      if (lane == 31) base = atomicAdd(&sm.count, incl);
+      if (lane == 31) base = atomicAdd(&sm.count[p], incl);
       base = __shfl_sync(kFull, base, 31);
       uint32_t at = base + incl - cnt;
+      const float* ep = sm.ee[s];
       while (mask) {
         const int b = __ffs(mask) - 1;
         mask &= mask - 1;
-        const int p = ((b >> 2) << 10) + (tid << 2) + (b & 3);
+        const int pos = ((b >> 2) << 10) + (tid << 2) + (b & 3);
         if (at < (uint32_t)kCandMax) {
-          sm.cand_key[at] = key_of(ep[p]);
-          sm.cand_pos[at] = (uint16_t)p;
+          sm.cand_key[p][at] = key_of(ep[pos]);
+          sm.cand_pos[p][at] = (uint16_t)pos;
         }
         ++at;
       }
+      __syncwarp();                               // bar.* is warp-aligned: reconverge first
+      __threadfence_block();
+      named_arrive(2 + p, kFastThreads);          // candidate list p is ready
     }
-    __syncthreads();                              // (2)
-    const uint32_t C = sm.count;
-    const float s = __uint_as_float(smax);
-    uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
-    uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
+  } else {
+    // ======================= selector ========================================
+    if (lane == 0) {
+      for (int r = 0; r < kStages && r < R; ++r) {
+        mbar_expect_tx(&sm.full[r], 2 * kBytes);
+        tma_load_1d(sm.tl[r], a.p.theta_local[r] + c.base, kBytes, &sm.full[r]);
+        tma_load_1d(sm.ee[r], a.p.err[r] + c.base, kBytes, &sm.full[r]);
+      }
+    }
+    __syncwarp();
     const int cwords = (k * bits) >> 5;
-
-    if (C > (uint32_t)kCandMax) {
-      // ---- overflow: block-wide exact selection on the whole chunk ---------
-      block_select_emit(ep, kC, k, bits, s, sm.sc, sm.cw, oidx, ocodes);
-      if (bits != 32 && tid < cwords) {
-        reinterpret_cast<uint32_t*>(ocodes)[tid] = sm.cw[tid];
-        sm.cw[tid] = 0;
-      }
-      if (tid == 0) sm.count = 0;
-    } else if (warp == 0) {
-      // ---- C: threshold with exactly k candidates at or above it -------------
-      uint32_t lo = T1, hi = smax + 1u, cnt_hi = 0;
-      uint32_t thr_ge = T1;                       // keep key >= thr_ge ...
-      uint32_t thr_eq = 0xFFFFFFFFu, pos_le = 0;  // ... and key == thr_eq with position <= pos_le
-      if (C != (uint32_t)k) {
-        bool exact = false;
-        while (hi - lo > 1u) {
-          const uint32_t mid = lo + ((hi - lo) >> 1);
-          uint32_t cnt = 0;
-          for (uint32_t i = lane; i < C; i += 32) cnt += sm.cand_key[i] >= mid ? 1u : 0u;
-          cnt = __reduce_add_sync(kFull, cnt);
-          if (cnt == (uint32_t)k) { thr_ge = mid; exact = true; break; }
-          if (cnt > (uint32_t)k) lo = mid; else { hi = mid; cnt_hi = cnt; }
-        }
-        if (!exact) {
-          // the k-th key is `lo` and it is tied: keep all keys above it and the
-          // (k - cnt_hi) lowest positions among the ties
-          thr_ge = lo + 1u;
-          thr_eq = lo;
-          const uint32_t need = (uint32_t)k - cnt_hi;
-          uint32_t plo = 0, phi = kC - 1;         // smallest P with #(ties at position <= P) >= need
-          while (plo < phi) {
-            const uint32_t pm = (plo + phi) >> 1;
-            uint32_t cnt = 0;
-            for (uint32_t i = lane; i < C; i += 32)
-              cnt += (sm.cand_key[i] == thr_eq && (uint32_t)sm.cand_pos[i] <= pm) ? 1u : 0u;
-            cnt = __reduce_add_sync(kFull, cnt);
-            if (cnt >= need) phi = pm; else plo = pm + 1;
-          }
-          pos_le = plo;
-        }
-      }
-      // ---- D: mark, walk in ascending position, emit ---------------------------
-      for (uint32_t i = lane; i < C; i += 32) {
-        const uint32_t ck = sm.cand_key[i];
-        const uint32_t cp = sm.cand_pos[i];
-        if (ck >= thr_ge || (ck == thr_eq && cp <= pos_le)) atomicOr(&sm.bitmap[cp >> 5], 1u << (cp & 31u));
-      }
+#pragma unroll 1
+    for (int r = 0; r < R; ++r) {
+      const int s = r % kStages, p = r & 1;
+      float* ep = sm.ee[s];
+      named_sync(2 + p, kFastThreads);            // candidate list p is ready
+      const uint32_t C = sm.count[p];
+      uint32_t T1 = 0xFFFFFFFFu, smax = 0;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) { T1 = min(T1, sm.wmin[s][w]); smax = max(smax, sm.wmax[s][w]); }
+      const float sc = __uint_as_float(smax);
+      uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
+      uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
+#ifdef SL_STATS
+      if (lane == 0) { atomicAdd(&a.flags[4], C); atomicAdd(&a.flags[7], 1u); if (C > kCandMax) atomicAdd(&a.flags[8], 1u); }
+#endif
+      // ---- C ----
+      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist, sm.bitmap, lane);
+      else if (C <= 32u * kCandReg)
+        select_candidates<kCandReg>(sm.cand_key[p], sm.cand_pos[p], C, (uint32_t)k, T1, smax, sm.bitmap, lane, a.flags + 4);
+      else
+        select_candidates<0>(sm.cand_key[p], sm.cand_pos[p], C, (uint32_t)k, T1, smax, sm.bitmap, lane, a.flags + 4);
       __syncwarp();
+      if (lane == 0) sm.count[p] = 0;
+      __threadfence_block();
+      __syncwarp();
+      if (r + 2 < R) named_arrive(4 + p, kFastThreads);   // candidate list p may be refilled
+      // ---- D ----
       uint4 bm = reinterpret_cast<uint4*>(sm.bitmap)[lane];
       const uint32_t mine = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
       uint32_t incl = mine;
@@ -407,40 +588,45 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         while (m) {
           const int b = __ffs(m) - 1;
           m &= m - 1;
-          const int p = lane * 128 + w * 32 + b;
-          const float v = ep[p];
-          oidx[slot] = (uint16_t)p;
+          const int pos = lane * 128 + w * 32 + b;
+          const float v = ep[pos];
+          oidx[slot] = (uint16_t)pos;
           float sent;
           if (bits == 32) {
             reinterpret_cast<float*>(ocodes)[slot] = v;
             sent = v;
           } else {
-            const uint32_t code = quant_code(v, s, bits);
+            const uint32_t code = quant_code(v, sc, bits);
             atomicOr(&sm.cw[(slot * (uint32_t)bits) >> 5], code << ((slot * (uint32_t)bits) & 31u));
-            sent = dequant(code, s, bits);
+            sent = dequant(code, sc, bits);
           }
-          ep[p] = __fsub_rn(v, sent);             // line 4: the residual
+          ep[pos] = __fsub_rn(v, sent);           // line 4: the residual
           ++slot;
         }
       }
       reinterpret_cast<uint4*>(sm.bitmap)[lane] = make_uint4(0, 0, 0, 0);
+      fence_async_smem();
       __syncwarp();
+      // ---- E ----
+      if (lane == 0) tma_store_1d(a.p.err[r] + c.base, ep, kBytes);
       if (bits != 32 && lane < cwords) {
         reinterpret_cast<uint32_t*>(ocodes)[lane] = sm.cw[lane];
         sm.cw[lane] = 0;
       }
-      if (lane == 0) sm.count = 0;
+      if (lane == 0) {
+        a.p.scales[r][g] = sc;
+        if (smax >= 0x7F800000u && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_NONFINITE);
+        tma_store_wait_read();                    // the stage has been read: it may be refilled
+        if (r + kStages < R) {
+          mbar_expect_tx(&sm.full[s], 2 * kBytes);
+          tma_load_1d(sm.tl[s], a.p.theta_local[r + kStages] + c.base, kBytes, &sm.full[s]);
+          tma_load_1d(sm.ee[s], a.p.err[r + kStages] + c.base, kBytes, &sm.full[s]);
+        }
+      }
+      __syncwarp();
     }
-    if (tid == 0) {
-      a.p.scales[r][g] = s;
-      if (smax >= 0x7F800000u && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_NONFINITE);
-    }
-    __syncthreads();                              // (3)
-
-    // ---- E: residual back to the error buffer -------------------------------
-#pragma unroll
-    for (int j = 0; j < 4; ++j) __stcs(er4 + tid + 256 * j, reinterpret_cast<const float4*>(ep)[tid + 256 * j]);
   }
+  if (timed_out && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 }  // namespace
@@ -461,7 +647,7 @@ cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream
     e = cudaFuncSetAttribute(compress_c4096_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)sizeof(FastSmem));
     if (e != cudaSuccess) return e;
-    compress_c4096_kernel<T><<<a.tb.n_chunks, kThreads, sizeof(FastSmem), st>>>(a);
+    compress_c4096_kernel<T><<<a.tb.n_chunks, kFastThreads, sizeof(FastSmem), st>>>(a);
     bool tails = false;
     for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
       tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)kC) != 0;
