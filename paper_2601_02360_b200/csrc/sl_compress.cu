@@ -211,17 +211,19 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 // Tuned kernel: chunk = 4096, k <= 128, (k * bits) % 32 == 0, 16-byte aligned arena.
 //
 // One CTA per chunk walks all R replicas; theta_global stays in registers.  The CTA is warp
-// specialised: 8 producer warps (256 threads) and one selector warp.
+// specialised: 8 producer warps (256 threads) and kSel selector warps; selector q handles the
+// replicas r with r % kSel == q, so two selections are in flight while the producers run ahead.
 //
-//  * theta_local and e of replica r arrive by TMA bulk copies (cp.async.bulk + mbarrier) in a
-//    3-deep ring of 32 KB stages, issued up to three replicas ahead by the selector's lane 0.
+//  * theta_local and e of replica r arrive by TMA bulk copies (cp.async.bulk + mbarrier):
+//    theta_local in a 2-deep ring (dead after phase A, refilled by producer thread 0), e in a
+//    4-deep ring (alive until its bulk store has read it, refilled by the selector that owns it).
 //  * Producers, per replica (thread t owns float4s t, t+256, t+512, t+768 of the chunk):
 //      A  e' = fma(beta, e, theta_global - theta_local), written in place of e in the stage;
 //         per-thread maximum key.  The chunk is cut into kp >= k groups of whole threads
 //         (kp a power of two); at least k keys are >= the smallest group maximum T1, so T1 is
 //         a lower bound of the k-th largest key.
 //      B  the keys >= T1 (a few hundred) are compacted into a candidate list.
-//  * Selector, per replica, concurrently with the producers' next replica:
+//  * Selector, per replica:
 //      C  bisects the key range [T1, max] for a threshold that leaves exactly k candidates;
 //         if the range collapses first the k-th key is tied, and the lowest positions among
 //         its ties are found by a second bisection over positions.
@@ -229,21 +231,24 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 //         lane owns 128 positions, slots from a prefix sum of popcounts), writes idx and
 //         codes, patches the residual into the stage.
 //      E  one TMA bulk store sends the stage's 16 KB of e' to the error buffer; when the
-//         store has read the stage, the loads of replica r+3 are issued into it.
+//         store has read the stage, e of replica r+4 is loaded into it.
 //  If the candidate list overflows (tie-heavy or constant chunks) the selector runs an exact
 //  warp-wide radix select over the whole chunk instead of C.
 //
-// Hand-offs: named barrier 1 = producers only; 2,3 = candidate list [parity] ready
-// (producers arrive, selector waits); 4,5 = candidate list [parity] free again (selector
-// arrives, producers wait).  Every mbarrier wait is bounded; running out raises
-// SL_FLAG_TIMEOUT and the kernel carries on (no trap, no hang).
+// Hand-offs: named barrier 1 = producers only; 2+q = candidate list q ready (producers
+// arrive, selector q waits); 4+q = candidate list q free again (selector q arrives, producers
+// wait).  Every mbarrier wait is bounded; running out raises SL_FLAG_TIMEOUT and the kernel
+// carries on (no trap, no hang).
 // ---------------------------------------------------------------------------
 constexpr int kC = 4096;
-constexpr int kStages = 3;
+constexpr int kSel = 2;               // selector warps
+constexpr int kTlStages = 2;
+constexpr int kEeStages = 4;
 constexpr int kCandMax = 1024;
 constexpr int kCandReg = 12;          // candidates per lane held in registers (C <= 384)
 constexpr int kMaxCodeWords = 32;     // k * bits / 32 <= 128 * 8 / 32
-constexpr int kFastThreads = kThreads + 32;
+constexpr int kFastThreads = kThreads + 32 * kSel;
+constexpr int kPairThreads = kThreads + 32;   // producers + one selector
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -283,16 +288,17 @@ __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sy
 __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
 struct alignas(16) FastSmem {
-  float tl[kStages][kC];              // theta_local of replica r in stage r % 3
-  float ee[kStages][kC];              // e, then e' in place, then the source of the bulk store
-  uint32_t cand_key[2][kCandMax];
-  uint16_t cand_pos[2][kCandMax];
-  uint32_t bitmap[kC / 32];
-  uint32_t hist[256];
-  uint32_t cw[kMaxCodeWords];
-  uint32_t wmin[kStages][kWarps], wmax[kStages][kWarps];   // ring: producers run up to two replicas ahead
-  uint32_t count[2];
-  uint64_t full[kStages];
+  float tl[kTlStages][kC];            // theta_local of replica r in stage r % 2
+  float ee[kEeStages][kC];            // e of replica r in stage r % 4, then e' in place, then the store's source
+  uint32_t cand_key[kSel][kCandMax];
+  uint16_t cand_pos[kSel][kCandMax];
+  uint32_t bitmap[kSel][kC / 32];
+  uint32_t hist[kSel][256];
+  uint32_t cw[kSel][kMaxCodeWords];
+  uint32_t wmin[kEeStages][kWarps], wmax[kEeStages][kWarps];   // ring: producers run up to three replicas ahead
+  uint32_t count[kSel];
+  uint64_t full_tl[kTlStages];
+  uint64_t full_ee[kEeStages];
 };
 
 // number of candidate keys >= mid; keys either in registers (NREG > 0) or in shared memory
@@ -444,13 +450,15 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   const int k = a.k, bits = a.bits, R = a.R;
   constexpr uint32_t kBytes = kC * 4;
 
-  if (tid < kC / 32) sm.bitmap[tid] = 0;
-  if (tid < kMaxCodeWords) sm.cw[tid] = 0;
+  for (int i = tid; i < kSel * (kC / 32); i += kFastThreads) (&sm.bitmap[0][0])[i] = 0;
+  if (tid < kSel * kMaxCodeWords) (&sm.cw[0][0])[tid] = 0;
   if (tid == 0) {
-    sm.count[0] = 0;
-    sm.count[1] = 0;
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) mbar_init(&sm.full[s], 1);
+    for (int q = 0; q < kSel; ++q) sm.count[q] = 0;
+#pragma unroll
+    for (int s = 0; s < kTlStages; ++s) mbar_init(&sm.full_tl[s], 1);
+#pragma unroll
+    for (int s = 0; s < kEeStages; ++s) mbar_init(&sm.full_ee[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -459,6 +467,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 
   if (warp < kWarps) {
     // ======================= producers =======================================
+    if (tid == 0) {
+      for (int r = 0; r < kTlStages && r < R; ++r) {
+        mbar_expect_tx(&sm.full_tl[r], kBytes);
+        tma_load_1d(sm.tl[r], a.p.theta_local[r] + c.base, kBytes, &sm.full_tl[r]);
+      }
+    }
     int kp = 8;                                   // kp = max(8, pow2ceil(k)) groups of 256/kp threads
     while (kp < k) kp <<= 1;
     const int group_lanes = kThreads / kp;        // 32, 16, 8, 4 or 2 lanes
@@ -467,13 +481,15 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     float4 G[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) G[j] = __ldcs(tg4 + tid + 256 * j);
+    __syncwarp();
 
 #pragma unroll 1
     for (int r = 0; r < R; ++r) {
-      const int s = r % kStages, p = r & 1;
-      if (!mbar_wait(&sm.full[s], (uint32_t)((r / kStages) & 1))) timed_out = true;
-      const float4* tl4 = reinterpret_cast<const float4*>(sm.tl[s]);
-      float4* ee4 = reinterpret_cast<float4*>(sm.ee[s]);
+      const int st = r % kTlStages, se = r % kEeStages, q = r % kSel;
+      if (!mbar_wait(&sm.full_tl[st], (uint32_t)((r / kTlStages) & 1))) timed_out = true;
+      if (!mbar_wait(&sm.full_ee[se], (uint32_t)((r / kEeStages) & 1))) timed_out = true;
+      const float4* tl4 = reinterpret_cast<const float4*>(sm.tl[st]);
+      float4* ee4 = reinterpret_cast<float4*>(sm.ee[se]);
       // ---- A ----
       uint32_t key[16];
       uint32_t tmax = 0;
@@ -498,13 +514,18 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       for (int d = 1; d < group_lanes; d <<= 1) gmax = max(gmax, __shfl_xor_sync(kFull, gmax, d));
       const uint32_t wmin = __reduce_min_sync(kFull, gmax);
       const uint32_t wmax = __reduce_max_sync(kFull, tmax);
-      if (lane == 0) { sm.wmin[s][warp] = wmin; sm.wmax[s][warp] = wmax; }
+      if (lane == 0) { sm.wmin[se][warp] = wmin; sm.wmax[se][warp] = wmax; }
       named_sync(1, kThreads);
+      if (tid == 0 && r + kTlStages < R) {        // every producer has read theta_local(r): refill its stage
+        mbar_expect_tx(&sm.full_tl[st], kBytes);
+        tma_load_1d(sm.tl[st], a.p.theta_local[r + kTlStages] + c.base, kBytes, &sm.full_tl[st]);
+      }
       uint32_t T1 = 0xFFFFFFFFu;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) T1 = min(T1, sm.wmin[s][w]);
+      for (int w = 0; w < kWarps; ++w) T1 = min(T1, sm.wmin[se][w]);
       // ---- B ----
-      if (r >= 2) named_sync(4 + p, kFastThreads);   // the selector is done with candidate list p
+      __syncwarp();
+      if (r >= kSel) named_sync(4 + q, kPairThreads);   // selector q is done with its candidate list
       uint32_t mask = 0;
 #pragma unroll
       for (int e = 0; e < 16; ++e) mask |= (key[e] >= T1 ? 1u : 0u) << e;
@@ -516,44 +537,46 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         if (lane >= d) incl += o;
       }
       uint32_t base = 0;
-      if (lane == 31) base = atomicAdd(&sm.count[p], incl);
+      if (lane == 31) base = atomicAdd(&sm.count[q], incl);
       base = __shfl_sync(kFull, base, 31);
       uint32_t at = base + incl - cnt;
-      const float* ep = sm.ee[s];
+      const float* ep = sm.ee[se];
       while (mask) {
         const int b = __ffs(mask) - 1;
         mask &= mask - 1;
         const int pos = ((b >> 2) << 10) + (tid << 2) + (b & 3);
         if (at < (uint32_t)kCandMax) {
-          sm.cand_key[p][at] = key_of(ep[pos]);
-          sm.cand_pos[p][at] = (uint16_t)pos;
+          sm.cand_key[q][at] = key_of(ep[pos]);
+          sm.cand_pos[q][at] = (uint16_t)pos;
         }
         ++at;
       }
       __syncwarp();                               // bar.* is warp-aligned: reconverge first
       __threadfence_block();
-      named_arrive(2 + p, kFastThreads);          // candidate list p is ready
+      named_arrive(2 + q, kPairThreads);          // candidate list q is ready
     }
   } else {
-    // ======================= selector ========================================
+    // ======================= selectors =======================================
+    const int q = warp - kWarps;
     if (lane == 0) {
-      for (int r = 0; r < kStages && r < R; ++r) {
-        mbar_expect_tx(&sm.full[r], 2 * kBytes);
-        tma_load_1d(sm.tl[r], a.p.theta_local[r] + c.base, kBytes, &sm.full[r]);
-        tma_load_1d(sm.ee[r], a.p.err[r] + c.base, kBytes, &sm.full[r]);
+      for (int r = q; r < kEeStages && r < R; r += kSel) {
+        mbar_expect_tx(&sm.full_ee[r], kBytes);
+        tma_load_1d(sm.ee[r], a.p.err[r] + c.base, kBytes, &sm.full_ee[r]);
       }
     }
     __syncwarp();
     const int cwords = (k * bits) >> 5;
+    uint32_t* bitmap = sm.bitmap[q];
+    uint32_t* cw = sm.cw[q];
 #pragma unroll 1
-    for (int r = 0; r < R; ++r) {
-      const int s = r % kStages, p = r & 1;
-      float* ep = sm.ee[s];
-      named_sync(2 + p, kFastThreads);            // candidate list p is ready
-      const uint32_t C = sm.count[p];
+    for (int r = q; r < R; r += kSel) {
+      const int se = r % kEeStages;
+      float* ep = sm.ee[se];
+      named_sync(2 + q, kPairThreads);            // candidate list q is ready
+      const uint32_t C = sm.count[q];
       uint32_t T1 = 0xFFFFFFFFu, smax = 0;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) { T1 = min(T1, sm.wmin[s][w]); smax = max(smax, sm.wmax[s][w]); }
+      for (int w = 0; w < kWarps; ++w) { T1 = min(T1, sm.wmin[se][w]); smax = max(smax, sm.wmax[se][w]); }
       const float sc = __uint_as_float(smax);
       uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
       uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
@@ -561,18 +584,18 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       if (lane == 0) { atomicAdd(&a.flags[4], C); atomicAdd(&a.flags[7], 1u); if (C > kCandMax) atomicAdd(&a.flags[8], 1u); }
 #endif
       // ---- C ----
-      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist, sm.bitmap, lane);
+      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist[q], bitmap, lane);
       else if (C <= 32u * kCandReg)
-        select_candidates<kCandReg>(sm.cand_key[p], sm.cand_pos[p], C, (uint32_t)k, T1, smax, sm.bitmap, lane, a.flags + 4);
+        select_candidates<kCandReg>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, bitmap, lane, a.flags + 4);
       else
-        select_candidates<0>(sm.cand_key[p], sm.cand_pos[p], C, (uint32_t)k, T1, smax, sm.bitmap, lane, a.flags + 4);
+        select_candidates<0>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, bitmap, lane, a.flags + 4);
       __syncwarp();
-      if (lane == 0) sm.count[p] = 0;
+      if (lane == 0) sm.count[q] = 0;
       __threadfence_block();
       __syncwarp();
-      if (r + 2 < R) named_arrive(4 + p, kFastThreads);   // candidate list p may be refilled
+      if (r + kSel < R) named_arrive(4 + q, kPairThreads);   // candidate list q may be refilled
       // ---- D ----
-      uint4 bm = reinterpret_cast<uint4*>(sm.bitmap)[lane];
+      uint4 bm = reinterpret_cast<uint4*>(bitmap)[lane];
       const uint32_t mine = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
       uint32_t incl = mine;
 #pragma unroll
@@ -597,30 +620,29 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
             sent = v;
           } else {
             const uint32_t code = quant_code(v, sc, bits);
-            atomicOr(&sm.cw[(slot * (uint32_t)bits) >> 5], code << ((slot * (uint32_t)bits) & 31u));
+            atomicOr(&cw[(slot * (uint32_t)bits) >> 5], code << ((slot * (uint32_t)bits) & 31u));
             sent = dequant(code, sc, bits);
           }
           ep[pos] = __fsub_rn(v, sent);           // line 4: the residual
           ++slot;
         }
       }
-      reinterpret_cast<uint4*>(sm.bitmap)[lane] = make_uint4(0, 0, 0, 0);
+      reinterpret_cast<uint4*>(bitmap)[lane] = make_uint4(0, 0, 0, 0);
       fence_async_smem();
       __syncwarp();
       // ---- E ----
       if (lane == 0) tma_store_1d(a.p.err[r] + c.base, ep, kBytes);
       if (bits != 32 && lane < cwords) {
-        reinterpret_cast<uint32_t*>(ocodes)[lane] = sm.cw[lane];
-        sm.cw[lane] = 0;
+        reinterpret_cast<uint32_t*>(ocodes)[lane] = cw[lane];
+        cw[lane] = 0;
       }
       if (lane == 0) {
         a.p.scales[r][g] = sc;
         if (smax >= 0x7F800000u && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_NONFINITE);
         tma_store_wait_read();                    // the stage has been read: it may be refilled
-        if (r + kStages < R) {
-          mbar_expect_tx(&sm.full[s], 2 * kBytes);
-          tma_load_1d(sm.tl[s], a.p.theta_local[r + kStages] + c.base, kBytes, &sm.full[s]);
-          tma_load_1d(sm.ee[s], a.p.err[r + kStages] + c.base, kBytes, &sm.full[s]);
+        if (r + kEeStages < R) {
+          mbar_expect_tx(&sm.full_ee[se], kBytes);
+          tma_load_1d(sm.ee[se], a.p.err[r + kEeStages] + c.base, kBytes, &sm.full_ee[se]);
         }
       }
       __syncwarp();
