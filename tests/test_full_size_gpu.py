@@ -1,0 +1,80 @@
+"""Parity at the benchmark's full size, in the launch configuration bench.py times: the ~1B
+parameter set (164 tensors, 241,829 chunks, R = 8, k = 64, 2-bit), two outer rounds carrying the
+error buffers.  The checker cannot do 8 x 1e9 elements in a test, so it is run on sampled chunks
+(every kind of tensor, first and last chunks, all-short tails, random interior chunks), each
+compared bit for bit; properties that hold at any size are checked on every chunk on the device."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle import slo
+from paper_2601_02360_b200 import synth
+from parity_util import assert_close, assert_exact
+
+pytestmark = pytest.mark.gpu
+f32 = np.float32
+
+
+def _gather(t, picks):
+    return [t[s:s + ln].cpu().numpy() for _, s, ln in picks]
+
+
+def _check_properties(st, wl):
+    nc = wl.n_chunks()
+    # chunk lengths in chunk order
+    lens = []
+    for sz in wl.sizes:
+        full, rem = divmod(sz, wl.chunk)
+        lens += [wl.chunk] * full + ([rem] if rem else [])
+    lens = torch.tensor(lens, dtype=torch.int32, device=st.dev)
+    keff = torch.clamp(lens, max=wl.k)
+    for r in range(wl.R):
+        idx = (st.idx[r].view(torch.int16).to(torch.int32) & 0xFFFF).view(nc, wl.k)
+        used = idx != 0xFFFF
+        assert torch.equal(used.sum(dim=1).to(torch.int32), keff), "kept count per chunk"
+        slot = torch.arange(wl.k, device=st.dev).view(1, -1)
+        assert torch.equal(used, slot < keff.view(-1, 1)), "padding only after the used slots"
+        nxt = torch.where(used[:, 1:], idx[:, 1:], torch.full_like(idx[:, 1:], 1 << 20))
+        assert bool((nxt > idx[:, :-1]).all()), "positions strictly ascending"
+        assert bool((torch.where(used, idx, torch.zeros_like(idx)) < lens.view(-1, 1)).all()), "positions inside the chunk"
+        assert bool((st.scales[r] >= 0).all()) and bool(torch.isfinite(st.scales[r]).all())
+
+
+def test_1b_workload_sampled_chunks_two_rounds():
+    free, _ = torch.cuda.mem_get_info()
+    wl = synth.workload("1b")
+    need = (2 * wl.R + 1) * wl.n_total * 4 + (2 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    dev = torch.device("cuda", 0)
+    st = bench.DeviceState(wl, 0, dev)
+    picks = synth.sample_chunks(wl, 220, seed=1)
+    assert sum(1 for _, _, ln in picks if ln < wl.chunk) >= 30      # the short tails are in
+    stride = st.api.sl_codes_stride(wl.k, wl.bits)
+    for rnd in range(2):
+        st.redraw_locals(rnd)
+        tg_in = _gather(st.theta_global, picks)
+        tl_in = [_gather(st.theta_local[r], picks) for r in range(wl.R)]
+        e_in = [_gather(st.err[r], picks) for r in range(wl.R)]
+        st.compress()
+        st.aggregate_apply()
+        torch.cuda.synchronize()
+        assert int(st.flags.item()) == 0
+        _check_properties(st, wl)
+        tg_out = _gather(st.theta_global, picks)
+        for ci, (g, s, ln) in enumerate(picks):
+            msgs = []
+            for r in range(wl.R):
+                e = e_in[r][ci].copy()
+                i_o, c_o, s_o, _ = slo.compress(tl_in[r][ci], tg_in[ci], e, [0, ln], wl.beta, wl.chunk, wl.k, wl.bits)
+                msgs.append((i_o, c_o, s_o))
+                what = f"round {rnd} chunk {g} replica {r}"
+                assert_exact(st.idx[r][g * wl.k:(g + 1) * wl.k].cpu().numpy(), i_o[0], what + " idx")
+                assert_exact(st.codes[r][g * stride:(g + 1) * stride].cpu().numpy(), c_o[0], what + " codes")
+                assert_close(st.scales[r][g:g + 1].cpu().numpy(), s_o, what + " scale")
+                assert_close(st.err[r][s:s + ln].cpu().numpy(), e, what + " err")
+            upd = slo.aggregate(msgs, [0, ln], wl.chunk, wl.k, wl.bits)
+            want = tg_in[ci].copy()
+            slo.outer_apply(want, upd, wl.outer_lr)
+            assert_close(tg_out[ci], want, f"round {rnd} chunk {g} theta_global")
