@@ -206,15 +206,18 @@ def sample_chunks(wl: Workload, n: int, seed: int = 0) -> List[Tuple[int, int, i
         g += nc
     n_c = g
     rng = np.random.default_rng(_mix(seed, 77) % (1 << 32))
-    picks = set()
-    for g0, lo, sz, nc in table:  # tails and first chunks of every tensor
-        picks.add(g0)
-        picks.add(g0 + nc - 1)
+    short = [g0 + nc - 1 for g0, lo, sz, nc in table if nc and sz % wl.chunk]
+    edges = sorted({g0 for g0, lo, sz, nc in table if nc} | {g0 + nc - 1 for g0, lo, sz, nc in table if nc})
+    picks = set(short[:n])
+    room = n - len(picks)
+    if room > 0:
+        rest = [e for e in edges if e not in picks]
+        if len(rest) > room // 2:
+            rest = list(rng.choice(rest, size=room // 2, replace=False))
+        picks |= set(int(x) for x in rest)
+    while len(picks) < min(n, n_c):
+        picks.add(int(rng.integers(0, n_c)))
     picks = sorted(picks)
-    if len(picks) > n:
-        picks = list(rng.choice(picks, size=n, replace=False))
-    extra = rng.integers(0, n_c, size=max(0, n - len(picks)))
-    picks = sorted(set(int(x) for x in picks) | set(int(x) for x in extra))
     out = []
     starts = np.asarray([t[0] for t in table])
     for gc in picks:
