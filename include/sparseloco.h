@@ -124,6 +124,14 @@ int sl_aggregate_apply(int R, const uint16_t* const* idx, const uint8_t* const* 
                        const float* const* scales, const sl_layout* layout, int chunk, int k,
                        int bits, float* theta_global, float outer_lr, uint32_t* flags, void* stream);
 
+/* The whole of Eq. 2 in one call, for R replicas that live on this device: sl_compress_batch
+ * followed by sl_aggregate_apply on the messages it wrote, on the same stream (err, idx, codes,
+ * scales and theta_global all updated). */
+int sl_outer_step(int R, const float* const* theta_local, float* theta_global, float* const* err,
+                  const sl_layout* layout, float beta, int chunk, int k, int bits, float outer_lr,
+                  uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
+                  void* stream);
+
 /* Static description of an SL_* return code. */
 const char* sl_strerror(int code);
 

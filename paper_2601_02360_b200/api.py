@@ -18,11 +18,11 @@ import torch
 from . import build as _build
 
 SL_OK, SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_CUDA = 0, -1, -2, -3, -4
-SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX = 1, 2
+SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
 SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 2048, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
-           "sl_outer_apply", "sl_aggregate_apply", "sl_strerror")
+           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_strerror")
 
 
 class SlLayout(ctypes.Structure):
@@ -65,6 +65,8 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_outer_apply.argtypes = [vp, vp, u64, f32, vp]
     L.sl_aggregate_apply.restype = i32
     L.sl_aggregate_apply.argtypes = [i32, vp, vp, vp, lp, i32, i32, i32, vp, f32, vp, vp]
+    L.sl_outer_step.restype = i32
+    L.sl_outer_step.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.sl_strerror.restype = ctypes.c_char_p
     L.sl_strerror.argtypes = [i32]
     if path is None:
@@ -172,6 +174,17 @@ def sl_aggregate_apply(idx: Sequence, codes: Sequence, scales: Sequence, layout,
     _check(load().sl_aggregate_apply(R, _ptr_table(idx), _ptr_table(codes), _ptr_table(scales),
                                      _layout(layout).ref(), chunk, k, bits, _ptr(theta_global), outer_lr,
                                      _ptr(flags), _stream(stream)), "sl_aggregate_apply")
+
+
+def sl_outer_step(theta_local: Sequence, theta_global, err: Sequence, layout, beta: float, chunk: int,
+                  k: int, bits: int, outer_lr: float, idx: Sequence, codes: Sequence, scales: Sequence,
+                  flags=None, stream=None) -> None:
+    R = len(theta_local)
+    assert len(err) == len(idx) == len(codes) == len(scales) == R
+    _check(load().sl_outer_step(R, _ptr_table(theta_local), _ptr(theta_global), _ptr_table(err),
+                                _layout(layout).ref(), beta, chunk, k, bits, outer_lr, _ptr_table(idx),
+                                _ptr_table(codes), _ptr_table(scales), _ptr(flags), _stream(stream)),
+           "sl_outer_step")
 
 
 def alloc_messages(layout, chunk: int, k: int, bits: int, R: int, device="cuda"):

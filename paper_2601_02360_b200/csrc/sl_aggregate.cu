@@ -61,19 +61,10 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
 
-// Tuned kernel for full 4096-element chunks of a 16-byte aligned arena.  One CTA per chunk:
-//  * theta_global's 16 KB are requested first (four 128-bit loads per thread) so that they fly
-//    while the messages are handled;
-//  * the (replica, slot) pairs of the chunk are spread over all threads, up to kPairs per
-//    thread and round, and every pair's position and value are fetched before any is applied,
-//    so the R messages cost one memory round trip instead of R;
-//  * the pairs are then applied to the shared-memory accumulator replica by replica (a barrier
-//    between replicas keeps the additions in replica order; inside one message positions are
-//    distinct, so there are no conflicts);
-//  * division by R is a multiplication by the exact reciprocal when R is a power of two (bit
-//    identical), an IEEE division otherwise.
+// Tuned kernel for full 4096-element chunks of a 16-byte aligned arena.  One CTA per chunk;
+// theta_global's 16 KB are requested first (four 128-bit loads per thread) so that they fly
+// while the messages are handled; the rest is aggregate_chunk_c4096().
 constexpr int kAC = 4096;
-constexpr int kPairs = 4;
 
 template <int T, bool APPLY>
 __global__ void __launch_bounds__(kThreads)
@@ -83,76 +74,11 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const uint32_t g = blockIdx.x;
   const ChunkRef c = locate(a.tb, g, kAC);
   if (c.len != kAC) return;                       // short chunks go to the generic tail launch
-  const int k = a.k, bits = a.bits, R = a.R;
-
-  float4* __restrict__ out4 = reinterpret_cast<float4*>(a.out + c.base);
+  float4* out4 = reinterpret_cast<float4*>(a.out + c.base);
   float4 G[4];
-  if (APPLY) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) G[j] = __ldcs(out4 + tid + 256 * j);
-  }
-#pragma unroll
-  for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(acc)[tid + 256 * j] = make_float4(0.f, 0.f, 0.f, 0.f);
-
-  bool bad = false;
-  const int total = R * k;
-  for (int q0 = 0; q0 < total; q0 += kThreads * kPairs) {
-    // fetch this round's pairs: pair q = (replica q / k, slot q % k); q grows with the replica
-    uint32_t pos[kPairs];
-    float val[kPairs];
-    int rep[kPairs];
-#pragma unroll
-    for (int i = 0; i < kPairs; ++i) {
-      const int q = q0 + tid + kThreads * i;
-      pos[i] = 0xFFFFu;
-      val[i] = 0.0f;
-      rep[i] = -1;
-      if (q < total) {
-        const int r = q / k, j = q - r * k;
-        rep[i] = r;
-        const uint32_t p = __ldg(a.m.idx[r] + (uint64_t)g * (uint64_t)k + j);
-        const uint8_t* __restrict__ codes = a.m.codes[r] + (uint64_t)g * (uint64_t)a.stride;
-        if (bits == 32) {
-          val[i] = __ldg(reinterpret_cast<const float*>(codes) + j);
-        } else {
-          const float s = __ldg(a.m.scales[r] + g);
-          const uint32_t bit = (uint32_t)j * (uint32_t)bits;
-          const uint32_t code = ((uint32_t)__ldg(codes + (bit >> 3)) >> (bit & 7u)) & ((1u << bits) - 1u);
-          val[i] = dequant(code, s, bits);
-        }
-        if (p != 0xFFFFu && p >= (uint32_t)kAC) bad = true; else pos[i] = p;
-      }
-    }
-    const int r_lo = q0 / k;
-    const int r_hi = min(R - 1, (q0 + kThreads * kPairs - 1) / k);
-    __syncthreads();                              // accumulator zeroed / previous round applied
-    for (int r = r_lo; r <= r_hi; ++r) {
-#pragma unroll
-      for (int i = 0; i < kPairs; ++i)
-        if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
-      __syncthreads();
-    }
-  }
-  if (total == 0) __syncthreads();
-
-  const bool pow2 = (R & (R - 1)) == 0;
-  const float Rf = (float)R, invR = 1.0f / Rf;
-  const float nlr = -a.outer_lr;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float4 s4 = reinterpret_cast<const float4*>(acc)[tid + 256 * j];
-    float4 u;
-    if (pow2) {
-      u.x = __fmul_rn(s4.x, invR); u.y = __fmul_rn(s4.y, invR); u.z = __fmul_rn(s4.z, invR); u.w = __fmul_rn(s4.w, invR);
-    } else {
-      u.x = __fdiv_rn(s4.x, Rf); u.y = __fdiv_rn(s4.y, Rf); u.z = __fdiv_rn(s4.z, Rf); u.w = __fdiv_rn(s4.w, Rf);
-    }
-    if (APPLY) {
-      u.x = __fmaf_rn(nlr, u.x, G[j].x); u.y = __fmaf_rn(nlr, u.y, G[j].y);
-      u.z = __fmaf_rn(nlr, u.z, G[j].z); u.w = __fmaf_rn(nlr, u.w, G[j].w);
-    }
-    __stcs(out4 + tid + 256 * j, u);
-  }
+  for (int j = 0; j < 4; ++j) G[j] = APPLY ? __ldcs(out4 + tid + 256 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool bad = aggregate_chunk_c4096<APPLY>(acc, G, a.m, g, a.k, a.bits, a.R, a.stride, out4, a.outer_lr, tid, 0);
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
 
@@ -190,13 +116,8 @@ cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned
   if (aligned16 && a.chunk == kAC) {
     if (apply) aggregate_c4096_kernel<T, true><<<a.tb.n_chunks, kThreads, 0, st>>>(a);
     else aggregate_c4096_kernel<T, false><<<a.tb.n_chunks, kThreads, 0, st>>>(a);
-    bool tails = false;
-    for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
-      tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)kAC) != 0;
-    if (tails) {
-      if (apply) aggregate_generic_kernel<T, true, true><<<a.tb.n_tensors, kThreads, smem, st>>>(a);
-      else aggregate_generic_kernel<T, false, true><<<a.tb.n_tensors, kThreads, smem, st>>>(a);
-    }
+    const cudaError_t e = launch_aggregate_tails<T>(a, apply, st);
+    if (e != cudaSuccess) return e;
     return cudaPeekAtLastError();
   }
   if (apply) aggregate_generic_kernel<T, true, false><<<a.tb.n_chunks, kThreads, smem, st>>>(a);
@@ -204,6 +125,20 @@ cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned
   return cudaPeekAtLastError();
 }
 
+template <int T>
+cudaError_t launch_aggregate_tails(const AggregateArgs<T>& a, bool apply, cudaStream_t st) {
+  bool tails = false;
+  for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
+    tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)a.chunk) != 0;
+  if (!tails) return cudaSuccess;
+  const size_t smem = (size_t)a.chunk * 4;
+  if (apply) aggregate_generic_kernel<T, true, true><<<a.tb.n_tensors, kThreads, smem, st>>>(a);
+  else aggregate_generic_kernel<T, false, true><<<a.tb.n_tensors, kThreads, smem, st>>>(a);
+  return cudaPeekAtLastError();
+}
+
+template cudaError_t launch_aggregate_tails<256>(const AggregateArgs<256>&, bool, cudaStream_t);
+template cudaError_t launch_aggregate_tails<SL_MAX_TENSORS>(const AggregateArgs<SL_MAX_TENSORS>&, bool, cudaStream_t);
 template cudaError_t launch_aggregate<256>(const AggregateArgs<256>&, bool, bool, cudaStream_t);
 template cudaError_t launch_aggregate<SL_MAX_TENSORS>(const AggregateArgs<SL_MAX_TENSORS>&, bool, bool, cudaStream_t);
 

@@ -51,10 +51,13 @@ void fill_table(Table<T>& tb, const sl_layout* L, int chunk, bool* offsets_mult4
   *offsets_mult4 = m4;
 }
 
+// step = false: Eq. 2 lines 1-4 only.  step = true: the whole of Eq. 2 (theta_global is updated):
+// compress followed by aggregate-apply on the same stream.
 template <int T>
-int compress_impl(int R, const float* const* theta_local, const float* theta_global, float* const* err,
+int compress_impl(int R, const float* const* theta_local, float* theta_global, float* const* err,
                   const sl_layout* L, float beta, int chunk, int k, int bits, uint16_t* const* idx,
-                  uint8_t* const* codes, float* const* scales, uint32_t* flags, cudaStream_t st) {
+                  uint8_t* const* codes, float* const* scales, uint32_t* flags, cudaStream_t st,
+                  bool step, float outer_lr) {
   std::unique_ptr<CompressArgs<T>> a(new (std::nothrow) CompressArgs<T>);
   if (!a) return SL_ERR_CUDA;
   bool m4;
@@ -70,23 +73,45 @@ int compress_impl(int R, const float* const* theta_local, const float* theta_glo
            aligned(codes[r], 16) && aligned(scales[r], 4);
   }
   a->theta_global = theta_global;
+  a->theta_out = theta_global;
   a->flags = flags;
   a->beta = beta;
+  a->outer_lr = outer_lr;
+  a->fused = 0;
   a->chunk = chunk;
   a->k = k;
   a->bits = bits;
   a->R = R;
   a->stride = (uint32_t)codes_stride(k, bits);
-  return launch_compress<T>(*a, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+  if (!step) return launch_compress<T>(*a, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+
+  std::unique_ptr<AggregateArgs<T>> g(new (std::nothrow) AggregateArgs<T>);
+  if (!g) return SL_ERR_CUDA;
+  g->tb = a->tb;
+  for (int r = 0; r < R; ++r) {
+    g->m.idx[r] = idx[r];
+    g->m.codes[r] = codes[r];
+    g->m.scales[r] = scales[r];
+  }
+  g->out = theta_global;
+  g->flags = flags;
+  g->outer_lr = outer_lr;
+  g->chunk = chunk;
+  g->k = k;
+  g->bits = bits;
+  g->R = R;
+  g->stride = a->stride;
+  if (launch_compress<T>(*a, al16, st) != cudaSuccess) return SL_ERR_CUDA;
+  return launch_aggregate<T>(*g, true, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 }
 
-int compress_checked(int R, const float* const* theta_local, const float* theta_global,
+int compress_checked(int R, const float* const* theta_local, float* theta_global,
                      float* const* err, const sl_layout* L, float beta, int chunk, int k, int bits,
                      uint16_t* const* idx, uint8_t* const* codes, float* const* scales,
-                     uint32_t* flags, void* stream) {
+                     uint32_t* flags, void* stream, bool step = false, float outer_lr = 0.0f) {
   if (R < 1 || R > SL_MAX_REPLICAS) return SL_ERR_INVALID_ARG;
   if (!theta_local || !theta_global || !err || !idx || !codes || !scales) return SL_ERR_INVALID_ARG;
-  if (!std::isfinite(beta)) return SL_ERR_INVALID_ARG;
+  if (!std::isfinite(beta) || !std::isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
   const int rc = check_common(L, chunk, k, bits);
   if (rc != SL_OK) return rc;
   if (!aligned(theta_global, 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
@@ -99,9 +124,9 @@ int compress_checked(int R, const float* const* theta_local, const float* theta_
   cudaStream_t st = (cudaStream_t)stream;
   if (L->n_tensors <= 256)
     return compress_impl<256>(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx, codes,
-                              scales, flags, st);
+                              scales, flags, st, step, outer_lr);
   return compress_impl<SL_MAX_TENSORS>(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx,
-                                       codes, scales, flags, st);
+                                       codes, scales, flags, st, step, outer_lr);
 }
 
 template <int T>
@@ -173,16 +198,25 @@ uint64_t sl_codes_stride(int k, int bits) {
 int sl_compress(const float* theta_local, const float* theta_global, float* err, const sl_layout* L,
                 float beta, int chunk, int k, int bits, uint16_t* idx, uint8_t* codes, float* scales,
                 uint32_t* flags, void* stream) {
-  return compress_checked(1, &theta_local, theta_global, &err, L, beta, chunk, k, bits, &idx, &codes,
-                          &scales, flags, stream);
+  // theta_global is only read when no step is asked for
+  return compress_checked(1, &theta_local, const_cast<float*>(theta_global), &err, L, beta, chunk, k, bits,
+                          &idx, &codes, &scales, flags, stream);
 }
 
 int sl_compress_batch(int R, const float* const* theta_local, const float* theta_global,
                       float* const* err, const sl_layout* L, float beta, int chunk, int k, int bits,
                       uint16_t* const* idx, uint8_t* const* codes, float* const* scales,
                       uint32_t* flags, void* stream) {
+  return compress_checked(R, theta_local, const_cast<float*>(theta_global), err, L, beta, chunk, k, bits, idx,
+                          codes, scales, flags, stream);
+}
+
+int sl_outer_step(int R, const float* const* theta_local, float* theta_global, float* const* err,
+                  const sl_layout* L, float beta, int chunk, int k, int bits, float outer_lr,
+                  uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
+                  void* stream) {
   return compress_checked(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx, codes, scales,
-                          flags, stream);
+                          flags, stream, true, outer_lr);
 }
 
 int sl_aggregate(int R, const uint16_t* const* idx, const uint8_t* const* codes,

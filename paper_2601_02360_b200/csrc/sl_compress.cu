@@ -8,6 +8,8 @@
 //                            chunk walks all R replicas with theta_global held in registers, a
 //                            cheap lower bound on the k-th magnitude prunes the chunk to a few
 //                            hundred candidates, one warp finishes the exact selection.
+#include <algorithm>
+
 #include "sl_common.cuh"
 
 namespace sl {
@@ -214,39 +216,49 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 // specialised: 8 producer warps (256 threads) and kSel selector warps; selector q handles the
 // replicas r with r % kSel == q, so two selections are in flight while the producers run ahead.
 //
-//  * theta_local and e of replica r arrive by TMA bulk copies (cp.async.bulk + mbarrier):
-//    theta_local in a 2-deep ring (dead after phase A, refilled by producer thread 0), e in a
-//    4-deep ring (alive until its bulk store has read it, refilled by the selector that owns it).
+//  * All bulk data moves by TMA (cp.async.bulk, no multicast), issued by producer thread 0:
+//    theta_local of replica r is loaded two replicas ahead into a 2-deep ring (dead after phase
+//    A); e lives in a 4-deep ring whose stages cycle through load -> produce -> select -> drain:
+//    e(r+1) is loaded while replica r is produced, replica r-1 is being selected, and the stage
+//    of replica r-2, patched with the residual, drains to the error buffer as one bulk store.
+//    Nobody waits for a store it has just issued: under a saturated memory system a 16 KB store
+//    takes microseconds to drain, and a warp with ordinary global stores in flight also stalls
+//    on its next shared-memory access.  So the selectors issue no global stores at all.
 //  * Producers, per replica (thread t owns float4s t, t+256, t+512, t+768 of the chunk):
 //      A  e' = fma(beta, e, theta_global - theta_local), written in place of e in the stage;
-//         per-thread maximum key.  The chunk is cut into kp >= k groups of whole threads
-//         (kp a power of two); at least k keys are >= the smallest group maximum T1, so T1 is
-//         a lower bound of the k-th largest key.
-//      B  the keys >= T1 (a few hundred) are compacted into a candidate list.
+//         per-thread maximum key.  Every warp sorts its 32 thread maxima (bitonic network of
+//         shuffles) and takes the j-th largest, j = ceil(k/8): at least j keys of the warp's 512
+//         are >= it, so at least 8j >= k keys of the chunk are >= T1 = the smallest of the eight
+//         values: T1 is a lower bound of the k-th largest key.
+//      B  the keys >= T1 (about a hundred for k = 64) are compacted into a candidate list and
+//         counted in a 256-bin histogram of the key range [T1, max].
+//      E  replica r-2, finished by its selector in the meantime: warp 0 copies its message from
+//         shared memory to idx / codes / scales, thread 0 issues the bulk store of its stage.
 //  * Selector, per replica:
-//      C  bisects the key range [T1, max] for a threshold that leaves exactly k candidates;
-//         if the range collapses first the k-th key is tied, and the lowest positions among
-//         its ties are found by a second bisection over positions.
-//      D  marks the kept positions in a 4096-bit map, walks it in ascending position (each
-//         lane owns 128 positions, slots from a prefix sum of popcounts), writes idx and
-//         codes, patches the residual into the stage.
-//      E  one TMA bulk store sends the stage's 16 KB of e' to the error buffer; when the
-//         store has read the stage, e of replica r+4 is loaded into it.
+//      C  a suffix scan of the histogram finds the bin that holds the k-th largest key; a
+//         bisection inside that bin (candidates in registers) finds a threshold that leaves
+//         exactly k candidates; if the range collapses first the k-th key is tied, and the
+//         lowest positions among its ties are found by a second bisection over positions.
+//      D  kept positions are marked in a 4096-bit map and compacted (ballots); a prefix sum of
+//         the map's popcounts turns a position into its rank = message slot; each lane then
+//         handles k/32 kept elements: idx and code into a shared-memory copy of the message,
+//         residual patched into the stage.
 //  If the candidate list overflows (tie-heavy or constant chunks) the selector runs an exact
 //  warp-wide radix select over the whole chunk instead of C.
 //
 // Hand-offs: named barrier 1 = producers only; 2+q = candidate list q ready (producers
-// arrive, selector q waits); 4+q = candidate list q free again (selector q arrives, producers
-// wait).  Every mbarrier wait is bounded; running out raises SL_FLAG_TIMEOUT and the kernel
+// arrive, selector q waits); 4+q = selector q has finished a replica: its candidate list is free
+// and the stage holds the final residual (selector q arrives, producers wait).  Every mbarrier wait is bounded; running out raises SL_FLAG_TIMEOUT and the kernel
 // carries on (no trap, no hang).
 // ---------------------------------------------------------------------------
 constexpr int kC = 4096;
 constexpr int kSel = 2;               // selector warps
 constexpr int kTlStages = 2;
 constexpr int kEeStages = 4;
-constexpr int kCandMax = 1024;
-constexpr int kCandReg = 12;          // candidates per lane held in registers (C <= 384)
-constexpr int kMaxCodeWords = 32;     // k * bits / 32 <= 128 * 8 / 32
+constexpr int kCandMax = 512;
+constexpr int kCandReg = 6;           // candidates per lane held in registers (C <= 192)
+
+constexpr int kPtrCache = 16;         // replicas whose pointers are staged in shared memory
 constexpr int kFastThreads = kThreads + 32 * kSel;
 constexpr int kPairThreads = kThreads + 32;   // producers + one selector
 constexpr uint32_t kWaitLimit = 1u << 22;
@@ -259,17 +271,19 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// bounded wait on a phase; false = gave up
+// bounded wait on a phase; false = gave up.  test_wait + nanosleep rather than try_wait: a
+// suspended try_wait was seen to delay the shared-memory instructions of other warps.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   const uint32_t addr = smem_u32(bar);
   for (uint32_t it = 0; it < kWaitLimit; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
     if (ok) return true;
+    __nanosleep(40);
   }
   return false;
 }
@@ -282,63 +296,117 @@ __device__ __forceinline__ void tma_store_1d(void* dst, const void* src, uint32_
                ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// wait until all bulk stores of this thread have read their source
+__device__ __forceinline__ void tma_store_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
-__device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
 struct alignas(16) FastSmem {
   float tl[kTlStages][kC];            // theta_local of replica r in stage r % 2
   float ee[kEeStages][kC];            // e of replica r in stage r % 4, then e' in place, then the store's source
   uint32_t cand_key[kSel][kCandMax];
   uint16_t cand_pos[kSel][kCandMax];
-  uint32_t bitmap[kSel][kC / 32];
-  uint32_t hist[kSel][256];
-  uint32_t cw[kSel][kMaxCodeWords];
+  uint32_t bitmap[kSel][kC / 32];     // kept positions of the selection in progress
+  uint32_t hist[kSel][256];           // candidates per bin of [T1, max]; radix histogram in the overflow path
+  uint16_t msg_idx[kEeStages][128];   // the message of the replica in each stage: positions,
+  uint32_t msg_codes[kEeStages][128]; // packed codes (or k raw floats when bits == 32),
+  float msg_scale[kEeStages];         // scale
+  uint16_t kept_pos[kSel][128];
+  uint8_t prefix[kSel][kC / 32];      // kept positions before each bitmap word
   uint32_t wmin[kEeStages][kWarps], wmax[kEeStages][kWarps];   // ring: producers run up to three replicas ahead
   uint32_t count[kSel];
+  const float* p_tl[kPtrCache];       // the first kPtrCache replicas' pointers (parameter-space reads
+  float* p_err[kPtrCache];            // with a run-time index are slow)
+  uint16_t* p_idx[kPtrCache];
+  uint8_t* p_codes[kPtrCache];
+  float* p_scales[kPtrCache];
   uint64_t full_tl[kTlStages];
   uint64_t full_ee[kEeStages];
 };
+static_assert(sizeof(FastSmem) <= 115712, "two CTAs per SM need 2 * (smem + 1 KB) <= 228 KB");
+
+// bins of the candidate histogram: bin = (key - T1) >> sh with (max - T1) >> sh <= 255
+__device__ __forceinline__ int hist_shift(uint32_t T1, uint32_t smax) {
+  const uint32_t range = smax - T1;
+  return range < 256u ? 0 : (32 - __clz(range)) - 8;
+}
 
 // number of candidate keys >= mid; keys either in registers (NREG > 0) or in shared memory
 template <int NREG>
-__device__ __forceinline__ uint32_t count_ge(const uint32_t* ck_reg, const uint32_t* ck_smem, uint32_t C,
-                                             uint32_t mid, int lane) {
-  uint32_t cnt = 0;
+__device__ __forceinline__ uint32_t count_ge(const uint32_t (&ck)[NREG > 0 ? NREG : 1], const uint32_t* ck_smem,
+                                             uint32_t C, uint32_t mid, int lane) {
+  uint32_t c0 = 0, c1 = 0, c2 = 0;
   if (NREG > 0) {
 #pragma unroll
-    for (int i = 0; i < NREG; ++i) cnt += ck_reg[i] >= mid ? 1u : 0u;
+    for (int i = 0; i < NREG; i += 3) {
+      c0 += ck[i] >= mid ? 1u : 0u;
+      if (i + 1 < NREG) c1 += ck[i + 1] >= mid ? 1u : 0u;
+      if (i + 2 < NREG) c2 += ck[i + 2] >= mid ? 1u : 0u;
+    }
   } else {
-    for (uint32_t i = lane; i < C; i += 32) cnt += ck_smem[i] >= mid ? 1u : 0u;
+    for (uint32_t i = lane; i < C; i += 32) c0 += ck_smem[i] >= mid ? 1u : 0u;
   }
-  return __reduce_add_sync(kFull, cnt);
+  return __reduce_add_sync(kFull, c0 + c1 + c2);
 }
 
-// Phase C + marking: threshold among C candidates, kept positions OR-ed into the bitmap.
+// Phase C and the first half of D for a candidate list that did not overflow: threshold, then
+// kept positions marked in `bitmap` and compacted into `kept_pos` (any order).
 template <int NREG>
 __device__ __forceinline__ void select_candidates(const uint32_t* cand_key, const uint16_t* cand_pos, uint32_t C,
-                                                  uint32_t k, uint32_t T1, uint32_t smax, uint32_t* bitmap,
-                                                  int lane, uint32_t* stats) {
+                                                  uint32_t k, uint32_t T1, uint32_t smax, uint32_t* hist,
+                                                  uint32_t* bitmap, uint16_t* kept_pos, int lane) {
   uint32_t ck[NREG > 0 ? NREG : 1];
+  uint32_t cp[NREG > 0 ? NREG : 1];
   if (NREG > 0) {
 #pragma unroll
     for (int i = 0; i < NREG; ++i) {
       const uint32_t at = (uint32_t)lane + 32u * (uint32_t)i;
       ck[i] = at < C ? cand_key[at] : 0u;          // padding 0 is below every probe (probes are > T1 >= 0)
+      cp[i] = at < C ? (uint32_t)cand_pos[at] : 0u;
     }
   }
-  uint32_t lo = T1, hi = smax + 1u, cnt_hi = 0;
-  uint32_t thr_ge = T1;                            // keep key >= thr_ge ...
+  // ---- the bin of the k-th largest key: suffix sums of the histogram, top bin first
+  const int sh = hist_shift(T1, smax);
+  uint32_t lo, hi, cnt_hi;
+  bool exact;
+  {
+    const uint4 h0 = reinterpret_cast<const uint4*>(hist)[2 * lane];
+    const uint4 h1 = reinterpret_cast<const uint4*>(hist)[2 * lane + 1];
+    reinterpret_cast<uint4*>(hist)[2 * lane] = make_uint4(0, 0, 0, 0);       // ready for the next replica
+    reinterpret_cast<uint4*>(hist)[2 * lane + 1] = make_uint4(0, 0, 0, 0);
+    const uint32_t h[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+    uint32_t mine = 0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) mine += h[b];
+    uint32_t suf = mine;                          // candidates in this lane's bins and above
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t o = __shfl_down_sync(kFull, suf, d);
+      if (lane + d < 32) suf += o;
+    }
+    const uint32_t vote = __ballot_sync(kFull, suf >= k);
+    const int sel = 31 - __clz(vote);             // highest lane whose suffix still reaches k (C >= k: lane 0 does)
+    uint32_t above = suf - mine, bin = (uint32_t)lane * 8u, in_bin = 0;
+    bool found = false;
+#pragma unroll
+    for (int bb = 7; bb >= 0; --bb) {
+      if (!found) {
+        if (above + h[bb] >= k) { found = true; bin = (uint32_t)(lane * 8 + bb); in_bin = h[bb]; }
+        else above += h[bb];
+      }
+    }
+    bin = __shfl_sync(kFull, bin, sel);
+    in_bin = __shfl_sync(kFull, in_bin, sel);
+    cnt_hi = __shfl_sync(kFull, above, sel);      // candidates in the bins above: all kept, fewer than k
+    lo = T1 + (bin << sh);                        // keys of the bin: lo <= key < lo + 2^sh
+    hi = lo + (1u << sh);
+    exact = cnt_hi + in_bin == k;                 // the whole bin is kept: threshold = its lower edge
+  }
+  uint32_t thr_ge = lo;                            // keep key >= thr_ge ...
   uint32_t thr_eq = 0xFFFFFFFFu, pos_le = 0;       // ... and key == thr_eq at position <= pos_le
-  if (C != k) {
-    bool exact = false;
-    while (hi - lo > 1u) {
+  if (!exact) {
+    while (hi - lo > 1u) {                         // count(key >= lo) > k > count(key >= hi) = cnt_hi
       const uint32_t mid = lo + ((hi - lo) >> 1);
       const uint32_t cnt = count_ge<NREG>(ck, cand_key, C, mid, lane);
-#ifdef SL_STATS
-      if (lane == 0) atomicAdd(&stats[1], 1u);
-#endif
       if (cnt == k) { thr_ge = mid; exact = true; break; }
       if (cnt > k) lo = mid; else { hi = mid; cnt_hi = cnt; }
     }
@@ -358,33 +426,44 @@ __device__ __forceinline__ void select_candidates(const uint32_t* cand_key, cons
         if (cnt >= need) phi = pm; else plo = pm + 1;
       }
       pos_le = plo;
-#ifdef SL_STATS
-      if (lane == 0) atomicAdd(&stats[2], 1u);
-#endif
     }
   }
+  // ---- mark and compact the kept candidates
+  uint32_t base = 0;
   if (NREG > 0) {
 #pragma unroll
     for (int i = 0; i < NREG; ++i) {
-      const uint32_t at = (uint32_t)lane + 32u * (uint32_t)i;
-      if (at < C) {
-        const uint32_t cp = cand_pos[at];
-        if (ck[i] >= thr_ge || (ck[i] == thr_eq && cp <= pos_le)) atomicOr(&bitmap[cp >> 5], 1u << (cp & 31u));
+      if (32u * (uint32_t)i < C) {
+        const bool keep = ((uint32_t)lane + 32u * (uint32_t)i < C) &&
+                          (ck[i] >= thr_ge || (ck[i] == thr_eq && cp[i] <= pos_le));
+        const uint32_t bal = __ballot_sync(kFull, keep);
+        if (keep) {
+          atomicOr(&bitmap[cp[i] >> 5], 1u << (cp[i] & 31u));
+          kept_pos[base + __popc(bal & lanemask_lt())] = (uint16_t)cp[i];
+        }
+        base += __popc(bal);
       }
     }
   } else {
-    for (uint32_t i = lane; i < C; i += 32) {
-      const uint32_t k_i = cand_key[i];
-      const uint32_t cp = cand_pos[i];
-      if (k_i >= thr_ge || (k_i == thr_eq && cp <= pos_le)) atomicOr(&bitmap[cp >> 5], 1u << (cp & 31u));
+    for (uint32_t i0 = 0; i0 < C; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      const uint32_t k_i = i < C ? cand_key[i] : 0u;
+      const uint32_t p_i = i < C ? (uint32_t)cand_pos[i] : 0u;
+      const bool keep = i < C && (k_i >= thr_ge || (k_i == thr_eq && p_i <= pos_le));
+      const uint32_t bal = __ballot_sync(kFull, keep);
+      if (keep) {
+        atomicOr(&bitmap[p_i >> 5], 1u << (p_i & 31u));
+        kept_pos[base + __popc(bal & lanemask_lt())] = (uint16_t)p_i;
+      }
+      base += __popc(bal);
     }
   }
 }
 
-// Overflow path of the selector: exact radix select over the whole chunk by one warp, kept
-// positions written to the bitmap (one ballot = one bitmap word).
+// Overflow path of the selector: exact radix select over the whole chunk by one warp; kept
+// positions go to the bitmap (one ballot = one bitmap word) and to kept_pos.
 __device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, uint32_t* hist, uint32_t* bitmap,
-                                                 int lane) {
+                                                 uint16_t* kept_pos, int lane) {
   uint32_t prefix = 0, need = k;
 #pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
@@ -424,8 +503,10 @@ __device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, ui
     prefix |= digit << shift;
     __syncwarp();
   }
+#pragma unroll
+  for (int b = 0; b < 8; ++b) hist[lane * 8 + b] = 0;     // leave the histogram clean for phase B
   const uint32_t kth = prefix;
-  uint32_t eq_seen = 0;
+  uint32_t eq_seen = 0, base = 0;
   for (int w = 0; w < kC / 32; ++w) {
     const uint32_t key = key_of(ep[w * 32 + lane]);
     const bool eq = key == kth;
@@ -433,9 +514,37 @@ __device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, ui
     const bool keep = key > kth || (eq && eq_seen + __popc(eqm & lanemask_lt()) < need);
     const uint32_t km = __ballot_sync(kFull, keep);
     if (lane == 0) bitmap[w] = km;
+    if (keep) kept_pos[base + __popc(km & lanemask_lt())] = (uint16_t)(w * 32 + lane);
     eq_seen += __popc(eqm);
+    base += __popc(km);
   }
 }
+
+// One work item = one (full chunk, replica) pair.  CTA b of G owns the full chunks among
+// b, b+G, b+2G, ... and walks their items in order: item w is replica w % R of its (w / R)-th chunk.
+template <int T>
+struct ItemCursor {
+  uint32_t g;      // chunk number in the arena
+  uint64_t base;   // element offset of the chunk
+  int r;           // replica
+  bool valid;
+
+  // first full chunk at or after g0 (stepping by the grid size)
+  __device__ __forceinline__ void seek(const Table<T>& tb, uint32_t g0, uint32_t step) {
+    g = g0;
+    valid = false;
+    while (g < tb.n_chunks) {
+      const ChunkRef c = locate(tb, g, kC);
+      if (c.len == kC) { base = c.base; valid = true; return; }
+      g += step;                                   // short chunks belong to the tail launch
+    }
+  }
+  __device__ __forceinline__ void start(const Table<T>& tb, uint32_t b, uint32_t step) { r = 0; seek(tb, b, step); }
+  __device__ __forceinline__ void advance(const Table<T>& tb, int n, int R, uint32_t step) {
+    r += n;
+    while (valid && r >= R) { r -= R; seek(tb, g + step, step); }
+  }
+};
 
 template <int T>
 __global__ void __launch_bounds__(kFastThreads, 2)
@@ -444,14 +553,20 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   FastSmem& sm = *reinterpret_cast<FastSmem*>(smem_raw);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t g = blockIdx.x;
-  const ChunkRef c = locate(a.tb, g, kC);
-  if (c.len != kC) return;                        // short chunks go to the generic tail launch
+  const uint32_t G = gridDim.x;
   const int k = a.k, bits = a.bits, R = a.R;
   constexpr uint32_t kBytes = kC * 4;
 
   for (int i = tid; i < kSel * (kC / 32); i += kFastThreads) (&sm.bitmap[0][0])[i] = 0;
-  if (tid < kSel * kMaxCodeWords) (&sm.cw[0][0])[tid] = 0;
+  for (int i = tid; i < kSel * 256; i += kFastThreads) (&sm.hist[0][0])[i] = 0;
+  for (int i = tid; i < kEeStages * 128; i += kFastThreads) (&sm.msg_codes[0][0])[i] = 0;
+  if (tid < kPtrCache && tid < R) {
+    sm.p_tl[tid] = a.p.theta_local[tid];
+    sm.p_err[tid] = a.p.err[tid];
+    sm.p_idx[tid] = a.p.idx[tid];
+    sm.p_codes[tid] = a.p.codes[tid];
+    sm.p_scales[tid] = a.p.scales[tid];
+  }
   if (tid == 0) {
 #pragma unroll
     for (int q = 0; q < kSel; ++q) sm.count[q] = 0;
@@ -467,27 +582,35 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 
   if (warp < kWarps) {
     // ======================= producers =======================================
+    ItemCursor<T> cur;                            // item w
+    cur.start(a.tb, blockIdx.x, G);
+    ItemCursor<T> pf = cur;                       // thread 0: the item whose theta_local is loaded next
     if (tid == 0) {
-      for (int r = 0; r < kTlStages && r < R; ++r) {
-        mbar_expect_tx(&sm.full_tl[r], kBytes);
-        tma_load_1d(sm.tl[r], a.p.theta_local[r] + c.base, kBytes, &sm.full_tl[r]);
+      for (int i = 0; i < kTlStages && pf.valid; ++i) {
+        mbar_expect_tx(&sm.full_tl[i], kBytes);
+        tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
+        pf.advance(a.tb, 1, R, G);
       }
     }
-    int kp = 8;                                   // kp = max(8, pow2ceil(k)) groups of 256/kp threads
-    while (kp < k) kp <<= 1;
-    const int group_lanes = kThreads / kp;        // 32, 16, 8, 4 or 2 lanes
+    const int cwords = bits == 32 ? k : (k * bits) >> 5;   // 32-bit words of codes per chunk
+    const int jsel = 32 - (k + kWarps - 1) / kWarps;   // lane holding the ceil(k/8)-th largest after an ascending sort
     const float beta = a.beta;
-    const float4* __restrict__ tg4 = reinterpret_cast<const float4*>(a.theta_global + c.base);
-    float4 G[4];
+    float4 G4[4];                                 // this thread's 16 elements of theta_global
+    if (cur.valid) {
+      const float4* tg4 = reinterpret_cast<const float4*>(a.theta_global + cur.base);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) G[j] = __ldcs(tg4 + tid + 256 * j);
+      for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + tid + 256 * j);
+    }
+    uint32_t g_m1 = 0, g_m2 = 0;                  // chunk and replica of items w-1 and w-2
+    int r_m1 = 0, r_m2 = 0;
     __syncwarp();
 
+    uint32_t w = 0;
 #pragma unroll 1
-    for (int r = 0; r < R; ++r) {
-      const int st = r % kTlStages, se = r % kEeStages, q = r % kSel;
-      if (!mbar_wait(&sm.full_tl[st], (uint32_t)((r / kTlStages) & 1))) timed_out = true;
-      if (!mbar_wait(&sm.full_ee[se], (uint32_t)((r / kEeStages) & 1))) timed_out = true;
+    for (; cur.valid; ++w) {
+      const int st = w % kTlStages, se = w % kEeStages, q = w % kSel;
+      if (!mbar_wait(&sm.full_tl[st], (w / kTlStages) & 1u)) timed_out = true;
+      if (!mbar_wait(&sm.full_ee[se], (w / kEeStages) & 1u)) timed_out = true;
       const float4* tl4 = reinterpret_cast<const float4*>(sm.tl[st]);
       float4* ee4 = reinterpret_cast<float4*>(sm.ee[se]);
       // ---- A ----
@@ -498,10 +621,10 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         const float4 L = tl4[tid + 256 * j];
         const float4 E = ee4[tid + 256 * j];
         float4 v;
-        v.x = __fmaf_rn(beta, E.x, __fsub_rn(G[j].x, L.x));
-        v.y = __fmaf_rn(beta, E.y, __fsub_rn(G[j].y, L.y));
-        v.z = __fmaf_rn(beta, E.z, __fsub_rn(G[j].z, L.z));
-        v.w = __fmaf_rn(beta, E.w, __fsub_rn(G[j].w, L.w));
+        v.x = __fmaf_rn(beta, E.x, __fsub_rn(G4[j].x, L.x));
+        v.y = __fmaf_rn(beta, E.y, __fsub_rn(G4[j].y, L.y));
+        v.z = __fmaf_rn(beta, E.z, __fsub_rn(G4[j].z, L.z));
+        v.w = __fmaf_rn(beta, E.w, __fsub_rn(G4[j].w, L.w));
         ee4[tid + 256 * j] = v;
         key[4 * j + 0] = key_of(v.x);
         key[4 * j + 1] = key_of(v.y);
@@ -509,149 +632,225 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         key[4 * j + 3] = key_of(v.w);
         tmax = max(tmax, max(max(key[4 * j], key[4 * j + 1]), max(key[4 * j + 2], key[4 * j + 3])));
       }
-      fence_async_smem();                         // e' must be visible to the later bulk store
-      uint32_t gmax = tmax;
-      for (int d = 1; d < group_lanes; d <<= 1) gmax = max(gmax, __shfl_xor_sync(kFull, gmax, d));
-      const uint32_t wmin = __reduce_min_sync(kFull, gmax);
-      const uint32_t wmax = __reduce_max_sync(kFull, tmax);
-      if (lane == 0) { sm.wmin[se][warp] = wmin; sm.wmax[se][warp] = wmax; }
-      named_sync(1, kThreads);
-      if (tid == 0 && r + kTlStages < R) {        // every producer has read theta_local(r): refill its stage
-        mbar_expect_tx(&sm.full_tl[st], kBytes);
-        tma_load_1d(sm.tl[st], a.p.theta_local[r + kTlStages] + c.base, kBytes, &sm.full_tl[st]);
-      }
-      uint32_t T1 = 0xFFFFFFFFu;
+      fence_async_smem();                         // e' must be visible to the bulk store that drains this stage
+      // the next item: same chunk, or the next chunk, whose theta_global is requested now (the
+      // registers are free) so that it arrives while this item is finished
+      ItemCursor<T> nxt = cur;
+      nxt.advance(a.tb, 1, R, G);
+      if (nxt.valid && nxt.r == 0) {
+        const float4* tg4 = reinterpret_cast<const float4*>(a.theta_global + nxt.base);
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) T1 = min(T1, sm.wmin[se][w]);
+        for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + tid + 256 * j);
+      }
+      uint32_t v = tmax;                           // bitonic sort of the 32 thread maxima, ascending over lanes
+#pragma unroll
+      for (int size = 2; size <= 32; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+          const uint32_t o = __shfl_xor_sync(kFull, v, stride);
+          const bool up = (lane & size) == 0, lower = (lane & stride) == 0;
+          v = (up == lower) ? min(v, o) : max(v, o);
+        }
+      }
+      const uint32_t wmin = __shfl_sync(kFull, v, jsel);     // this warp's ceil(k/8)-th largest thread maximum
+      const uint32_t wmax = __shfl_sync(kFull, v, 31);
+      if (lane == 0) { sm.wmin[se][warp] = wmin; sm.wmax[se][warp] = wmax; }
+      if (w >= (uint32_t)kSel) {
+        __syncwarp();
+        named_sync(4 + q, kPairThreads);          // selector q has finished item w-2
+        // ---- E (item w-2): its message leaves shared memory (warp 0, three coalesced stores) ----
+        if (warp == 0) {
+          const int sp = (w - kSel) % kEeStages;
+          const bool pc = r_m2 < kPtrCache;
+          uint16_t* oidx = (pc ? sm.p_idx[r_m2] : a.p.idx[r_m2]) + (uint64_t)g_m2 * (uint64_t)k;
+          uint32_t* ocodes = reinterpret_cast<uint32_t*>((pc ? sm.p_codes[r_m2] : a.p.codes[r_m2]) + (uint64_t)g_m2 * (uint64_t)a.stride);
+          for (int i = lane; i < (k >> 1); i += 32)
+            reinterpret_cast<uint32_t*>(oidx)[i] = reinterpret_cast<const uint32_t*>(sm.msg_idx[sp])[i];
+          for (int i = lane; i < cwords; i += 32) {
+            ocodes[i] = sm.msg_codes[sp][i];
+            sm.msg_codes[sp][i] = 0;              // the next message in this stage ORs its codes into zeros
+          }
+          if (lane == 0) (pc ? sm.p_scales[r_m2] : a.p.scales[r_m2])[g_m2] = sm.msg_scale[sp];
+        }
+      }
+      named_sync(1, kThreads);
+      if (tid == 0 && pf.valid) {                 // every producer has read theta_local(w): its stage takes item w+2's
+        mbar_expect_tx(&sm.full_tl[st], kBytes);
+        tma_load_1d(sm.tl[st], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[st]);
+        pf.advance(a.tb, 1, R, G);
+      }
+      uint32_t T1, smax;
+      {
+        const uint4 m0 = reinterpret_cast<const uint4*>(sm.wmin[se])[0], m1 = reinterpret_cast<const uint4*>(sm.wmin[se])[1];
+        const uint4 x0 = reinterpret_cast<const uint4*>(sm.wmax[se])[0], x1 = reinterpret_cast<const uint4*>(sm.wmax[se])[1];
+        T1 = min(min(min(m0.x, m0.y), min(m0.z, m0.w)), min(min(m1.x, m1.y), min(m1.z, m1.w)));
+        smax = max(max(max(x0.x, x0.y), max(x0.z, x0.w)), max(max(x1.x, x1.y), max(x1.z, x1.w)));
+      }
+      const int sh = hist_shift(T1, smax);
       // ---- B ----
-      __syncwarp();
-      if (r >= kSel) named_sync(4 + q, kPairThreads);   // selector q is done with its candidate list
       uint32_t mask = 0;
 #pragma unroll
       for (int e = 0; e < 16; ++e) mask |= (key[e] >= T1 ? 1u : 0u) << e;
-      const uint32_t cnt = __popc(mask);
-      uint32_t incl = cnt;
+      if (mask) {
+        uint32_t at = atomicAdd(&sm.count[q], (uint32_t)__popc(mask));
+        uint32_t* ckey = sm.cand_key[q];
+        uint16_t* cpos = sm.cand_pos[q];
+        uint32_t* hist = sm.hist[q];
 #pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t o = __shfl_up_sync(kFull, incl, d);
-        if (lane >= d) incl += o;
-      }
-      uint32_t base = 0;
-      if (lane == 31) base = atomicAdd(&sm.count[q], incl);
-      base = __shfl_sync(kFull, base, 31);
-      uint32_t at = base + incl - cnt;
-      const float* ep = sm.ee[se];
-      while (mask) {
-        const int b = __ffs(mask) - 1;
-        mask &= mask - 1;
-        const int pos = ((b >> 2) << 10) + (tid << 2) + (b & 3);
-        if (at < (uint32_t)kCandMax) {
-          sm.cand_key[q][at] = key_of(ep[pos]);
-          sm.cand_pos[q][at] = (uint16_t)pos;
+        for (int e = 0; e < 16; ++e) {
+          if (mask & (1u << e)) {
+            if (at < (uint32_t)kCandMax) {
+              ckey[at] = key[e];
+              cpos[at] = (uint16_t)(((e >> 2) << 10) + (tid << 2) + (e & 3));
+            }
+            atomicAdd(&hist[(key[e] - T1) >> sh], 1u);
+            ++at;
+          }
         }
-        ++at;
       }
       __syncwarp();                               // bar.* is warp-aligned: reconverge first
-      __threadfence_block();
-      named_arrive(2 + q, kPairThreads);          // candidate list q is ready
+      named_arrive(2 + q, kPairThreads);          // candidate list q is ready (bar.arrive orders the shared-memory
+                                                  // writes before it; a membar here would also wait for global stores)
+      g_m2 = g_m1; r_m2 = r_m1;
+      g_m1 = cur.g; r_m1 = cur.r;
+      cur = nxt;
+    }
+    // the last kSel items' messages
+    const uint32_t W = w;
+    for (uint32_t wp = (W > (uint32_t)kSel ? W - kSel : 0); wp < W; ++wp) {
+      const bool last = wp + 1 == W;
+      const uint32_t gp = last ? g_m1 : g_m2;
+      const int rp = last ? r_m1 : r_m2;
+      __syncwarp();
+      named_sync(4 + wp % kSel, kPairThreads);
+      if (warp == 0) {
+        const int sp = wp % kEeStages;
+        const bool pc = rp < kPtrCache;
+        uint16_t* oidx = (pc ? sm.p_idx[rp] : a.p.idx[rp]) + (uint64_t)gp * (uint64_t)k;
+        uint32_t* ocodes = reinterpret_cast<uint32_t*>((pc ? sm.p_codes[rp] : a.p.codes[rp]) + (uint64_t)gp * (uint64_t)a.stride);
+        for (int i = lane; i < (k >> 1); i += 32)
+          reinterpret_cast<uint32_t*>(oidx)[i] = reinterpret_cast<const uint32_t*>(sm.msg_idx[sp])[i];
+        for (int i = lane; i < cwords; i += 32) ocodes[i] = sm.msg_codes[sp][i];
+        if (lane == 0) (pc ? sm.p_scales[rp] : a.p.scales[rp])[gp] = sm.msg_scale[sp];
+      }
     }
   } else {
     // ======================= selectors =======================================
     const int q = warp - kWarps;
+    ItemCursor<T> cur;                            // item w = q, q+2, q+4, ...
+    cur.start(a.tb, blockIdx.x, G);
+    cur.advance(a.tb, q, R, G);
+    ItemCursor<T> pf = cur;                       // the item whose e is loaded next by this selector: w, w+2 at start, then w+4
     if (lane == 0) {
-      for (int r = q; r < kEeStages && r < R; r += kSel) {
-        mbar_expect_tx(&sm.full_ee[r], kBytes);
-        tma_load_1d(sm.ee[r], a.p.err[r] + c.base, kBytes, &sm.full_ee[r]);
+      for (int i = q; i < kEeStages && pf.valid; i += kSel) {
+        mbar_expect_tx(&sm.full_ee[i], kBytes);
+        tma_load_1d(sm.ee[i], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes, &sm.full_ee[i]);
+        pf.advance(a.tb, kSel, R, G);
       }
+    } else {
+      for (int i = q; i < kEeStages && pf.valid; i += kSel) pf.advance(a.tb, kSel, R, G);
     }
     __syncwarp();
-    const int cwords = (k * bits) >> 5;
     uint32_t* bitmap = sm.bitmap[q];
-    uint32_t* cw = sm.cw[q];
+    uint16_t* kept_pos = sm.kept_pos[q];
+    uint8_t* prefix = sm.prefix[q];
+    int pending_stage = -1;                       // stage whose bulk store is in flight
 #pragma unroll 1
-    for (int r = q; r < R; r += kSel) {
-      const int se = r % kEeStages;
+    for (uint32_t w = q; cur.valid; w += kSel) {
+      const int se = w % kEeStages;
       float* ep = sm.ee[se];
       named_sync(2 + q, kPairThreads);            // candidate list q is ready
+      // The store of this selector's previous item was issued a whole hand-off ago; once it has
+      // read its stage, e of the item four ahead is loaded into it.
+      if (pending_stage >= 0) {
+        if (lane == 0) {
+          tma_store_wait_read_all();
+          if (pf.valid) {
+            mbar_expect_tx(&sm.full_ee[pending_stage], kBytes);
+            tma_load_1d(sm.ee[pending_stage], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes,
+                        &sm.full_ee[pending_stage]);
+          }
+        }
+        pf.advance(a.tb, kSel, R, G);
+        __syncwarp();
+      }
       const uint32_t C = sm.count[q];
-      uint32_t T1 = 0xFFFFFFFFu, smax = 0;
-#pragma unroll
-      for (int w = 0; w < kWarps; ++w) { T1 = min(T1, sm.wmin[se][w]); smax = max(smax, sm.wmax[se][w]); }
+      uint32_t T1, smax;
+      {
+        const uint4 m0 = reinterpret_cast<const uint4*>(sm.wmin[se])[0], m1 = reinterpret_cast<const uint4*>(sm.wmin[se])[1];
+        const uint4 x0 = reinterpret_cast<const uint4*>(sm.wmax[se])[0], x1 = reinterpret_cast<const uint4*>(sm.wmax[se])[1];
+        T1 = min(min(min(m0.x, m0.y), min(m0.z, m0.w)), min(min(m1.x, m1.y), min(m1.z, m1.w)));
+        smax = max(max(max(x0.x, x0.y), max(x0.z, x0.w)), max(max(x1.x, x1.y), max(x1.z, x1.w)));
+      }
       const float sc = __uint_as_float(smax);
-      uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
-      uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
-#ifdef SL_STATS
-      if (lane == 0) { atomicAdd(&a.flags[4], C); atomicAdd(&a.flags[7], 1u); if (C > kCandMax) atomicAdd(&a.flags[8], 1u); }
-#endif
+      uint16_t* midx = sm.msg_idx[se];
+      uint32_t* mcodes = sm.msg_codes[se];
       // ---- C ----
-      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist[q], bitmap, lane);
+      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist[q], bitmap, kept_pos, lane);
       else if (C <= 32u * kCandReg)
-        select_candidates<kCandReg>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, bitmap, lane, a.flags + 4);
+        select_candidates<kCandReg>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
       else
-        select_candidates<0>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, bitmap, lane, a.flags + 4);
+        select_candidates<0>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
       __syncwarp();
       if (lane == 0) sm.count[q] = 0;
-      __threadfence_block();
-      __syncwarp();
-      if (r + kSel < R) named_arrive(4 + q, kPairThreads);   // candidate list q may be refilled
       // ---- D ----
-      uint4 bm = reinterpret_cast<uint4*>(bitmap)[lane];
-      const uint32_t mine = __popc(bm.x) + __popc(bm.y) + __popc(bm.z) + __popc(bm.w);
-      uint32_t incl = mine;
+      {
+        const uint4 bm = reinterpret_cast<const uint4*>(bitmap)[lane];
+        const uint32_t c0 = __popc(bm.x), c1 = __popc(bm.y), c2 = __popc(bm.z), c3 = __popc(bm.w);
+        const uint32_t mine = c0 + c1 + c2 + c3;
+        uint32_t incl = mine;
 #pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t o = __shfl_up_sync(kFull, incl, d);
-        if (lane >= d) incl += o;
-      }
-      uint32_t slot = incl - mine;
-      const uint32_t words[4] = {bm.x, bm.y, bm.z, bm.w};
-#pragma unroll
-      for (int w = 0; w < 4; ++w) {
-        uint32_t m = words[w];
-        while (m) {
-          const int b = __ffs(m) - 1;
-          m &= m - 1;
-          const int pos = lane * 128 + w * 32 + b;
-          const float v = ep[pos];
-          oidx[slot] = (uint16_t)pos;
-          float sent;
-          if (bits == 32) {
-            reinterpret_cast<float*>(ocodes)[slot] = v;
-            sent = v;
-          } else {
-            const uint32_t code = quant_code(v, sc, bits);
-            atomicOr(&cw[(slot * (uint32_t)bits) >> 5], code << ((slot * (uint32_t)bits) & 31u));
-            sent = dequant(code, sc, bits);
-          }
-          ep[pos] = __fsub_rn(v, sent);           // line 4: the residual
-          ++slot;
+        for (int d = 1; d < 32; d <<= 1) {
+          const uint32_t o = __shfl_up_sync(kFull, incl, d);
+          if (lane >= d) incl += o;
         }
+        const uint32_t ex = incl - mine;           // kept positions before this lane's 128 positions (<= 128)
+        reinterpret_cast<uint32_t*>(prefix)[lane] = ex | ((ex + c0) << 8) | ((ex + c0 + c1) << 16) | ((ex + c0 + c1 + c2) << 24);
       }
-      reinterpret_cast<uint4*>(bitmap)[lane] = make_uint4(0, 0, 0, 0);
-      fence_async_smem();
       __syncwarp();
-      // ---- E ----
-      if (lane == 0) tma_store_1d(a.p.err[r] + c.base, ep, kBytes);
-      if (bits != 32 && lane < cwords) {
-        reinterpret_cast<uint32_t*>(ocodes)[lane] = cw[lane];
-        cw[lane] = 0;
+      for (int t = lane; t < k; t += 32) {
+        const uint32_t pos = kept_pos[t];
+        const uint32_t wd = pos >> 5;
+        const uint32_t slot = (uint32_t)prefix[wd] + __popc(bitmap[wd] & ((1u << (pos & 31u)) - 1u));
+        const float v = ep[pos];
+        midx[slot] = (uint16_t)pos;
+        float sent;
+        if (bits == 32) {
+          mcodes[slot] = __float_as_uint(v);
+          sent = v;
+        } else {
+          const uint32_t code = quant_code(v, sc, bits);
+          atomicOr(&mcodes[(slot * (uint32_t)bits) >> 5], code << ((slot * (uint32_t)bits) & 31u));
+          sent = dequant(code, sc, bits);
+        }
+        ep[pos] = __fsub_rn(v, sent);             // line 4: the residual
       }
       if (lane == 0) {
-        a.p.scales[r][g] = sc;
+        sm.msg_scale[se] = sc;
         if (smax >= 0x7F800000u && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_NONFINITE);
-        tma_store_wait_read();                    // the stage has been read: it may be refilled
-        if (r + kEeStages < R) {
-          mbar_expect_tx(&sm.full_ee[se], kBytes);
-          tma_load_1d(sm.ee[se], a.p.err[r + kEeStages] + c.base, kBytes, &sm.full_ee[se]);
-        }
       }
+      fence_async_smem();                         // the patched stage is read by a bulk store
       __syncwarp();
+      reinterpret_cast<uint4*>(bitmap)[lane] = make_uint4(0, 0, 0, 0);
+      // ---- E: the stage drains to the error buffer ----
+      if (lane == 0)
+        tma_store_1d((cur.r < kPtrCache ? sm.p_err[cur.r] : a.p.err[cur.r]) + cur.base, ep, kBytes);
+      pending_stage = se;
+      __syncwarp();
+      named_arrive(4 + q, kPairThreads);          // item w is finished: message final, candidate list free
+      cur.advance(a.tb, kSel, R, G);
     }
+    if (lane == 0) tma_store_wait_read_all();      // shared memory must outlive the bulk stores' reads
   }
   if (timed_out && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 }  // namespace
+
+template <int T>
+bool compress_is_tuned(const CompressArgs<T>& a, bool aligned16) {
+  return aligned16 && a.chunk == kC && a.k <= 128 && ((a.k * a.bits) % 32) == 0;
+}
 
 template <int T>
 cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream_t st) {
@@ -664,12 +863,16 @@ cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream
     e = cudaFuncSetAttribute(compress_generic_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gsmem);
     if (e != cudaSuccess) return e;
   }
-  const bool fast = aligned16 && a.chunk == kC && a.k <= 128 && ((a.k * a.bits) % 32) == 0;
-  if (fast) {
+  if (compress_is_tuned(a, aligned16)) {
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     e = cudaFuncSetAttribute(compress_c4096_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)sizeof(FastSmem));
     if (e != cudaSuccess) return e;
-    compress_c4096_kernel<T><<<a.tb.n_chunks, kFastThreads, sizeof(FastSmem), st>>>(a);
+    // persistent grid: two CTAs per SM, each walking its share of the chunks
+    const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * 2u);
+    compress_c4096_kernel<T><<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
     bool tails = false;
     for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
       tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)kC) != 0;
@@ -683,6 +886,8 @@ cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream
   return cudaPeekAtLastError();
 }
 
+template bool compress_is_tuned<256>(const CompressArgs<256>&, bool);
+template bool compress_is_tuned<SL_MAX_TENSORS>(const CompressArgs<SL_MAX_TENSORS>&, bool);
 template cudaError_t launch_compress<256>(const CompressArgs<256>&, bool, cudaStream_t);
 template cudaError_t launch_compress<SL_MAX_TENSORS>(const CompressArgs<SL_MAX_TENSORS>&, bool, cudaStream_t);
 

@@ -95,6 +95,10 @@ class GpuStep:
         api.sl_aggregate_apply(self.idx, self.codes, self.scales, self.layout, self.chunk, self.k,
                                self.bits, self.theta_global, outer_lr, self.flags)
 
+    def outer_step(self, beta, outer_lr):
+        api.sl_outer_step(self.theta_local, self.theta_global, self.err, self.layout, beta, self.chunk,
+                          self.k, self.bits, outer_lr, self.idx, self.codes, self.scales, self.flags)
+
     def messages_host(self):
         torch.cuda.synchronize()
         out = []
@@ -113,10 +117,11 @@ def compare_messages(gpu_msgs, ora_msgs, what=""):
 
 
 def run_and_compare(offsets, tg, tls, errs, beta, chunk, k, bits, outer_lr, rounds=1, next_locals=None,
-                    batched=True, what=""):
+                    batched=True, what="", fused=False):
     """Runs `rounds` outer steps on the GPU and on the checker from the same inputs and compares
     everything after every round.  `next_locals(round, theta_global_numpy)` supplies the replicas'
-    parameters for the rounds after the first."""
+    parameters for the rounds after the first.  fused=True drives the GPU through the single
+    sl_outer_step call instead of sl_compress_batch + sl_aggregate_apply."""
     R = len(tls)
     gs = GpuStep(offsets, R, chunk, k, bits)
     tg_o = tg.copy()
@@ -127,7 +132,10 @@ def run_and_compare(offsets, tg, tls, errs, beta, chunk, k, bits, outer_lr, roun
         if t > 0:
             tls = next_locals(t, tg_o)
             gs.upload(None, tls)   # theta_global stays what each side computed itself
-        gs.compress(beta, batched=batched)
+        if fused:
+            gs.outer_step(beta, outer_lr)
+        else:
+            gs.compress(beta, batched=batched)
         res = oracle_compress_all(tls, tg_o, errs_o, offsets, beta, chunk, k, bits)
         ora_msgs = [(i, c, s) for i, c, s, _ in res]
         for _, _, _, f in res:
@@ -138,7 +146,8 @@ def run_and_compare(offsets, tg, tls, errs, beta, chunk, k, bits, outer_lr, roun
             assert_close(gs.err[r].cpu().numpy(), errs_o[r], f"{what} round {t} err[r={r}]")
         upd = slo.aggregate(ora_msgs, offsets, chunk, k, bits)
         slo.outer_apply(tg_o, upd, outer_lr)
-        gs.aggregate_apply(outer_lr)
+        if not fused:
+            gs.aggregate_apply(outer_lr)
         assert_close(gs.theta_global.cpu().numpy(), tg_o, f"{what} round {t} theta_global")
     assert int(gs.flags.item()) == flags_o, (what, int(gs.flags.item()), flags_o)
     return gs, tg_o, errs_o

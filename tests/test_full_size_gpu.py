@@ -41,7 +41,8 @@ def _check_properties(st, wl):
         assert bool((st.scales[r] >= 0).all()) and bool(torch.isfinite(st.scales[r]).all())
 
 
-def test_1b_workload_sampled_chunks_two_rounds():
+@pytest.mark.parametrize("fused", [False, True], ids=["two_calls", "outer_step"])
+def test_1b_workload_sampled_chunks_two_rounds(fused):
     free, _ = torch.cuda.mem_get_info()
     wl = synth.workload("1b")
     need = (2 * wl.R + 1) * wl.n_total * 4 + (2 << 30)
@@ -57,8 +58,11 @@ def test_1b_workload_sampled_chunks_two_rounds():
         tg_in = _gather(st.theta_global, picks)
         tl_in = [_gather(st.theta_local[r], picks) for r in range(wl.R)]
         e_in = [_gather(st.err[r], picks) for r in range(wl.R)]
-        st.compress()
-        st.aggregate_apply()
+        if fused:
+            st.outer_step()
+        else:
+            st.compress()
+            st.aggregate_apply()
         torch.cuda.synchronize()
         assert int(st.flags.item()) == 0
         _check_properties(st, wl)

@@ -288,3 +288,54 @@ def test_density_sweep_cells_on_sub_arena(k, R):
     errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
     run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
                     what=f"sweep k{k} R{R}")
+
+
+# ---------------------------------------------------------------- the one-call step (sl_outer_step)
+def test_outer_step_tiny_three_rounds():
+    wl = synth.workload("tiny")
+    tgt = synth.gen_theta_global(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r).numpy() for r in range(wl.R)]
+    errs = [synth.gen_error(wl, r).numpy() for r in range(wl.R)]
+    nxt = lambda t, tg: [synth.gen_theta_local(wl, torch.from_numpy(tg), t, r).numpy() for r in range(wl.R)]
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    rounds=3, next_locals=nxt, what="outer_step tiny", fused=True)
+
+
+@pytest.mark.parametrize("k,bits,R", [(64, 2, 8), (16, 2, 3), (128, 2, 5), (64, 8, 2), (32, 32, 1), (64, 4, 16)])
+def test_outer_step_aligned_arena(k, bits, R):
+    sizes = [5 * 4096, 1024, 4096 + 2048, 512, 4, 3 * 4096 + 4092, 4096]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), R, seed=k + bits + R)
+    run_and_compare(off, tg, tls, errs, 0.95, 4096, k, bits, 0.8, what=f"outer_step k{k} b{bits} R{R}", fused=True)
+
+
+@pytest.mark.parametrize("chunk,k,bits", [(4096, 60, 2), (256, 8, 2), (100, 7, 8), (8192, 100, 4)])
+def test_outer_step_falls_back_on_other_shapes(chunk, k, bits):
+    sizes = [3 * chunk + 5, 1, chunk, 7, 2 * chunk + chunk // 2 + 3]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), 3, seed=chunk + k)
+    run_and_compare(off, tg, tls, errs, 0.95, chunk, k, bits, 1.0, what=f"outer_step generic C{chunk}", fused=True)
+
+
+def test_outer_step_adversarial_chunks():
+    chunk, k, bits = 4096, 64, 2
+    cases = _adversarial_chunks(chunk, k)
+    n = chunk * len(cases)
+    ep = np.concatenate(list(cases.values()))
+    tg = np.zeros(n, f32)
+    tls = [(-ep).astype(f32), np.roll(-ep, chunk).astype(f32), np.roll(-ep, 3 * chunk).astype(f32)]
+    errs = [np.zeros(n, f32) for _ in range(3)]
+    run_and_compare([0, n], tg, tls, errs, 0.0, chunk, k, bits, 1.0, what="outer_step adversarial", fused=True)
+
+
+def test_outer_step_180m_sub_arena_three_rounds():
+    full = synth.workload("180m")
+    wl = synth.sub_arena(full, list(range(9)) + [len(full.tensors) - 1])
+    tgt = synth.gen_theta_global(wl)
+    rho = synth.row_scales(wl)
+    tls = [synth.gen_theta_local(wl, tgt, 0, r, rho=rho).numpy() for r in range(wl.R)]
+    errs = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    nxt = lambda t, tg: [synth.gen_theta_local(wl, torch.from_numpy(tg), t, r, rho=rho).numpy()
+                         for r in range(wl.R)]
+    run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
+                    rounds=3, next_locals=nxt, what="outer_step 180m sub-arena", fused=True)
