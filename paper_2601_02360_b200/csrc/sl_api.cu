@@ -73,11 +73,8 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
            aligned(codes[r], 16) && aligned(scales[r], 4);
   }
   a->theta_global = theta_global;
-  a->theta_out = theta_global;
   a->flags = flags;
   a->beta = beta;
-  a->outer_lr = outer_lr;
-  a->fused = 0;
   a->chunk = chunk;
   a->k = k;
   a->bits = bits;

@@ -60,11 +60,8 @@ struct CompressArgs {
   Table<T> tb;
   CompressPtrs p;
   const float* theta_global;
-  float* theta_out;   // fused step only: theta_global again, written with the outer update
   uint32_t* flags;
   float beta;
-  float outer_lr;     // fused step only
-  int fused;          // 1: the tuned kernel finishes every chunk with the average and the outer update
   int chunk, k, bits, R;
   uint32_t stride;  // bytes of codes per chunk
 };
@@ -117,90 +114,6 @@ __device__ __forceinline__ float dequant(uint32_t code, float s, int bits) {
 
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
-
-// ---------------------------------------------------------------------------
-// Eq. 2 line 5 for one full 4096-element chunk, run by 256 threads (tid 0..255) that
-// synchronise on named barrier `bar`.  `acc` is a 16 KB shared accumulator, G the thread's
-// four float4s of theta_global (APPLY only), P any struct with idx[], codes[], scales[].
-//  * the (replica, slot) pairs of the chunk are spread over the threads, up to kAggPairs per
-//    thread and round; every pair's position and value are fetched before any is applied, so
-//    the R messages cost one memory round trip instead of R (loads are ld.global.cg: the fused
-//    step reads messages its own CTA has just written);
-//  * the pairs are applied replica by replica (a barrier between replicas keeps the additions
-//    in replica order; inside one message positions are distinct: no conflicts, no atomics);
-//  * division by R is a multiplication by the exact reciprocal when R is a power of two (bit
-//    identical), an IEEE division otherwise.
-// Returns true if a slot named a position outside the chunk (skipped).
-// ---------------------------------------------------------------------------
-constexpr int kAggPairs = 4;
-
-template <bool APPLY, typename P>
-__device__ __forceinline__ bool aggregate_chunk_c4096(float* acc, const float4 (&G)[4], const P& m, uint32_t g,
-                                                      int k, int bits, int R, uint32_t stride,
-                                                      float4* out4, float outer_lr, int tid, int bar) {
-#pragma unroll
-  for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(acc)[tid + 256 * j] = make_float4(0.f, 0.f, 0.f, 0.f);
-  bool bad = false;
-  const int total = R * k;
-  const int kshift = (k & (k - 1)) == 0 ? 31 - __clz(k) : -1;
-  for (int q0 = 0; q0 < total; q0 += 256 * kAggPairs) {
-    uint32_t pos[kAggPairs];
-    float val[kAggPairs];
-    int rep[kAggPairs];
-#pragma unroll
-    for (int i = 0; i < kAggPairs; ++i) {
-      const int q = q0 + tid + 256 * i;            // pair q = (replica q / k, slot q % k)
-      pos[i] = 0xFFFFu;
-      val[i] = 0.0f;
-      rep[i] = -1;
-      if (q < total) {
-        const int r = kshift >= 0 ? (q >> kshift) : q / k;
-        const int j = q - r * k;
-        rep[i] = r;
-        const uint32_t p = __ldcg(m.idx[r] + (uint64_t)g * (uint64_t)k + j);
-        const uint8_t* codes = m.codes[r] + (uint64_t)g * (uint64_t)stride;
-        if (bits == 32) {
-          val[i] = __ldcg(reinterpret_cast<const float*>(codes) + j);
-        } else {
-          const float s = __ldcg(m.scales[r] + g);
-          const uint32_t bit = (uint32_t)j * (uint32_t)bits;
-          const uint32_t code = ((uint32_t)__ldcg(codes + (bit >> 3)) >> (bit & 7u)) & ((1u << bits) - 1u);
-          val[i] = dequant(code, s, bits);
-        }
-        if (p != 0xFFFFu && p >= 4096u) bad = true; else pos[i] = p;
-      }
-    }
-    const int r_lo = kshift >= 0 ? (q0 >> kshift) : q0 / k;
-    const int r_hi = min(R - 1, (q0 + 256 * kAggPairs - 1) / k);
-    named_sync(bar, 256);                          // accumulator zeroed / previous round applied
-    for (int r = r_lo; r <= r_hi; ++r) {
-#pragma unroll
-      for (int i = 0; i < kAggPairs; ++i)
-        if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
-      named_sync(bar, 256);
-    }
-  }
-  if (total == 0) named_sync(bar, 256);
-  const bool pow2 = (R & (R - 1)) == 0;
-  const float Rf = (float)R, invR = 1.0f / Rf;
-  const float nlr = -outer_lr;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float4 s4 = reinterpret_cast<const float4*>(acc)[tid + 256 * j];
-    float4 u;
-    if (pow2) {
-      u.x = __fmul_rn(s4.x, invR); u.y = __fmul_rn(s4.y, invR); u.z = __fmul_rn(s4.z, invR); u.w = __fmul_rn(s4.w, invR);
-    } else {
-      u.x = __fdiv_rn(s4.x, Rf); u.y = __fdiv_rn(s4.y, Rf); u.z = __fdiv_rn(s4.z, Rf); u.w = __fdiv_rn(s4.w, Rf);
-    }
-    if (APPLY) {
-      u.x = __fmaf_rn(nlr, u.x, G[j].x); u.y = __fmaf_rn(nlr, u.y, G[j].y);
-      u.z = __fmaf_rn(nlr, u.z, G[j].z); u.w = __fmaf_rn(nlr, u.w, G[j].w);
-    }
-    __stcs(out4 + tid + 256 * j, u);
-  }
-  return bad;
-}
 
 // ---------------------------------------------------------------------------
 // launchers implemented in the kernel files (host side, return cudaError_t)
