@@ -64,28 +64,59 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
 }
 
 // Tuned kernel for full 4096-element chunks of a 16-byte aligned arena.  Persistent grid: CTA b
-// walks chunks b, b+G, b+2G, ...  Per chunk:
-//  * theta_global's 16 KB are requested first (four 128-bit loads per thread) so that they fly
-//    while the messages are handled;
+// walks the full chunks among b, b+G, b+2G, ...  Software pipelined over chunks: while chunk i is
+// accumulated and written, the next chunk's theta_global is already on its way into shared memory
+// (one 16 KB TMA bulk copy, no multicast, double buffered, mbarrier completion) and its message
+// entries are on their way into registers.  Per chunk:
 //  * the (replica, slot) pairs of the chunk are spread over the threads, NP per thread: pair
 //    q = tid + 256 i is slot q % k of replica q / k.  What does not depend on the chunk (replica,
-//    slot, the three pointers, the bit offset of the code) is computed once per thread, outside
-//    the chunk loop.  Every pair's position and value are fetched before any is applied, so the R
-//    messages cost one memory round trip instead of R;
+//    slot, the three pointers, the bit offset of the code) is computed once per thread;
 //  * the pairs are applied to a 16 KB shared accumulator in replica order: one round per replica,
 //    a barrier between rounds (inside one message positions are distinct: no conflicts, no
 //    atomics; across messages the barrier fixes the order of the additions);
 //  * division by R is a multiplication by the exact reciprocal when R is a power of two (bit
-//    identical), an IEEE division otherwise; the outer update is one fused multiply-add.
+//    identical), an IEEE division otherwise; the outer update is one fused multiply-add; the
+//    result leaves with 128-bit streaming stores.
 constexpr int kAC = 4096;
+constexpr uint32_t kAggWaitLimit = 1u << 22;
+
+struct AggSmem {
+  float acc[kAC];
+  float gbuf[2][kAC];                // theta_global of the current / next chunk (APPLY only)
+  uint64_t full[2];
+};
+
+__device__ __forceinline__ uint32_t agg_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// first full chunk at or after g (stepping by `step`); t_lo caches the tensor of the last hit
+template <int T>
+__device__ __forceinline__ bool next_full_chunk(const Table<T>& tb, uint32_t& g, uint32_t step, uint32_t& t_lo,
+                                                uint64_t& base) {
+  for (; g < tb.n_chunks; g += step) {
+    if (!(tb.first_chunk[t_lo] <= g && g < tb.first_chunk[t_lo + 1])) {
+      uint32_t lo = 0, hi = tb.n_tensors;
+      while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
+      }
+      t_lo = lo;
+    }
+    base = tb.offset[t_lo] + (uint64_t)(g - tb.first_chunk[t_lo]) * (uint64_t)kAC;
+    if (tb.offset[t_lo + 1] - base >= (uint64_t)kAC) return true;   // short chunks go to the generic tail launch
+  }
+  return false;
+}
 
 template <int T, bool APPLY, int NP>
 __global__ void __launch_bounds__(kThreads)
 aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
-  __shared__ __align__(16) float acc[kAC];
+  extern __shared__ __align__(16) unsigned char agg_smem_raw[];
+  AggSmem& sm = *reinterpret_cast<AggSmem*>(agg_smem_raw);
+  float* acc = sm.acc;
   const int tid = threadIdx.x;
   const int k = a.k, bits = a.bits, R = a.R;
   const int total = R * k;
+  constexpr uint32_t kBytes = kAC * 4;
 
   // per-thread, chunk-independent description of its pairs
   const uint16_t* p_idx[NP];
@@ -112,26 +143,50 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const bool pow2 = (R & (R - 1)) == 0;
   const float Rf = (float)R, invR = 1.0f / Rf;
   const float nlr = -a.outer_lr;
-  bool bad = false;
-  uint32_t t_lo = 0;                               // tensor of the previous chunk: the next one is usually the same
+  bool bad = false, timed_out = false;
 
-  for (uint32_t g = blockIdx.x; g < a.tb.n_chunks; g += gridDim.x) {
-    // chunk -> (base, full?) with the previous tensor as the first guess
-    if (!(a.tb.first_chunk[t_lo] <= g && g < a.tb.first_chunk[t_lo + 1])) {
-      uint32_t lo = 0, hi = a.tb.n_tensors;
-      while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (a.tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
-      }
-      t_lo = lo;
-    }
-    const uint64_t base = a.tb.offset[t_lo] + (uint64_t)(g - a.tb.first_chunk[t_lo]) * (uint64_t)kAC;
-    if (a.tb.offset[t_lo + 1] - base < (uint64_t)kAC) continue;   // short chunks go to the generic tail launch
+  if (APPLY && tid == 0) {
+    for (int s = 0; s < 2; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(agg_smem_u32(&sm.full[s])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
 
-    float4* out4 = reinterpret_cast<float4*>(a.out + base);
-    float4 G[4];
+  // raw message entries of a chunk: position, code bits (or the float itself), scale
+  uint32_t rp[NP], rc[NP];
+  float rs[NP];
+  auto fetch = [&](uint32_t g) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) G[j] = APPLY ? __ldcs(out4 + tid + 256 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < NP; ++i) {
+      rp[i] = 0xFFFFu; rc[i] = 0; rs[i] = 0.0f;
+      if (rep[i] >= 0) {
+        rp[i] = __ldg(p_idx[i] + (uint64_t)g * (uint64_t)k);
+        if (bits == 32) {
+          rc[i] = __float_as_uint(__ldg(reinterpret_cast<const float*>(p_code[i] + (uint64_t)g * (uint64_t)a.stride)));
+        } else {
+          rc[i] = (uint32_t)__ldg(p_code[i] + (uint64_t)g * (uint64_t)a.stride);
+          rs[i] = __ldg(p_scale[i] + g);
+        }
+      }
+    }
+  };
+  auto load_theta = [&](uint64_t base, int buf) {      // thread 0 only
+    const uint32_t bar = agg_smem_u32(&sm.full[buf]);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(agg_smem_u32(sm.gbuf[buf])), "l"(a.out + base), "r"(kBytes), "r"(bar) : "memory");
+  };
+
+  uint32_t g = blockIdx.x, t_lo = 0;
+  uint64_t base = 0;
+  bool valid = next_full_chunk(a.tb, g, gridDim.x, t_lo, base);
+  if (valid) {
+    if (APPLY && tid == 0) load_theta(base, 0);
+    fetch(g);
+  }
+  for (uint32_t it = 0; valid; ++it) {
+    // this chunk's entries become values; then the next chunk's loads are issued
     uint32_t pos[NP];
     float val[NP];
 #pragma unroll
@@ -139,25 +194,41 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       pos[i] = 0xFFFFu;
       val[i] = 0.0f;
       if (rep[i] >= 0) {
-        const uint32_t p = __ldg(p_idx[i] + (uint64_t)g * (uint64_t)k);
-        if (bits == 32) {
-          val[i] = __ldg(reinterpret_cast<const float*>(p_code[i] + (uint64_t)g * (uint64_t)a.stride));
-        } else {
-          const uint32_t code = ((uint32_t)__ldg(p_code[i] + (uint64_t)g * (uint64_t)a.stride) >> cshift[i]) & cmask;
-          val[i] = dequant(code, __ldg(p_scale[i] + g), bits);
-        }
-        if (p != 0xFFFFu && p >= (uint32_t)kAC) bad = true; else pos[i] = p;
+        val[i] = bits == 32 ? __uint_as_float(rc[i]) : dequant((rc[i] >> cshift[i]) & cmask, rs[i], bits);
+        if (rp[i] != 0xFFFFu && rp[i] >= (uint32_t)kAC) bad = true; else pos[i] = rp[i];
       }
     }
+    const uint32_t g_cur = g;
+    const uint64_t base_cur = base;
+    g += gridDim.x;
+    valid = next_full_chunk(a.tb, g, gridDim.x, t_lo, base);
+    if (valid) {
+      if (APPLY && tid == 0) load_theta(base, (it + 1) & 1);   // that buffer was last read before the barrier ending iteration it-1
+      fetch(g);
+    }
+    (void)g_cur;
 #pragma unroll
     for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(acc)[tid + 256 * j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    __syncthreads();                               // accumulator zeroed (and the previous chunk's read of it done)
+    __syncthreads();
     for (int r = 0; r < R; ++r) {
 #pragma unroll
       for (int i = 0; i < NP; ++i)
         if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
       __syncthreads();
     }
+    const float4* g4 = reinterpret_cast<const float4*>(sm.gbuf[it & 1]);
+    if (APPLY) {                                   // bounded wait for this chunk's theta_global
+      const uint32_t bar = agg_smem_u32(&sm.full[it & 1]), parity = (it >> 1) & 1u;
+      bool ok = false;
+      for (uint32_t spin = 0; spin < kAggWaitLimit && !ok; ++spin) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        ok = done != 0;
+      }
+      if (!ok) timed_out = true;
+    }
+    float4* out4 = reinterpret_cast<float4*>(a.out + base_cur);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float4 s4 = reinterpret_cast<const float4*>(acc)[tid + 256 * j];
@@ -168,14 +239,16 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
         u.x = __fdiv_rn(s4.x, Rf); u.y = __fdiv_rn(s4.y, Rf); u.z = __fdiv_rn(s4.z, Rf); u.w = __fdiv_rn(s4.w, Rf);
       }
       if (APPLY) {
-        u.x = __fmaf_rn(nlr, u.x, G[j].x); u.y = __fmaf_rn(nlr, u.y, G[j].y);
-        u.z = __fmaf_rn(nlr, u.z, G[j].z); u.w = __fmaf_rn(nlr, u.w, G[j].w);
+        const float4 G = g4[tid + 256 * j];
+        u.x = __fmaf_rn(nlr, u.x, G.x); u.y = __fmaf_rn(nlr, u.y, G.y);
+        u.z = __fmaf_rn(nlr, u.z, G.z); u.w = __fmaf_rn(nlr, u.w, G.w);
       }
       __stcs(out4 + tid + 256 * j, u);
     }
-    __syncthreads();                               // everyone has read the accumulator before it is zeroed again
+    __syncthreads();                               // accumulator and theta buffer read by everyone before they are reused
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+  if (timed_out && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 template <int T, bool APPLY>
@@ -185,15 +258,18 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   const int pairs = (a.R * a.k + kThreads - 1) / kThreads;
+  const size_t smem = APPLY ? sizeof(AggSmem) : sizeof(float) * kAC;
   // persistent grid: exactly as many CTAs as are resident at once, so that every CTA walks the
   // same number of chunks
   auto launch = [&](auto kernel) -> cudaError_t {
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
     int per_sm = 0;
-    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0);
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * (uint64_t)per_sm);
-    kernel<<<grid, kThreads, 0, st>>>(a);
+    kernel<<<grid, kThreads, smem, st>>>(a);
     return cudaPeekAtLastError();
   };
   if (pairs <= 1) return launch(aggregate_c4096_kernel<T, APPLY, 1>);
