@@ -224,7 +224,7 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 //    Nobody waits for a store it has just issued: under a saturated memory system a 16 KB store
 //    takes microseconds to drain, and a warp with ordinary global stores in flight also stalls
 //    on its next shared-memory access.  So the selectors issue no global stores at all.
-//  * Producers, per replica (thread t owns float4s t, t+256, t+512, t+768 of the chunk):
+//  * Producers, per replica (a thread owns four float4s of the chunk, 256 float4s apart):
 //      A  e' = fma(beta, e, theta_global - theta_local), written in place of e in the stage;
 //         per-thread maximum key.  Every warp sorts its 32 thread maxima (bitonic network of
 //         shuffles) and takes the j-th largest, j = ceil(k/8): at least j keys of the warp's 512
@@ -593,13 +593,19 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       }
     }
     const int cwords = bits == 32 ? k : (k * bits) >> 5;   // 32-bit words of codes per chunk
+    // This thread's float4s are number t4 + 256 j (j = 0..3) of the chunk, with
+    // t4 = 64 (lane / 8) + 8 warp + lane % 8: every 8 lanes read 128 contiguous bytes (no bank
+    // conflicts), and every warp samples each of the sixteen 256-element regions of the chunk
+    // with 32 elements, so a row boundary inside the chunk (rows of very different scale) cannot
+    // leave a warp with small values only, which would ruin the lower bound below.
+    const int t4 = ((lane >> 3) << 6) + (warp << 3) + (lane & 7);
     const int jsel = 32 - (k + kWarps - 1) / kWarps;   // lane holding the ceil(k/8)-th largest after an ascending sort
     const float beta = a.beta;
     float4 G4[4];                                 // this thread's 16 elements of theta_global
     if (cur.valid) {
       const float4* tg4 = reinterpret_cast<const float4*>(a.theta_global + cur.base);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + tid + 256 * j);
+      for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + t4 + 256 * j);
     }
     uint32_t g_m1 = 0, g_m2 = 0;                  // chunk and replica of items w-1 and w-2
     int r_m1 = 0, r_m2 = 0;
@@ -618,14 +624,14 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       uint32_t tmax = 0;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float4 L = tl4[tid + 256 * j];
-        const float4 E = ee4[tid + 256 * j];
+        const float4 L = tl4[t4 + 256 * j];
+        const float4 E = ee4[t4 + 256 * j];
         float4 v;
         v.x = __fmaf_rn(beta, E.x, __fsub_rn(G4[j].x, L.x));
         v.y = __fmaf_rn(beta, E.y, __fsub_rn(G4[j].y, L.y));
         v.z = __fmaf_rn(beta, E.z, __fsub_rn(G4[j].z, L.z));
         v.w = __fmaf_rn(beta, E.w, __fsub_rn(G4[j].w, L.w));
-        ee4[tid + 256 * j] = v;
+        ee4[t4 + 256 * j] = v;
         key[4 * j + 0] = key_of(v.x);
         key[4 * j + 1] = key_of(v.y);
         key[4 * j + 2] = key_of(v.z);
@@ -640,7 +646,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       if (nxt.valid && nxt.r == 0) {
         const float4* tg4 = reinterpret_cast<const float4*>(a.theta_global + nxt.base);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + tid + 256 * j);
+        for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + t4 + 256 * j);
       }
       uint32_t v = tmax;                           // bitonic sort of the 32 thread maxima, ascending over lanes
 #pragma unroll
@@ -701,7 +707,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
           if (mask & (1u << e)) {
             if (at < (uint32_t)kCandMax) {
               ckey[at] = key[e];
-              cpos[at] = (uint16_t)(((e >> 2) << 10) + (tid << 2) + (e & 3));
+              cpos[at] = (uint16_t)(((e >> 2) << 10) + (t4 << 2) + (e & 3));
             }
             atomicAdd(&hist[(key[e] - T1) >> sh], 1u);
             ++at;
