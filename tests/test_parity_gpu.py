@@ -339,3 +339,43 @@ def test_outer_step_180m_sub_arena_three_rounds():
                          for r in range(wl.R)]
     run_and_compare(wl.offsets(), tgt.numpy(), tls, errs, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr,
                     rounds=3, next_locals=nxt, what="outer_step 180m sub-arena", fused=True)
+
+
+# ---------------------------------------------------------------- less travelled code paths
+@pytest.mark.parametrize("R,k", [(20, 64), (64, 16), (17, 128), (1, 64), (2, 128)])
+def test_many_replicas_beyond_the_pointer_cache(R, k):
+    # R > 16 reads the replicas' pointers from the kernel parameters instead of shared memory;
+    # R * k > 2048 sends the aggregate to the generic kernel
+    sizes = [6 * 4096, 2048, 3 * 4096 + 1024]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), R, seed=R * 7 + k)
+    run_and_compare(off, tg, tls, errs, 0.95, 4096, k, 2, 1.0, rounds=1, what=f"R{R} k{k}")
+
+
+def test_arena_with_more_than_256_tensors():
+    # 300 tensors select the large by-value table (up to 2048 tensors)
+    rng = np.random.default_rng(4)
+    sizes = [int(x) * 4 for x in rng.integers(1, 3000, size=300)]
+    sizes[10] = 4096 * 3
+    sizes[200] = 4096 * 2 + 512
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), 3, seed=17)
+    run_and_compare(off, tg, tls, errs, 0.95, 4096, 64, 2, 1.0, rounds=2,
+                    next_locals=lambda t, g: [(g + np.random.default_rng(t * 10 + r).normal(0, 1e-3, g.size)).astype(f32)
+                                              for r in range(3)], what="300 tensors")
+
+
+def test_empty_tensors_inside_the_arena():
+    sizes = [4096, 0, 0, 8192 + 100, 0, 512]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), 2, seed=23)
+    run_and_compare(off, tg, tls, errs, 0.95, 4096, 64, 2, 1.0, what="empty tensors")
+
+
+def test_more_chunks_than_resident_ctas():
+    # the persistent grids hold 296 / 592 CTAs: 1500 chunks give every CTA several chunks and a ragged last wave
+    n = 1500 * 4096 + 2048
+    tg, tls, errs = _case(n, 3, seed=31)
+    run_and_compare([0, n], tg, tls, errs, 0.95, 4096, 64, 2, 1.0, rounds=2,
+                    next_locals=lambda t, g: [(g + np.random.default_rng(t * 10 + r).normal(0, 1e-3, g.size)).astype(f32)
+                                              for r in range(3)], what="1500 chunks")
