@@ -353,6 +353,8 @@ def run_ours(args) -> None:
         wl = wl.replace(R=args.R)
     if args.k:
         wl = wl.replace(k=args.k)
+    if args.variant != "plain":
+        wl = wl.replace(variant=args.variant)
     if args.first_tensors:
         wl = synth.sub_arena(wl, list(range(args.first_tensors)), f"{wl.name}[:{args.first_tensors}]")
     st = DeviceState(wl, rank_seed(args.seed, rank), dev)
@@ -410,7 +412,7 @@ def run_ours(args) -> None:
         "data": "synthetic",
         "config": {"workload": wl.name, "params": wl.n_total, "tensors": len(wl.tensors),
                    "chunks": wl.n_chunks(), "R": wl.R, "k": wl.k, "bits": wl.bits, "chunk": wl.chunk,
-                   "beta": wl.beta, "outer_lr": wl.outer_lr,
+                   "beta": wl.beta, "outer_lr": wl.outer_lr, "variant": wl.variant,
                    "l2": "inputs (GBs per launch) far larger than the 126 MB L2; no flush needed",
                    "sharding": "none: every rank runs an independent parameter set" if world > 1 else "single GPU",
                    "step": "sl_compress_batch + sl_aggregate_apply; theta_local re-drawn between steps (untimed)"},
@@ -452,6 +454,8 @@ def main() -> None:
     ap.add_argument("--k", type=int, default=0)
     ap.add_argument("--first-tensors", type=int, default=0,
                     help="keep only the first N tensors of the workload (small cases for profiling)")
+    ap.add_argument("--variant", default="plain", choices=["plain", "ties_literal", "ties_dyadic"],
+                    help="tie-heavy value laws of the density-sweep configuration")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")

@@ -256,7 +256,8 @@ constexpr int kSel = 2;               // selector warps
 constexpr int kTlStages = 2;
 constexpr int kEeStages = 4;
 constexpr int kCandMax = 512;
-constexpr int kCandReg = 6;           // candidates per lane held in registers (C <= 192)
+constexpr int kCandReg = 6;           // candidates per lane held in registers: C <= 192 (k <= 64) ...
+constexpr int kCandRegBig = 11;       // ... or C <= 352 (k = 128); longer lists are walked in shared memory
 
 constexpr int kPtrCache = 16;         // replicas whose pointers are staged in shared memory
 constexpr int kFastThreads = kThreads + 32 * kSel;
@@ -795,6 +796,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist[q], bitmap, kept_pos, lane);
       else if (C <= 32u * kCandReg)
         select_candidates<kCandReg>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
+      else if (C <= 32u * kCandRegBig)
+        select_candidates<kCandRegBig>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
       else
         select_candidates<0>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
       __syncwarp();
