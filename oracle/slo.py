@@ -44,6 +44,12 @@ def lib():
         L.slo_compress.argtypes = [vp, vp, vp, vp, u32, f32, i32, i32, i32, vp, vp, vp, vp]
         L.slo_aggregate.restype = i32
         L.slo_aggregate.argtypes = [i32, vp, vp, vp, vp, u32, i32, i32, i32, vp]
+        L.slo_num_chunks_tiled.restype = u64
+        L.slo_num_chunks_tiled.argtypes = [vp, vp, u32, i32]
+        L.slo_compress_tiled.restype = i32
+        L.slo_compress_tiled.argtypes = [vp, vp, vp, vp, vp, u32, f32, i32, i32, i32, vp, vp, vp, vp]
+        L.slo_aggregate_tiled.restype = i32
+        L.slo_aggregate_tiled.argtypes = [i32, vp, vp, vp, vp, vp, u32, i32, i32, i32, vp]
         L.slo_outer_apply.restype = i32
         L.slo_outer_apply.argtypes = [vp, vp, u64, f32]
         L.slo_quantise.restype = u32
@@ -62,9 +68,21 @@ def _off(offsets) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(offsets, dtype=np.uint64))
 
 
-def num_chunks(offsets, chunk: int) -> int:
+def _cols(cols, n_tensors):
+    """None = consecutive chunks everywhere; else per-tensor column counts (0 = consecutive)."""
+    if cols is None:
+        return None
+    c = np.ascontiguousarray(np.asarray(cols, dtype=np.uint64))
+    assert c.shape == (n_tensors,)
+    return c
+
+
+def num_chunks(offsets, chunk: int, cols=None) -> int:
     off = _off(offsets)
-    return int(lib().slo_num_chunks(_p(off), len(off) - 1, chunk))
+    c = _cols(cols, len(off) - 1)
+    if c is None:
+        return int(lib().slo_num_chunks(_p(off), len(off) - 1, chunk))
+    return int(lib().slo_num_chunks_tiled(_p(off), _p(c), len(off) - 1, chunk))
 
 
 def codes_stride(k: int, bits: int) -> int:
@@ -72,26 +90,30 @@ def codes_stride(k: int, bits: int) -> int:
 
 
 def compress(theta_local: np.ndarray, theta_global: np.ndarray, err: np.ndarray, offsets,
-             beta: float, chunk: int, k: int, bits: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, int]:
-    """Eq. 2 lines 1-4 for one replica.  `err` is updated in place.
-    Returns (idx[n_c, k] u16, codes[n_c, stride] u8, scales[n_c] f32, flags)."""
+             beta: float, chunk: int, k: int, bits: int, cols=None) -> Tuple[np.ndarray, np.ndarray, np.ndarray, int]:
+    """Eq. 2 lines 1-4 for one replica.  `err` is updated in place.  `cols` switches matrices
+    to square-tile chunks.  Returns (idx[n_c, k] u16, codes[n_c, stride] u8, scales[n_c] f32, flags)."""
     off = _off(offsets)
+    c = _cols(cols, len(off) - 1)
     for a in (theta_local, theta_global, err):
         assert a.dtype == np.float32 and a.flags.c_contiguous
-    nc = num_chunks(off, chunk)
+    if chunk < 1:
+        raise ValueError("slo_compress rejected its arguments (chunk)")
+    nc = num_chunks(off, chunk, cols)
     idx = np.empty((nc, k), dtype=np.uint16)
     codes = np.empty((nc, codes_stride(k, bits)), dtype=np.uint8)
     scales = np.empty(nc, dtype=np.float32)
     flags = np.zeros(1, dtype=np.uint32)
-    rc = lib().slo_compress(_p(theta_local), _p(theta_global), _p(err), _p(off), len(off) - 1,
-                            beta, chunk, k, bits, _p(idx), _p(codes), _p(scales), _p(flags))
+    rc = lib().slo_compress_tiled(_p(theta_local), _p(theta_global), _p(err), _p(off),
+                                  _p(c) if c is not None else None, len(off) - 1,
+                                  beta, chunk, k, bits, _p(idx), _p(codes), _p(scales), _p(flags))
     if rc != 0:
         raise ValueError(f"slo_compress rejected its arguments ({rc})")
     return idx, codes, scales, int(flags[0])
 
 
 def aggregate(msgs: Sequence[Tuple[np.ndarray, np.ndarray, np.ndarray]], offsets, chunk: int, k: int,
-              bits: int) -> np.ndarray:
+              bits: int, cols=None) -> np.ndarray:
     """Dense mean update from the messages of the replicas, added in the order
     given; the divisor is always len(msgs)."""
     off = _off(offsets)
@@ -106,7 +128,9 @@ def aggregate(msgs: Sequence[Tuple[np.ndarray, np.ndarray, np.ndarray]], offsets
         return a
     pi, pc, ps = arr(0), arr(1), arr(2)
     update = np.empty(int(off[-1]), dtype=np.float32)
-    rc = lib().slo_aggregate(n, pi, pc, ps, _p(off), len(off) - 1, chunk, k, bits, _p(update))
+    c = _cols(cols, len(off) - 1)
+    rc = lib().slo_aggregate_tiled(n, pi, pc, ps, _p(off), _p(c) if c is not None else None, len(off) - 1,
+                                   chunk, k, bits, _p(update))
     if rc != 0:
         raise ValueError(f"slo_aggregate rejected its arguments ({rc})")
     return update
@@ -128,15 +152,15 @@ def dequantise(code: int, s: float, bits: int) -> float:
 
 
 def outer_round(theta_locals: Sequence[np.ndarray], theta_global: np.ndarray, errs: Sequence[np.ndarray],
-                offsets, beta: float, chunk: int, k: int, bits: int, outer_lr: float):
+                offsets, beta: float, chunk: int, k: int, bits: int, outer_lr: float, cols=None):
     """One whole outer step (all of Eq. 2) for R replicas; theta_global and the
     error buffers are updated in place.  Returns the R messages and the update."""
     msgs = []
     flags = 0
     for tl, e in zip(theta_locals, errs):
-        i, c, s, f = compress(tl, theta_global, e, offsets, beta, chunk, k, bits)
+        i, c, s, f = compress(tl, theta_global, e, offsets, beta, chunk, k, bits, cols)
         msgs.append((i, c, s))
         flags |= f
-    upd = aggregate(msgs, offsets, chunk, k, bits)
+    upd = aggregate(msgs, offsets, chunk, k, bits, cols)
     outer_apply(theta_global, upd, outer_lr)
     return msgs, upd, flags

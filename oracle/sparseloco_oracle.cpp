@@ -10,6 +10,13 @@
 // any fast-math flag; the only fused operations are the explicit std::fmaf
 // calls.  The selection is a full std::sort of every chunk on purpose.
 //
+// Chunk geometry.  By default a chunk is `chunk` consecutive elements of one tensor.  With a
+// `cols` array (tile mode, the paper's literal "64 x 64" chunks, section 3 and Table 8) a tensor
+// with cols[t] > 0 is a row-major matrix of cols[t] columns cut into s x s tiles, s*s = chunk,
+// tiles numbered row-major over the tile grid; position p of a tile is row p / s, column p % s
+// of the tile, and only positions inside the matrix exist (edge tiles are smaller).  Tensors with
+// cols[t] == 0 keep the consecutive chunks.
+//
 // Parity status of each function (what pins it is in tests/test_oracle_*.py):
 //   slo_compress / selection, error feedback, residual : pinned
 //   slo_compress / quantiser Q                         : the paper never defines
@@ -76,6 +83,61 @@ inline uint32_t get_code(const uint8_t* chunk_codes, int slot, int bits) {
   return code;
 }
 
+// One chunk's elements: arena offsets of its existing positions, in ascending position order.
+struct ChunkGeom {
+  std::vector<uint64_t> addr;   // arena element offset of every existing position
+  std::vector<uint32_t> pos;    // the chunk-local position it has
+};
+
+inline int tile_side(int chunk) {
+  int s = 1;
+  while ((int64_t)s * s < chunk) ++s;
+  return (int64_t)s * s == chunk ? s : 0;
+}
+
+// calls f(g, geom) for every chunk of the arena, in chunk order
+template <class F>
+void for_each_chunk(const uint64_t* offset, const uint64_t* cols, uint32_t n_tensors, int chunk, F f) {
+  ChunkGeom cg;
+  uint64_t g = 0;
+  const int s = tile_side(chunk);
+  for (uint32_t t = 0; t < n_tensors; ++t) {
+    const uint64_t n_t = offset[t + 1] - offset[t];
+    const uint64_t c_t = cols ? cols[t] : 0;
+    if (c_t == 0) {
+      for (uint64_t c0 = 0; c0 < n_t; c0 += (uint64_t)chunk, ++g) {
+        const int len = (int)std::min<uint64_t>((uint64_t)chunk, n_t - c0);
+        cg.addr.clear(); cg.pos.clear();
+        for (int i = 0; i < len; ++i) { cg.addr.push_back(offset[t] + c0 + i); cg.pos.push_back((uint32_t)i); }
+        f(g, cg);
+      }
+    } else {
+      const uint64_t rows = n_t / c_t;
+      for (uint64_t r0 = 0; r0 < rows; r0 += (uint64_t)s)
+        for (uint64_t q0 = 0; q0 < c_t; q0 += (uint64_t)s, ++g) {
+          cg.addr.clear(); cg.pos.clear();
+          for (int lr = 0; lr < s && r0 + lr < rows; ++lr)
+            for (int lc = 0; lc < s && q0 + lc < c_t; ++lc) {
+              cg.addr.push_back(offset[t] + (r0 + lr) * c_t + q0 + lc);
+              cg.pos.push_back((uint32_t)(lr * s + lc));
+            }
+          f(g, cg);
+        }
+    }
+  }
+}
+
+inline bool geometry_ok(const uint64_t* offset, const uint64_t* cols, uint32_t n_tensors, int chunk) {
+  if (!cols) return true;
+  bool any = false;
+  for (uint32_t t = 0; t < n_tensors; ++t) {
+    if (cols[t] == 0) continue;
+    any = true;
+    if ((offset[t + 1] - offset[t]) % cols[t] != 0) return false;   // a matrix is rows x cols exactly
+  }
+  return !any || tile_side(chunk) > 0;
+}
+
 }  // namespace
 
 extern "C" {
@@ -92,6 +154,14 @@ uint64_t slo_num_chunks(const uint64_t* offset, uint32_t n_tensors, int chunk) {
   return n;
 }
 
+// the same with the tile geometry (cols may be null)
+uint64_t slo_num_chunks_tiled(const uint64_t* offset, const uint64_t* cols, uint32_t n_tensors, int chunk) {
+  if (chunk < 1 || !geometry_ok(offset, cols, n_tensors, chunk)) return 0;
+  uint64_t n = 0;
+  for_each_chunk(offset, cols, n_tensors, chunk, [&](uint64_t, const ChunkGeom&) { ++n; });
+  return n;
+}
+
 uint64_t slo_codes_stride(int k, int bits) { return codes_stride(k, bits); }
 
 // Eq. 2 lines 1-4 for one replica over a whole arena.
@@ -101,106 +171,116 @@ uint64_t slo_codes_stride(int k, int bits) { return codes_stride(k, bits); }
 //   codes  : [n_c * codes_stride] packed codes (float[k] per chunk when bits == 32)
 //   scales : [n_c]
 //   flags  : optional single word, OR of SLO_FLAG_*
+int slo_compress_tiled(const float* theta_local, const float* theta_global, float* err,
+                       const uint64_t* offset, const uint64_t* cols, uint32_t n_tensors, float beta, int chunk,
+                       int k, int bits, uint16_t* idx, uint8_t* codes, float* scales, uint32_t* flags) {
+  if (!theta_local || !theta_global || !err || !offset || !idx || !codes || !scales) return SLO_ERR_INVALID_ARG;
+  if (chunk < 1 || chunk > 65535 || k < 1 || k > chunk || !bits_ok(bits)) return SLO_ERR_INVALID_ARG;
+  if (!geometry_ok(offset, cols, n_tensors, chunk)) return SLO_ERR_INVALID_ARG;
+  const uint64_t cs = codes_stride(k, bits);
+  std::vector<float> ep((size_t)chunk);
+  std::vector<std::pair<uint32_t, uint32_t>> order((size_t)chunk);  // (magnitude key, index into the chunk's element list)
+  std::vector<uint32_t> kept;
+  for_each_chunk(offset, cols, n_tensors, chunk, [&](uint64_t g, const ChunkGeom& cg) {
+    const int len = (int)cg.addr.size();
+    const int k_eff = std::min(k, len);
+
+    // line 1: pseudo-gradient, global minus local; line 2: error feedback, one fused rounding
+    for (int i = 0; i < len; ++i) {
+      const float delta = theta_global[cg.addr[i]] - theta_local[cg.addr[i]];
+      ep[i] = std::fmaf(beta, err[cg.addr[i]], delta);
+    }
+
+    // line 3, Top-k: total order "larger magnitude first, then lower position"; magnitude compared
+    // through the 31 low bits of the float (so +0 and -0 tie).  The element list is in ascending
+    // position order, so its index orders ties like the position does.
+    for (int i = 0; i < len; ++i) order[i] = {f2u(ep[i]) & 0x7FFFFFFFu, (uint32_t)i};
+    std::sort(order.begin(), order.begin() + len,
+              [](const std::pair<uint32_t, uint32_t>& a, const std::pair<uint32_t, uint32_t>& b) {
+                if (a.first != b.first) return a.first > b.first;
+                return a.second < b.second;
+              });
+    kept.clear();
+    for (int j = 0; j < k_eff; ++j) kept.push_back(order[j].second);
+    std::sort(kept.begin(), kept.end());   // message order: ascending position
+
+    // scale: the largest magnitude of the chunk (always a kept element)
+    const uint32_t smax = order[0].first;
+    const float s = u2f(smax);
+    if (smax >= 0x7F800000u && flags) *flags |= SLO_FLAG_NONFINITE;
+    scales[g] = s;
+
+    // line 3, Q, and line 4, residual; message slots k_eff..k-1 are padding
+    uint16_t* cidx = idx + g * (uint64_t)k;
+    uint8_t* ccodes = codes + g * cs;
+    std::memset(ccodes, 0, cs);
+    for (int j = 0; j < k; ++j) cidx[j] = 0xFFFF;
+    for (int j = 0; j < k_eff; ++j) {
+      const uint32_t i = kept[j];
+      float sent;
+      if (bits == 32) {
+        sent = ep[i];
+        std::memcpy(ccodes + 4 * (size_t)j, &sent, 4);
+      } else {
+        const uint32_t code = quantise(ep[i], s, bits);
+        put_code(ccodes, j, bits, code);
+        sent = dequantise(code, s, bits);
+      }
+      cidx[j] = (uint16_t)cg.pos[i];
+      ep[i] = ep[i] - sent;
+    }
+    for (int i = 0; i < len; ++i) err[cg.addr[i]] = ep[i];
+  });
+  return SLO_OK;
+}
+
 int slo_compress(const float* theta_local, const float* theta_global, float* err,
                  const uint64_t* offset, uint32_t n_tensors, float beta, int chunk, int k, int bits,
                  uint16_t* idx, uint8_t* codes, float* scales, uint32_t* flags) {
-  if (!theta_local || !theta_global || !err || !offset || !idx || !codes || !scales) return SLO_ERR_INVALID_ARG;
-  if (chunk < 1 || chunk > 65535 || k < 1 || k > chunk || !bits_ok(bits)) return SLO_ERR_INVALID_ARG;
-  const uint64_t cs = codes_stride(k, bits);
-  std::vector<float> ep((size_t)chunk);
-  std::vector<std::pair<uint32_t, uint32_t>> order((size_t)chunk);  // (magnitude key, position)
-  std::vector<uint32_t> kept;
-  uint64_t g = 0;  // global chunk number
-  for (uint32_t t = 0; t < n_tensors; ++t) {
-    const uint64_t n_t = offset[t + 1] - offset[t];
-    for (uint64_t c0 = 0; c0 < n_t; c0 += (uint64_t)chunk, ++g) {
-      const uint64_t base = offset[t] + c0;
-      const int len = (int)std::min<uint64_t>((uint64_t)chunk, n_t - c0);
-      const int k_eff = std::min(k, len);
-
-      // line 1: pseudo-gradient, global minus local; line 2: error feedback, one fused rounding
-      for (int i = 0; i < len; ++i) {
-        const float delta = theta_global[base + i] - theta_local[base + i];
-        ep[i] = std::fmaf(beta, err[base + i], delta);
-      }
-
-      // line 3, Top-k: total order "larger magnitude first, then lower position";
-      // magnitude compared through the 31 low bits of the float (so +0 and -0 tie)
-      for (int i = 0; i < len; ++i) order[i] = {f2u(ep[i]) & 0x7FFFFFFFu, (uint32_t)i};
-      std::sort(order.begin(), order.begin() + len,
-                [](const std::pair<uint32_t, uint32_t>& a, const std::pair<uint32_t, uint32_t>& b) {
-                  if (a.first != b.first) return a.first > b.first;
-                  return a.second < b.second;
-                });
-      kept.clear();
-      for (int j = 0; j < k_eff; ++j) kept.push_back(order[j].second);
-      std::sort(kept.begin(), kept.end());   // message order: ascending position
-
-      // scale: the largest magnitude of the chunk (always a kept element)
-      const uint32_t smax = order[0].first;
-      const float s = u2f(smax);
-      if (smax >= 0x7F800000u && flags) *flags |= SLO_FLAG_NONFINITE;
-      scales[g] = s;
-
-      // line 3, Q, and line 4, residual; message slots k_eff..k-1 are padding
-      uint16_t* cidx = idx + g * (uint64_t)k;
-      uint8_t* ccodes = codes + g * cs;
-      std::memset(ccodes, 0, cs);
-      for (int j = 0; j < k; ++j) cidx[j] = 0xFFFF;
-      for (int j = 0; j < k_eff; ++j) {
-        const uint32_t i = kept[j];
-        float sent;
-        if (bits == 32) {
-          sent = ep[i];
-          std::memcpy(ccodes + 4 * (size_t)j, &sent, 4);
-        } else {
-          const uint32_t code = quantise(ep[i], s, bits);
-          put_code(ccodes, j, bits, code);
-          sent = dequantise(code, s, bits);
-        }
-        cidx[j] = (uint16_t)i;
-        ep[i] = ep[i] - sent;
-      }
-      for (int i = 0; i < len; ++i) err[base + i] = ep[i];
-    }
-  }
-  return SLO_OK;
+  return slo_compress_tiled(theta_local, theta_global, err, offset, nullptr, n_tensors, beta, chunk, k, bits,
+                            idx, codes, scales, flags);
 }
 
 // Eq. 2 line 5, first half: dense mean over R replicas' messages, replicas
 // added in the order 0..R-1 starting from +0, divisor always R.
+int slo_aggregate_tiled(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                        const float* const* scales, const uint64_t* offset, const uint64_t* cols,
+                        uint32_t n_tensors, int chunk, int k, int bits, float* update) {
+  if (R < 1 || !idx || !codes || !scales || !offset || !update) return SLO_ERR_INVALID_ARG;
+  if (chunk < 1 || chunk > 65535 || k < 1 || k > chunk || !bits_ok(bits)) return SLO_ERR_INVALID_ARG;
+  if (!geometry_ok(offset, cols, n_tensors, chunk)) return SLO_ERR_INVALID_ARG;
+  const uint64_t cs = codes_stride(k, bits);
+  std::vector<int64_t> where((size_t)chunk);   // position -> index into the chunk's element list, -1 = no such position
+  int rc = SLO_OK;
+  for_each_chunk(offset, cols, n_tensors, chunk, [&](uint64_t g, const ChunkGeom& cg) {
+    const int len = (int)cg.addr.size();
+    std::fill(where.begin(), where.end(), -1);
+    for (int i = 0; i < len; ++i) { where[cg.pos[i]] = i; update[cg.addr[i]] = 0.0f; }
+    for (int r = 0; r < R; ++r) {
+      const uint16_t* cidx = idx[r] + g * (uint64_t)k;
+      const uint8_t* ccodes = codes[r] + g * cs;
+      const float s = scales[r][g];
+      for (int j = 0; j < k; ++j) {
+        const uint32_t p = cidx[j];
+        if (p == 0xFFFFu) continue;          // padding slot
+        if ((int)p >= chunk || where[p] < 0) { rc = SLO_ERR_INVALID_ARG; continue; }
+        float v;
+        if (bits == 32) std::memcpy(&v, ccodes + 4 * (size_t)j, 4);
+        else v = dequantise(get_code(ccodes, j, bits), s, bits);
+        const uint64_t at = cg.addr[where[p]];
+        update[at] = update[at] + v;
+      }
+    }
+    const float Rf = (float)R;
+    for (int i = 0; i < len; ++i) update[cg.addr[i]] = update[cg.addr[i]] / Rf;
+  });
+  return rc;
+}
+
 int slo_aggregate(int R, const uint16_t* const* idx, const uint8_t* const* codes,
                   const float* const* scales, const uint64_t* offset, uint32_t n_tensors,
                   int chunk, int k, int bits, float* update) {
-  if (R < 1 || !idx || !codes || !scales || !offset || !update) return SLO_ERR_INVALID_ARG;
-  if (chunk < 1 || chunk > 65535 || k < 1 || k > chunk || !bits_ok(bits)) return SLO_ERR_INVALID_ARG;
-  const uint64_t cs = codes_stride(k, bits);
-  uint64_t g = 0;
-  for (uint32_t t = 0; t < n_tensors; ++t) {
-    const uint64_t n_t = offset[t + 1] - offset[t];
-    for (uint64_t c0 = 0; c0 < n_t; c0 += (uint64_t)chunk, ++g) {
-      const uint64_t base = offset[t] + c0;
-      const int len = (int)std::min<uint64_t>((uint64_t)chunk, n_t - c0);
-      for (int i = 0; i < len; ++i) update[base + i] = 0.0f;
-      for (int r = 0; r < R; ++r) {
-        const uint16_t* cidx = idx[r] + g * (uint64_t)k;
-        const uint8_t* ccodes = codes[r] + g * cs;
-        const float s = scales[r][g];
-        for (int j = 0; j < k; ++j) {
-          const uint32_t i = cidx[j];
-          if (i == 0xFFFFu) continue;          // padding slot
-          if ((int)i >= len) return SLO_ERR_INVALID_ARG;
-          float v;
-          if (bits == 32) std::memcpy(&v, ccodes + 4 * (size_t)j, 4);
-          else v = dequantise(get_code(ccodes, j, bits), s, bits);
-          update[base + i] = update[base + i] + v;
-        }
-      }
-      const float Rf = (float)R;
-      for (int i = 0; i < len; ++i) update[base + i] = update[base + i] / Rf;
-    }
-  }
-  return SLO_OK;
+  return slo_aggregate_tiled(R, idx, codes, scales, offset, nullptr, n_tensors, chunk, k, bits, update);
 }
 
 // Eq. 2 line 5, second half: plain SGD outer step, theta <- theta - lr * update (one fused rounding)
