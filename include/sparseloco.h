@@ -24,10 +24,17 @@
  * Arena and chunks
  * ----------------
  *  Parameters live in a flat fp32 arena of `n_total` elements holding `n_tensors` tensors back
- *  to back (row-major).  Chunks are runs of `chunk` consecutive elements of ONE tensor (the
- *  paper's 64 x 64 = 4096 elements, §3 "Training Configuration", Table 8); the last chunk of a
- *  tensor may be short and keeps k_eff = min(k, its length).  Chunks are numbered through the
- *  arena in order: chunk g owns idx[g*k .. g*k+k), codes[g*stride .. (g+1)*stride), scales[g].
+ *  to back (row-major).  Two chunk geometries (the paper says "64 x 64 (i.e., 4096 elements per
+ *  chunk)", §3 "Training Configuration", Table 8, which can be read either way):
+ *   - consecutive (default): a chunk is a run of `chunk` consecutive elements of ONE tensor; the
+ *     last chunk of a tensor may be short.  Position p of a chunk is its p-th element.
+ *   - square tiles (sl_layout.cols[t] > 0): tensor t is a matrix of cols[t] columns cut into
+ *     s x s tiles, s*s = chunk, numbered row-major over the tile grid.  Position p of a tile is
+ *     its row p / s, column p % s; tiles on the matrix's right and bottom edges are smaller and
+ *     only the positions inside the matrix exist.
+ *  A chunk with fewer than k elements keeps them all (k_eff = min(k, its size)).  Chunks are
+ *  numbered through the arena in order: chunk g owns idx[g*k .. g*k+k), codes[g*stride ..
+ *  (g+1)*stride), scales[g].
  *
  * Message of one chunk
  * --------------------
@@ -54,7 +61,9 @@ extern "C" {
 enum {
   SL_OK = 0,
   SL_ERR_INVALID_ARG = -1, /* null pointer, k < 1, k > chunk, bits not in {2,4,8,32}, R out of range,
-                              beta / outer_lr not finite, offsets not ascending or not ending at n_total */
+                              beta / outer_lr not finite, offsets not ascending or not ending at n_total,
+                              tiles asked for with a chunk that is not a square or a tensor that is not
+                              a whole number of rows */
   SL_ERR_ALIGNMENT = -2,   /* a float pointer not 4-byte aligned or idx not 2-byte aligned */
   SL_ERR_UNSUPPORTED = -3, /* chunk > SL_MAX_CHUNK, n_tensors > SL_MAX_TENSORS, more than 2^31 chunks */
   SL_ERR_CUDA = -4         /* a CUDA runtime call or a launch failed (the error is not cleared) */
@@ -67,7 +76,7 @@ enum {
 };
 
 #define SL_MAX_CHUNK 8192     /* elements; any chunk size in [1, SL_MAX_CHUNK] is accepted */
-#define SL_MAX_TENSORS 2048   /* tensors per call; split larger arenas into several calls */
+#define SL_MAX_TENSORS 1536   /* tensors per call; split larger arenas into several calls */
 #define SL_MAX_REPLICAS 64    /* replicas per batched / aggregate call */
 
 /* HOST description of an arena.  offset[0] = 0 < ... (non-decreasing) ... offset[n_tensors] =
@@ -78,9 +87,12 @@ typedef struct sl_layout {
   uint64_t n_total;
   uint32_t n_tensors;
   const uint64_t* offset; /* HOST, [n_tensors + 1] */
+  const uint64_t* cols;   /* HOST, [n_tensors], or NULL: columns of every tensor that is cut into square
+                             tiles, 0 for tensors (and NULL for arenas) with consecutive chunks */
 } sl_layout;
 
-/* Number of chunks of the arena, sum over tensors of ceil(n_t / chunk).  0 on bad arguments. */
+/* Number of chunks of the arena: per tensor ceil(n_t / chunk), or ceil(rows / s) * ceil(cols / s)
+ * for a tensor cut into tiles.  0 on bad arguments. */
 uint64_t sl_num_chunks(const sl_layout* layout, int chunk);
 
 /* Bytes of `codes` ONE chunk owns: ceil(k*bits/8), or 4*k when bits == 32.  0 on bad arguments.

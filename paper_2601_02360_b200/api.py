@@ -19,7 +19,7 @@ from . import build as _build
 
 SL_OK, SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_CUDA = 0, -1, -2, -3, -4
 SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
-SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 2048, 64
+SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1536, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
            "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_strerror")
@@ -27,7 +27,7 @@ EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch
 
 class SlLayout(ctypes.Structure):
     _fields_ = [("n_total", ctypes.c_uint64), ("n_tensors", ctypes.c_uint32),
-                ("offset", ctypes.POINTER(ctypes.c_uint64))]
+                ("offset", ctypes.POINTER(ctypes.c_uint64)), ("cols", ctypes.POINTER(ctypes.c_uint64))]
 
 
 class SparseLoCoError(RuntimeError):
@@ -79,13 +79,20 @@ def strerror(code: int) -> str:
 
 
 class Layout:
-    """Host description of an arena (`sl_layout`): element offsets of its tensors."""
+    """Host description of an arena (`sl_layout`): element offsets of its tensors and, for the
+    tensors cut into square tiles, their number of columns (`cols`, 0 = consecutive chunks)."""
 
-    def __init__(self, offsets: Sequence[int]):
+    def __init__(self, offsets: Sequence[int], cols: Optional[Sequence[int]] = None):
         self.offsets = np.ascontiguousarray(np.asarray(offsets, dtype=np.uint64))
         assert self.offsets.ndim == 1 and len(self.offsets) >= 1
-        self.c = SlLayout(int(self.offsets[-1]), len(self.offsets) - 1,
-                          self.offsets.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)))
+        u64p = ctypes.POINTER(ctypes.c_uint64)
+        self.cols = None
+        cols_p = ctypes.cast(None, u64p)
+        if cols is not None:
+            self.cols = np.ascontiguousarray(np.asarray(cols, dtype=np.uint64))
+            assert self.cols.shape == (len(self.offsets) - 1,)
+            cols_p = self.cols.ctypes.data_as(u64p)
+        self.c = SlLayout(int(self.offsets[-1]), len(self.offsets) - 1, self.offsets.ctypes.data_as(u64p), cols_p)
 
     @property
     def n_total(self) -> int:

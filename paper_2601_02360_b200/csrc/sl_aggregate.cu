@@ -31,7 +31,7 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const ChunkRef c = locate(a.tb, g, a.chunk);
   const int len = c.len, k = a.k, bits = a.bits;
 
-  for (int i = tid; i < len; i += kThreads) acc[i] = 0.0f;
+  for (int i = tid; i < len; i += kThreads) acc[i] = 0.0f;   // one accumulator per element of the chunk
   __syncthreads();
   bool bad = false;
   for (int r = 0; r < a.R; ++r) {
@@ -39,9 +39,10 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
     const uint8_t* __restrict__ codes = a.m.codes[r] + (uint64_t)g * (uint64_t)a.stride;
     const float s = a.m.scales[r][g];
     for (int j = tid; j < k; j += kThreads) {
-      const uint32_t i = idx[j];
-      if (i == 0xFFFFu) continue;                 // padding slot
-      if (i >= (uint32_t)len) { bad = true; continue; }
+      const uint32_t p = idx[j];
+      if (p == 0xFFFFu) continue;                 // padding slot
+      const int i = c.elem(p);                    // position -> element number (they differ in edge tiles)
+      if (i < 0) { bad = true; continue; }
       float v;
       if (bits == 32) {
         v = reinterpret_cast<const float*>(codes)[j];
@@ -55,10 +56,11 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
     __syncthreads();
   }
   const float Rf = (float)a.R;
-  float* __restrict__ out = a.out + c.base;
+  float* __restrict__ out = a.out;
   for (int i = tid; i < len; i += kThreads) {
     const float u = __fdiv_rn(acc[i], Rf);
-    out[i] = APPLY ? __fmaf_rn(-a.outer_lr, u, out[i]) : u;
+    const uint64_t at = c.addr(i);
+    out[at] = APPLY ? __fmaf_rn(-a.outer_lr, u, out[at]) : u;
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }

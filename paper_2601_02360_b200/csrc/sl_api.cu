@@ -17,6 +17,25 @@ inline uint64_t codes_stride(int k, int bits) {
   return bits == 32 ? (uint64_t)k * 4u : ((uint64_t)k * (uint64_t)bits + 7u) / 8u;
 }
 
+// side of the square tile with `chunk` elements, 0 if chunk is not a square
+inline uint32_t tile_side(int chunk) {
+  uint32_t s = 1;
+  while ((uint64_t)s * s < (uint64_t)chunk) ++s;
+  return (uint64_t)s * s == (uint64_t)chunk ? s : 0;
+}
+
+// chunks of tensor t; false if its description is inconsistent
+inline bool tensor_chunks(const sl_layout* L, uint32_t t, int chunk, uint32_t side, uint64_t* out) {
+  if (L->offset[t + 1] < L->offset[t]) return false;
+  const uint64_t n_t = L->offset[t + 1] - L->offset[t];
+  const uint64_t c_t = L->cols ? L->cols[t] : 0;
+  if (c_t == 0) { *out = (n_t + (uint64_t)chunk - 1) / (uint64_t)chunk; return true; }
+  if (side == 0 || c_t > 0xFFFFFFFFull || n_t % c_t != 0) return false;
+  const uint64_t rows = n_t / c_t;
+  *out = ((rows + side - 1) / side) * ((c_t + side - 1) / side);
+  return true;
+}
+
 int check_common(const sl_layout* L, int chunk, int k, int bits) {
   if (!L || !L->offset) return SL_ERR_INVALID_ARG;
   if (chunk < 1 || k < 1 || k > chunk || !bits_ok(bits)) return SL_ERR_INVALID_ARG;
@@ -24,31 +43,42 @@ int check_common(const sl_layout* L, int chunk, int k, int bits) {
   if (L->n_tensors < 1) return SL_ERR_INVALID_ARG;
   if (L->n_tensors > SL_MAX_TENSORS) return SL_ERR_UNSUPPORTED;
   if (L->offset[0] != 0 || L->offset[L->n_tensors] != L->n_total) return SL_ERR_INVALID_ARG;
+  const uint32_t side = tile_side(chunk);
   uint64_t nc = 0;
   for (uint32_t t = 0; t < L->n_tensors; ++t) {
-    if (L->offset[t + 1] < L->offset[t]) return SL_ERR_INVALID_ARG;
-    nc += (L->offset[t + 1] - L->offset[t] + (uint64_t)chunk - 1) / (uint64_t)chunk;
+    uint64_t c;
+    if (!tensor_chunks(L, t, chunk, side, &c)) return SL_ERR_INVALID_ARG;
+    nc += c;
   }
   if (nc > 0x7FFFFFFFull) return SL_ERR_UNSUPPORTED;
   return SL_OK;
 }
 
+// *tuned_ok: the layout is one the tuned kernels take (consecutive chunks only, every offset a
+// multiple of 4 elements)
 template <int T>
-void fill_table(Table<T>& tb, const sl_layout* L, int chunk, bool* offsets_mult4) {
+void fill_table(Table<T>& tb, const sl_layout* L, int chunk, bool* tuned_ok) {
   tb.n_tensors = L->n_tensors;
+  const uint32_t side = tile_side(chunk);
   uint32_t nc = 0;
-  bool m4 = true;
+  bool m4 = true, tiled = false;
   for (uint32_t t = 0; t < L->n_tensors; ++t) {
     tb.first_chunk[t] = nc;
     tb.offset[t] = L->offset[t];
+    tb.cols[t] = L->cols ? (uint32_t)L->cols[t] : 0u;
+    tiled = tiled || tb.cols[t] != 0;
     m4 = m4 && (L->offset[t] % 4 == 0);
-    nc += (uint32_t)((L->offset[t + 1] - L->offset[t] + (uint64_t)chunk - 1) / (uint64_t)chunk);
+    uint64_t c = 0;
+    tensor_chunks(L, t, chunk, side, &c);
+    nc += (uint32_t)c;
   }
   tb.first_chunk[L->n_tensors] = nc;
   tb.offset[L->n_tensors] = L->n_total;
+  tb.cols[L->n_tensors] = 0;
+  tb.side = tiled ? side : 0;
   m4 = m4 && (L->n_total % 4 == 0);
   tb.n_chunks = nc;
-  *offsets_mult4 = m4;
+  *tuned_ok = m4 && !tiled;
 }
 
 // step = false: Eq. 2 lines 1-4 only.  step = true: the whole of Eq. 2 (theta_global is updated):
@@ -179,10 +209,12 @@ extern "C" {
 
 uint64_t sl_num_chunks(const sl_layout* L, int chunk) {
   if (!L || !L->offset || chunk < 1) return 0;
+  const uint32_t side = tile_side(chunk);
   uint64_t nc = 0;
   for (uint32_t t = 0; t < L->n_tensors; ++t) {
-    if (L->offset[t + 1] < L->offset[t]) return 0;
-    nc += (L->offset[t + 1] - L->offset[t] + (uint64_t)chunk - 1) / (uint64_t)chunk;
+    uint64_t c;
+    if (!tensor_chunks(L, t, chunk, side, &c)) return 0;
+    nc += c;
   }
   return nc;
 }

@@ -12,20 +12,44 @@ namespace sl {
 // constant bank), so that the library needs no device-side table and no state.
 // first_chunk[t] = number of chunks owned by tensors before t.
 // ---------------------------------------------------------------------------
+// cols[t] > 0: tensor t is a matrix of cols[t] columns cut into side x side tiles (side*side = chunk).
 template <int T>
 struct Table {
   uint32_t n_tensors;
   uint32_t n_chunks;
+  uint32_t side;      // tile side, 0 when no tensor is tiled
   uint32_t first_chunk[T + 1];
+  uint32_t cols[T + 1];
   uint64_t offset[T + 1];
 };
 
 struct ChunkRef {
-  uint64_t base;  // element offset of the chunk in the arena
-  int len;        // elements in the chunk (1..chunk)
+  uint64_t base;    // element offset of the chunk's first element in the arena
+  int len;          // elements in the chunk (1..chunk)
+  uint32_t stride;  // 0: consecutive chunk; else the matrix's row length (the chunk is a tile)
+  uint32_t w;       // tile: columns of this tile (<= side)
+  uint32_t side;    // tile: side of a full tile
+
+  // the d-th element of the chunk (ascending position): its arena offset and its position
+  __device__ __forceinline__ uint64_t addr(int d) const {
+    if (stride == 0) return base + (uint64_t)d;
+    const uint32_t lr = (uint32_t)d / w, lc = (uint32_t)d - lr * w;
+    return base + (uint64_t)lr * stride + lc;
+  }
+  __device__ __forceinline__ uint32_t pos(int d) const {
+    if (stride == 0) return (uint32_t)d;
+    const uint32_t lr = (uint32_t)d / w, lc = (uint32_t)d - lr * w;
+    return lr * side + lc;
+  }
+  // position -> element number, or -1 if the chunk has no such position
+  __device__ __forceinline__ int elem(uint32_t p) const {
+    if (stride == 0) return p < (uint32_t)len ? (int)p : -1;
+    const uint32_t lr = p / side, lc = p - lr * side;
+    return (lc < w && lr * w + lc < (uint32_t)len) ? (int)(lr * w + lc) : -1;
+  }
 };
 
-// chunk g -> (base, len): binary search over the tensors' first chunks
+// chunk g -> its geometry: binary search over the tensors' first chunks
 template <int T>
 __device__ __forceinline__ ChunkRef locate(const Table<T>& tb, uint32_t g, int chunk) {
   uint32_t lo = 0, hi = tb.n_tensors;  // first_chunk[lo] <= g < first_chunk[hi]
@@ -34,9 +58,26 @@ __device__ __forceinline__ ChunkRef locate(const Table<T>& tb, uint32_t g, int c
     if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
   }
   ChunkRef c;
-  c.base = tb.offset[lo] + (uint64_t)(g - tb.first_chunk[lo]) * (uint64_t)chunk;
-  const uint64_t left = tb.offset[lo + 1] - c.base;
-  c.len = left < (uint64_t)chunk ? (int)left : chunk;
+  const uint32_t nc = tb.cols[lo];
+  const uint32_t in_t = g - tb.first_chunk[lo];
+  if (nc == 0) {
+    c.base = tb.offset[lo] + (uint64_t)in_t * (uint64_t)chunk;
+    const uint64_t left = tb.offset[lo + 1] - c.base;
+    c.len = left < (uint64_t)chunk ? (int)left : chunk;
+    c.stride = 0; c.w = 0; c.side = 0;
+  } else {
+    const uint32_t s = tb.side;
+    const uint32_t tiles_c = (nc + s - 1) / s;
+    const uint32_t tr = in_t / tiles_c, tc = in_t - tr * tiles_c;
+    const uint64_t rows = (tb.offset[lo + 1] - tb.offset[lo]) / nc;
+    const uint64_t r0 = (uint64_t)tr * s, c0 = (uint64_t)tc * s;
+    const uint32_t h = (uint32_t)(rows - r0 < s ? rows - r0 : s);
+    c.w = (uint32_t)(nc - c0 < s ? nc - c0 : s);
+    c.base = tb.offset[lo] + r0 * nc + c0;
+    c.len = (int)(h * c.w);
+    c.stride = nc;
+    c.side = s;
+  }
   return c;
 }
 

@@ -2,8 +2,9 @@
 // quantisation, residual.
 //
 // Two kernels with identical results:
-//   compress_generic_kernel  any chunk length / k / code width / alignment; one CTA per
-//                            (chunk, replica); exact 4-pass radix select in shared memory.
+//   compress_generic_kernel  any chunk length / k / code width / alignment, consecutive chunks or
+//                            square tiles; one CTA per (chunk, replica); exact 4-pass radix
+//                            select in shared memory.
 //   compress_c4096_kernel    the tuned path for full 4096-element chunks, k <= 128: one CTA per
 //                            chunk walks all R replicas with theta_global held in registers, a
 //                            cheap lower bound on the k-th magnitude prunes the chunk to a few
@@ -42,9 +43,10 @@ struct SelectScratch {
 //   * codes OR-ed into `cw` (zeroed by the caller), residual patched into `ep`.
 // All threads of the CTA must call it; it ends with a barrier.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void block_select_emit(float* ep, int len, int k_eff, int bits, float s,
+__device__ __forceinline__ void block_select_emit(float* ep, const ChunkRef& c, int k_eff, int bits, float s,
                                                   SelectScratch& sc, uint32_t* cw,
                                                   uint16_t* __restrict__ oidx, uint8_t* __restrict__ ocodes) {
+  const int len = c.len;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t prefix = 0, need = (uint32_t)k_eff;
 #pragma unroll 1
@@ -121,7 +123,7 @@ __device__ __forceinline__ void block_select_emit(float* ep, int len, int k_eff,
     const uint32_t km = __ballot_sync(kFull, keep);
     if (keep) {
       const uint32_t slot = out_base + __popc(km & lanemask_lt());
-      oidx[slot] = (uint16_t)i;
+      oidx[slot] = (uint16_t)c.pos(i);            // element number -> position (they differ in edge tiles)
       float sent;
       if (bits == 32) {
         reinterpret_cast<float*>(ocodes)[slot] = v;
@@ -167,15 +169,16 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   const int k = a.k, bits = a.bits;
   const int k_eff = k < len ? k : len;
 
-  const float* __restrict__ tl = a.p.theta_local[r] + c.base;
-  const float* __restrict__ tg = a.theta_global + c.base;
-  float* __restrict__ er = a.p.err[r] + c.base;
+  const float* __restrict__ tl = a.p.theta_local[r];
+  const float* __restrict__ tg = a.theta_global;
+  float* __restrict__ er = a.p.err[r];
 
-  // pseudo-gradient and error feedback
+  // pseudo-gradient and error feedback; element i of the chunk (ascending position) sits at c.addr(i)
   uint32_t tmax = 0;
   for (int i = tid; i < len; i += kThreads) {
-    const float d = __fsub_rn(tg[i], tl[i]);
-    const float e = __fmaf_rn(a.beta, er[i], d);
+    const uint64_t at = c.addr(i);
+    const float d = __fsub_rn(tg[at], tl[at]);
+    const float e = __fmaf_rn(a.beta, er[at], d);
     ep[i] = e;
     tmax = max(tmax, key_of(e));
   }
@@ -192,10 +195,10 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 
   uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
   uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
-  block_select_emit(ep, len, k_eff, bits, s, sc, cw, oidx, ocodes);
+  block_select_emit(ep, c, k_eff, bits, s, sc, cw, oidx, ocodes);
 
   // write-back
-  for (int i = tid; i < len; i += kThreads) er[i] = ep[i];
+  for (int i = tid; i < len; i += kThreads) er[c.addr(i)] = ep[i];
   for (int j = k_eff + tid; j < k; j += kThreads) oidx[j] = 0xFFFFu;
   if (bits != 32) {
     const uint8_t* cb = reinterpret_cast<const uint8_t*>(cw);

@@ -47,10 +47,10 @@ def assert_exact(a: np.ndarray, b: np.ndarray, what: str) -> None:
                              f"{a[tuple(w[0])]} vs {b[tuple(w[0])]}")
 
 
-def oracle_compress_all(tls, tg, errs, offsets, beta, chunk, k, bits, threads: int = 8):
+def oracle_compress_all(tls, tg, errs, offsets, beta, chunk, k, bits, threads: int = 8, cols=None):
     """Checker side of Eq. 2 lines 1-4 for every replica (errs updated in place)."""
     def one(r):
-        return slo.compress(tls[r], tg, errs[r], offsets, beta, chunk, k, bits)
+        return slo.compress(tls[r], tg, errs[r], offsets, beta, chunk, k, bits, cols)
     with ThreadPoolExecutor(max_workers=max(1, min(threads, len(tls)))) as ex:
         return list(ex.map(one, range(len(tls))))
 
@@ -58,8 +58,8 @@ def oracle_compress_all(tls, tg, errs, offsets, beta, chunk, k, bits, threads: i
 class GpuStep:
     """Device buffers for one arena and R replicas, driven through the binding."""
 
-    def __init__(self, offsets, R, chunk, k, bits, device="cuda"):
-        self.layout = api.Layout(offsets)
+    def __init__(self, offsets, R, chunk, k, bits, device="cuda", cols=None):
+        self.layout = api.Layout(offsets, cols)
         self.R, self.chunk, self.k, self.bits = R, chunk, k, bits
         n = self.layout.n_total
         self.n = n
@@ -117,13 +117,13 @@ def compare_messages(gpu_msgs, ora_msgs, what=""):
 
 
 def run_and_compare(offsets, tg, tls, errs, beta, chunk, k, bits, outer_lr, rounds=1, next_locals=None,
-                    batched=True, what="", fused=False):
+                    batched=True, what="", fused=False, cols=None):
     """Runs `rounds` outer steps on the GPU and on the checker from the same inputs and compares
     everything after every round.  `next_locals(round, theta_global_numpy)` supplies the replicas'
     parameters for the rounds after the first.  fused=True drives the GPU through the single
     sl_outer_step call instead of sl_compress_batch + sl_aggregate_apply."""
     R = len(tls)
-    gs = GpuStep(offsets, R, chunk, k, bits)
+    gs = GpuStep(offsets, R, chunk, k, bits, cols=cols)
     tg_o = tg.copy()
     errs_o = [e.copy() for e in errs]
     gs.upload(tg, tls, errs)
@@ -136,7 +136,7 @@ def run_and_compare(offsets, tg, tls, errs, beta, chunk, k, bits, outer_lr, roun
             gs.outer_step(beta, outer_lr)
         else:
             gs.compress(beta, batched=batched)
-        res = oracle_compress_all(tls, tg_o, errs_o, offsets, beta, chunk, k, bits)
+        res = oracle_compress_all(tls, tg_o, errs_o, offsets, beta, chunk, k, bits, cols=cols)
         ora_msgs = [(i, c, s) for i, c, s, _ in res]
         for _, _, _, f in res:
             flags_o |= f
@@ -144,7 +144,7 @@ def run_and_compare(offsets, tg, tls, errs, beta, chunk, k, bits, outer_lr, roun
         compare_messages(gpu_msgs, ora_msgs, f"{what} round {t}")
         for r in range(R):
             assert_close(gs.err[r].cpu().numpy(), errs_o[r], f"{what} round {t} err[r={r}]")
-        upd = slo.aggregate(ora_msgs, offsets, chunk, k, bits)
+        upd = slo.aggregate(ora_msgs, offsets, chunk, k, bits, cols)
         slo.outer_apply(tg_o, upd, outer_lr)
         if not fused:
             gs.aggregate_apply(outer_lr)

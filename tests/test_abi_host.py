@@ -49,6 +49,16 @@ def test_sizes(lib):
     assert api.strerror(api.SL_OK) == "ok" and "align" in api.strerror(api.SL_ERR_ALIGNMENT)
 
 
+def test_tile_geometry_sizes(lib):
+    lay = api.Layout([0, 24], cols=[6])                 # a 4 x 6 matrix
+    assert api.sl_num_chunks(lay, 16) == 1 * 2          # 4 x 4 tiles: one tile row, two tile columns
+    assert api.sl_num_chunks(lay, 4) == 2 * 3
+    assert api.sl_num_chunks(lay, 8) == 0               # 8 is not a square
+    assert api.sl_num_chunks(api.Layout([0, 24], cols=[5]), 16) == 0   # 24 elements are not rows of 5
+    assert api.sl_num_chunks(api.Layout([0, 24, 30], cols=[6, 0]), 16) == 2 + 1
+    assert api.sl_num_chunks(api.Layout([0, 24], cols=[0]), 8) == 3    # no tiles: any chunk size
+
+
 def _call_compress(lib, lay, chunk=4096, k=64, bits=2, beta=0.95, ptr=0x1000, idx=0x1000, R=None):
     if R is None:
         return lib.sl_compress(ptr, 0x1000, 0x1000, lay.ref(), beta, chunk, k, bits, idx, 0x1000, 0x1000, 0, 0)
@@ -81,6 +91,8 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert _call_compress(lib, wrong_total) == E.SL_ERR_INVALID_ARG
     many = api.Layout(np.arange(api.SL_MAX_TENSORS + 2) * 4)
     assert _call_compress(lib, many) == E.SL_ERR_UNSUPPORTED
+    assert _call_compress(lib, api.Layout([0, 24], cols=[6]), chunk=8, k=2) == E.SL_ERR_INVALID_ARG    # not a square
+    assert _call_compress(lib, api.Layout([0, 24], cols=[5]), chunk=16, k=2) == E.SL_ERR_INVALID_ARG   # not whole rows
     tab = (ctypes.c_void_p * 2)(0x1000, 0x1000)
     assert lib.sl_aggregate(2, tab, tab, tab, lay.ref(), 4096, 64, 2, 0, 0, 0) == E.SL_ERR_INVALID_ARG
     assert lib.sl_aggregate(0, tab, tab, tab, lay.ref(), 4096, 64, 2, 0x1000, 0, 0) == E.SL_ERR_INVALID_ARG
