@@ -241,13 +241,17 @@ def run_reference(args) -> None:
 
 # --------------------------------------------------------------------------- the CUDA path, timed
 class DeviceState:
-    def __init__(self, wl: synth.Workload, seed: int, device):
+    def __init__(self, wl: synth.Workload, seed: int, device, tiles: bool = False):
         from paper_2601_02360_b200 import api
         self.api = api
         self.wl = wl
         self.seed = seed
         self.dev = device
-        self.layout = api.Layout(wl.offsets())
+        # --tiles: matrices are cut into sqrt(chunk) x sqrt(chunk) tiles (the paper's literal 64 x 64
+        # chunks); vectors keep consecutive chunks
+        cols = [c if r > 1 else 0 for _, r, c in wl.tensors] if tiles else None
+        self.layout = api.Layout(wl.offsets(), cols)
+        self.n_chunks = api.sl_num_chunks(self.layout, wl.chunk)
         n = wl.n_total
         self.theta_global = synth.gen_theta_global(wl, device, seed)
         self.rho = synth.row_scales(wl, seed)
@@ -357,7 +361,7 @@ def run_ours(args) -> None:
         wl = wl.replace(variant=args.variant)
     if args.first_tensors:
         wl = synth.sub_arena(wl, list(range(args.first_tensors)), f"{wl.name}[:{args.first_tensors}]")
-    st = DeviceState(wl, rank_seed(args.seed, rank), dev)
+    st = DeviceState(wl, rank_seed(args.seed, rank), dev, tiles=args.tiles)
     stream = torch.cuda.current_stream()
 
     sampler = ClockSampler(local)
@@ -413,6 +417,7 @@ def run_ours(args) -> None:
         "config": {"workload": wl.name, "params": wl.n_total, "tensors": len(wl.tensors),
                    "chunks": wl.n_chunks(), "R": wl.R, "k": wl.k, "bits": wl.bits, "chunk": wl.chunk,
                    "beta": wl.beta, "outer_lr": wl.outer_lr, "variant": wl.variant,
+                   "geometry": "64x64 tiles of each matrix" if args.tiles else "consecutive chunks",
                    "l2": "inputs (GBs per launch) far larger than the 126 MB L2; no flush needed",
                    "sharding": "none: every rank runs an independent parameter set" if world > 1 else "single GPU",
                    "step": "sl_compress_batch + sl_aggregate_apply; theta_local re-drawn between steps (untimed)"},
@@ -454,6 +459,8 @@ def main() -> None:
     ap.add_argument("--k", type=int, default=0)
     ap.add_argument("--first-tensors", type=int, default=0,
                     help="keep only the first N tensors of the workload (small cases for profiling)")
+    ap.add_argument("--tiles", action="store_true",
+                    help="cut matrices into square tiles of `chunk` elements instead of consecutive chunks")
     ap.add_argument("--variant", default="plain", choices=["plain", "ties_literal", "ties_dyadic"],
                     help="tie-heavy value laws of the density-sweep configuration")
     ap.add_argument("--seed", type=int, default=0)

@@ -76,13 +76,14 @@ enum {
 };
 
 #define SL_MAX_CHUNK 8192     /* elements; any chunk size in [1, SL_MAX_CHUNK] is accepted */
-#define SL_MAX_TENSORS 1536   /* tensors per call; split larger arenas into several calls */
+#define SL_MAX_TENSORS 1280   /* tensors per call; split larger arenas into several calls */
 #define SL_MAX_REPLICAS 64    /* replicas per batched / aggregate call */
 
 /* HOST description of an arena.  offset[0] = 0 < ... (non-decreasing) ... offset[n_tensors] =
  * n_total.  A single tensor is n_tensors = 1, offset = {0, n}.  The tuned kernels need every
- * offset to be a multiple of 4 elements and every arena pointer 16-byte aligned; otherwise the
- * calls fall back to a slower kernel with identical results. */
+ * offset (and every tiled tensor's column count) to be a multiple of 4 elements and every arena
+ * pointer 16-byte aligned; otherwise the calls fall back to a slower kernel with identical
+ * results. */
 typedef struct sl_layout {
   uint64_t n_total;
   uint32_t n_tensors;

@@ -19,7 +19,7 @@ from . import build as _build
 
 SL_OK, SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_CUDA = 0, -1, -2, -3, -4
 SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
-SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1536, 64
+SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1280, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
            "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_strerror")

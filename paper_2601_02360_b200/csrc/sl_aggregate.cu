@@ -13,8 +13,8 @@ constexpr int kThreads = 256;
 // in replica order (positions inside one message are distinct, so a pass has no conflicts and
 // needs no atomics; a barrier separates the passes), then divided by R and either written out
 // (APPLY = false) or folded straight into theta_global (APPLY = true).
-// TAILS = false: CTA b handles chunk b.  TAILS = true: CTA b handles the short last chunk of
-// tensor b (if it has one), which is how the tuned kernel delegates the tensors' ragged ends.
+// TAILS = false: CTA b handles chunk b.  TAILS = true: CTA b handles the b-th chunk that is not
+// full (short last chunks, edge tiles), which is how the tuned kernel delegates the ragged ends.
 template <int T, bool APPLY, bool TAILS>
 __global__ void __launch_bounds__(kThreads)
 aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
@@ -22,12 +22,7 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
   float* acc = reinterpret_cast<float*>(smem_raw);  // [chunk]
   const int tid = threadIdx.x;
   uint32_t g = blockIdx.x;
-  if (TAILS) {
-    const uint32_t t = g;
-    const uint64_t n_t = a.tb.offset[t + 1] - a.tb.offset[t];
-    if (n_t % (uint64_t)a.chunk == 0) return;
-    g = a.tb.first_chunk[t + 1] - 1;
-  }
+  if (TAILS) g = tail_chunk(a.tb, g, a.chunk);    // the g-th chunk that is not full
   const ChunkRef c = locate(a.tb, g, a.chunk);
   const int len = c.len, k = a.k, bits = a.bits;
 
@@ -90,26 +85,22 @@ struct AggSmem {
 
 __device__ __forceinline__ uint32_t agg_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// first full chunk at or after g (stepping by `step`); t_lo caches the tensor of the last hit
+// first full chunk at or after g (stepping by `step`); t_lo caches the tensor of the last hit;
+// stride = elements between the chunk's rows of 64 (64 for a consecutive chunk)
 template <int T>
 __device__ __forceinline__ bool next_full_chunk(const Table<T>& tb, uint32_t& g, uint32_t step, uint32_t& t_lo,
-                                                uint64_t& base) {
+                                                uint64_t& base, uint32_t& stride) {
   for (; g < tb.n_chunks; g += step) {
-    if (!(tb.first_chunk[t_lo] <= g && g < tb.first_chunk[t_lo + 1])) {
-      uint32_t lo = 0, hi = tb.n_tensors;
-      while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
-      }
-      t_lo = lo;
-    }
-    base = tb.offset[t_lo] + (uint64_t)(g - tb.first_chunk[t_lo]) * (uint64_t)kAC;
-    if (tb.offset[t_lo + 1] - base >= (uint64_t)kAC) return true;   // short chunks go to the generic tail launch
+    const ChunkRef c = locate_cached(tb, g, kAC, t_lo);
+    if (c.len == kAC) { base = c.base; stride = c.stride ? c.stride : 64u; return true; }
   }
-  return false;
+  return false;                                    // chunks that are not full go to the generic tail launch
 }
 
-template <int T, bool APPLY, int NP>
+// TILED (arenas with matrices cut into 64 x 64 tiles): a chunk is 64 rows of 256 bytes `stride`
+// elements apart; theta_global then comes in by 16-byte cp.async copies of all threads instead
+// of one bulk copy, and the stores follow the same geometry.
+template <int T, bool APPLY, int NP, bool TILED>
 __global__ void __launch_bounds__(kThreads)
 aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   extern __shared__ __align__(16) unsigned char agg_smem_raw[];
@@ -149,7 +140,7 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
 
   if (APPLY && tid == 0) {
     for (int s = 0; s < 2; ++s)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(agg_smem_u32(&sm.full[s])) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(agg_smem_u32(&sm.full[s])), "r"(TILED ? kThreads : 1) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -173,18 +164,29 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       }
     }
   };
-  auto load_theta = [&](uint64_t base, int buf) {      // thread 0 only
+  auto load_theta = [&](uint64_t base, uint32_t stride, int buf) {
     const uint32_t bar = agg_smem_u32(&sm.full[buf]);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBytes) : "memory");
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(agg_smem_u32(sm.gbuf[buf])), "l"(a.out + base), "r"(kBytes), "r"(bar) : "memory");
+    if (TILED) {                                   // every thread: four 16-byte copies, then one arrival
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int f = tid + 256 * j;
+        const float* src = a.out + base + (size_t)(f >> 4) * stride + (size_t)((f & 15) << 2);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                     ::"r"(agg_smem_u32(reinterpret_cast<float4*>(sm.gbuf[buf]) + f)), "l"(src) : "memory");
+      }
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+    } else if (tid == 0) {                         // one 16 KB bulk copy
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBytes) : "memory");
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(agg_smem_u32(sm.gbuf[buf])), "l"(a.out + base), "r"(kBytes), "r"(bar) : "memory");
+    }
   };
 
-  uint32_t g = blockIdx.x, t_lo = 0;
+  uint32_t g = blockIdx.x, t_lo = 0, stride = 64;
   uint64_t base = 0;
-  bool valid = next_full_chunk(a.tb, g, gridDim.x, t_lo, base);
+  bool valid = next_full_chunk(a.tb, g, gridDim.x, t_lo, base, stride);
   if (valid) {
-    if (APPLY && tid == 0) load_theta(base, 0);
+    if (APPLY) load_theta(base, stride, 0);
     fetch(g);
   }
   for (uint32_t it = 0; valid; ++it) {
@@ -200,15 +202,14 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
         if (rp[i] != 0xFFFFu && rp[i] >= (uint32_t)kAC) bad = true; else pos[i] = rp[i];
       }
     }
-    const uint32_t g_cur = g;
     const uint64_t base_cur = base;
+    const uint32_t stride_cur = stride;
     g += gridDim.x;
-    valid = next_full_chunk(a.tb, g, gridDim.x, t_lo, base);
+    valid = next_full_chunk(a.tb, g, gridDim.x, t_lo, base, stride);
     if (valid) {
-      if (APPLY && tid == 0) load_theta(base, (it + 1) & 1);   // that buffer was last read before the barrier ending iteration it-1
+      if (APPLY) load_theta(base, stride, (it + 1) & 1);   // that buffer was last read before the barrier ending iteration it-1
       fetch(g);
     }
-    (void)g_cur;
 #pragma unroll
     for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(acc)[tid + 256 * j] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
@@ -230,9 +231,12 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       }
       if (!ok) timed_out = true;
     }
-    float4* out4 = reinterpret_cast<float4*>(a.out + base_cur);
+    float* out_cur = a.out + base_cur;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
+      const int f = tid + 256 * j;                 // float4 f of the chunk: row f / 16 of a tile
+      float4* dst = reinterpret_cast<float4*>(TILED ? out_cur + (size_t)(f >> 4) * stride_cur + (size_t)((f & 15) << 2)
+                                                    : out_cur + (size_t)f * 4);
       const float4 s4 = reinterpret_cast<const float4*>(acc)[tid + 256 * j];
       float4 u;
       if (pow2) {
@@ -245,7 +249,7 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
         u.x = __fmaf_rn(nlr, u.x, G.x); u.y = __fmaf_rn(nlr, u.y, G.y);
         u.z = __fmaf_rn(nlr, u.z, G.z); u.w = __fmaf_rn(nlr, u.w, G.w);
       }
-      __stcs(out4 + tid + 256 * j, u);
+      __stcs(dst, u);
     }
     __syncthreads();                               // accumulator and theta buffer read by everyone before they are reused
   }
@@ -274,10 +278,16 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
     kernel<<<grid, kThreads, smem, st>>>(a);
     return cudaPeekAtLastError();
   };
-  if (pairs <= 1) return launch(aggregate_c4096_kernel<T, APPLY, 1>);
-  if (pairs <= 2) return launch(aggregate_c4096_kernel<T, APPLY, 2>);
-  if (pairs <= 4) return launch(aggregate_c4096_kernel<T, APPLY, 4>);
-  return launch(aggregate_c4096_kernel<T, APPLY, 8>);
+  if (a.tb.side != 0) {
+    if (pairs <= 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, true>);
+    if (pairs <= 2) return launch(aggregate_c4096_kernel<T, APPLY, 2, true>);
+    if (pairs <= 4) return launch(aggregate_c4096_kernel<T, APPLY, 4, true>);
+    return launch(aggregate_c4096_kernel<T, APPLY, 8, true>);
+  }
+  if (pairs <= 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, false>);
+  if (pairs <= 2) return launch(aggregate_c4096_kernel<T, APPLY, 2, false>);
+  if (pairs <= 4) return launch(aggregate_c4096_kernel<T, APPLY, 4, false>);
+  return launch(aggregate_c4096_kernel<T, APPLY, 8, false>);
 }
 
 __global__ void __launch_bounds__(256)
@@ -325,13 +335,10 @@ cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned
 
 template <int T>
 cudaError_t launch_aggregate_tails(const AggregateArgs<T>& a, bool apply, cudaStream_t st) {
-  bool tails = false;
-  for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
-    tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)a.chunk) != 0;
-  if (!tails) return cudaSuccess;
+  if (a.tb.n_tails == 0) return cudaSuccess;
   const size_t smem = (size_t)a.chunk * 4;
-  if (apply) aggregate_generic_kernel<T, true, true><<<a.tb.n_tensors, kThreads, smem, st>>>(a);
-  else aggregate_generic_kernel<T, false, true><<<a.tb.n_tensors, kThreads, smem, st>>>(a);
+  if (apply) aggregate_generic_kernel<T, true, true><<<a.tb.n_tails, kThreads, smem, st>>>(a);
+  else aggregate_generic_kernel<T, false, true><<<a.tb.n_tails, kThreads, smem, st>>>(a);
   return cudaPeekAtLastError();
 }
 

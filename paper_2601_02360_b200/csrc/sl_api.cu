@@ -54,31 +54,42 @@ int check_common(const sl_layout* L, int chunk, int k, int bits) {
   return SL_OK;
 }
 
-// *tuned_ok: the layout is one the tuned kernels take (consecutive chunks only, every offset a
-// multiple of 4 elements)
+// *tuned_ok: the layout is one the tuned kernels take (every offset, and every tiled tensor's
+// column count, a multiple of 4 elements)
 template <int T>
 void fill_table(Table<T>& tb, const sl_layout* L, int chunk, bool* tuned_ok) {
   tb.n_tensors = L->n_tensors;
   const uint32_t side = tile_side(chunk);
-  uint32_t nc = 0;
+  uint32_t nc = 0, nt = 0;
   bool m4 = true, tiled = false;
   for (uint32_t t = 0; t < L->n_tensors; ++t) {
     tb.first_chunk[t] = nc;
+    tb.first_tail[t] = nt;
     tb.offset[t] = L->offset[t];
     tb.cols[t] = L->cols ? (uint32_t)L->cols[t] : 0u;
-    tiled = tiled || tb.cols[t] != 0;
-    m4 = m4 && (L->offset[t] % 4 == 0);
+    m4 = m4 && (L->offset[t] % 4 == 0) && (tb.cols[t] % 4 == 0);
     uint64_t c = 0;
     tensor_chunks(L, t, chunk, side, &c);
     nc += (uint32_t)c;
+    const uint64_t n_t = L->offset[t + 1] - L->offset[t];
+    if (tb.cols[t] == 0) {
+      nt += (n_t % (uint64_t)chunk) != 0 ? 1u : 0u;
+    } else {
+      tiled = true;
+      const uint64_t rows = n_t / tb.cols[t];
+      const uint64_t full = (rows / side) * (tb.cols[t] / side);
+      nt += (uint32_t)(c - full);
+    }
   }
   tb.first_chunk[L->n_tensors] = nc;
+  tb.first_tail[L->n_tensors] = nt;
   tb.offset[L->n_tensors] = L->n_total;
   tb.cols[L->n_tensors] = 0;
   tb.side = tiled ? side : 0;
   m4 = m4 && (L->n_total % 4 == 0);
   tb.n_chunks = nc;
-  *tuned_ok = m4 && !tiled;
+  tb.n_tails = nt;
+  *tuned_ok = m4;
 }
 
 // step = false: Eq. 2 lines 1-4 only.  step = true: the whole of Eq. 2 (theta_global is updated):

@@ -18,7 +18,9 @@ struct Table {
   uint32_t n_tensors;
   uint32_t n_chunks;
   uint32_t side;      // tile side, 0 when no tensor is tiled
+  uint32_t n_tails;   // chunks that are not full (short last chunks, edge tiles)
   uint32_t first_chunk[T + 1];
+  uint32_t first_tail[T + 1];   // not-full chunks owned by tensors before t
   uint32_t cols[T + 1];
   uint64_t offset[T + 1];
 };
@@ -49,14 +51,9 @@ struct ChunkRef {
   }
 };
 
-// chunk g -> its geometry: binary search over the tensors' first chunks
+// geometry of chunk g, which belongs to tensor lo
 template <int T>
-__device__ __forceinline__ ChunkRef locate(const Table<T>& tb, uint32_t g, int chunk) {
-  uint32_t lo = 0, hi = tb.n_tensors;  // first_chunk[lo] <= g < first_chunk[hi]
-  while (hi - lo > 1) {
-    const uint32_t mid = (lo + hi) >> 1;
-    if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
-  }
+__device__ __forceinline__ ChunkRef chunk_of_tensor(const Table<T>& tb, uint32_t lo, uint32_t g, int chunk) {
   ChunkRef c;
   const uint32_t nc = tb.cols[lo];
   const uint32_t in_t = g - tb.first_chunk[lo];
@@ -79,6 +76,54 @@ __device__ __forceinline__ ChunkRef locate(const Table<T>& tb, uint32_t g, int c
     c.side = s;
   }
   return c;
+}
+
+// chunk g -> its geometry: binary search over the tensors' first chunks
+template <int T>
+__device__ __forceinline__ ChunkRef locate(const Table<T>& tb, uint32_t g, int chunk) {
+  uint32_t lo = 0, hi = tb.n_tensors;  // first_chunk[lo] <= g < first_chunk[hi]
+  while (hi - lo > 1) {
+    const uint32_t mid = (lo + hi) >> 1;
+    if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
+  }
+  return chunk_of_tensor(tb, lo, g, chunk);
+}
+
+// the same, trying the tensor of the caller's previous chunk first (t_lo is updated)
+template <int T>
+__device__ __forceinline__ ChunkRef locate_cached(const Table<T>& tb, uint32_t g, int chunk, uint32_t& t_lo) {
+  if (!(tb.first_chunk[t_lo] <= g && g < tb.first_chunk[t_lo + 1])) {
+    uint32_t lo = 0, hi = tb.n_tensors;
+    while (hi - lo > 1) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (tb.first_chunk[mid] <= g) lo = mid; else hi = mid;
+    }
+    t_lo = lo;
+  }
+  return chunk_of_tensor(tb, t_lo, g, chunk);
+}
+
+// the e-th chunk of the arena that is not full (e < n_tails) -> its chunk number.  A tensor with
+// consecutive chunks has at most one (its last); a tiled matrix has its right edge column of
+// tiles (if cols is not a multiple of the side), then its bottom edge row.
+template <int T>
+__device__ __forceinline__ uint32_t tail_chunk(const Table<T>& tb, uint32_t e, int chunk) {
+  uint32_t lo = 0, hi = tb.n_tensors;  // first_tail[lo] <= e < first_tail[hi]
+  while (hi - lo > 1) {
+    const uint32_t mid = (lo + hi) >> 1;
+    if (tb.first_tail[mid] <= e) lo = mid; else hi = mid;
+  }
+  const uint32_t j = e - tb.first_tail[lo];
+  const uint32_t nc = tb.cols[lo];
+  if (nc == 0) return tb.first_chunk[lo + 1] - 1;
+  const uint32_t s = tb.side;
+  const uint64_t rows = (tb.offset[lo + 1] - tb.offset[lo]) / nc;
+  const uint32_t fr = (uint32_t)(rows / s), fc = nc / s;
+  const uint32_t tr = (uint32_t)((rows + s - 1) / s), tc = (nc + s - 1) / s;
+  const uint32_t right = tc > fc ? tr : 0;      // tiles of the right edge column
+  uint32_t tile_r, tile_c;
+  if (j < right) { tile_r = j; tile_c = fc; } else { tile_r = fr; tile_c = j - right; }
+  return tb.first_chunk[lo] + tile_r * tc + tile_c;
 }
 
 // per-replica pointer tables, by value as well

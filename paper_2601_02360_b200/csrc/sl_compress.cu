@@ -143,8 +143,8 @@ __device__ __forceinline__ void block_select_emit(float* ep, const ChunkRef& c, 
 
 // ---------------------------------------------------------------------------
 // Generic kernel.  TAILS = false: CTA b handles chunk b / R of replica b % R.
-// TAILS = true: CTA b handles the short last chunk of tensor b / R (if it has one); this is
-// how the tuned path delegates the ragged ends of the tensors.
+// TAILS = true: CTA b handles the (b / R)-th chunk that is not full (short last chunks, edge
+// tiles); this is how the tuned path delegates the ragged ends of the tensors.
 // ---------------------------------------------------------------------------
 template <int T, bool TAILS>
 __global__ void __launch_bounds__(kThreads)
@@ -158,12 +158,7 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = (int)(blockIdx.x % (uint32_t)a.R);
   uint32_t g = blockIdx.x / (uint32_t)a.R;
-  if (TAILS) {
-    const uint32_t t = g;
-    const uint64_t n_t = a.tb.offset[t + 1] - a.tb.offset[t];
-    if (n_t % (uint64_t)a.chunk == 0) return;     // no short chunk in this tensor
-    g = a.tb.first_chunk[t + 1] - 1;
-  }
+  if (TAILS) g = tail_chunk(a.tb, g, a.chunk);    // the g-th chunk that is not full
   const ChunkRef c = locate(a.tb, g, a.chunk);
   const int len = c.len;
   const int k = a.k, bits = a.bits;
@@ -294,6 +289,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// 16-byte asynchronous copy global -> shared (per thread, any address pattern), and the arrival
+// that makes an mbarrier wait for this thread's copies issued so far
+__device__ __forceinline__ void cp_async_16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void tma_store_1d(void* dst, const void* src, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
@@ -528,9 +531,12 @@ __device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, ui
 // b, b+G, b+2G, ... and walks their items in order: item w is replica w % R of its (w / R)-th chunk.
 template <int T>
 struct ItemCursor {
-  uint32_t g;      // chunk number in the arena
-  uint64_t base;   // element offset of the chunk
-  int r;           // replica
+  uint32_t g;       // chunk number in the arena
+  uint64_t base;    // element offset of the chunk's first element
+  uint32_t stride;  // elements between the chunk's rows of 64: 64 for a consecutive chunk, the matrix's
+                    // row length for a tile
+  uint32_t t_lo;    // tensor of the chunk (lookup cache)
+  int r;            // replica
   bool valid;
 
   // first full chunk at or after g0 (stepping by the grid size)
@@ -538,19 +544,26 @@ struct ItemCursor {
     g = g0;
     valid = false;
     while (g < tb.n_chunks) {
-      const ChunkRef c = locate(tb, g, kC);
-      if (c.len == kC) { base = c.base; valid = true; return; }
-      g += step;                                   // short chunks belong to the tail launch
+      const ChunkRef c = locate_cached(tb, g, kC, t_lo);
+      if (c.len == kC) { base = c.base; stride = c.stride ? c.stride : 64u; valid = true; return; }
+      g += step;                                   // chunks that are not full belong to the tail launch
     }
   }
-  __device__ __forceinline__ void start(const Table<T>& tb, uint32_t b, uint32_t step) { r = 0; seek(tb, b, step); }
+  __device__ __forceinline__ void start(const Table<T>& tb, uint32_t b, uint32_t step) { r = 0; t_lo = 0; seek(tb, b, step); }
   __device__ __forceinline__ void advance(const Table<T>& tb, int n, int R, uint32_t step) {
     r += n;
     while (valid && r >= R) { r -= R; seek(tb, g + step, step); }
   }
 };
 
-template <int T>
+// TILED = false: every full chunk is 16 KB of consecutive memory and moves by TMA bulk copies as
+// described above.  TILED = true (arenas with matrices cut into 64 x 64 tiles): a chunk is 64 rows
+// of 256 bytes, `stride` elements apart.  Bulk copies of 256 bytes run at a third of the rate of
+// 16 KB ones, so here the 256 producer threads fetch theta_local and e themselves with 16-byte
+// cp.async copies (completion through the same mbarriers), two items ahead, and write the
+// residual back with 128-bit streaming stores; the selectors touch shared memory only.  In
+// shared memory a tile is stored row after row, so everything between load and store is the same.
+template <int T, bool TILED>
 __global__ void __launch_bounds__(kFastThreads, 2)
 compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -575,9 +588,9 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 #pragma unroll
     for (int q = 0; q < kSel; ++q) sm.count[q] = 0;
 #pragma unroll
-    for (int s = 0; s < kTlStages; ++s) mbar_init(&sm.full_tl[s], 1);
-#pragma unroll
-    for (int s = 0; s < kEeStages; ++s) mbar_init(&sm.full_ee[s], 1);
+    for (int s = 0; s < kTlStages; ++s) mbar_init(&sm.full_tl[s], TILED ? kThreads : 1);   // TILED: one arrival per
+#pragma unroll                                                                           // producer thread's copies
+    for (int s = 0; s < kEeStages; ++s) mbar_init(&sm.full_ee[s], TILED ? kThreads : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -588,13 +601,29 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     // ======================= producers =======================================
     ItemCursor<T> cur;                            // item w
     cur.start(a.tb, blockIdx.x, G);
-    ItemCursor<T> pf = cur;                       // thread 0: the item whose theta_local is loaded next
-    if (tid == 0) {
-      for (int i = 0; i < kTlStages && pf.valid; ++i) {
+    ItemCursor<T> pf = cur;                       // the item whose theta_local (TILED: and e) is loaded next
+    // TILED: float4 f of a chunk (f = tid + 256 j) is columns 4 (f % 16) .. +3 of row f / 16
+    auto tile_load = [&](const ItemCursor<T>& it, int st_tl, int st_ee) {
+      const float* src_tl = (it.r < kPtrCache ? sm.p_tl[it.r] : a.p.theta_local[it.r]) + it.base;
+      const float* src_ee = (it.r < kPtrCache ? sm.p_err[it.r] : a.p.err[it.r]) + it.base;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int f = tid + 256 * j;
+        const size_t off = (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2);
+        cp_async_16(reinterpret_cast<float4*>(sm.tl[st_tl]) + f, src_tl + off);
+        cp_async_16(reinterpret_cast<float4*>(sm.ee[st_ee]) + f, src_ee + off);
+      }
+      cp_async_arrive(&sm.full_tl[st_tl]);
+      cp_async_arrive(&sm.full_ee[st_ee]);
+    };
+    for (int i = 0; i < kTlStages && pf.valid; ++i) {
+      if (TILED) {
+        tile_load(pf, i, i);
+      } else if (tid == 0) {
         mbar_expect_tx(&sm.full_tl[i], kBytes);
         tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
-        pf.advance(a.tb, 1, R, G);
       }
+      pf.advance(a.tb, 1, R, G);
     }
     const int cwords = bits == 32 ? k : (k * bits) >> 5;   // 32-bit words of codes per chunk
     // This thread's float4s are number t4 + 256 j (j = 0..3) of the chunk, with
@@ -606,13 +635,31 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     const int jsel = 32 - (k + kWarps - 1) / kWarps;   // lane holding the ceil(k/8)-th largest after an ascending sort
     const float beta = a.beta;
     float4 G4[4];                                 // this thread's 16 elements of theta_global
-    if (cur.valid) {
-      const float4* tg4 = reinterpret_cast<const float4*>(a.theta_global + cur.base);
+    // theta_global of a chunk into this thread's registers (float4 f = t4 + 256 j; row f / 16 of a tile)
+    auto load_theta = [&](const ItemCursor<T>& it) {
+      const float* tg = a.theta_global + it.base;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + t4 + 256 * j);
-    }
-    uint32_t g_m1 = 0, g_m2 = 0;                  // chunk and replica of items w-1 and w-2
+      for (int j = 0; j < 4; ++j) {
+        const int f = t4 + 256 * j;
+        const size_t off = TILED ? (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2) : (size_t)f * 4;
+        G4[j] = __ldcs(reinterpret_cast<const float4*>(tg + off));
+      }
+    };
+    if (cur.valid) load_theta(cur);
+    uint32_t g_m1 = 0, g_m2 = 0;                  // chunk, replica (TILED: and place) of items w-1 and w-2
     int r_m1 = 0, r_m2 = 0;
+    uint64_t base_m1 = 0, base_m2 = 0;
+    uint32_t stride_m1 = 64, stride_m2 = 64;
+    // TILED: the residual of a finished item goes back to the error buffer from its stage
+    auto tile_store = [&](int rp, uint64_t base, uint32_t stride, int st_ee) {
+      float* dst = (rp < kPtrCache ? sm.p_err[rp] : a.p.err[rp]) + base;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int f = tid + 256 * j;
+        __stcs(reinterpret_cast<float4*>(dst + (size_t)(f >> 4) * stride + (size_t)((f & 15) << 2)),
+               reinterpret_cast<const float4*>(sm.ee[st_ee])[f]);
+      }
+    };
     __syncwarp();
 
     uint32_t w = 0;
@@ -642,16 +689,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         key[4 * j + 3] = key_of(v.w);
         tmax = max(tmax, max(max(key[4 * j], key[4 * j + 1]), max(key[4 * j + 2], key[4 * j + 3])));
       }
-      fence_async_smem();                         // e' must be visible to the bulk store that drains this stage
+      if (!TILED) fence_async_smem();             // e' must be visible to the bulk store that drains this stage
       // the next item: same chunk, or the next chunk, whose theta_global is requested now (the
       // registers are free) so that it arrives while this item is finished
       ItemCursor<T> nxt = cur;
       nxt.advance(a.tb, 1, R, G);
-      if (nxt.valid && nxt.r == 0) {
-        const float4* tg4 = reinterpret_cast<const float4*>(a.theta_global + nxt.base);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) G4[j] = __ldcs(tg4 + t4 + 256 * j);
-      }
+      if (nxt.valid && nxt.r == 0) load_theta(nxt);
       uint32_t v = tmax;                           // bitonic sort of the 32 thread maxima, ascending over lanes
 #pragma unroll
       for (int size = 2; size <= 32; size <<= 1) {
@@ -682,11 +725,18 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
           }
           if (lane == 0) (pc ? sm.p_scales[r_m2] : a.p.scales[r_m2])[g_m2] = sm.msg_scale[sp];
         }
+        if (TILED) tile_store(r_m2, base_m2, stride_m2, (w - kSel) % kEeStages);
       }
       named_sync(1, kThreads);
-      if (tid == 0 && pf.valid) {                 // every producer has read theta_local(w): its stage takes item w+2's
-        mbar_expect_tx(&sm.full_tl[st], kBytes);
-        tma_load_1d(sm.tl[st], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[st]);
+      if (pf.valid) {
+        // every producer has read theta_local(w) (TILED: and written back the stage of e(w-2)):
+        // the stages take item w+2's
+        if (TILED) {
+          tile_load(pf, st, (w + kTlStages) % kEeStages);
+        } else if (tid == 0) {
+          mbar_expect_tx(&sm.full_tl[st], kBytes);
+          tma_load_1d(sm.tl[st], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[st]);
+        }
         pf.advance(a.tb, 1, R, G);
       }
       uint32_t T1, smax;
@@ -721,8 +771,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       __syncwarp();                               // bar.* is warp-aligned: reconverge first
       named_arrive(2 + q, kPairThreads);          // candidate list q is ready (bar.arrive orders the shared-memory
                                                   // writes before it; a membar here would also wait for global stores)
-      g_m2 = g_m1; r_m2 = r_m1;
-      g_m1 = cur.g; r_m1 = cur.r;
+      g_m2 = g_m1; r_m2 = r_m1; base_m2 = base_m1; stride_m2 = stride_m1;
+      g_m1 = cur.g; r_m1 = cur.r; base_m1 = cur.base; stride_m1 = cur.stride;
       cur = nxt;
     }
     // the last kSel items' messages
@@ -743,6 +793,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         for (int i = lane; i < cwords; i += 32) ocodes[i] = sm.msg_codes[sp][i];
         if (lane == 0) (pc ? sm.p_scales[rp] : a.p.scales[rp])[gp] = sm.msg_scale[sp];
       }
+      if (TILED) tile_store(rp, last ? base_m1 : base_m2, last ? stride_m1 : stride_m2, wp % kEeStages);
     }
   } else {
     // ======================= selectors =======================================
@@ -751,7 +802,9 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     cur.start(a.tb, blockIdx.x, G);
     cur.advance(a.tb, q, R, G);
     ItemCursor<T> pf = cur;                       // the item whose e is loaded next by this selector: w, w+2 at start, then w+4
-    if (lane == 0) {
+    if (TILED) {
+      pf.valid = false;                           // the producers move all the data
+    } else if (lane == 0) {
       for (int i = q; i < kEeStages && pf.valid; i += kSel) {
         mbar_expect_tx(&sm.full_ee[i], kBytes);
         tma_load_1d(sm.ee[i], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes, &sm.full_ee[i]);
@@ -772,7 +825,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       named_sync(2 + q, kPairThreads);            // candidate list q is ready
       // The store of this selector's previous item was issued a whole hand-off ago; once it has
       // read its stage, e of the item four ahead is loaded into it.
-      if (pending_stage >= 0) {
+      if (!TILED && pending_stage >= 0) {
         if (lane == 0) {
           tma_store_wait_read_all();
           if (pf.valid) {
@@ -841,18 +894,18 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         sm.msg_scale[se] = sc;
         if (smax >= 0x7F800000u && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_NONFINITE);
       }
-      fence_async_smem();                         // the patched stage is read by a bulk store
+      if (!TILED) fence_async_smem();             // the patched stage is read by a bulk store
       __syncwarp();
       reinterpret_cast<uint4*>(bitmap)[lane] = make_uint4(0, 0, 0, 0);
-      // ---- E: the stage drains to the error buffer ----
-      if (lane == 0)
+      // ---- E: the stage drains to the error buffer (TILED: the producers write it back) ----
+      if (!TILED && lane == 0)
         tma_store_1d((cur.r < kPtrCache ? sm.p_err[cur.r] : a.p.err[cur.r]) + cur.base, ep, kBytes);
       pending_stage = se;
       __syncwarp();
       named_arrive(4 + q, kPairThreads);          // item w is finished: message final, candidate list free
       cur.advance(a.tb, kSel, R, G);
     }
-    if (lane == 0) tma_store_wait_read_all();      // shared memory must outlive the bulk stores' reads
+    if (!TILED && lane == 0) tma_store_wait_read_all();   // shared memory must outlive the bulk stores' reads
   }
   if (timed_out && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
@@ -879,17 +932,21 @@ cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream
     int dev = 0, sms = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(compress_c4096_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)sizeof(FastSmem));
-    if (e != cudaSuccess) return e;
     // persistent grid: two CTAs per SM, each walking its share of the chunks
     const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * 2u);
-    compress_c4096_kernel<T><<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
-    bool tails = false;
-    for (uint32_t t = 0; t < a.tb.n_tensors; ++t)
-      tails = tails || ((a.tb.offset[t + 1] - a.tb.offset[t]) % (uint64_t)kC) != 0;
-    if (tails)
-      compress_generic_kernel<T, true><<<a.tb.n_tensors * (unsigned)a.R, kThreads, gsmem, st>>>(a);
+    if (a.tb.side != 0) {
+      e = cudaFuncSetAttribute(compress_c4096_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)sizeof(FastSmem));
+      if (e != cudaSuccess) return e;
+      compress_c4096_kernel<T, true><<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
+    } else {
+      e = cudaFuncSetAttribute(compress_c4096_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)sizeof(FastSmem));
+      if (e != cudaSuccess) return e;
+      compress_c4096_kernel<T, false><<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
+    }
+    if (a.tb.n_tails)
+      compress_generic_kernel<T, true><<<a.tb.n_tails * (unsigned)a.R, kThreads, gsmem, st>>>(a);
     return cudaPeekAtLastError();
   }
   const uint64_t blocks = (uint64_t)a.tb.n_chunks * (uint64_t)a.R;
