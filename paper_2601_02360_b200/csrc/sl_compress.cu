@@ -290,14 +290,13 @@ __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-// 16-byte asynchronous copy global -> shared (per thread, any address pattern), and the arrival
-// that makes an mbarrier wait for this thread's copies issued so far
+// 16-byte asynchronous copy global -> shared (per thread, any address pattern); copies are
+// grouped per thread, and a thread can wait until all but its newest N groups have landed
 __device__ __forceinline__ void cp_async_16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_arrive(uint64_t* bar) {
-  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_1d(void* dst, const void* src, uint32_t bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
@@ -320,6 +319,7 @@ struct alignas(16) FastSmem {
   uint16_t kept_pos[kSel][128];
   uint8_t prefix[kSel][kC / 32];      // kept positions before each bitmap word
   uint32_t wmin[kEeStages][kWarps], wmax[kEeStages][kWarps];   // ring: producers run up to three replicas ahead
+  uint32_t tmax_x[kThreads];          // TILED: thread maxima, regrouped before the lower bound is taken
   uint32_t count[kSel];
   const float* p_tl[kPtrCache];       // the first kPtrCache replicas' pointers (parameter-space reads
   float* p_err[kPtrCache];            // with a run-time index are slow)
@@ -560,9 +560,12 @@ struct ItemCursor {
 // described above.  TILED = true (arenas with matrices cut into 64 x 64 tiles): a chunk is 64 rows
 // of 256 bytes, `stride` elements apart.  Bulk copies of 256 bytes run at a third of the rate of
 // 16 KB ones, so here the 256 producer threads fetch theta_local and e themselves with 16-byte
-// cp.async copies (completion through the same mbarriers), two items ahead, and write the
-// residual back with 128-bit streaming stores; the selectors touch shared memory only.  In
-// shared memory a tile is stored row after row, so everything between load and store is the same.
+// cp.async copies, two items ahead, and write the residual back with 128-bit streaming stores;
+// the selectors touch shared memory only.  Every thread copies exactly the float4s it will read
+// in phase A, so completion is a per-thread cp.async.wait_group and needs no barrier (256
+// per-thread arrivals on one mbarrier were tried first: they serialise and cost more than the
+// copies).  In shared memory a tile is stored row after row, so everything between load and
+// store is the same.
 template <int T, bool TILED>
 __global__ void __launch_bounds__(kFastThreads, 2)
 compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
@@ -588,9 +591,9 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 #pragma unroll
     for (int q = 0; q < kSel; ++q) sm.count[q] = 0;
 #pragma unroll
-    for (int s = 0; s < kTlStages; ++s) mbar_init(&sm.full_tl[s], TILED ? kThreads : 1);   // TILED: one arrival per
-#pragma unroll                                                                           // producer thread's copies
-    for (int s = 0; s < kEeStages; ++s) mbar_init(&sm.full_ee[s], TILED ? kThreads : 1);
+    for (int s = 0; s < kTlStages; ++s) mbar_init(&sm.full_tl[s], 1);
+#pragma unroll
+    for (int s = 0; s < kEeStages; ++s) mbar_init(&sm.full_ee[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -601,37 +604,39 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     // ======================= producers =======================================
     ItemCursor<T> cur;                            // item w
     cur.start(a.tb, blockIdx.x, G);
-    ItemCursor<T> pf = cur;                       // the item whose theta_local (TILED: and e) is loaded next
-    // TILED: float4 f of a chunk (f = tid + 256 j) is columns 4 (f % 16) .. +3 of row f / 16
-    auto tile_load = [&](const ItemCursor<T>& it, int st_tl, int st_ee) {
-      const float* src_tl = (it.r < kPtrCache ? sm.p_tl[it.r] : a.p.theta_local[it.r]) + it.base;
-      const float* src_ee = (it.r < kPtrCache ? sm.p_err[it.r] : a.p.err[it.r]) + it.base;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int f = tid + 256 * j;
-        const size_t off = (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2);
-        cp_async_16(reinterpret_cast<float4*>(sm.tl[st_tl]) + f, src_tl + off);
-        cp_async_16(reinterpret_cast<float4*>(sm.ee[st_ee]) + f, src_ee + off);
-      }
-      cp_async_arrive(&sm.full_tl[st_tl]);
-      cp_async_arrive(&sm.full_ee[st_ee]);
-    };
-    for (int i = 0; i < kTlStages && pf.valid; ++i) {
-      if (TILED) {
-        tile_load(pf, i, i);
-      } else if (tid == 0) {
-        mbar_expect_tx(&sm.full_tl[i], kBytes);
-        tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
-      }
-      pf.advance(a.tb, 1, R, G);
-    }
-    const int cwords = bits == 32 ? k : (k * bits) >> 5;   // 32-bit words of codes per chunk
     // This thread's float4s are number t4 + 256 j (j = 0..3) of the chunk, with
     // t4 = 64 (lane / 8) + 8 warp + lane % 8: every 8 lanes read 128 contiguous bytes (no bank
     // conflicts), and every warp samples each of the sixteen 256-element regions of the chunk
     // with 32 elements, so a row boundary inside the chunk (rows of very different scale) cannot
     // leave a warp with small values only, which would ruin the lower bound below.
     const int t4 = ((lane >> 3) << 6) + (warp << 3) + (lane & 7);
+    ItemCursor<T> pf = cur;                       // the item whose theta_local (TILED: and e) is loaded next
+    // TILED: float4 f of a chunk is columns 4 (f % 16) .. +3 of row f / 16; a thread copies the
+    // float4s t4 + 256 j it will read itself (one group of copies per item)
+    auto tile_load = [&](const ItemCursor<T>& it, int st_tl, int st_ee) {
+      const float* src_tl = (it.r < kPtrCache ? sm.p_tl[it.r] : a.p.theta_local[it.r]) + it.base;
+      const float* src_ee = (it.r < kPtrCache ? sm.p_err[it.r] : a.p.err[it.r]) + it.base;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int f = t4 + 256 * j;
+        const size_t off = (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2);
+        cp_async_16(reinterpret_cast<float4*>(sm.tl[st_tl]) + f, src_tl + off);
+        cp_async_16(reinterpret_cast<float4*>(sm.ee[st_ee]) + f, src_ee + off);
+      }
+    };
+    for (int i = 0; i < kTlStages; ++i) {
+      if (pf.valid) {
+        if (TILED) {
+          tile_load(pf, i, i);
+        } else if (tid == 0) {
+          mbar_expect_tx(&sm.full_tl[i], kBytes);
+          tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
+        }
+        pf.advance(a.tb, 1, R, G);
+      }
+      if (TILED) cp_async_commit();               // one group per item, empty ones included, keeps the count uniform
+    }
+    const int cwords = bits == 32 ? k : (k * bits) >> 5;   // 32-bit words of codes per chunk
     const int jsel = 32 - (k + kWarps - 1) / kWarps;   // lane holding the ceil(k/8)-th largest after an ascending sort
     const float beta = a.beta;
     float4 G4[4];                                 // this thread's 16 elements of theta_global
@@ -666,8 +671,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 #pragma unroll 1
     for (; cur.valid; ++w) {
       const int st = w % kTlStages, se = w % kEeStages, q = w % kSel;
-      if (!mbar_wait(&sm.full_tl[st], (w / kTlStages) & 1u)) timed_out = true;
-      if (!mbar_wait(&sm.full_ee[se], (w / kEeStages) & 1u)) timed_out = true;
+      if (TILED) {
+        cp_async_wait_but_one();                  // this thread's copies for item w have landed (item w+1's may fly)
+      } else {
+        if (!mbar_wait(&sm.full_tl[st], (w / kTlStages) & 1u)) timed_out = true;
+        if (!mbar_wait(&sm.full_ee[se], (w / kEeStages) & 1u)) timed_out = true;
+      }
       const float4* tl4 = reinterpret_cast<const float4*>(sm.tl[st]);
       float4* ee4 = reinterpret_cast<float4*>(sm.ee[se]);
       // ---- A ----
@@ -695,7 +704,17 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       ItemCursor<T> nxt = cur;
       nxt.advance(a.tb, 1, R, G);
       if (nxt.valid && nxt.r == 0) load_theta(nxt);
-      uint32_t v = tmax;                           // bitonic sort of the 32 thread maxima, ascending over lanes
+      uint32_t v = tmax;
+      if (TILED) {
+        // In a tile every row of the matrix has its own scale and a warp's float4s cover only 16 of
+        // the 64 rows, so the per-warp bound below could be taken over small rows only.  Regroup:
+        // group `warp` takes the maxima of threads 8 lane + warp, one from every warp and every
+        // row phase, so each group samples all 64 rows.
+        sm.tmax_x[tid] = tmax;
+        named_sync(1, kThreads);
+        v = sm.tmax_x[8 * lane + warp];
+      }
+      // bitonic sort of the group's 32 thread maxima, ascending over lanes
 #pragma unroll
       for (int size = 2; size <= 32; size <<= 1) {
 #pragma unroll
@@ -705,7 +724,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
           v = (up == lower) ? min(v, o) : max(v, o);
         }
       }
-      const uint32_t wmin = __shfl_sync(kFull, v, jsel);     // this warp's ceil(k/8)-th largest thread maximum
+      const uint32_t wmin = __shfl_sync(kFull, v, jsel);     // this group's ceil(k/8)-th largest thread maximum
       const uint32_t wmax = __shfl_sync(kFull, v, 31);
       if (lane == 0) { sm.wmin[se][warp] = wmin; sm.wmax[se][warp] = wmax; }
       if (w >= (uint32_t)kSel) {
@@ -739,6 +758,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         }
         pf.advance(a.tb, 1, R, G);
       }
+      if (TILED) cp_async_commit();
       uint32_t T1, smax;
       {
         const uint4 m0 = reinterpret_cast<const uint4*>(sm.wmin[se])[0], m1 = reinterpret_cast<const uint4*>(sm.wmin[se])[1];
