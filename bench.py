@@ -345,6 +345,68 @@ def run_e2e(st: DeviceState, steps: int, world: int):
     return float(np.mean(times)), h2d, d2h, note
 
 
+def run_exchange(args) -> None:
+    """Replica-per-GPU form (the paper's deployment): every rank hosts ONE replica of the same
+    parameter set; a step = sl_compress of the own replica, NCCL all-gather of the sparse
+    messages, sl_aggregate_apply on the own copy of theta_global.  R = number of ranks."""
+    import torch.distributed as dist
+    from paper_2601_02360_b200 import api, exchange
+    rank, local, world = dist_env()
+    assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torchrun"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29500")
+    if not dist.is_initialized():
+        dist.init_process_group(backend="nccl", rank=rank, world_size=world, device_id=dev)
+    wl = synth.workload(args.workload).replace(R=world)
+    if args.k:
+        wl = wl.replace(k=args.k)
+    if args.first_tensors:
+        wl = synth.sub_arena(wl, list(range(args.first_tensors)), f"{wl.name}[:{args.first_tensors}]")
+    lay = api.Layout(wl.offsets())
+    theta_global = synth.gen_theta_global(wl, dev, args.seed)          # the same on every rank
+    rho = synth.row_scales(wl, args.seed)
+    theta_local = torch.empty_like(theta_global)
+    err = torch.zeros_like(theta_global)
+    idx, codes, scales = api.alloc_messages(lay, wl.chunk, wl.k, wl.bits, 1, dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    times = []
+    for s in range(args.warmup + args.steps):
+        synth.gen_theta_local(wl, theta_global, s, rank, args.seed, out=theta_local, rho=rho)
+        if s == args.warmup:
+            dist.barrier()
+            torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        exchange.outer_step_replica(theta_local, theta_global, err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
+                                    wl.outer_lr, idx[0], codes[0], scales[0], flags)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            times.append(e0.elapsed_time(e1))
+    dist.barrier()
+    ms = max_over_ranks(float(np.sum(times)), world, dev) / args.steps
+    # every rank must hold the same parameters after the step
+    chk = theta_global.double().sum().reshape(1)
+    lo, hi = chk.clone(), chk.clone()
+    dist.all_reduce(lo, op=dist.ReduceOp.MIN)
+    dist.all_reduce(hi, op=dist.ReduceOp.MAX)
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": wl.n_total / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "params": wl.n_total, "R": world, "k": wl.k, "bits": wl.bits,
+                       "chunk": wl.chunk, "mode": "one replica per GPU, NCCL all-gather of the sparse messages",
+                       "message_bytes_per_replica": exchange.message_bytes(idx[0], codes[0], scales[0])},
+            "replicas_agree": bool(lo.item() == hi.item()), "device_flags": int(flags.item()),
+            "gpu_launches": 4 * args.steps}))
+    dist.destroy_process_group()
+
+
 def run_ours(args) -> None:
     from paper_2601_02360_b200 import api
     rank, local, world = init_dist("nccl")
@@ -459,6 +521,9 @@ def main() -> None:
     ap.add_argument("--k", type=int, default=0)
     ap.add_argument("--first-tensors", type=int, default=0,
                     help="keep only the first N tensors of the workload (small cases for profiling)")
+    ap.add_argument("--exchange", action="store_true",
+                    help="replica-per-GPU form: every rank hosts one replica and the sparse messages are "
+                         "all-gathered over NCCL (R = number of ranks); not the default bench line")
     ap.add_argument("--tiles", action="store_true",
                     help="cut matrices into square tiles of `chunk` elements instead of consecutive chunks")
     ap.add_argument("--variant", default="plain", choices=["plain", "ties_literal", "ties_dyadic"],
@@ -470,6 +535,8 @@ def main() -> None:
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.exchange:
+        run_exchange(args)
     else:
         run_ours(args)
 

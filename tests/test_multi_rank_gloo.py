@@ -65,3 +65,55 @@ def test_reference_arm_prints_once_under_two_ranks():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
+
+
+def _exchange_worker(rank, world, port, out):
+    """Each rank hosts one replica: its message is made by the CPU checker, exchanged with the
+    package's gather, and averaged by the checker on every rank."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from oracle import slo
+    from paper_2601_02360_b200 import exchange, synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = synth.workload("tiny").replace(R=world)
+    off = wl.offsets()
+    tg = synth.gen_theta_global(wl).numpy().copy()
+    tl = synth.gen_theta_local(wl, torch.from_numpy(tg), 0, rank).numpy()
+    err = np.zeros(wl.n_total, np.float32)
+    i, c, s, _ = slo.compress(tl, tg, err, off, wl.beta, wl.chunk, wl.k, wl.bits)
+    gi, gc, gs = exchange.all_gather_messages(torch.from_numpy(i), torch.from_numpy(c), torch.from_numpy(s))
+    msgs = [(a.numpy(), b.numpy(), d.numpy()) for a, b, d in zip(gi, gc, gs)]
+    upd = slo.aggregate(msgs, off, wl.chunk, wl.k, wl.bits)
+    slo.outer_apply(tg, upd, wl.outer_lr)
+    sent = exchange.message_bytes(torch.from_numpy(i), torch.from_numpy(c), torch.from_numpy(s))
+    out.put((rank, tg.tobytes(), sent))
+    dist.barrier()
+
+
+def test_replica_per_rank_exchange_gives_every_rank_the_single_process_result():
+    import numpy as np
+    import torch
+    from oracle import slo
+    from paper_2601_02360_b200 import synth
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_exchange_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=180) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    # the same step in one process
+    wl = synth.workload("tiny").replace(R=2)
+    tg = synth.gen_theta_global(wl).numpy().copy()
+    tls = [synth.gen_theta_local(wl, torch.from_numpy(tg), 0, r).numpy() for r in range(2)]
+    errs = [np.zeros(wl.n_total, np.float32) for _ in range(2)]
+    slo.outer_round(tls, tg, errs, wl.offsets(), wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr)
+    assert res[0][1] == res[1][1] == tg.tobytes()
+    assert res[0][2] == wl.n_chunks() * (2 * wl.k + wl.k * wl.bits // 8 + 4)

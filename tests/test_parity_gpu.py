@@ -379,3 +379,31 @@ def test_more_chunks_than_resident_ctas():
     run_and_compare([0, n], tg, tls, errs, 0.95, 4096, 64, 2, 1.0, rounds=2,
                     next_locals=lambda t, g: [(g + np.random.default_rng(t * 10 + r).normal(0, 1e-3, g.size)).astype(f32)
                                               for r in range(3)], what="1500 chunks")
+
+
+def test_replica_per_rank_step_on_one_gpu():
+    # world size 1: the exchange degenerates to a copy, the step must equal the single-replica step
+    import torch.distributed as dist
+    from paper_2601_02360_b200 import exchange
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    try:
+        wl = synth.workload("tiny").replace(R=1)
+        tgt = synth.gen_theta_global(wl)
+        tl = synth.gen_theta_local(wl, tgt, 0, 0)
+        gs = GpuStep(wl.offsets(), 1, wl.chunk, wl.k, wl.bits)
+        gs.upload(tgt.numpy(), [tl.numpy()])
+        # gloo moves host tensors: gather through the host, aggregate on the device
+        api.sl_compress(gs.theta_local[0], gs.theta_global, gs.err[0], gs.layout, wl.beta, wl.chunk, wl.k, wl.bits,
+                        gs.idx[0], gs.codes[0], gs.scales[0], gs.flags)
+        torch.cuda.synchronize()
+        gi, gc, gsc = exchange.all_gather_messages(gs.idx[0].cpu(), gs.codes[0].cpu(), gs.scales[0].cpu())
+        d = lambda ts: [t.cuda() for t in ts]
+        api.sl_aggregate_apply(d(gi), d(gc), d(gsc), gs.layout, wl.chunk, wl.k, wl.bits, gs.theta_global, wl.outer_lr, gs.flags)
+        want = tgt.numpy().copy()
+        slo.outer_round([tl.numpy()], want, [np.zeros(wl.n_total, f32)], wl.offsets(), wl.beta, wl.chunk, wl.k,
+                        wl.bits, wl.outer_lr)
+        assert_close(gs.theta_global.cpu().numpy(), want, "replica-per-rank, world 1")
+    finally:
+        dist.destroy_process_group()
