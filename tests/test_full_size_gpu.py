@@ -82,3 +82,68 @@ def test_1b_workload_sampled_chunks_two_rounds(fused):
             want = tg_in[ci].copy()
             slo.outer_apply(want, upd, wl.outer_lr)
             assert_close(tg_out[ci], want, f"round {rnd} chunk {g} theta_global")
+
+
+def test_1b_workload_with_tiles_sampled_tiles():
+    """The same workload with every matrix cut into 64 x 64 tiles (the tuned tile kernels at full
+    size): sampled tiles of every kind of matrix against the checker, one replica set, one round."""
+    free, _ = torch.cuda.mem_get_info()
+    wl = synth.workload("1b")
+    need = (2 * wl.R + 1) * wl.n_total * 4 + (2 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    dev = torch.device("cuda", 0)
+    st = bench.DeviceState(wl, 0, dev, tiles=True)
+    st.redraw_locals(0)
+    for r in range(wl.R):                      # a non-trivial error buffer
+        st.err[r].normal_(0.0, 5e-4)
+    off = wl.offsets()
+    rng = np.random.default_rng(3)
+    # (tensor, tile row, tile col) samples: first / last / random tiles of the first layer's matrices and the embedding
+    picks = []
+    first_chunk = 0
+    chunk_of = {}
+    for ti, (_, rows, cols) in enumerate(wl.tensors):
+        n_t = rows * cols
+        if rows > 1:
+            tr, tc = rows // 64, cols // 64
+            chunk_of[ti] = (first_chunk, tr, tc)
+            first_chunk += tr * tc
+        else:
+            first_chunk += -(-n_t // wl.chunk)
+    for ti in [0, 4, 6, len(wl.tensors) - 2, 9 * 7 + 5]:
+        fc, tr, tc = chunk_of[ti]
+        cand = {(0, 0), (tr - 1, tc - 1), (0, tc - 1)} | {(int(rng.integers(tr)), int(rng.integers(tc))) for _ in range(5)}
+        picks += [(ti, a, b) for a, b in sorted(cand)]
+    stride = st.api.sl_codes_stride(wl.k, wl.bits)
+
+    def block(t, ti, a, b):
+        _, rows, cols = wl.tensors[ti]
+        m = t[int(off[ti]):int(off[ti + 1])].view(rows, cols)
+        return m[a * 64:(a + 1) * 64, b * 64:(b + 1) * 64]
+
+    ins = [(block(st.theta_global, *p).cpu().numpy().copy(),
+            [block(st.theta_local[r], *p).cpu().numpy().copy() for r in range(wl.R)],
+            [block(st.err[r], *p).cpu().numpy().copy() for r in range(wl.R)]) for p in picks]
+    st.compress()
+    st.aggregate_apply()
+    torch.cuda.synchronize()
+    assert int(st.flags.item()) == 0
+    for (ti, a, b), (tg_in, tl_in, e_in) in zip(picks, ins):
+        fc, tr, tc = chunk_of[ti]
+        g = fc + a * tc + b
+        msgs = []
+        for r in range(wl.R):
+            e = e_in[r].reshape(-1).copy()
+            i_o, c_o, s_o, _ = slo.compress(tl_in[r].reshape(-1), tg_in.reshape(-1), e, [0, 4096], wl.beta, wl.chunk,
+                                            wl.k, wl.bits, cols=[64])
+            msgs.append((i_o, c_o, s_o))
+            what = f"tensor {ti} tile ({a},{b}) replica {r}"
+            assert_exact(st.idx[r][g * wl.k:(g + 1) * wl.k].cpu().numpy(), i_o[0], what + " idx")
+            assert_exact(st.codes[r][g * stride:(g + 1) * stride].cpu().numpy(), c_o[0], what + " codes")
+            assert_close(st.scales[r][g:g + 1].cpu().numpy(), s_o, what + " scale")
+            assert_close(block(st.err[r], ti, a, b).cpu().numpy().reshape(-1), e, what + " err")
+        upd = slo.aggregate(msgs, [0, 4096], wl.chunk, wl.k, wl.bits, cols=[64])
+        want = tg_in.reshape(-1).copy()
+        slo.outer_apply(want, upd, wl.outer_lr)
+        assert_close(block(st.theta_global, ti, a, b).cpu().numpy().reshape(-1), want, f"tensor {ti} tile ({a},{b}) theta_global")
