@@ -5,10 +5,11 @@
 //   compress_generic_kernel  any chunk length / k / code width / alignment, consecutive chunks or
 //                            square tiles; one CTA per (chunk, replica); exact 4-pass radix
 //                            select in shared memory.
-//   compress_c4096_kernel    the tuned path for full 4096-element chunks, k <= 128: one CTA per
-//                            chunk walks all R replicas with theta_global held in registers, a
-//                            cheap lower bound on the k-th magnitude prunes the chunk to a few
-//                            hundred candidates, one warp finishes the exact selection.
+//   compress_c4096_kernel    the tuned path for full 4096-element chunks, k <= 128: persistent
+//                            warp-specialised CTAs walk (chunk, replica) items with theta_global
+//                            held in registers, a cheap lower bound on the k-th magnitude prunes
+//                            the chunk to about a hundred candidates, a selector warp finishes
+//                            the exact selection while the producers work on the next items.
 #include <algorithm>
 
 #include "sl_common.cuh"
@@ -210,29 +211,35 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 // ---------------------------------------------------------------------------
 // Tuned kernel: chunk = 4096, k <= 128, (k * bits) % 32 == 0, 16-byte aligned arena.
 //
-// One CTA per chunk walks all R replicas; theta_global stays in registers.  The CTA is warp
-// specialised: 8 producer warps (256 threads) and kSel selector warps; selector q handles the
-// replicas r with r % kSel == q, so two selections are in flight while the producers run ahead.
+// Persistent grid of two CTAs per SM.  CTA b of G owns the full chunks among b, b+G, b+2G, ... and
+// walks their (chunk, replica) pairs - "items" - as one continuous stream: item w is replica
+// w % R of the CTA's (w / R)-th chunk, so the pipeline below never drains between chunks.
+// theta_global of the current chunk stays in registers (one trip through memory per chunk for
+// all R replicas); the next chunk's is requested as soon as the last replica has used them.
+// The CTA is warp specialised: 8 producer warps (256 threads) and kSel selector warps; selector q
+// handles the items w with w % kSel == q, so two selections are in flight while the producers
+// run ahead.
 //
-//  * All bulk data moves by TMA (cp.async.bulk, no multicast), issued by producer thread 0:
-//    theta_local of replica r is loaded two replicas ahead into a 2-deep ring (dead after phase
-//    A); e lives in a 4-deep ring whose stages cycle through load -> produce -> select -> drain:
-//    e(r+1) is loaded while replica r is produced, replica r-1 is being selected, and the stage
-//    of replica r-2, patched with the residual, drains to the error buffer as one bulk store.
-//    Nobody waits for a store it has just issued: under a saturated memory system a 16 KB store
-//    takes microseconds to drain, and a warp with ordinary global stores in flight also stalls
-//    on its next shared-memory access.  So the selectors issue no global stores at all.
-//  * Producers, per replica (a thread owns four float4s of the chunk, 256 float4s apart):
+//  * Bulk data moves by TMA (cp.async.bulk + mbarrier complete_tx, no multicast).  theta_local of
+//    item w+2 is loaded by producer thread 0 into a 2-deep ring (a stage is dead after phase A).
+//    e lives in a 4-deep ring: loaded four items ahead by the selector that owns the stage,
+//    overwritten in place with e' by the producers, patched with the residual by the selector,
+//    and sent back to the error buffer as ONE bulk store by that selector.  Under a saturated
+//    memory system such a store takes microseconds to drain, so nobody waits for a store it has
+//    just issued: the selector checks it only at the start of its next item, where it idles at a
+//    barrier anyway, and then refills the stage.
+//  * Producers, per item (a thread owns four float4s of the chunk, 256 float4s apart):
 //      A  e' = fma(beta, e, theta_global - theta_local), written in place of e in the stage;
 //         per-thread maximum key.  Every warp sorts its 32 thread maxima (bitonic network of
 //         shuffles) and takes the j-th largest, j = ceil(k/8): at least j keys of the warp's 512
 //         are >= it, so at least 8j >= k keys of the chunk are >= T1 = the smallest of the eight
 //         values: T1 is a lower bound of the k-th largest key.
-//      B  the keys >= T1 (about a hundred for k = 64) are compacted into a candidate list and
+//      B  the keys >= T1 (about a hundred for k = 64) are appended to a candidate list and
 //         counted in a 256-bin histogram of the key range [T1, max].
-//      E  replica r-2, finished by its selector in the meantime: warp 0 copies its message from
-//         shared memory to idx / codes / scales, thread 0 issues the bulk store of its stage.
-//  * Selector, per replica:
+//      E  item w-2, finished by its selector in the meantime: warp 0 copies its message from
+//         shared memory to idx / codes / scales (three coalesced stores; the selectors issue no
+//         ordinary global stores).
+//  * Selector, per item:
 //      C  a suffix scan of the histogram finds the bin that holds the k-th largest key; a
 //         bisection inside that bin (candidates in registers) finds a threshold that leaves
 //         exactly k candidates; if the range collapses first the k-th key is tied, and the
@@ -244,10 +251,12 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 //  If the candidate list overflows (tie-heavy or constant chunks) the selector runs an exact
 //  warp-wide radix select over the whole chunk instead of C.
 //
-// Hand-offs: named barrier 1 = producers only; 2+q = candidate list q ready (producers
-// arrive, selector q waits); 4+q = selector q has finished a replica: its candidate list is free
-// and the stage holds the final residual (selector q arrives, producers wait).  Every mbarrier wait is bounded; running out raises SL_FLAG_TIMEOUT and the kernel
-// carries on (no trap, no hang).
+// Hand-offs: named barrier 1 = producers only; 2+q = candidate list q ready (producers arrive,
+// selector q waits); 4+q = selector q has finished an item: message final, candidate list free
+// (selector q arrives, producers wait).  bar.arrive / bar.sync order the shared-memory accesses
+// around them (the producer/consumer idiom of the PTX manual), so no membar is used: it would
+// also wait for global stores in flight.  Every mbarrier wait is bounded; running out raises
+// SL_FLAG_TIMEOUT and the kernel carries on (no trap, no hang).
 // ---------------------------------------------------------------------------
 constexpr int kC = 4096;
 constexpr int kSel = 2;               // selector warps
@@ -270,8 +279,7 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// bounded wait on a phase; false = gave up.  test_wait + nanosleep rather than try_wait: a
-// suspended try_wait was seen to delay the shared-memory instructions of other warps.
+// bounded wait on a phase; false = gave up (non-blocking test_wait with a short sleep between polls)
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   const uint32_t addr = smem_u32(bar);
   for (uint32_t it = 0; it < kWaitLimit; ++it) {
