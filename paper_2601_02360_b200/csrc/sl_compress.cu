@@ -942,7 +942,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 
 template <int T>
 bool compress_is_tuned(const CompressArgs<T>& a, bool aligned16) {
-  return aligned16 && a.chunk == kC && a.k <= 128 && ((a.k * a.bits) % 32) == 0;
+  // even k: the message's positions leave shared memory as 32-bit words
+  return aligned16 && a.chunk == kC && a.k <= 128 && ((a.k * a.bits) % 32) == 0 && (a.k % 2) == 0;
 }
 
 template <int T>

@@ -80,7 +80,8 @@ def test_ragged_multi_tensor_arena(chunk, k, bits):
     run_and_compare(off, tg, tls, errs, 0.95, chunk, k, bits, 0.8, what=f"ragged C{chunk} k{k} b{bits}")
 
 
-@pytest.mark.parametrize("k,bits", [(16, 2), (32, 2), (64, 2), (128, 2), (64, 4), (64, 8), (32, 32)])
+@pytest.mark.parametrize("k,bits", [(16, 2), (32, 2), (64, 2), (128, 2), (64, 4), (64, 8), (32, 32), (5, 32), (7, 32),
+                                    (6, 32), (8, 4), (4, 8), (2, 32), (128, 32), (128, 8)])
 def test_aligned_arena_fast_path_shapes(k, bits):
     # every tensor a multiple of 4 elements (the layout the tuned kernels accept), short tails included
     sizes = [5 * 4096, 1024, 4096 + 2048, 512, 4, 3 * 4096 + 4092, 4096]
