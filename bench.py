@@ -407,6 +407,81 @@ def run_exchange(args) -> None:
     dist.destroy_process_group()
 
 
+def run_embed(args) -> None:
+    """The step right after the outer step for replicas that compress activations (§2.4, Eqs. 3-4):
+    sl_embed_reproject on the token-embedding table of the chosen model (vocab x d, k = d/8, the
+    paper's 87.5 % setting).  One GPU; its own JSON line, not the default bench line."""
+    from paper_2601_02360_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = synth.workload(args.workload)
+    name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
+    k = args.k or d // 8
+    U = torch.from_numpy(synth.gen_subspace_basis(d, k, args.seed)).to(dev)
+    T_S_h, T_perp_h = synth.gen_embedding_pair(V, d, args.seed)
+    T_S0 = torch.from_numpy(T_S_h).to(dev)
+    T_S, T_perp = T_S0.clone(), torch.from_numpy(T_perp_h).to(dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(0)
+    times = []
+    for s in range(args.warmup + args.steps):
+        T_S.copy_(T_S0)                      # a table that has drifted out of the subspace again
+        torch.cuda.synchronize()
+        if s == args.warmup:
+            sampler.start()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        api.sl_embed_reproject(T_S, T_perp, U, V, d, k, flags)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            times.append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
+    ms = float(np.mean(times))
+    alg_bytes = 16 * V * d + 4 * d * k      # read T_S and T_perp, write both, read U once
+    flops = 4 * V * d * k
+    peak, peak_src = measured_peak_gbs()
+    line = {
+        "metric": "embed_reproject_rows_per_s", "value": V / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "tf32 contraction, f32 update", "data": "synthetic",
+        "config": {"workload": f"{wl.name} token embedding {V}x{d}, k={k}",
+                   "l2": "the two tables (2 x %.0f MB) exceed the 126 MB L2" % (V * d * 4 / 1e6)},
+        "roofline": {"bound": "hbm", "achieved": alg_bytes / (ms * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak, "traffic": None, "peak_source": peak_src,
+                     "algorithmic_bytes": alg_bytes, "tensor_tflops": flops / (ms * 1e-3) / 1e12},
+        "clocks": clocks, "device_flags": int(flags.item()), "gpu_launches": args.steps,
+    }
+    if not args.no_e2e:
+        hs, hp = torch.from_numpy(T_S_h).pin_memory(), torch.from_numpy(T_perp_h).pin_memory()
+        t_e2e = []
+        for _ in range(max(1, args.e2e_steps)):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            T_S.copy_(hs, non_blocking=True)
+            T_perp.copy_(hp, non_blocking=True)
+            api.sl_embed_reproject(T_S, T_perp, U, V, d, k, flags)
+            hs.copy_(T_S, non_blocking=True)
+            hp.copy_(T_perp, non_blocking=True)
+            torch.cuda.synchronize()
+            t_e2e.append(time.perf_counter() - t0)
+        e = float(np.mean(t_e2e))
+        line["e2e"] = {"value": V / e, "unit": "rows/s", "ms": e * 1e3, "h2d_bytes_per_step": 8 * V * d,
+                       "d2h_bytes_per_step": 8 * V * d}
+    if not args.no_cpu:
+        from oracle import embed as oe
+        rows = min(V, 4000)
+        Uh = U.cpu().numpy()
+        t0 = time.perf_counter()
+        oe.embed_reproject(T_S_h[:rows], T_perp_h[:rows], Uh)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": rows / dt, "unit": "rows/s", "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"first {rows} rows of the table, float64 numpy"}
+    print(json.dumps(line))
+
+
 def run_ours(args) -> None:
     from paper_2601_02360_b200 import api
     rank, local, world = init_dist("nccl")
@@ -524,6 +599,9 @@ def main() -> None:
     ap.add_argument("--exchange", action="store_true",
                     help="replica-per-GPU form: every rank hosts one replica and the sparse messages are "
                          "all-gathered over NCCL (R = number of ranks); not the default bench line")
+    ap.add_argument("--embed", action="store_true",
+                    help="time sl_embed_reproject (token-embedding adaptation, Eqs. 3-4) on the model's "
+                         "embedding table instead of the outer step; one GPU, its own JSON line")
     ap.add_argument("--tiles", action="store_true",
                     help="cut matrices into square tiles of `chunk` elements instead of consecutive chunks")
     ap.add_argument("--variant", default="plain", choices=["plain", "ties_literal", "ties_dyadic"],
@@ -535,6 +613,8 @@ def main() -> None:
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.embed:
+        run_embed(args)
     elif args.exchange:
         run_exchange(args)
     else:

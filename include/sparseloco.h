@@ -145,6 +145,22 @@ int sl_outer_step(int R, const float* const* theta_local, float* theta_global, f
                   uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
                   void* stream);
 
+/* Token-embedding adaptation applied after every outer synchronisation (paper section 2.4,
+ * Eqs. 3-4).  The embedding table is kept as TE = T_S + T_perp; U (section 2.3) spans the
+ * compression subspace S, and Pi_S(t) = t U U^T for a row t.  In place:
+ *     T_perp[v,:] <- T_perp[v,:] + (T_S[v,:] - Pi_S(T_S[v,:]))
+ *     T_S[v,:]    <- Pi_S(T_S[v,:])                                  for v < V.
+ * T_S, T_perp: DEVICE, float32, V x d row-major, read and written.  U: DEVICE, float32, d x k
+ * row-major (orthonormal columns; not checked), read only.  All three 16-byte aligned.
+ * The two contractions run on the tensor cores in TF32 (operands cut to 10 mantissa bits,
+ * float32 accumulation); the subtraction and the addition are float32, each rounded once, and
+ * use the very value that is stored to T_S, so T_S + T_perp is conserved to float32 rounding.
+ * Needs d % 4 == 0, k % 4 == 0, 4 <= k <= 256, V >= 1 (else SL_ERR_UNSUPPORTED); V = 0 is a
+ * no-op.  `flags` (DEVICE, may be NULL) receives SL_FLAG_TIMEOUT if an internal wait gave up,
+ * in which case the tables' contents are unspecified.  Asynchronous on `stream`. */
+int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
+                       uint32_t* flags, void* stream);
+
 /* Static description of an SL_* return code. */
 const char* sl_strerror(int code);
 

@@ -209,5 +209,7 @@ template <int T> bool compress_is_tuned(const CompressArgs<T>& a, bool aligned16
 template <int T> cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned16, cudaStream_t st);
 template <int T> cudaError_t launch_aggregate_tails(const AggregateArgs<T>& a, bool apply, cudaStream_t st);
 cudaError_t launch_outer_apply(float* theta, const float* update, uint64_t n, float lr, cudaStream_t st);
+cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
+                                   uint32_t* flags, cudaStream_t st);
 
 }  // namespace sl

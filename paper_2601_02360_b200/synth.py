@@ -227,3 +227,23 @@ def sample_chunks(wl: Workload, n: int, seed: int = 0) -> List[Tuple[int, int, i
         s = lo + c * wl.chunk
         out.append((gc, s, min(wl.chunk, lo + sz - s)))
     return out
+
+
+# ---------------------------------------------------------------------------
+# inputs of the token-embedding adaptation (paper §2.3-2.4)
+# ---------------------------------------------------------------------------
+def gen_subspace_basis(d: int, k: int, seed: int = 0) -> np.ndarray:
+    """U (d x k, float32): a Gaussian matrix orthonormalised by QR, as §2.3 describes its creation."""
+    rng = np.random.default_rng(_mix(0x5B5, d, k, seed))
+    q, r = np.linalg.qr(rng.standard_normal((d, k)))
+    q = q * np.sign(np.diag(r))  # fixes the sign convention of the factorisation
+    return np.ascontiguousarray(q.astype(np.float32))
+
+
+def gen_embedding_pair(V: int, d: int, seed: int = 0, std: float = 0.02) -> Tuple[np.ndarray, np.ndarray]:
+    """(T_S, T_perp), V x d float32 each, N(0, std) i.i.d.: after an outer synchronisation with
+    replicas that do not compress, T_S is a generic table with components outside the subspace."""
+    rng = np.random.default_rng(_mix(0xE3B, V, d, seed))
+    T_S = (rng.standard_normal((V, d), dtype=np.float32) * np.float32(std))
+    T_perp = (rng.standard_normal((V, d), dtype=np.float32) * np.float32(std))
+    return T_S, T_perp

@@ -108,3 +108,16 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
 def test_binding_raises_with_the_library_message(lib):
     with pytest.raises(api.SparseLoCoError, match="invalid argument"):
         api.sl_compress(0x1000, 0x1000, 0x1000, [0, 8192], 0.9, 4096, 0, 2, 0x1000, 0x1000, 0x1000, None, 0)
+
+
+def test_embed_reproject_argument_checks():
+    L = api.load()
+    fake = 0x10000
+    call = lambda ts, tp, u, V, d, k: L.sl_embed_reproject(ts, tp, u, V, d, k, None, None)
+    assert call(None, fake, fake, 8, 64, 8) == api.SL_ERR_INVALID_ARG
+    assert call(fake, fake, None, 8, 64, 8) == api.SL_ERR_INVALID_ARG
+    assert call(fake + 4, fake, fake, 8, 64, 8) == api.SL_ERR_ALIGNMENT
+    assert call(fake, fake, fake + 8, 8, 64, 8) == api.SL_ERR_ALIGNMENT
+    for d, k in [(62, 8), (64, 6), (64, 0), (64, 260), (0, 4)]:
+        assert call(fake, fake, fake, 8, d, k) == api.SL_ERR_UNSUPPORTED
+    assert call(fake, fake, fake, 0, 64, 8) == api.SL_OK        # an empty table is a no-op

@@ -1,0 +1,117 @@
+"""Parity of sl_embed_reproject (paper §2.4, Eqs. 3-4) with the float64 CPU checker.
+
+Tolerance (derived from the arithmetic): each contraction takes its operands in TF32, i.e. with a
+relative error of at most 2^-10 each (whether the hardware rounds or cuts), and accumulates in
+float32.  An entry of Pi_S(T_S) is a sum of products t*u*u'; the first contraction perturbs each
+t*u by <= (2*2^-10 + 2^-20)|t||u|, the second takes the (already perturbed) coordinate and u' in
+TF32 again, another 2*2^-10, and float32 accumulation over d and k terms adds far less than
+2^-10.  With B = sum_j (sum_i |t_i||u_ij|)|u_nj| (the sum of the magnitudes of all products) the
+error is therefore below 5 * 2^-10 * B; the tests allow 2^-7 * B.  The element-wise part (the
+subtraction and the addition of Eq. 3) is float32 with one rounding each and is checked
+bit for bit from the kernel's own T_S output.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import embed as oe
+from paper_2601_02360_b200 import api, synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2.0 ** -7
+
+
+def _run(T_S, T_perp, U):
+    T_S, T_perp, U = (np.ascontiguousarray(a, dtype=np.float32) for a in (T_S, T_perp, U))
+    V, d = T_S.shape
+    k = U.shape[1]
+    ts = torch.from_numpy(T_S).cuda()
+    tp = torch.from_numpy(T_perp).cuda()
+    u = torch.from_numpy(U).cuda()
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.sl_embed_reproject(ts, tp, u, V, d, k, flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    assert torch.equal(u.cpu(), torch.from_numpy(U))
+    return ts.cpu().numpy(), tp.cpu().numpy()
+
+
+def _check(T_S, T_perp, U, ts_gpu, tp_gpu):
+    ref_ts, ref_tp = oe.embed_reproject(T_S, T_perp, U)
+    B = oe.abs_bound(T_S, U)
+    tiny = 1e-30
+    err_ts = np.abs(ts_gpu.astype(np.float64) - ref_ts)
+    assert np.all(err_ts <= TOL * B + tiny), float((err_ts / (B + tiny)).max())
+    ulp = 2.0 ** -23 * (np.abs(ref_tp) + np.abs(T_S) + np.abs(ref_ts))
+    err_tp = np.abs(tp_gpu.astype(np.float64) - ref_tp)
+    assert np.all(err_tp <= TOL * B + 2 * ulp + tiny)
+    # Eq. 3 in float32, one rounding per operation, from the very T_S that was stored
+    expect_tp = (T_perp + (T_S - ts_gpu)).astype(np.float32)
+    assert np.array_equal(expect_tp.view(np.uint32), tp_gpu.view(np.uint32))
+    # the table T_S + T_perp is conserved to float32 rounding
+    te_err = np.abs((ts_gpu.astype(np.float64) + tp_gpu) - (T_S.astype(np.float64) + T_perp))
+    assert np.all(te_err <= 2 * ulp + tiny)
+    return err_ts, ref_ts
+
+
+@pytest.mark.parametrize("V,d,k", [(1000, 512, 64), (333, 2048, 256), (129, 132, 12), (5, 64, 4),
+                                   (260, 1536, 192), (128, 128, 32), (257, 1000, 200), (64, 2048, 8)])
+def test_parity_random(V, d, k):
+    U = synth.gen_subspace_basis(d, k, seed=1)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=2)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, U)
+    err, ref = _check(T_S, T_perp, U, ts_gpu, tp_gpu)
+    # typical (not worst-case) accuracy: random signs make the error far smaller than the bound
+    assert np.sqrt((err ** 2).mean()) <= 2.0 ** -9 * np.sqrt((ref ** 2).mean())
+
+
+@pytest.mark.parametrize("V,d,k", [(300, 256, 8), (130, 512, 32), (128, 2048, 256), (77, 384, 100)])
+def test_exact_when_tf32_is_exact(V, d, k):
+    # U = k columns of the identity and dyadic table entries with <= 10 significant bits: every
+    # product and every sum is exact in TF32 / float32, so the result must match bit for bit.
+    rng = np.random.default_rng(3)
+    cols = rng.permutation(d)[:k]
+    U = np.zeros((d, k), dtype=np.float32)
+    U[cols, np.arange(k)] = 1.0
+    T_S = (rng.integers(-512, 513, size=(V, d)) / 64.0).astype(np.float32)
+    T_perp = (rng.integers(-512, 513, size=(V, d)) / 64.0).astype(np.float32)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, U)
+    ref_ts, ref_tp = oe.embed_reproject(T_S, T_perp, U)
+    assert np.array_equal(ts_gpu, ref_ts.astype(np.float32))
+    assert np.array_equal(tp_gpu, ref_tp.astype(np.float32))
+
+
+def test_signed_basis_exact():
+    # columns of +-1/2-scaled Hadamard-like vectors keep everything dyadic: catches a transposed or
+    # mis-swizzled operand that the identity columns (symmetric in their own way) could hide
+    d, k, V = 64, 4, 200
+    H = np.array([[1.0]])
+    while H.shape[0] < d:
+        H = np.block([[H, H], [H, -H]])
+    U = (H[:, [1, 6, 11, 40]] / 8.0).astype(np.float32)          # orthonormal: |column|^2 = 64/64
+    rng = np.random.default_rng(4)
+    T_S = (rng.integers(-8, 9, size=(V, d)) / 4.0).astype(np.float32)
+    T_perp = (rng.integers(-8, 9, size=(V, d)) / 4.0).astype(np.float32)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, U)
+    ref_ts, ref_tp = oe.embed_reproject(T_S, T_perp, U)
+    assert np.array_equal(ts_gpu, ref_ts.astype(np.float32))
+    assert np.array_equal(tp_gpu, ref_tp.astype(np.float32))
+
+
+def test_second_application_is_a_fixed_point_up_to_tf32():
+    V, d, k = 256, 1024, 128
+    U = synth.gen_subspace_basis(d, k, seed=5)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=6)
+    ts1, tp1 = _run(T_S, T_perp, U)
+    ts2, tp2 = _run(ts1, tp1, U)
+    B = oe.abs_bound(ts1, U)
+    assert np.all(np.abs(ts2.astype(np.float64) - ts1) <= TOL * B + 1e-30)
+
+
+def test_full_table_of_the_1b_model():
+    V, d, k = 32000, 2048, 256
+    U = synth.gen_subspace_basis(d, k, seed=7)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=8)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, U)
+    _check(T_S, T_perp, U, ts_gpu, tp_gpu)
