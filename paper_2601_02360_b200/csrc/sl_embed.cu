@@ -1,25 +1,27 @@
 // Token-embedding re-projection after an outer synchronisation (paper §2.4, Eqs. 3-4):
 //     T_perp <- T_perp + (T_S - Pi_S(T_S)),   T_S <- Pi_S(T_S),   Pi_S(t) = t U U^T.
 //
-// One CTA owns 128 rows of the table.  Both contractions run on the 5th-generation tensor
-// cores (tcgen05.mma, kind::tf32) with their accumulators in tensor memory:
+// The table's rows are dealt out in groups of 32, evenly over one CTA per SM; a CTA walks its
+// rows in sub-tiles of up to 128 rows.  Both contractions of a sub-tile run on the
+// 5th-generation tensor cores (tcgen05.mma, kind::tf32) with accumulators in tensor memory:
 //
-//   pass 1   P[128 x k]  = T_S[128 x d] . U[d x k]        K-loop over d in steps of 32 columns.
-//            A = a T_S tile (K-major, 128-byte swizzle), B = 32 rows of U (N-major: U is stored
-//            with k contiguous, so the operand is fed "MN-major", which for 32-bit elements
-//            exists only in the 128-byte swizzle with 32-byte atoms).  P stays in tensor memory.
+//   pass 1   P[128 x k]  = T_S[rows x d] . U[d x k]        K-loop over d in steps of 32 columns.
+//            A = a T_S tile (K-major, 128-byte swizzle), B = 32 rows of U (U is stored with k
+//            contiguous, so the operand is fed "MN-major", which for 32-bit elements exists only
+//            in the 128-byte swizzle with 32-byte atoms).  P stays in tensor memory.
 //   pass 2   O[128 x 128] = P[128 x k] . U[n0.., :]^T      for each block of 128 output columns.
-//            A = P read straight from tensor memory (no round trip through shared memory),
-//            B = 128 rows of U (K-major).  O is double buffered in tensor memory, so the
-//            element-wise update of block c overlaps the contraction of block c+1.
+//            A = P read straight from tensor memory, B = 128 rows of U (K-major).  O is double
+//            buffered in tensor memory.  (An MMA of N = 64 costs as many cycles as one of
+//            N = 128, so the blocks are 128 wide; the epilogue takes them in halves of 64.)
 //
-// Warp roles: warp 0 issues the bulk tensor copies (TMA) into a 3-slot ring, warp 1 owns tensor
-// memory and issues the MMAs, warps 2-9 are the epilogue: each reads 32 lanes x 64 columns of O
-// from tensor memory, turns them through a padded shared-memory tile so that global accesses are
-// whole 256-byte row segments (a batch of 16 rows in flight per warp), and applies Eqs. 3-4 with explicitly rounded float32 operations.
-// Out-of-range rows and columns (V, d, k not multiples of the tile) are zero-filled by the
-// copies and masked in the epilogue.  Every wait is bounded; a wait that gives up raises
-// SL_FLAG_TIMEOUT and all roles fall through to the common exit, which frees tensor memory.
+// All global traffic is bulk tensor copies (TMA): warp 0 loads the MMA operands; warp 6 loads,
+// for pass 2, the T_S / T_perp tiles of each half block into swizzled shared-memory buffers;
+// warp 1 owns tensor memory and issues the MMAs; warps 2-5 (one thread per row) read O from
+// tensor memory and apply Eqs. 3-4 in place in those buffers with explicitly rounded float32
+// operations (the 128-byte swizzle makes the row-per-thread accesses conflict-free); warp 7
+// stores the buffers back with bulk tensor stores, which clip at the table's edges.  The pass-1 operand ring shares its shared memory with the pass-2 buffers.  Rows a sub-tile does
+// not own (its height is a multiple of 32 below 128) are never stored.  Every wait is bounded;
+// a wait that gives up raises SL_FLAG_TIMEOUT and all roles fall through to the common exit.
 #include <cuda.h>   // CUtensorMap and its enums only: the encoder is fetched through the runtime
 #include <mutex>
 
@@ -28,22 +30,29 @@
 namespace sl {
 namespace {
 
-constexpr int kRows = 128;        // rows of the table per CTA (MMA M)
+constexpr int kRows = 128;        // rows per sub-tile (MMA M)
 constexpr int kTileK = 32;        // floats per 128-byte swizzle row
-constexpr int kBlockN = 128;      // output columns per pass-2 block
-constexpr int kStages = 3;
-constexpr int kSlotA = kRows * kTileK * 4;          // 16 KB
-constexpr int kSlotB = 256 * kTileK * 4;            // 32 KB
-constexpr int kSlot = kSlotA + kSlotB;
-constexpr int kEpiWarps = 8;      // two warps per 32-lane window of tensor memory, 64 columns each
-constexpr int kStageStride = 64 + 4;                // floats; 272-byte rows keep 16-byte stores conflict-free
-constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kBlockN = 128;      // output columns per pass-2 MMA block
+constexpr int kHalfN = 64;        // ... which the epilogue takes in two halves
+constexpr int kRing1 = 4;         // pass-1 ring: T_S tile (16 KB) + 32 rows of U (up to 32 KB) per slot
+constexpr int kSlotA = kRows * kTileK * 4;
+constexpr int kSlot1 = kSlotA + 256 * kTileK * 4;
+constexpr int kEBufs = 2;         // pass-2 tile buffers: T_S half block (32 KB) + T_perp half block (32 KB)
+constexpr int kEHalf = 2 * kRows * kTileK * 4;
+constexpr int kESize = 2 * kEHalf;
+constexpr int kRing2 = 6;         // pass-2 ring: 128 rows of U x 32 columns per slot
+constexpr int kSlot2 = kBlockN * kTileK * 4;
+constexpr int kRing2InX = 4;      // its first slots lie behind the tile buffers, the others in `y`
+constexpr int kThreads = 256;
 constexpr long long kWaitClocks = 2000000000ll;     // about a second
+static_assert(kEBufs * kESize + kRing2InX * kSlot2 == kRing1 * kSlot1, "pass-2 buffers fill the pass-1 ring");
 
 struct EmbedSmem {
-  uint8_t slot[kStages][kSlot];
-  float stage[kEpiWarps][32][kStageStride];
-  uint64_t full[kStages], empty[kStages], o_full[2], o_empty[2];
+  uint8_t x[kRing1 * kSlot1];                   // pass 1: operand ring; pass 2: tile buffers + ring slots
+  uint8_t y[kRing2 - kRing2InX][kSlot2];
+  uint64_t full1[kRing1], empty1[kRing1], full2[kRing2], empty2[kRing2];
+  uint64_t o_full[2], o_empty[2], e_full[kEBufs], e_empty[kEBufs], e_done[kEBufs];
+  uint64_t p_done, x_free;   // per sub-tile: pass 1 has read its ring / pass 2 has left the shared region
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
@@ -108,24 +117,59 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"((uint64_t)map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ float4 lds128(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, float4 v) {
+  asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+// number of uses so far of slot s of an n-slot ring after `it` round-robin uses in total
+__device__ __forceinline__ uint32_t ring_uses(uint32_t it, uint32_t s, uint32_t n) { return (it + n - 1 - s) / n; }
+
+struct Maps {
+  CUtensorMap ts128, ts32, tp128, tp32;   // T_S / T_perp, boxes of 128 and of 32 rows x 32 floats
+  CUtensorMap u_n;                        // U, box 32 rows (d) x 32 floats (k), 32-byte-atom swizzle
+  CUtensorMap u_k;                        // U, box 128 rows (d) x 32 floats (k)
+};
+
+__device__ __forceinline__ uint8_t* ring2_slot(EmbedSmem& sm, uint32_t s) {
+  return s < (uint32_t)kRing2InX ? sm.x + kEBufs * kESize + s * kSlot2 : sm.y[s - kRing2InX];
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-embed_reproject_kernel(const __grid_constant__ CUtensorMap map_ts, const __grid_constant__ CUtensorMap map_u_n,
-                       const __grid_constant__ CUtensorMap map_u_k, float* __restrict__ T_S,
-                       float* __restrict__ T_perp, uint64_t V, uint32_t d, uint32_t kp, uint32_t* flags) {
+embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d, uint32_t kp, uint32_t* flags) {
   extern __shared__ uint8_t raw[];
   EmbedSmem& sm = *reinterpret_cast<EmbedSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const uint64_t m0 = (uint64_t)blockIdx.x * kRows;
   const uint32_t k_tiles1 = (d + kTileK - 1) / kTileK;      // pass 1: steps over d
   const uint32_t k_tiles2 = kp / kTileK;                    // pass 2: steps over k (padded)
   const uint32_t n_blocks = (d + kBlockN - 1) / kBlockN;
+  const uint32_t n_halves = (d + kHalfN - 1) / kHalfN;
+  // this CTA's rows: groups [g0, g1) of 32 rows
+  const uint64_t G = (V + 31) / 32;
+  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], kEpiWarps); }
+    for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 1); mbar_init(&sm.empty1[s], 1); }
+    for (int s = 0; s < kRing2; ++s) { mbar_init(&sm.full2[s], 1); mbar_init(&sm.empty2[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
+    for (int b = 0; b < kEBufs; ++b) {
+      mbar_init(&sm.e_full[b], 1); mbar_init(&sm.e_empty[b], 1); mbar_init(&sm.e_done[b], 4);
+    }
+    mbar_init(&sm.p_done, 1);
+    mbar_init(&sm.x_free, 1);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -140,139 +184,236 @@ embed_reproject_kernel(const __grid_constant__ CUtensorMap map_ts, const __grid_
   const uint32_t t_p = tbase;            // P: columns [0, kp)
   const uint32_t t_o = tbase + 256;      // O: two buffers of 128 columns
 
+  // bounded wait for the last of `uses` uses of a barrier (nothing to wait for when it was never used)
+  auto wait_last = [&](uint64_t* bar, uint32_t uses) { return uses == 0 || mbar_wait(bar, (uses - 1) & 1u, sm); };
+  // after an abort: give the copies this thread issued the time to land before the CTA exits
+  auto landed = [&](uint64_t* bar, uint32_t uses) {
+    const long long t0 = clock64();
+    while (uses) {
+      uint32_t done;
+      asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                   : "=r"(done) : "r"(smem_u32(bar)), "r"((uses - 1) & 1u) : "memory");
+      if (done || clock64() - t0 > kWaitClocks) break;
+      __nanosleep(64);
+    }
+  };
+
   if (warp == 0) {
     if (lane == 0) {
-      // ---- producer: one ring over both passes ----
-      uint32_t it = 0;
+      // ---- operand producer: T_S tiles and U for pass 1, U for pass 2 ----
+      uint32_t it1 = 0, it2 = 0, t = 0;
       bool ok = true;
-      for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it) {
-        const uint32_t s = it % kStages;
-        ok = mbar_wait(&sm.empty[s], ((it / kStages) & 1u) ^ 1u, sm);
-        if (!ok) break;
-        mbar_expect_tx(&sm.full[s], kSlotA + kp * kTileK * 4);
-        tma_load_2d(sm.slot[s], &map_ts, (int)(kt * kTileK), (int)m0, &sm.full[s]);
-        for (uint32_t g = 0; g < kp / 32; ++g)
-          tma_load_2d(sm.slot[s] + kSlotA + g * 4096, &map_u_n, (int)(g * 32), (int)(kt * kTileK), &sm.full[s]);
-      }
-      for (uint32_t c = 0; ok && c < n_blocks; ++c)
-        for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it) {
-          const uint32_t s = it % kStages;
-          ok = mbar_wait(&sm.empty[s], ((it / kStages) & 1u) ^ 1u, sm);
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+        const int r0 = (int)(g * 32);
+        // the pass-1 ring lies over the pass-2 buffers of the previous sub-tile: wait until its last tile
+        // store has left shared memory (by then its MMAs have long read their ring slots).  Waits that
+        // cross roles go through barriers with one phase per sub-tile, so that a waiter can never be
+        // two phases away and be fooled by the parity.
+        if (t > 0) ok = mbar_wait(&sm.x_free, (t - 1) & 1u, sm);
+        for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
+          const uint32_t s = it1 % kRing1;
+          ok = mbar_wait(&sm.empty1[s], ((it1 / kRing1) & 1u) ^ 1u, sm);
           if (!ok) break;
-          mbar_expect_tx(&sm.full[s], kBlockN * kTileK * 4);
-          tma_load_2d(sm.slot[s] + kSlotA, &map_u_k, (int)(kt * kTileK), (int)(c * kBlockN), &sm.full[s]);
+          uint8_t* slot = sm.x + s * kSlot1;
+          mbar_expect_tx(&sm.full1[s], h * 128 + kp * 128);
+          if (hg == 4) {
+            tma_load_2d(slot, &maps.ts128, (int)(kt * kTileK), r0, &sm.full1[s]);
+          } else {
+            for (uint32_t i = 0; i < hg; ++i)
+              tma_load_2d(slot + i * 4096, &maps.ts32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full1[s]);
+          }
+          for (uint32_t n = 0; n < kp / 32; ++n)
+            tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
         }
-      // no copy of this CTA may still be in flight when it exits
-      const uint32_t last = it < (uint32_t)kStages ? it : (uint32_t)kStages;
-      for (uint32_t b = 0; b < last; ++b) {
-        const uint32_t j = it - 1 - b;
-        const long long t0 = clock64();
-        for (;;) {
-          uint32_t done;
-          asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                       : "=r"(done) : "r"(smem_u32(&sm.full[j % kStages])), "r"((j / kStages) & 1u) : "memory");
-          if (done || clock64() - t0 > kWaitClocks) break;
-          __nanosleep(64);
+        // ... and the pass-2 ring lies over the pass-1 ring: its last MMAs must have read it
+        ok = ok && mbar_wait(&sm.p_done, t & 1u, sm);
+        for (uint32_t c = 0; ok && c < n_blocks; ++c)
+          for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it2) {
+            const uint32_t s = it2 % kRing2;
+            ok = mbar_wait(&sm.empty2[s], ((it2 / kRing2) & 1u) ^ 1u, sm);
+            if (!ok) break;
+            mbar_expect_tx(&sm.full2[s], kSlot2);
+            tma_load_2d(ring2_slot(sm, s), &maps.u_k, (int)(kt * kTileK), (int)(c * kBlockN), &sm.full2[s]);
+          }
+      }
+      if (!ok) {
+        for (uint32_t s = 0; s < (uint32_t)kRing1; ++s) landed(&sm.full1[s], ring_uses(it1, s, kRing1));
+        for (uint32_t s = 0; s < (uint32_t)kRing2; ++s) landed(&sm.full2[s], ring_uses(it2, s, kRing2));
+      }
+    }
+  } else if (warp == 6) {
+    if (lane == 0) {
+      // ---- tile producer: the T_S / T_perp tiles of each half block of pass 2 ----
+      uint32_t hcg = 0, t = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+        const int r0 = (int)(g * 32);
+        // the tile buffers lie over the pass-1 ring: wait until this sub-tile's pass 1 has read it
+        ok = mbar_wait(&sm.p_done, t & 1u, sm);
+        for (uint32_t hb = 0; ok && hb < n_halves; ++hb, ++hcg) {
+          const uint32_t b = hcg % kEBufs;
+          ok = wait_last(&sm.e_empty[b], hcg / kEBufs);
+          if (!ok) break;
+          const uint32_t ngrp = (hb * kHalfN + 32 < d) ? 2 : 1;
+          uint8_t* e = sm.x + b * kESize;
+          mbar_expect_tx(&sm.e_full[b], 2 * ngrp * h * 128);
+          for (uint32_t grp = 0; grp < ngrp; ++grp) {
+            const int x = (int)(hb * kHalfN + 32 * grp);
+            uint8_t* ets = e + grp * (kEHalf / 2);
+            uint8_t* etp = ets + kEHalf;
+            if (hg == 4) {
+              tma_load_2d(ets, &maps.ts128, x, r0, &sm.e_full[b]);
+              tma_load_2d(etp, &maps.tp128, x, r0, &sm.e_full[b]);
+            } else {
+              for (uint32_t i = 0; i < hg; ++i) {
+                tma_load_2d(ets + i * 4096, &maps.ts32, x, r0 + 32 * (int)i, &sm.e_full[b]);
+                tma_load_2d(etp + i * 4096, &maps.tp32, x, r0 + 32 * (int)i, &sm.e_full[b]);
+              }
+            }
+          }
         }
       }
+      if (!ok)
+        for (uint32_t b = 0; b < (uint32_t)kEBufs; ++b) landed(&sm.e_full[b], ring_uses(hcg, b, kEBufs));
+    }
+  } else if (warp == 7) {
+    if (lane == 0) {
+      // ---- tile store: writes each finished half block back and frees its buffer ----
+      uint32_t hcg = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
+        const int r0 = (int)(g * 32);
+        for (uint32_t hb = 0; ok && hb < n_halves; ++hb, ++hcg) {
+          const uint32_t b = hcg % kEBufs;
+          ok = mbar_wait(&sm.e_done[b], (hcg / kEBufs) & 1u, sm);
+          if (!ok) break;
+          const uint32_t ngrp = (hb * kHalfN + 32 < d) ? 2 : 1;
+          const uint32_t e = smem_u32(sm.x + b * kESize);
+          for (uint32_t grp = 0; grp < ngrp; ++grp) {
+            const int x = (int)(hb * kHalfN + 32 * grp);
+            for (uint32_t i = 0; i < hg; ++i) {
+              tma_store_2d(&maps.ts32, x, r0 + 32 * (int)i, e + grp * (kEHalf / 2) + i * 4096);
+              tma_store_2d(&maps.tp32, x, r0 + 32 * (int)i, e + kEHalf + grp * (kEHalf / 2) + i * 4096);
+            }
+          }
+          bulk_commit();
+          bulk_wait_read_all();          // the copies have read the buffer: the tile producer may refill it
+          mbar_arrive(&sm.e_empty[b]);
+        }
+        if (ok) mbar_arrive(&sm.x_free);  // the next sub-tile's operand ring may overwrite the buffers
+      }
+      bulk_wait_all();
     }
   } else if (warp == 1) {
     if (lane == 0) {
       // ---- MMA issuer ----
-      uint32_t it = 0;
+      uint32_t it1 = 0, it2 = 0, cg = 0;
       bool ok = true;
       const uint32_t idesc1 = instr_desc(kRows, (int)kp, 1);
       const uint32_t idesc2 = instr_desc(kRows, kBlockN, 0);
-      for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it) {
-        const uint32_t s = it % kStages;
-        ok = mbar_wait(&sm.full[s], (it / kStages) & 1u, sm);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t a0 = smem_u32(sm.slot[s]), b0 = a0 + kSlotA;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)   // K = 8 per instruction: 32 bytes along a swizzled row of A, 8 rows of U
-          mma_ss(t_p, smem_desc(a0 + 32 * j, 16, 1024, 2), smem_desc(b0 + 1024 * j, 4096, 512, 1), idesc1,
-                 (kt | (uint32_t)j) != 0);
-        mma_commit(&sm.empty[s]);
-      }
-      for (uint32_t c = 0; ok && c < n_blocks; ++c) {
-        const uint32_t buf = c & 1u;
-        if (c >= 2) {
-          ok = mbar_wait(&sm.o_empty[buf], ((c >> 1) - 1u) & 1u, sm);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2);      // K-major tile, rows of 128 bytes
+      const uint64_t desc_n = smem_desc(0, 4096, 512, 1);     // U rows as N-major operand
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
+        for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
+          const uint32_t s = it1 % kRing1;
+          ok = mbar_wait(&sm.full1[s], (it1 / kRing1) & 1u, sm);
           if (!ok) break;
           tc_fence_after();
+          const uint32_t a0 = smem_u32(sm.x + s * kSlot1);
+          const uint64_t da = desc_k | (uint64_t)((a0 >> 4) & 0x3FFF);
+          const uint64_t db = desc_n | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+#pragma unroll
+          for (int j = 0; j < 4; ++j)   // K = 8 per instruction: 32 bytes along a swizzled row of A, 8 rows of U
+            mma_ss(t_p, da + 2 * j, db + 64 * j, idesc1, (kt | (uint32_t)j) != 0);
+          mma_commit(&sm.empty1[s]);
         }
-        for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it) {
-          const uint32_t s = it % kStages;
-          ok = mbar_wait(&sm.full[s], (it / kStages) & 1u, sm);
+        if (ok) mma_commit(&sm.p_done);
+        for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+          const uint32_t buf = cg & 1u;
+          ok = wait_last(&sm.o_empty[buf], cg >> 1);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t b0 = smem_u32(sm.slot[s]) + kSlotA;
+          for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it2) {
+            const uint32_t s = it2 % kRing2;
+            ok = mbar_wait(&sm.full2[s], (it2 / kRing2) & 1u, sm);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t db = desc_k | (uint64_t)((smem_u32(ring2_slot(sm, s)) >> 4) & 0x3FFF);
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            mma_ts(t_o + buf * kBlockN, t_p + kt * kTileK + 8 * j, smem_desc(b0 + 32 * j, 16, 1024, 2), idesc2,
-                   (kt | (uint32_t)j) != 0);
-          mma_commit(&sm.empty[s]);
+            for (int j = 0; j < 4; ++j)
+              mma_ts(t_o + buf * kBlockN, t_p + kt * kTileK + 8 * j, db + 2 * j, idesc2, (kt | (uint32_t)j) != 0);
+            mma_commit(&sm.empty2[s]);
+          }
+          if (!ok) break;
+          mma_commit(&sm.o_full[buf]);
         }
-        if (!ok) break;
-        mma_commit(&sm.o_full[buf]);
       }
     }
   } else {
-    // ---- epilogue: warp w may read tensor-memory lanes 32*(w%4).. only (the hardware's lane window
-    // of a warp); the two warps of a window take 64 columns of the block each ----
-    const int q = warp & 3, h = (warp - 2) >> 2;
-    float (*st)[kStageStride] = sm.stage[warp - 2];
-    const int sub = lane >> 4, c4 = (lane & 15) * 4;   // read-back: half a warp per row
+    // ---- epilogue: one thread per row; warp w may read tensor-memory lanes 32*(w%4).. only ----
+    const int q = warp & 3;
+    const uint32_t row = (uint32_t)(32 * q + lane);
+    const uint32_t sw = row & 7u;
+    uint32_t cg = 0, hcg = 0;
     bool ok = true;
-    for (uint32_t c = 0; ok && c < n_blocks; ++c) {
-      const uint32_t buf = c & 1u;
-      ok = mbar_wait(&sm.o_full[buf], (c >> 1) & 1u, sm);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after();
+    for (uint64_t g = g0; ok && g < g1; g += 4) {
+      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+      for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+        const uint32_t buf = cg & 1u;
+        const uint32_t nh = (c * kBlockN + kHalfN < d) ? 2 : 1;
+        ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm);
+        for (uint32_t half = 0; half < nh; ++half, ++hcg) {
+          const uint32_t b = hcg % kEBufs;
+          ok = ok && mbar_wait(&sm.e_full[b], (hcg / kEBufs) & 1u, sm);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          uint32_t o[64];
+          const uint32_t ta = t_o + buf * kBlockN + half * kHalfN + ((uint32_t)(32 * q) << 16);
+          tmem_ld32(ta, o);
+          tmem_ld32(ta + 32, o + 32);
+          tmem_ld_wait();
+          if (half + 1 == nh) {      // this warp has taken all it needs from the O buffer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.o_empty[buf]);
+          }
+          const uint32_t x0 = c * kBlockN + half * kHalfN;
+          const uint32_t ngrp = (x0 + 32 < d) ? 2 : 1;
+          const uint32_t e = smem_u32(sm.x + b * kESize);
+          if (row < h) {
 #pragma unroll
-      for (int cb = 0; cb < 2; ++cb) {
-        uint32_t r[32];
-        tmem_ld32(t_o + buf * kBlockN + 64 * h + cb * 32 + ((uint32_t)(32 * q) << 16), r);
+            for (uint32_t grp = 0; grp < 2; ++grp) {
+              if (grp < ngrp) {
 #pragma unroll
-        for (int i = 0; i < 32; i += 4)
-          *reinterpret_cast<uint4*>(&st[lane][cb * 32 + i]) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.o_empty[buf]);
-      const uint32_t col = c * kBlockN + 64 * h + c4;
-      if (col < d) {
-#pragma unroll 1
-        for (int rb = 0; rb < 32; rb += 16) {
-          float4 ts[8], tp[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {      // all loads of the batch first: 8 KB in flight per warp
-            const uint64_t row = m0 + (uint64_t)(32 * q + rb + 2 * i + sub);
-            if (row < V) {
-              ts[i] = __ldcs(reinterpret_cast<const float4*>(T_S + row * d + col));
-              tp[i] = __ldcs(reinterpret_cast<const float4*>(T_perp + row * d + col));
+                for (uint32_t ch = 0; ch < 8; ++ch) {
+                  const uint32_t a = e + grp * (kEHalf / 2) + row * 128 + ((ch ^ sw) << 4);
+                  const float4 ts = lds128(a);
+                  float4 tp = lds128(a + kEHalf);
+                  float4 pi;
+                  pi.x = __uint_as_float(o[grp * 32 + ch * 4 + 0]);
+                  pi.y = __uint_as_float(o[grp * 32 + ch * 4 + 1]);
+                  pi.z = __uint_as_float(o[grp * 32 + ch * 4 + 2]);
+                  pi.w = __uint_as_float(o[grp * 32 + ch * 4 + 3]);
+                  tp.x = __fadd_rn(tp.x, __fsub_rn(ts.x, pi.x));
+                  tp.y = __fadd_rn(tp.y, __fsub_rn(ts.y, pi.y));
+                  tp.z = __fadd_rn(tp.z, __fsub_rn(ts.z, pi.z));
+                  tp.w = __fadd_rn(tp.w, __fsub_rn(ts.w, pi.w));
+                  sts128(a, pi);
+                  sts128(a + kEHalf, tp);
+                }
+              }
             }
           }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int rr = rb + 2 * i + sub;
-            const uint64_t row = m0 + (uint64_t)(32 * q + rr);
-            if (row < V) {
-              const float4 o = *reinterpret_cast<const float4*>(&st[rr][c4]);
-              float4 t = tp[i];
-              t.x = __fadd_rn(t.x, __fsub_rn(ts[i].x, o.x));
-              t.y = __fadd_rn(t.y, __fsub_rn(ts[i].y, o.y));
-              t.z = __fadd_rn(t.z, __fsub_rn(ts[i].z, o.z));
-              t.w = __fadd_rn(t.w, __fsub_rn(ts[i].w, o.w));
-              __stcs(reinterpret_cast<float4*>(T_S + row * d + col), o);
-              __stcs(reinterpret_cast<float4*>(T_perp + row * d + col), t);
-            }
-          }
+          // hand the finished buffer to the storing warp
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.e_done[b]);
         }
       }
-      __syncwarp();
     }
   }
   tc_fence_before();
@@ -318,19 +459,24 @@ bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, ui
 
 cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                                    uint32_t* flags, cudaStream_t st) {
-  CUtensorMap map_ts, map_u_n, map_u_k;
-  if (!make_map(&map_ts, T_S, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map(&map_u_n, U, k, d, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
-      !make_map(&map_u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B))
+  Maps m;
+  if (!make_map(&m.ts128, T_S, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.ts32, T_S, d, V, 32, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.tp128, T_perp, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.tp32, T_perp, d, V, 32, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.u_n, U, k, d, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
+      !make_map(&m.u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B))
     return cudaErrorInvalidValue;
   const int smem = (int)sizeof(EmbedSmem) + 1024;
-  const cudaError_t attr =
-      cudaFuncSetAttribute(embed_reproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (attr != cudaSuccess) return attr;
+  cudaError_t e = cudaFuncSetAttribute(embed_reproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  int dev = 0, sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
   const uint32_t kp = (k + 31u) & ~31u;
-  const uint64_t grid = (V + kRows - 1) / kRows;
-  if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-  embed_reproject_kernel<<<(unsigned)grid, kThreads, smem, st>>>(map_ts, map_u_n, map_u_k, T_S, T_perp, V, d, kp, flags);
+  const uint64_t tiles = (V + kRows - 1) / kRows;          // never more CTAs than full sub-tiles
+  const unsigned grid = (unsigned)(tiles < (uint64_t)sms ? tiles : (uint64_t)sms);
+  embed_reproject_kernel<<<grid, kThreads, smem, st>>>(m, V, d, kp, flags);
   return cudaGetLastError();
 }
 
