@@ -12,10 +12,10 @@
 //   pass 2   O[128 x 128] = P[128 x k] . U[n0.., :]^T      for each block of 128 output columns.
 //            A = P read straight from tensor memory, B = 128 rows of U (K-major).  O is double
 //            buffered in tensor memory.  (An MMA of N = 64 costs as many cycles as one of
-//            N = 128, so the blocks are 128 wide; the epilogue takes them in halves of 64.)
+//            N = 128, so the blocks are 128 wide; the epilogue takes them in parts of 32.)
 //
 // All global traffic is bulk tensor copies (TMA): warp 0 loads the MMA operands; warp 6 loads,
-// for pass 2, the T_S / T_perp tiles of each half block into swizzled shared-memory buffers;
+// for pass 2, the T_S / T_perp tiles of each 32-column part into swizzled shared-memory buffers;
 // warp 1 owns tensor memory and issues the MMAs; warps 2-5 (one thread per row) read O from
 // tensor memory and apply Eqs. 3-4 in place in those buffers with explicitly rounded float32
 // operations (the 128-byte swizzle makes the row-per-thread accesses conflict-free); warp 7
@@ -33,16 +33,16 @@ namespace {
 constexpr int kRows = 128;        // rows per sub-tile (MMA M)
 constexpr int kTileK = 32;        // floats per 128-byte swizzle row
 constexpr int kBlockN = 128;      // output columns per pass-2 MMA block
-constexpr int kHalfN = 64;        // ... which the epilogue takes in two halves
+constexpr int kPartN = 32;        // ... which the epilogue takes in four parts of one swizzle row each
 constexpr int kRing1 = 4;         // pass-1 ring: T_S tile (16 KB) + 32 rows of U (up to 32 KB) per slot
 constexpr int kSlotA = kRows * kTileK * 4;
 constexpr int kSlot1 = kSlotA + 256 * kTileK * 4;
-constexpr int kEBufs = 2;         // pass-2 tile buffers: T_S half block (32 KB) + T_perp half block (32 KB)
-constexpr int kEHalf = 2 * kRows * kTileK * 4;
+constexpr int kEBufs = 5;         // pass-2 tile buffers: 128 x 32 of T_S (16 KB) + the same of T_perp
+constexpr int kEHalf = kRows * kTileK * 4;
 constexpr int kESize = 2 * kEHalf;
-constexpr int kRing2 = 6;         // pass-2 ring: 128 rows of U x 32 columns per slot
+constexpr int kRing2 = 4;         // pass-2 ring: 128 rows of U x 32 columns per slot
 constexpr int kSlot2 = kBlockN * kTileK * 4;
-constexpr int kRing2InX = 4;      // its first slots lie behind the tile buffers, the others in `y`
+constexpr int kRing2InX = 2;      // its first slots lie behind the tile buffers, the others in `y`
 constexpr int kThreads = 256;
 constexpr long long kWaitClocks = 2000000000ll;     // about a second
 static_assert(kEBufs * kESize + kRing2InX * kSlot2 == kRing1 * kSlot1, "pass-2 buffers fill the pass-1 ring");
@@ -156,7 +156,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
   const uint32_t k_tiles1 = (d + kTileK - 1) / kTileK;      // pass 1: steps over d
   const uint32_t k_tiles2 = kp / kTileK;                    // pass 2: steps over k (padded)
   const uint32_t n_blocks = (d + kBlockN - 1) / kBlockN;
-  const uint32_t n_halves = (d + kHalfN - 1) / kHalfN;
+  const uint32_t n_parts = (d + kPartN - 1) / kPartN;
   // this CTA's rows: groups [g0, g1) of 32 rows
   const uint64_t G = (V + 31) / 32;
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
@@ -244,7 +244,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     }
   } else if (warp == 6) {
     if (lane == 0) {
-      // ---- tile producer: the T_S / T_perp tiles of each half block of pass 2 ----
+      // ---- tile producer: the T_S / T_perp tiles of each 32-column part of pass 2 ----
       uint32_t hcg = 0, t = 0;
       bool ok = true;
       for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
@@ -252,25 +252,21 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
         const int r0 = (int)(g * 32);
         // the tile buffers lie over the pass-1 ring: wait until this sub-tile's pass 1 has read it
         ok = mbar_wait(&sm.p_done, t & 1u, sm);
-        for (uint32_t hb = 0; ok && hb < n_halves; ++hb, ++hcg) {
+        for (uint32_t hb = 0; ok && hb < n_parts; ++hb, ++hcg) {
           const uint32_t b = hcg % kEBufs;
           ok = wait_last(&sm.e_empty[b], hcg / kEBufs);
           if (!ok) break;
-          const uint32_t ngrp = (hb * kHalfN + 32 < d) ? 2 : 1;
-          uint8_t* e = sm.x + b * kESize;
-          mbar_expect_tx(&sm.e_full[b], 2 * ngrp * h * 128);
-          for (uint32_t grp = 0; grp < ngrp; ++grp) {
-            const int x = (int)(hb * kHalfN + 32 * grp);
-            uint8_t* ets = e + grp * (kEHalf / 2);
-            uint8_t* etp = ets + kEHalf;
-            if (hg == 4) {
-              tma_load_2d(ets, &maps.ts128, x, r0, &sm.e_full[b]);
-              tma_load_2d(etp, &maps.tp128, x, r0, &sm.e_full[b]);
-            } else {
-              for (uint32_t i = 0; i < hg; ++i) {
-                tma_load_2d(ets + i * 4096, &maps.ts32, x, r0 + 32 * (int)i, &sm.e_full[b]);
-                tma_load_2d(etp + i * 4096, &maps.tp32, x, r0 + 32 * (int)i, &sm.e_full[b]);
-              }
+          const int x = (int)(hb * kPartN);
+          uint8_t* ets = sm.x + b * kESize;
+          uint8_t* etp = ets + kEHalf;
+          mbar_expect_tx(&sm.e_full[b], 2 * h * 128);
+          if (hg == 4) {
+            tma_load_2d(ets, &maps.ts128, x, r0, &sm.e_full[b]);
+            tma_load_2d(etp, &maps.tp128, x, r0, &sm.e_full[b]);
+          } else {
+            for (uint32_t i = 0; i < hg; ++i) {
+              tma_load_2d(ets + i * 4096, &maps.ts32, x, r0 + 32 * (int)i, &sm.e_full[b]);
+              tma_load_2d(etp + i * 4096, &maps.tp32, x, r0 + 32 * (int)i, &sm.e_full[b]);
             }
           }
         }
@@ -280,24 +276,21 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     }
   } else if (warp == 7) {
     if (lane == 0) {
-      // ---- tile store: writes each finished half block back and frees its buffer ----
+      // ---- tile store: writes each finished part back and frees its buffer ----
       uint32_t hcg = 0;
       bool ok = true;
       for (uint64_t g = g0; ok && g < g1; g += 4) {
         const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
         const int r0 = (int)(g * 32);
-        for (uint32_t hb = 0; ok && hb < n_halves; ++hb, ++hcg) {
+        for (uint32_t hb = 0; ok && hb < n_parts; ++hb, ++hcg) {
           const uint32_t b = hcg % kEBufs;
           ok = mbar_wait(&sm.e_done[b], (hcg / kEBufs) & 1u, sm);
           if (!ok) break;
-          const uint32_t ngrp = (hb * kHalfN + 32 < d) ? 2 : 1;
+          const int x = (int)(hb * kPartN);
           const uint32_t e = smem_u32(sm.x + b * kESize);
-          for (uint32_t grp = 0; grp < ngrp; ++grp) {
-            const int x = (int)(hb * kHalfN + 32 * grp);
-            for (uint32_t i = 0; i < hg; ++i) {
-              tma_store_2d(&maps.ts32, x, r0 + 32 * (int)i, e + grp * (kEHalf / 2) + i * 4096);
-              tma_store_2d(&maps.tp32, x, r0 + 32 * (int)i, e + kEHalf + grp * (kEHalf / 2) + i * 4096);
-            }
+          for (uint32_t i = 0; i < hg; ++i) {
+            tma_store_2d(&maps.ts32, x, r0 + 32 * (int)i, e + i * 4096);
+            tma_store_2d(&maps.tp32, x, r0 + 32 * (int)i, e + kEHalf + i * 4096);
           }
           bulk_commit();
           bulk_wait_read_all();          // the copies have read the buffer: the tile producer may refill it
@@ -363,49 +356,41 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
       for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
         const uint32_t buf = cg & 1u;
-        const uint32_t nh = (c * kBlockN + kHalfN < d) ? 2 : 1;
+        const uint32_t left = (d - c * kBlockN + kPartN - 1) / kPartN;
+        const uint32_t np = left < 4 ? left : 4;      // parts of this block that exist
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm);
-        for (uint32_t half = 0; half < nh; ++half, ++hcg) {
+        for (uint32_t part = 0; part < np; ++part, ++hcg) {
           const uint32_t b = hcg % kEBufs;
           ok = ok && mbar_wait(&sm.e_full[b], (hcg / kEBufs) & 1u, sm);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
-          uint32_t o[64];
-          const uint32_t ta = t_o + buf * kBlockN + half * kHalfN + ((uint32_t)(32 * q) << 16);
-          tmem_ld32(ta, o);
-          tmem_ld32(ta + 32, o + 32);
+          uint32_t o[32];
+          tmem_ld32(t_o + buf * kBlockN + part * kPartN + ((uint32_t)(32 * q) << 16), o);
           tmem_ld_wait();
-          if (half + 1 == nh) {      // this warp has taken all it needs from the O buffer
+          if (part + 1 == np) {      // this warp has taken all it needs from the O buffer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.o_empty[buf]);
           }
-          const uint32_t x0 = c * kBlockN + half * kHalfN;
-          const uint32_t ngrp = (x0 + 32 < d) ? 2 : 1;
           const uint32_t e = smem_u32(sm.x + b * kESize);
           if (row < h) {
 #pragma unroll
-            for (uint32_t grp = 0; grp < 2; ++grp) {
-              if (grp < ngrp) {
-#pragma unroll
-                for (uint32_t ch = 0; ch < 8; ++ch) {
-                  const uint32_t a = e + grp * (kEHalf / 2) + row * 128 + ((ch ^ sw) << 4);
-                  const float4 ts = lds128(a);
-                  float4 tp = lds128(a + kEHalf);
-                  float4 pi;
-                  pi.x = __uint_as_float(o[grp * 32 + ch * 4 + 0]);
-                  pi.y = __uint_as_float(o[grp * 32 + ch * 4 + 1]);
-                  pi.z = __uint_as_float(o[grp * 32 + ch * 4 + 2]);
-                  pi.w = __uint_as_float(o[grp * 32 + ch * 4 + 3]);
-                  tp.x = __fadd_rn(tp.x, __fsub_rn(ts.x, pi.x));
-                  tp.y = __fadd_rn(tp.y, __fsub_rn(ts.y, pi.y));
-                  tp.z = __fadd_rn(tp.z, __fsub_rn(ts.z, pi.z));
-                  tp.w = __fadd_rn(tp.w, __fsub_rn(ts.w, pi.w));
-                  sts128(a, pi);
-                  sts128(a + kEHalf, tp);
-                }
-              }
+            for (uint32_t ch = 0; ch < 8; ++ch) {
+              const uint32_t a = e + row * 128 + ((ch ^ sw) << 4);
+              const float4 ts = lds128(a);
+              float4 tp = lds128(a + kEHalf);
+              float4 pi;
+              pi.x = __uint_as_float(o[ch * 4 + 0]);
+              pi.y = __uint_as_float(o[ch * 4 + 1]);
+              pi.z = __uint_as_float(o[ch * 4 + 2]);
+              pi.w = __uint_as_float(o[ch * 4 + 3]);
+              tp.x = __fadd_rn(tp.x, __fsub_rn(ts.x, pi.x));
+              tp.y = __fadd_rn(tp.y, __fsub_rn(ts.y, pi.y));
+              tp.z = __fadd_rn(tp.z, __fsub_rn(ts.z, pi.z));
+              tp.w = __fadd_rn(tp.w, __fsub_rn(ts.w, pi.w));
+              sts128(a, pi);
+              sts128(a + kEHalf, tp);
             }
           }
           // hand the finished buffer to the storing warp
@@ -443,7 +428,8 @@ EncodeTiledFn encoder() {
 }
 
 // row-major float32 matrix [outer][inner] -> a map whose box is box_outer rows of 32 floats
-bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, uint32_t box_outer, CUtensorMapSwizzle sw) {
+bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, uint32_t box_outer, CUtensorMapSwizzle sw,
+              CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_128B) {
   EncodeTiledFn enc = encoder();
   if (!enc) return false;
   const cuuint64_t dims[2] = {inner, outer};
@@ -451,7 +437,7 @@ bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, ui
   const cuuint32_t box[2] = {(cuuint32_t)kTileK, box_outer};
   const cuuint32_t es[2] = {1, 1};
   return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(p), dims, strides, box, es,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, promo,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -459,11 +445,14 @@ bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, ui
 
 cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                                    uint32_t* flags, cudaStream_t st) {
+  // a box row of the tables is 128 bytes of a much longer row whose neighbouring 128 bytes are wanted
+  // next (the next 32-column part, the next K step): fetch 256 bytes into L2 at a time
+  constexpr CUtensorMapL2promotion kTablePromo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
   Maps m;
-  if (!make_map(&m.ts128, T_S, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map(&m.ts32, T_S, d, V, 32, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map(&m.tp128, T_perp, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map(&m.tp32, T_perp, d, V, 32, CU_TENSOR_MAP_SWIZZLE_128B) ||
+  if (!make_map(&m.ts128, T_S, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B, kTablePromo) ||
+      !make_map(&m.ts32, T_S, d, V, 32, CU_TENSOR_MAP_SWIZZLE_128B, kTablePromo) ||
+      !make_map(&m.tp128, T_perp, d, V, kRows, CU_TENSOR_MAP_SWIZZLE_128B, kTablePromo) ||
+      !make_map(&m.tp32, T_perp, d, V, 32, CU_TENSOR_MAP_SWIZZLE_128B, kTablePromo) ||
       !make_map(&m.u_n, U, k, d, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
       !make_map(&m.u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B))
     return cudaErrorInvalidValue;
