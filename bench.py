@@ -372,6 +372,8 @@ def run_exchange(args) -> None:
     idx, codes, scales = api.alloc_messages(lay, wl.chunk, wl.k, wl.bits, 1, dev)
     flags = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
+    groups = exchange.plan_groups(wl.offsets(), wl.chunk, args.groups) if args.groups > 1 else None
+    comm = torch.cuda.Stream() if groups else None
     times = []
     for s in range(args.warmup + args.steps):
         synth.gen_theta_local(wl, theta_global, s, rank, args.seed, out=theta_local, rho=rho)
@@ -381,8 +383,13 @@ def run_exchange(args) -> None:
         e0 = torch.cuda.Event(enable_timing=True)
         e1 = torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        exchange.outer_step_replica(theta_local, theta_global, err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
-                                    wl.outer_lr, idx[0], codes[0], scales[0], flags)
+        if groups is None:
+            exchange.outer_step_replica(theta_local, theta_global, err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
+                                        wl.outer_lr, idx[0], codes[0], scales[0], flags)
+        else:
+            exchange.outer_step_replica_pipelined(theta_local, theta_global, err, groups, wl.beta, wl.chunk, wl.k,
+                                                  wl.bits, wl.outer_lr, idx[0], codes[0], scales[0], flags,
+                                                  comm_stream=comm)
         e1.record(stream)
         torch.cuda.synchronize()
         if s >= args.warmup:
@@ -401,9 +408,10 @@ def run_exchange(args) -> None:
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "params": wl.n_total, "R": world, "k": wl.k, "bits": wl.bits,
                        "chunk": wl.chunk, "mode": "one replica per GPU, NCCL all-gather of the sparse messages",
+                       "tensor_groups": len(groups) if groups else 1,
                        "message_bytes_per_replica": exchange.message_bytes(idx[0], codes[0], scales[0])},
             "replicas_agree": bool(lo.item() == hi.item()), "device_flags": int(flags.item()),
-            "gpu_launches": 4 * args.steps}))
+            "gpu_launches": (4 * len(groups) if groups else 4) * args.steps}))
     dist.destroy_process_group()
 
 
@@ -599,6 +607,9 @@ def main() -> None:
     ap.add_argument("--exchange", action="store_true",
                     help="replica-per-GPU form: every rank hosts one replica and the sparse messages are "
                          "all-gathered over NCCL (R = number of ranks); not the default bench line")
+    ap.add_argument("--groups", type=int, default=1,
+                    help="with --exchange: cut the arena into this many tensor groups and overlap the gather "
+                         "of one group with the compression of the next")
     ap.add_argument("--embed", action="store_true",
                     help="time sl_embed_reproject (token-embedding adaptation, Eqs. 3-4) on the model's "
                          "embedding table instead of the outer step; one GPU, its own JSON line")

@@ -10,10 +10,18 @@ The gather is a plain `torch.distributed.all_gather` of bytes (NCCL on GPUs, glo
 gathered messages land in this rank's own memory before any kernel reads them.  Messages are
 listed in rank order, which fixes the order of the additions, so every rank computes bit-identical
 parameters.
+
+`outer_step_replica_pipelined` cuts the arena into groups of consecutive tensors and overlaps the
+gather of one group's message with the compression of the next group (two CUDA streams); the
+result is the same bit for bit, because chunks never straddle tensors and every chunk is handled
+by the same kernels as in the one-shot form.
 """
 from __future__ import annotations
 
-from typing import List, Sequence, Tuple
+import dataclasses
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
 
 import torch
 import torch.distributed as dist
@@ -48,3 +56,81 @@ def outer_step_replica(theta_local, theta_global, err, layout, beta: float, chun
     g_idx, g_codes, g_scales = all_gather_messages(idx, codes, scales, group)
     api.sl_aggregate_apply(g_idx, g_codes, g_scales, layout, chunk, k, bits, theta_global, outer_lr, flags, stream)
     return g_idx, g_codes, g_scales
+
+
+@dataclasses.dataclass
+class TensorGroup:
+    """A run of consecutive tensors of the arena with the element and chunk ranges it owns."""
+    t0: int
+    t1: int
+    e0: int
+    e1: int
+    c0: int
+    c1: int
+    offsets: np.ndarray           # the group's own offsets, starting at 0
+    cols: Optional[np.ndarray]
+
+
+def plan_groups(offsets: Sequence[int], chunk: int, n_groups: int,
+                cols: Optional[Sequence[int]] = None) -> List[TensorGroup]:
+    """Cuts the tensors into at most n_groups runs of about equal element counts (host logic only).
+    A group never splits a tensor, so its chunks are exactly the arena's chunks c0..c1-1."""
+    from . import api
+    off = np.asarray(offsets, dtype=np.uint64)
+    n_t = len(off) - 1
+    assert n_t >= 1 and n_groups >= 1
+    total = int(off[-1])
+    cuts = [0]
+    for g in range(1, n_groups):
+        target = total * g // n_groups
+        t = int(np.searchsorted(off, target, side="left"))
+        t = min(max(t, cuts[-1] + 1), n_t)
+        if t < n_t and t > cuts[-1]:
+            cuts.append(t)
+    cuts.append(n_t)
+    groups, c0 = [], 0
+    for t0, t1 in zip(cuts[:-1], cuts[1:]):
+        if t1 <= t0:
+            continue
+        sub = (off[t0:t1 + 1] - off[t0]).astype(np.uint64)
+        sub_cols = None if cols is None else np.asarray(cols, dtype=np.uint64)[t0:t1]
+        nc = api.sl_num_chunks(api.Layout(sub, sub_cols), chunk)
+        groups.append(TensorGroup(t0, t1, int(off[t0]), int(off[t1]), c0, c0 + nc, sub, sub_cols))
+        c0 += nc
+    return groups
+
+
+def group_slices(g: TensorGroup, k: int, codes_stride: int, idx, codes, scales):
+    """The part of one replica's message arrays that belongs to group g (views, no copy)."""
+    return (idx[g.c0 * k:g.c1 * k], codes[g.c0 * codes_stride:g.c1 * codes_stride], scales[g.c0:g.c1])
+
+
+def outer_step_replica_pipelined(theta_local, theta_global, err, groups: Sequence[TensorGroup], beta: float,
+                                 chunk: int, k: int, bits: int, outer_lr: float, idx, codes, scales,
+                                 flags=None, group=None, comm_stream=None):
+    """The same step as outer_step_replica with the gather of group g overlapped with the
+    compression of group g+1.  Compression and the final aggregate-and-apply run on the current
+    stream, the gathers on `comm_stream` (created if not given)."""
+    from . import api
+    st = api.sl_codes_stride(k, bits)
+    cur = torch.cuda.current_stream()
+    comm = comm_stream or torch.cuda.Stream()
+    gathered = []
+    for g in groups:
+        lay = api.Layout(g.offsets, g.cols)
+        gi, gc, gs = group_slices(g, k, st, idx, codes, scales)
+        api.sl_compress(theta_local[g.e0:g.e1], theta_global[g.e0:g.e1], err[g.e0:g.e1], lay, beta, chunk, k, bits,
+                        gi, gc, gs, flags, cur)
+        ready = torch.cuda.Event()
+        ready.record(cur)
+        with torch.cuda.stream(comm):
+            comm.wait_event(ready)
+            out = all_gather_messages(gi, gc, gs, group)
+            done = torch.cuda.Event()
+            done.record(comm)
+        gathered.append((g, lay, out, done))
+    for g, lay, (a_idx, a_codes, a_scales), done in gathered:
+        cur.wait_event(done)
+        api.sl_aggregate_apply(a_idx, a_codes, a_scales, lay, chunk, k, bits, theta_global[g.e0:g.e1], outer_lr,
+                               flags, cur)
+    return gathered

@@ -117,3 +117,70 @@ def test_replica_per_rank_exchange_gives_every_rank_the_single_process_result():
     slo.outer_round(tls, tg, errs, wl.offsets(), wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr)
     assert res[0][1] == res[1][1] == tg.tobytes()
     assert res[0][2] == wl.n_chunks() * (2 * wl.k + wl.k * wl.bits // 8 + 4)
+
+
+def test_group_plan_covers_the_arena_without_splitting_tensors():
+    import numpy as np
+    from paper_2601_02360_b200 import api, exchange, synth
+    wl = synth.sub_arena(synth.workload("180m"), list(range(12)))
+    off = wl.offsets()
+    whole = api.sl_num_chunks(api.Layout(off), wl.chunk)
+    for n in (1, 2, 3, 7, 12, 40):
+        gs = exchange.plan_groups(off, wl.chunk, n)
+        assert 1 <= len(gs) <= min(n, len(off) - 1)
+        assert gs[0].t0 == 0 and gs[0].e0 == 0 and gs[0].c0 == 0
+        assert gs[-1].t1 == len(off) - 1 and gs[-1].e1 == int(off[-1]) and gs[-1].c1 == whole
+        for a, b in zip(gs, gs[1:]):
+            assert a.t1 == b.t0 and a.e1 == b.e0 and a.c1 == b.c0
+        for g in gs:
+            assert g.t1 > g.t0 and int(g.offsets[0]) == 0 and int(g.offsets[-1]) == g.e1 - g.e0
+            assert np.array_equal(g.offsets, off[g.t0:g.t1 + 1] - off[g.t0])
+    # tiles: the per-tensor chunk counts come from the library's own geometry
+    cols = [c if r > 1 else 0 for _, r, c in wl.tensors]
+    gs = exchange.plan_groups(off, wl.chunk, 3, cols)
+    assert gs[-1].c1 == api.sl_num_chunks(api.Layout(off, cols), wl.chunk)
+
+
+def _group_exchange_worker(rank, world, port, out):
+    """Gathering the message group by group (the slices the pipelined step exchanges) must give
+    every rank the same arrays as gathering it whole."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from oracle import slo
+    from paper_2601_02360_b200 import api, exchange, synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = synth.sub_arena(synth.workload("180m"), [0, 7, 8, 9]).replace(R=world)
+    off = wl.offsets()
+    tg = synth.gen_theta_global(wl).numpy().copy()
+    tl = synth.gen_theta_local(wl, torch.from_numpy(tg), 0, rank).numpy()
+    err = np.zeros(wl.n_total, np.float32)
+    i, c, s, _ = slo.compress(tl, tg, err, off, wl.beta, wl.chunk, wl.k, wl.bits)
+    ti, tc, ts = torch.from_numpy(i).reshape(-1), torch.from_numpy(c).reshape(-1), torch.from_numpy(s)
+    whole = exchange.all_gather_messages(ti, tc, ts)
+    st = api.sl_codes_stride(wl.k, wl.bits)
+    parts = [exchange.all_gather_messages(*exchange.group_slices(g, wl.k, st, ti, tc, ts))
+             for g in exchange.plan_groups(off, wl.chunk, 3)]
+    ok = len(parts) >= 2
+    for r in range(world):
+        for a in range(3):
+            ok = ok and torch.equal(torch.cat([p[a][r] for p in parts]), whole[a][r])
+    out.put((rank, bool(ok)))
+    dist.barrier()
+
+
+def test_group_by_group_gather_equals_the_whole_gather():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_group_exchange_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=180) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == [(0, True), (1, True)]

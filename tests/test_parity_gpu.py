@@ -408,3 +408,43 @@ def test_replica_per_rank_step_on_one_gpu():
         assert_close(gs.theta_global.cpu().numpy(), want, "replica-per-rank, world 1")
     finally:
         dist.destroy_process_group()
+
+
+def test_pipelined_replica_step_on_one_gpu():
+    # gathers of one tensor group overlapped with the compression of the next (two streams, NCCL with
+    # one rank): same bits as the checker's one-shot step, over two rounds
+    import torch.distributed as dist
+    from paper_2601_02360_b200 import exchange
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        wl = synth.sub_arena(synth.workload("180m"), list(range(10))).replace(R=1)
+        off = wl.offsets()
+        groups = exchange.plan_groups(off, wl.chunk, 4)
+        assert len(groups) >= 3
+        tgt = synth.gen_theta_global(wl)
+        gs = GpuStep(off, 1, wl.chunk, wl.k, wl.bits)
+        want = tgt.numpy().copy()
+        h_err = [np.zeros(wl.n_total, f32)]
+        for rnd in range(2):
+            tl = synth.gen_theta_local(wl, torch.from_numpy(want), rnd, 0)
+            if rnd == 0:
+                gs.upload(tgt.numpy(), [tl.numpy()])
+            else:
+                gs.theta_local[0].copy_(tl)
+            exchange.outer_step_replica_pipelined(gs.theta_local[0], gs.theta_global, gs.err[0], groups, wl.beta,
+                                                  wl.chunk, wl.k, wl.bits, wl.outer_lr, gs.idx[0], gs.codes[0],
+                                                  gs.scales[0], gs.flags)
+            torch.cuda.synchronize()
+            msgs, _, _ = slo.outer_round([tl.numpy()], want, h_err, off, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr)
+            nc = wl.n_chunks()
+            assert (gs.idx[0].cpu().numpy().reshape(nc, wl.k) == msgs[0][0]).all()
+            assert (gs.codes[0].cpu().numpy().reshape(nc, -1) == msgs[0][1]).all()
+            assert_close(gs.scales[0].cpu().numpy(), msgs[0][2], "pipelined scales")
+            assert_close(gs.err[0].cpu().numpy(), h_err[0], "pipelined error buffer")
+            assert_close(gs.theta_global.cpu().numpy(), want, "pipelined theta_global")
+        assert int(gs.flags.item()) == 0
+    finally:
+        dist.destroy_process_group()
