@@ -155,7 +155,7 @@ int sl_outer_step(int R, const float* const* theta_local, float* theta_global, f
  * The two contractions run on the tensor cores in TF32 (operands cut to 10 mantissa bits,
  * float32 accumulation); the subtraction and the addition are float32, each rounded once, and
  * use the very value that is stored to T_S, so T_S + T_perp is conserved to float32 rounding.
- * Needs d % 4 == 0, k % 4 == 0, 4 <= k <= 256, V >= 1 (else SL_ERR_UNSUPPORTED); V = 0 is a
+ * Needs d % 4 == 0, k % 4 == 0, 4 <= k <= 256, V < 2^31 (else SL_ERR_UNSUPPORTED); V = 0 is a
  * no-op.  `flags` (DEVICE, may be NULL) receives SL_FLAG_TIMEOUT if an internal wait gave up,
  * in which case the tables' contents are unspecified.  Asynchronous on `stream`. */
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,

@@ -284,7 +284,7 @@ int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, ui
   if (!T_S || !T_perp || !U) return SL_ERR_INVALID_ARG;
   if (!aligned(T_S, 16) || !aligned(T_perp, 16) || !aligned(U, 16) || (flags && !aligned(flags, 4)))
     return SL_ERR_ALIGNMENT;
-  if (d < 4 || d % 4 != 0 || k < 4 || k % 4 != 0 || k > 256 || V > 0xFFFFFFFFull) return SL_ERR_UNSUPPORTED;
+  if (d < 4 || d % 4 != 0 || k < 4 || k % 4 != 0 || k > 256 || V > 0x7FFFFFFFull) return SL_ERR_UNSUPPORTED;
   if (V == 0) return SL_OK;
   return launch_embed_reproject(T_S, T_perp, U, V, d, k, flags, (cudaStream_t)stream) == cudaSuccess
              ? SL_OK : SL_ERR_CUDA;
