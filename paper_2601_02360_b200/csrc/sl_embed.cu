@@ -19,9 +19,10 @@
 // warp 1 owns tensor memory and issues the MMAs; warps 2-5 (one thread per row) read O from
 // tensor memory and apply Eqs. 3-4 in place in those buffers with explicitly rounded float32
 // operations (the 128-byte swizzle makes the row-per-thread accesses conflict-free); warp 7
-// stores the buffers back with bulk tensor stores, which clip at the table's edges.  The pass-1 operand ring shares its shared memory with the pass-2 buffers.  Rows a sub-tile does
-// not own (its height is a multiple of 32 below 128) are never stored.  Every wait is bounded;
-// a wait that gives up raises SL_FLAG_TIMEOUT and all roles fall through to the common exit.
+// stores the buffers back with bulk tensor stores, which clip at the table's edges.  The pass-1
+// operand ring shares its shared memory with the pass-2 buffers.  Rows a sub-tile does not own
+// (its height is a multiple of 32 below 128) are never stored.  Every wait is bounded; a wait
+// that gives up raises SL_FLAG_TIMEOUT and all roles fall through to the common exit.
 #include <cuda.h>   // CUtensorMap and its enums only: the encoder is fetched through the runtime
 #include <mutex>
 
