@@ -14,7 +14,8 @@
  *    buffer; the library allocates nothing and keeps no state between calls.
  *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream)
  *    and use the current CUDA device.  Host arrays (layout offsets, pointer tables) are read
- *    before the call returns.
+ *    before the call returns.  A call only enqueues kernels on `stream` (its tables travel in the
+ *    kernels' parameters), so it may be recorded into a CUDA graph by stream capture.
  *  - Return value: SL_OK or a negative SL_ERR_*; nothing throws, aborts or prints.  All argument
  *    checks happen on the host before anything is launched.  Conditions met on the device never
  *    trap: they OR a bit into `*flags`.

@@ -115,3 +115,26 @@ def test_full_table_of_the_1b_model():
     T_S, T_perp = synth.gen_embedding_pair(V, d, seed=8)
     ts_gpu, tp_gpu = _run(T_S, T_perp, U)
     _check(T_S, T_perp, U, ts_gpu, tp_gpu)
+
+
+def test_captured_in_a_cuda_graph():
+    # the tensor maps are built on the host at call time and travel in the kernel parameters, so the
+    # call can be captured and replayed on the same buffers
+    V, d, k = 500, 512, 64
+    U = synth.gen_subspace_basis(d, k, seed=9)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=10)
+    ts, tp, u = torch.from_numpy(T_S).cuda(), torch.from_numpy(T_perp).cuda(), torch.from_numpy(U).cuda()
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            api.sl_embed_reproject(ts, tp, u, V, d, k, flags, stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    assert torch.equal(ts.cpu(), torch.from_numpy(T_S))
+    graph.replay()
+    torch.cuda.synchronize()
+    _check(T_S, T_perp, U, ts.cpu().numpy(), tp.cpu().numpy())
+    assert int(flags.item()) == 0

@@ -448,3 +448,43 @@ def test_pipelined_replica_step_on_one_gpu():
         assert int(gs.flags.item()) == 0
     finally:
         dist.destroy_process_group()
+
+
+def test_outer_step_captured_in_a_cuda_graph():
+    # every entry point only enqueues kernels on the caller's stream (tables travel by value in the
+    # kernel parameters), so a whole outer step can be captured once and replayed every H inner steps
+    wl = synth.sub_arena(synth.workload("180m"), [0, 1, 7, 8]).replace(R=3)
+    off = wl.offsets()
+    tgt = synth.gen_theta_global(wl)
+    gs = GpuStep(off, wl.R, wl.chunk, wl.k, wl.bits)
+    want = tgt.numpy().copy()
+    h_err = [np.zeros(wl.n_total, f32) for _ in range(wl.R)]
+    tls = [synth.gen_theta_local(wl, tgt, 0, r) for r in range(wl.R)]
+    gs.upload(tgt.numpy(), [t.numpy() for t in tls])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            api.sl_outer_step(gs.theta_local, gs.theta_global, gs.err, gs.layout, wl.beta, wl.chunk, wl.k, wl.bits,
+                              wl.outer_lr, gs.idx, gs.codes, gs.scales, gs.flags, stream=side)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    # capture does not execute: nothing has changed yet
+    assert_close(gs.theta_global.cpu().numpy(), want, "theta_global untouched by capture")
+    for rnd in range(3):
+        if rnd:
+            tls = [synth.gen_theta_local(wl, torch.from_numpy(want), rnd, r) for r in range(wl.R)]
+            for r in range(wl.R):
+                gs.theta_local[r].copy_(tls[r])
+        graph.replay()
+        torch.cuda.synchronize()
+        msgs, _, _ = slo.outer_round([t.numpy() for t in tls], want, h_err, off, wl.beta, wl.chunk, wl.k, wl.bits,
+                                     wl.outer_lr)
+        nc = wl.n_chunks()
+        for r in range(wl.R):
+            assert (gs.idx[r].cpu().numpy().reshape(nc, wl.k) == msgs[r][0]).all()
+            assert (gs.codes[r].cpu().numpy().reshape(nc, -1) == msgs[r][1]).all()
+            assert_close(gs.err[r].cpu().numpy(), h_err[r], f"graph replay {rnd}: error buffer {r}")
+        assert_close(gs.theta_global.cpu().numpy(), want, f"graph replay {rnd}: theta_global")
+    assert int(gs.flags.item()) == 0
