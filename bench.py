@@ -362,6 +362,8 @@ def run_exchange(args) -> None:
     wl = synth.workload(args.workload).replace(R=world)
     if args.k:
         wl = wl.replace(k=args.k)
+    if args.bits:
+        wl = wl.replace(bits=args.bits)
     if args.first_tensors:
         wl = synth.sub_arena(wl, list(range(args.first_tensors)), f"{wl.name}[:{args.first_tensors}]")
     lay = api.Layout(wl.offsets())
@@ -502,6 +504,8 @@ def run_ours(args) -> None:
         wl = wl.replace(R=args.R)
     if args.k:
         wl = wl.replace(k=args.k)
+    if args.bits:
+        wl = wl.replace(bits=args.bits)
     if args.variant != "plain":
         wl = wl.replace(variant=args.variant)
     if args.first_tensors:
@@ -602,6 +606,8 @@ def main() -> None:
     ap.add_argument("--workload", default="1b", choices=["tiny", "180m", "0p5b", "1b"])
     ap.add_argument("--R", type=int, default=0)
     ap.add_argument("--k", type=int, default=0)
+    ap.add_argument("--bits", type=int, default=0, choices=[0, 2, 4, 8, 32],
+                    help="bits per kept value (32 = no quantisation, the paper's own runs)")
     ap.add_argument("--first-tensors", type=int, default=0,
                     help="keep only the first N tensors of the workload (small cases for profiling)")
     ap.add_argument("--exchange", action="store_true",
