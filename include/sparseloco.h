@@ -151,6 +151,8 @@ int sl_outer_step(int R, const float* const* theta_local, float* theta_global, f
  * compression subspace S, and Pi_S(t) = t U U^T for a row t.  In place:
  *     T_perp[v,:] <- T_perp[v,:] + (T_S[v,:] - Pi_S(T_S[v,:]))
  *     T_S[v,:]    <- Pi_S(T_S[v,:])                                  for v < V.
+ * The split made before training (same section: T_S <- TE U U^T, T_perp <- TE - T_S) is the
+ * same call on T_S = TE and T_perp = 0.
  * T_S, T_perp: DEVICE, float32, V x d row-major, read and written.  U: DEVICE, float32, d x k
  * row-major (orthonormal columns; not checked), read only.  All three 16-byte aligned.
  * The two contractions run on the tensor cores in TF32 (operands cut to 10 mantissa bits,

@@ -44,6 +44,8 @@ def lib():
         L.slo_compress.argtypes = [vp, vp, vp, vp, u32, f32, i32, i32, i32, vp, vp, vp, vp]
         L.slo_aggregate.restype = i32
         L.slo_aggregate.argtypes = [i32, vp, vp, vp, vp, u32, i32, i32, i32, vp]
+        L.slo_chunk_lengths.restype = i32
+        L.slo_chunk_lengths.argtypes = [vp, vp, u32, i32, vp]
         L.slo_num_chunks_tiled.restype = u64
         L.slo_num_chunks_tiled.argtypes = [vp, vp, u32, i32]
         L.slo_compress_tiled.restype = i32
@@ -83,6 +85,17 @@ def num_chunks(offsets, chunk: int, cols=None) -> int:
     if c is None:
         return int(lib().slo_num_chunks(_p(off), len(off) - 1, chunk))
     return int(lib().slo_num_chunks_tiled(_p(off), _p(c), len(off) - 1, chunk))
+
+
+def chunk_lengths(offsets, chunk: int, cols=None) -> np.ndarray:
+    """Existing positions of every chunk of the arena (uint32[n_chunks])."""
+    off = _off(offsets)
+    c = _cols(cols, len(off) - 1)
+    out = np.zeros(num_chunks(off, chunk, cols), dtype=np.uint32)
+    rc = lib().slo_chunk_lengths(_p(off), _p(c) if c is not None else None, len(off) - 1, chunk, _p(out))
+    if rc != 0:
+        raise ValueError("slo_chunk_lengths: bad arguments")
+    return out
 
 
 def codes_stride(k: int, bits: int) -> int:

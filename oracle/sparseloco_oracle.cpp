@@ -290,6 +290,13 @@ int slo_outer_apply(float* theta_global, const float* update, uint64_t n, float 
   return SLO_OK;
 }
 
+// number of existing positions of every chunk (its length; an edge tile counts what lies inside the matrix)
+int slo_chunk_lengths(const uint64_t* offset, const uint64_t* cols, uint32_t n_tensors, int chunk, uint32_t* len) {
+  if (!offset || !len || chunk < 1 || !geometry_ok(offset, cols, n_tensors, chunk)) return SLO_ERR_INVALID_ARG;
+  for_each_chunk(offset, cols, n_tensors, chunk, [&](uint64_t g, const ChunkGeom& cg) { len[g] = (uint32_t)cg.addr.size(); });
+  return SLO_OK;
+}
+
 // the two halves of Q on their own, for the tests that pin the quantiser
 uint32_t slo_quantise(float v, float s, int bits) { return quantise(v, s, bits); }
 float slo_dequantise(uint32_t code, float s, int bits) { return dequantise(code, s, bits); }

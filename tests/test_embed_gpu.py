@@ -138,3 +138,19 @@ def test_captured_in_a_cuda_graph():
     torch.cuda.synchronize()
     _check(T_S, T_perp, U, ts.cpu().numpy(), tp.cpu().numpy())
     assert int(flags.item()) == 0
+
+
+def test_initial_split_is_the_same_call_on_a_zero_t_perp():
+    # §2.4, before training: T_S <- TE U U^T, T_perp <- TE - T_S.  With T_S = TE and T_perp = 0 the
+    # re-projection computes exactly that.
+    V, d, k = 640, 768, 96
+    U = synth.gen_subspace_basis(d, k, seed=11)
+    TE, _ = synth.gen_embedding_pair(V, d, seed=12)
+    ts_gpu, tp_gpu = _run(TE, np.zeros_like(TE), U)
+    ref_ts, ref_tp = oe.embed_init(TE, U)
+    B = oe.abs_bound(TE, U)
+    assert np.all(np.abs(ts_gpu - ref_ts) <= TOL * B + 1e-30)
+    assert np.all(np.abs(tp_gpu - ref_tp) <= TOL * B + 1e-30)
+    assert np.array_equal(tp_gpu, (TE - ts_gpu).astype(np.float32))
+    # and the table is back exactly: T_S + T_perp == TE wherever the subtraction was exact, else 1 ulp
+    assert np.all(np.abs((ts_gpu.astype(np.float64) + tp_gpu) - TE) <= 2.0 ** -23 * (np.abs(TE) + np.abs(ts_gpu)))
