@@ -387,7 +387,7 @@ def run_exchange(args) -> None:
         e0.record(stream)
         if groups is None:
             exchange.outer_step_replica(theta_local, theta_global, err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
-                                        wl.outer_lr, idx[0], codes[0], scales[0], flags)
+                                        wl.outer_lr, idx[0], codes[0], scales[0], flags, idx12=args.idx12)
         else:
             exchange.outer_step_replica_pipelined(theta_local, theta_global, err, groups, wl.beta, wl.chunk, wl.k,
                                                   wl.bits, wl.outer_lr, idx[0], codes[0], scales[0], flags,
@@ -411,7 +411,9 @@ def run_exchange(args) -> None:
             "config": {"workload": wl.name, "params": wl.n_total, "R": world, "k": wl.k, "bits": wl.bits,
                        "chunk": wl.chunk, "mode": "one replica per GPU, NCCL all-gather of the sparse messages",
                        "tensor_groups": len(groups) if groups else 1,
-                       "message_bytes_per_replica": exchange.message_bytes(idx[0], codes[0], scales[0])},
+                       "positions": "12 bits on the wire" if args.idx12 else "uint16",
+                       "message_bytes_per_replica": exchange.message_bytes(idx[0], codes[0], scales[0])
+                       - (idx[0].numel() * 2 - wl.n_chunks() * api.sl_idx12_stride(wl.k) if args.idx12 else 0)},
             "replicas_agree": bool(lo.item() == hi.item()), "device_flags": int(flags.item()),
             "gpu_launches": (4 * len(groups) if groups else 4) * args.steps}))
     dist.destroy_process_group()
@@ -613,6 +615,8 @@ def main() -> None:
     ap.add_argument("--exchange", action="store_true",
                     help="replica-per-GPU form: every rank hosts one replica and the sparse messages are "
                          "all-gathered over NCCL (R = number of ranks); not the default bench line")
+    ap.add_argument("--idx12", action="store_true",
+                    help="with --exchange: send the positions as 12 bits each")
     ap.add_argument("--groups", type=int, default=1,
                     help="with --exchange: cut the arena into this many tensor groups and overlap the gather "
                          "of one group with the compression of the next")

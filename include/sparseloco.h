@@ -146,6 +146,21 @@ int sl_outer_step(int R, const float* const* theta_local, float* theta_global, f
                   uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
                   void* stream);
 
+/* 12-bit wire form of the positions (the message of Eq. 2 line 3 carries "indices and values"; a
+ * position of a chunk of at most 4096 elements fits 12 bits, which takes a k = 64, 2-bit message
+ * from 148 to 116 bytes per chunk).  Slot j of a chunk occupies bits [12 j, 12 j + 12) of the
+ * chunk's sl_idx12_stride(k) = ceil(12 k / 8) bytes, least-significant bits first.  The padding
+ * 0xFFFF travels as 0xFFF; on the way back 0xFFF is position 4095 in a chunk that has all 4096
+ * positions (such a chunk has no padding) and padding in every other chunk, which is why
+ * unpacking needs the layout.  The kernels of this library work on the uint16 form; these two
+ * calls convert a replica's positions before and after they cross the network.
+ *   sl_pack_idx12:   idx [n_chunks * k] -> packed [n_chunks * stride].  A position above 4095
+ *                    (other than the padding) is cut to 12 bits and raises SL_FLAG_BAD_INDEX.
+ *   sl_unpack_idx12: packed -> idx, for the arena `layout` describes; chunk <= 4096. */
+uint64_t sl_idx12_stride(int k);
+int sl_pack_idx12(const uint16_t* idx, uint64_t n_chunks, int k, uint8_t* packed, uint32_t* flags, void* stream);
+int sl_unpack_idx12(const uint8_t* packed, const sl_layout* layout, int chunk, int k, uint16_t* idx, void* stream);
+
 /* Token-embedding adaptation applied after every outer synchronisation (paper section 2.4,
  * Eqs. 3-4).  The embedding table is kept as TE = T_S + T_perp; U (section 2.3) spans the
  * compression subspace S, and Pi_S(t) = t U U^T for a row t.  In place:

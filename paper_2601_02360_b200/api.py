@@ -22,7 +22,8 @@ SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
 SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1280, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
-           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_strerror")
+           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_idx12_stride",
+           "sl_pack_idx12", "sl_unpack_idx12", "sl_strerror")
 
 
 class SlLayout(ctypes.Structure):
@@ -69,6 +70,12 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_outer_step.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.sl_embed_reproject.restype = i32
     L.sl_embed_reproject.argtypes = [vp, vp, vp, u64, ctypes.c_uint32, ctypes.c_uint32, vp, vp]
+    L.sl_idx12_stride.restype = u64
+    L.sl_idx12_stride.argtypes = [i32]
+    L.sl_pack_idx12.restype = i32
+    L.sl_pack_idx12.argtypes = [vp, u64, i32, vp, vp, vp]
+    L.sl_unpack_idx12.restype = i32
+    L.sl_unpack_idx12.argtypes = [vp, lp, i32, i32, vp, vp]
     L.sl_strerror.restype = ctypes.c_char_p
     L.sl_strerror.argtypes = [i32]
     if path is None:
@@ -199,6 +206,19 @@ def sl_outer_step(theta_local: Sequence, theta_global, err: Sequence, layout, be
 def sl_embed_reproject(T_S, T_perp, U, V: int, d: int, k: int, flags=None, stream=None) -> None:
     _check(load().sl_embed_reproject(_ptr(T_S), _ptr(T_perp), _ptr(U), V, d, k, _ptr(flags), _stream(stream)),
            "sl_embed_reproject")
+
+
+def sl_idx12_stride(k: int) -> int:
+    return int(load().sl_idx12_stride(k))
+
+
+def sl_pack_idx12(idx, n_chunks: int, k: int, packed, flags=None, stream=None) -> None:
+    _check(load().sl_pack_idx12(_ptr(idx), n_chunks, k, _ptr(packed), _ptr(flags), _stream(stream)), "sl_pack_idx12")
+
+
+def sl_unpack_idx12(packed, layout, chunk: int, k: int, idx, stream=None) -> None:
+    _check(load().sl_unpack_idx12(_ptr(packed), _layout(layout).ref(), chunk, k, _ptr(idx), _stream(stream)),
+           "sl_unpack_idx12")
 
 
 def alloc_messages(layout, chunk: int, k: int, bits: int, R: int, device="cuda"):

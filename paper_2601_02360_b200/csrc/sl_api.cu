@@ -214,6 +214,15 @@ int aggregate_checked(int R, const uint16_t* const* idx, const uint8_t* const* c
                                         flags, st);
 }
 
+template <int T>
+int unpack_impl(const uint8_t* packed, const sl_layout* L, int chunk, int k, uint16_t* idx, cudaStream_t st) {
+  std::unique_ptr<Table<T>> tb(new (std::nothrow) Table<T>);
+  if (!tb) return SL_ERR_CUDA;
+  bool m4;
+  fill_table(*tb, L, chunk, &m4);
+  return launch_unpack_idx12(*tb, packed, chunk, k, idx, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -277,6 +286,26 @@ int sl_aggregate_apply(int R, const uint16_t* const* idx, const uint8_t* const* 
                        float* theta_global, float outer_lr, uint32_t* flags, void* stream) {
   return aggregate_checked(R, idx, codes, scales, L, chunk, k, bits, theta_global, outer_lr, true, flags,
                            stream);
+}
+
+uint64_t sl_idx12_stride(int k) { return k < 1 ? 0 : (12u * (uint64_t)k + 7u) / 8u; }
+
+int sl_pack_idx12(const uint16_t* idx, uint64_t n_chunks, int k, uint8_t* packed, uint32_t* flags, void* stream) {
+  if (!idx || !packed || k < 1 || k > 4096) return SL_ERR_INVALID_ARG;
+  if (!aligned(idx, 2) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
+  if (n_chunks > 0x7FFFFFFFull) return SL_ERR_UNSUPPORTED;
+  return launch_pack_idx12(idx, n_chunks, k, packed, flags, (cudaStream_t)stream) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+}
+
+int sl_unpack_idx12(const uint8_t* packed, const sl_layout* L, int chunk, int k, uint16_t* idx, void* stream) {
+  if (!packed || !idx) return SL_ERR_INVALID_ARG;
+  const int rc = check_common(L, chunk, k, 32);
+  if (rc != SL_OK) return rc;
+  if (chunk > 4096) return SL_ERR_UNSUPPORTED;
+  if (!aligned(idx, 2)) return SL_ERR_ALIGNMENT;
+  cudaStream_t st = (cudaStream_t)stream;
+  return L->n_tensors <= 256 ? unpack_impl<256>(packed, L, chunk, k, idx, st)
+                             : unpack_impl<SL_MAX_TENSORS>(packed, L, chunk, k, idx, st);
 }
 
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,

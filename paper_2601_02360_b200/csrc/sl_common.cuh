@@ -209,6 +209,10 @@ template <int T> bool compress_is_tuned(const CompressArgs<T>& a, bool aligned16
 template <int T> cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned16, cudaStream_t st);
 template <int T> cudaError_t launch_aggregate_tails(const AggregateArgs<T>& a, bool apply, cudaStream_t st);
 cudaError_t launch_outer_apply(float* theta, const float* update, uint64_t n, float lr, cudaStream_t st);
+cudaError_t launch_pack_idx12(const uint16_t* idx, uint64_t n_chunks, int k, uint8_t* packed, uint32_t* flags,
+                              cudaStream_t st);
+template <int T> cudaError_t launch_unpack_idx12(const Table<T>& tb, const uint8_t* packed, int chunk, int k,
+                                                 uint16_t* idx, cudaStream_t st);
 cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                                    uint32_t* flags, cudaStream_t st);
 

@@ -47,13 +47,36 @@ def message_bytes(idx: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor) 
     return sum(t.numel() * t.element_size() for t in (idx, codes, scales))
 
 
+def all_gather_messages_idx12(idx: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, layout, chunk: int,
+                              k: int, group=None, flags=None):
+    """The same exchange with the positions sent as 12 bits each (sl_pack_idx12 before the gather,
+    sl_unpack_idx12 of every rank's part after it, both on the current stream).  Returns the lists in
+    rank order (positions back in their uint16 form) and the bytes this rank sent."""
+    from . import api
+    world = dist.get_world_size(group)
+    nc = scales.numel()
+    packed = torch.empty(nc * api.sl_idx12_stride(k), dtype=torch.uint8, device=idx.device)
+    api.sl_pack_idx12(idx, nc, k, packed, flags)
+    g_packed = _gather_bytes(packed, world, group)
+    g_codes = _gather_bytes(codes, world, group)
+    g_scales = _gather_bytes(scales, world, group)
+    g_idx = [torch.empty_like(idx) for _ in range(world)]
+    for r in range(world):
+        api.sl_unpack_idx12(g_packed[r], layout, chunk, k, g_idx[r])
+    return g_idx, g_codes, g_scales, message_bytes(packed, codes, scales)
+
+
 def outer_step_replica(theta_local, theta_global, err, layout, beta: float, chunk: int, k: int, bits: int,
-                       outer_lr: float, idx, codes, scales, flags=None, group=None, stream=None):
+                       outer_lr: float, idx, codes, scales, flags=None, group=None, stream=None, idx12: bool = False):
     """One outer step of the replica this rank hosts.  err, idx, codes, scales and theta_global are
-    updated; returns the gathered messages (idx, codes, scales lists in rank order)."""
+    updated; returns the gathered messages (idx, codes, scales lists in rank order).  idx12: send the
+    positions as 12 bits each (chunk <= 4096; `stream` must then be the current stream)."""
     from . import api
     api.sl_compress(theta_local, theta_global, err, layout, beta, chunk, k, bits, idx, codes, scales, flags, stream)
-    g_idx, g_codes, g_scales = all_gather_messages(idx, codes, scales, group)
+    if idx12:
+        g_idx, g_codes, g_scales, _ = all_gather_messages_idx12(idx, codes, scales, layout, chunk, k, group, flags)
+    else:
+        g_idx, g_codes, g_scales = all_gather_messages(idx, codes, scales, group)
     api.sl_aggregate_apply(g_idx, g_codes, g_scales, layout, chunk, k, bits, theta_global, outer_lr, flags, stream)
     return g_idx, g_codes, g_scales
 

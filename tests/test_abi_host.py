@@ -22,7 +22,7 @@ def lib():
 def _declared():
     src = open(HEADER).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(sl_[a-z_]+)\s*\(", src)))
+    return sorted(set(re.findall(r"\b(sl_[a-z0-9_]+)\s*\(", src)))
 
 
 def test_every_declared_symbol_is_exported(lib):
@@ -121,3 +121,17 @@ def test_embed_reproject_argument_checks():
     for d, k in [(62, 8), (64, 6), (64, 0), (64, 260), (0, 4)]:
         assert call(fake, fake, fake, 8, d, k) == api.SL_ERR_UNSUPPORTED
     assert call(fake, fake, fake, 0, 64, 8) == api.SL_OK        # an empty table is a no-op
+
+
+def test_idx12_argument_checks():
+    L = api.load()
+    assert [api.sl_idx12_stride(k) for k in (0, 1, 2, 3, 64)] == [0, 2, 3, 5, 96]
+    fake = 0x10000
+    assert L.sl_pack_idx12(None, 4, 64, fake, None, None) == api.SL_ERR_INVALID_ARG
+    assert L.sl_pack_idx12(fake, 4, 0, fake, None, None) == api.SL_ERR_INVALID_ARG
+    assert L.sl_pack_idx12(fake + 1, 4, 64, fake, None, None) == api.SL_ERR_ALIGNMENT
+    assert L.sl_pack_idx12(fake, 0, 64, fake, None, None) == api.SL_OK        # nothing to do
+    lay = api.Layout([0, 100])
+    assert L.sl_unpack_idx12(None, lay.ref(), 4096, 64, fake, None) == api.SL_ERR_INVALID_ARG
+    assert L.sl_unpack_idx12(fake, lay.ref(), 8192, 64, fake, None) == api.SL_ERR_UNSUPPORTED   # 13-bit positions
+    assert L.sl_unpack_idx12(fake, lay.ref(), 4096, 64, fake + 1, None) == api.SL_ERR_ALIGNMENT
