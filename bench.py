@@ -376,6 +376,9 @@ def run_exchange(args) -> None:
     stream = torch.cuda.current_stream()
     groups = exchange.plan_groups(wl.offsets(), wl.chunk, args.groups) if args.groups > 1 else None
     comm = torch.cuda.Stream() if groups else None
+    pm = exchange.PeerMessages(lay, wl.chunk, wl.k, wl.bits) if args.peer else None
+    if pm is not None:
+        idx, codes, scales = [pm.idx[rank]], [pm.codes[rank]], [pm.scales[rank]]
     times = []
     for s in range(args.warmup + args.steps):
         synth.gen_theta_local(wl, theta_global, s, rank, args.seed, out=theta_local, rho=rho)
@@ -385,7 +388,10 @@ def run_exchange(args) -> None:
         e0 = torch.cuda.Event(enable_timing=True)
         e1 = torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        if groups is None:
+        if pm is not None:
+            exchange.outer_step_replica_peer(theta_local, theta_global, err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
+                                             wl.outer_lr, pm, flags)
+        elif groups is None:
             exchange.outer_step_replica(theta_local, theta_global, err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
                                         wl.outer_lr, idx[0], codes[0], scales[0], flags, idx12=args.idx12)
         else:
@@ -409,7 +415,10 @@ def run_exchange(args) -> None:
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "params": wl.n_total, "R": world, "k": wl.k, "bits": wl.bits,
-                       "chunk": wl.chunk, "mode": "one replica per GPU, NCCL all-gather of the sparse messages",
+                       "chunk": wl.chunk,
+                       "mode": ("one replica per GPU, messages in symmetric memory, the averaging kernel reads "
+                                "the peers' buffers over NVLink (no gather)") if args.peer else
+                               "one replica per GPU, NCCL all-gather of the sparse messages",
                        "tensor_groups": len(groups) if groups else 1,
                        "positions": "12 bits on the wire" if args.idx12 else "uint16",
                        "message_bytes_per_replica": exchange.message_bytes(idx[0], codes[0], scales[0])
@@ -615,6 +624,9 @@ def main() -> None:
     ap.add_argument("--exchange", action="store_true",
                     help="replica-per-GPU form: every rank hosts one replica and the sparse messages are "
                          "all-gathered over NCCL (R = number of ranks); not the default bench line")
+    ap.add_argument("--peer", action="store_true",
+                    help="with --exchange: no gather; messages live in symmetric memory and the averaging "
+                         "kernel reads every rank's buffer through its NVLink peer mapping")
     ap.add_argument("--idx12", action="store_true",
                     help="with --exchange: send the positions as 12 bits each")
     ap.add_argument("--groups", type=int, default=1,

@@ -11,6 +11,13 @@ gathered messages land in this rank's own memory before any kernel reads them.  
 listed in rank order, which fixes the order of the additions, so every rank computes bit-identical
 parameters.
 
+`outer_step_replica_peer` is the form without a gather: every rank writes its message into a
+buffer that all ranks of the node have mapped (symmetric memory over NVLink), and after one
+barrier `sl_aggregate_apply` is handed the PEERS' buffers as its message tables, so the
+averaging kernel pulls each chunk's messages over NVLink with plain loads while it works through
+the chunks - the transfer and the arithmetic overlap chunk by chunk, nothing is staged, and no
+load from a peer uses TMA multicast (the kernels read messages with ordinary read-only loads).
+
 `outer_step_replica_pipelined` cuts the arena into groups of consecutive tensors and overlaps the
 gather of one group's message with the compression of the next group (two CUDA streams); the
 result is the same bit for bit, because chunks never straddle tensors and every chunk is handled
@@ -157,3 +164,63 @@ def outer_step_replica_pipelined(theta_local, theta_global, err, groups: Sequenc
         api.sl_aggregate_apply(a_idx, a_codes, a_scales, lay, chunk, k, bits, theta_global[g.e0:g.e1], outer_lr,
                                flags, cur)
     return gathered
+
+
+def _align(n: int, a: int = 256) -> int:
+    return (n + a - 1) // a * a
+
+
+class PeerMessages:
+    """One replica's message buffers in symmetric memory, with views of every peer's copy.
+
+    The three arrays of a message sit in one flat buffer (256-byte aligned sections) that
+    `torch.distributed._symmetric_memory` maps into every rank of `group` (one node: NVLink peer
+    mappings).  idx[r] / codes[r] / scales[r] are views of rank r's buffer; this rank writes only
+    its own (index `rank`) and reads all of them after `barrier()`."""
+
+    def __init__(self, layout, chunk: int, k: int, bits: int, group=None, device=None):
+        import torch.distributed._symmetric_memory as symm
+        from . import api
+        group = group or dist.group.WORLD
+        device = device or torch.device("cuda", torch.cuda.current_device())
+        nc = api.sl_num_chunks(layout, chunk)
+        st = api.sl_codes_stride(k, bits)
+        self.sections = self.plan(nc, k, st)
+        total = self.sections[-1][1]
+        self.buf = symm.empty(total, dtype=torch.uint8, device=device)
+        self.handle = symm.rendezvous(self.buf, group)
+        self.rank, self.world = self.handle.rank, self.handle.world_size
+        self.idx, self.codes, self.scales = [], [], []
+        for r in range(self.world):
+            b = self.buf if r == self.rank else self.handle.get_buffer(r, (total,), torch.uint8)
+            (i0, i1), (c0, c1), (s0, s1) = self.sections
+            self.idx.append(b[i0:i0 + nc * k * 2].view(torch.uint16))
+            self.codes.append(b[c0:c0 + nc * st])
+            self.scales.append(b[s0:s0 + nc * 4].view(torch.float32))
+
+    @staticmethod
+    def plan(n_chunks: int, k: int, codes_stride: int):
+        """Byte ranges (start, end) of idx, codes, scales in the flat buffer (host logic only)."""
+        i1 = _align(n_chunks * k * 2)
+        c1 = i1 + _align(n_chunks * codes_stride)
+        s1 = c1 + _align(n_chunks * 4)
+        return (0, i1), (i1, c1), (c1, s1)
+
+    def barrier(self) -> None:
+        """All ranks' work enqueued so far on their current streams is complete and visible."""
+        self.handle.barrier()
+
+
+def outer_step_replica_peer(theta_local, theta_global, err, layout, beta: float, chunk: int, k: int, bits: int,
+                            outer_lr: float, pm: PeerMessages, flags=None):
+    """One outer step of the replica this rank hosts, with the exchange folded into the averaging
+    kernel: compress into this rank's symmetric buffer, barrier, aggregate-and-apply reading every
+    rank's message in place through its peer mapping (rank order, so all ranks end bit-identical),
+    barrier again so that nobody overwrites a message a peer may still be reading."""
+    from . import api
+    r = pm.rank
+    api.sl_compress(theta_local, theta_global, err, layout, beta, chunk, k, bits, pm.idx[r], pm.codes[r],
+                    pm.scales[r], flags)
+    pm.barrier()
+    api.sl_aggregate_apply(pm.idx, pm.codes, pm.scales, layout, chunk, k, bits, theta_global, outer_lr, flags)
+    pm.barrier()

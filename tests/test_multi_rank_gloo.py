@@ -184,3 +184,16 @@ def test_group_by_group_gather_equals_the_whole_gather():
         p.join(timeout=60)
         assert p.exitcode == 0
     assert res == [(0, True), (1, True)]
+
+
+def test_peer_message_buffer_plan():
+    # the flat symmetric buffer: three aligned, non-overlapping sections that hold the three arrays
+    from paper_2601_02360_b200 import api, exchange, synth
+    wl = synth.workload("tiny")
+    nc = api.sl_num_chunks(api.Layout(wl.offsets()), wl.chunk)
+    for k, bits in ((64, 2), (5, 4), (32, 32), (1, 8)):
+        st = api.sl_codes_stride(k, bits)
+        (i0, i1), (c0, c1), (s0, s1) = exchange.PeerMessages.plan(nc, k, st)
+        assert i0 == 0 and c0 == i1 and s0 == c1
+        assert i1 - i0 >= nc * k * 2 and c1 - c0 >= nc * st and s1 - s0 >= nc * 4
+        assert all(x % 256 == 0 for x in (i0, c0, s0, s1))      # 16-byte alignment of every array and more

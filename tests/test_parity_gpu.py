@@ -488,3 +488,40 @@ def test_outer_step_captured_in_a_cuda_graph():
             assert_close(gs.err[r].cpu().numpy(), h_err[r], f"graph replay {rnd}: error buffer {r}")
         assert_close(gs.theta_global.cpu().numpy(), want, f"graph replay {rnd}: theta_global")
     assert int(gs.flags.item()) == 0
+
+
+def test_peer_memory_replica_step_on_one_gpu():
+    # the gather-free form: the message lives in symmetric memory and the averaging kernel reads the
+    # ranks' buffers through their peer mappings (with one rank: its own mapping).  Two rounds.
+    import torch.distributed as dist
+    from paper_2601_02360_b200 import exchange
+    import socket
+    s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        wl = synth.sub_arena(synth.workload("180m"), list(range(10))).replace(R=1)
+        off = wl.offsets()
+        lay = api.Layout(off)
+        pm = exchange.PeerMessages(lay, wl.chunk, wl.k, wl.bits)
+        assert pm.world == 1 and pm.idx[0].data_ptr() % 16 == 0 and pm.scales[0].data_ptr() % 16 == 0
+        tgt = synth.gen_theta_global(wl)
+        d_tg = tgt.cuda()
+        d_err = torch.zeros_like(d_tg)
+        flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+        want = tgt.numpy().copy()
+        h_err = [np.zeros(wl.n_total, f32)]
+        for rnd in range(2):
+            tl = synth.gen_theta_local(wl, torch.from_numpy(want), rnd, 0)
+            exchange.outer_step_replica_peer(tl.cuda(), d_tg, d_err, lay, wl.beta, wl.chunk, wl.k, wl.bits,
+                                             wl.outer_lr, pm, flags)
+            torch.cuda.synchronize()
+            msgs, _, _ = slo.outer_round([tl.numpy()], want, h_err, off, wl.beta, wl.chunk, wl.k, wl.bits, wl.outer_lr)
+            nc = wl.n_chunks()
+            assert (pm.idx[0].cpu().numpy().reshape(nc, wl.k) == msgs[0][0]).all()
+            assert (pm.codes[0].cpu().numpy().reshape(nc, -1) == msgs[0][1]).all()
+            assert_close(d_err.cpu().numpy(), h_err[0], "peer form: error buffer")
+            assert_close(d_tg.cpu().numpy(), want, "peer form: theta_global")
+        assert int(flags.item()) == 0
+    finally:
+        dist.destroy_process_group()
