@@ -154,3 +154,31 @@ def test_initial_split_is_the_same_call_on_a_zero_t_perp():
     assert np.array_equal(tp_gpu, (TE - ts_gpu).astype(np.float32))
     # and the table is back exactly: T_S + T_perp == TE wherever the subtraction was exact, else 1 ulp
     assert np.all(np.abs((ts_gpu.astype(np.float64) + tp_gpu) - TE) <= 2.0 ** -23 * (np.abs(TE) + np.abs(ts_gpu)))
+
+
+@pytest.mark.parametrize("V,d,k", [(1, 4, 4), (2, 8, 8), (31, 36, 4), (33, 60, 16), (127, 260, 256), (200, 124, 100),
+                                   (96, 4096, 32), (385, 96, 96), (1000, 64, 64), (160, 2052, 252)])
+def test_odd_shapes(V, d, k):
+    # sizes below one tile, k = d (the projection is the identity up to TF32), d and k off the
+    # 32 / 128 grids: everything outside the matrices is zero-filled on load and clipped on store
+    U = synth.gen_subspace_basis(d, k, seed=21)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=22)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, U)
+    _check(T_S, T_perp, U, ts_gpu, tp_gpu)
+
+
+def test_neighbouring_memory_is_untouched():
+    # the table sits in the middle of a larger allocation: rows before and after it must not change
+    V, d, k = 130, 200, 40
+    U = synth.gen_subspace_basis(d, k, seed=23)
+    T_S, T_perp = synth.gen_embedding_pair(V + 64, d, seed=24)
+    big_s, big_p = torch.from_numpy(T_S).cuda(), torch.from_numpy(T_perp).cuda()
+    u = torch.from_numpy(U).cuda()
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.sl_embed_reproject(big_s[32:32 + V], big_p[32:32 + V], u, V, d, k, flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    hs, hp = big_s.cpu().numpy(), big_p.cpu().numpy()
+    assert np.array_equal(hs[:32], T_S[:32]) and np.array_equal(hs[32 + V:], T_S[32 + V:])
+    assert np.array_equal(hp[:32], T_perp[:32]) and np.array_equal(hp[32 + V:], T_perp[32 + V:])
+    _check(T_S[32:32 + V], T_perp[32:32 + V], U, hs[32:32 + V], hp[32:32 + V])
