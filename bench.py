@@ -310,7 +310,7 @@ def run_e2e(st: DeviceState, steps: int, world: int):
     wl = st.wl
     n = wl.n_total
     need = n * 4
-    budget = int(host_memory_available() * 0.5)
+    budget = int(host_memory_available() * 0.5 / max(1, world))   # the ranks of a node share its memory
     pool = max(1, min(wl.R, budget // need - 1))
     host_tl = [torch.empty(n, dtype=torch.float32).pin_memory() for _ in range(pool)]
     for p in range(pool):
