@@ -68,9 +68,10 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
 //  * the (replica, slot) pairs of the chunk are spread over the threads, NP per thread: pair
 //    q = tid + 256 i is slot q % k of replica q / k.  What does not depend on the chunk (replica,
 //    slot, the three pointers, the bit offset of the code) is computed once per thread;
-//  * the pairs are applied to a 16 KB shared accumulator in replica order: one round per replica,
-//    a barrier between rounds (inside one message positions are distinct: no conflicts, no
-//    atomics; across messages the barrier fixes the order of the additions);
+//  * the pairs are applied to a 16 KB shared accumulator in replica order: one round per replica
+//    (and per group of 256 pairs it has entries in), a barrier between rounds (inside one message
+//    positions are distinct: no conflicts, no atomics; across messages the barrier fixes the order
+//    of the additions);
 //  * division by R is a multiplication by the exact reciprocal when R is a power of two (bit
 //    identical), an IEEE division otherwise; the outer update is one fused multiply-add; the
 //    result leaves with 128-bit streaming stores.
@@ -213,11 +214,19 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(acc)[tid + 256 * j] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
-    for (int r = 0; r < R; ++r) {
+    // pair i of all threads covers pairs 256 i .. 256 i + 255, i.e. the replicas r_lo..r_hi below (non-
+    // decreasing with i): one round per (i, replica) in that order applies every replica's entries
+    // after all entries of the replicas before it, with one predicated add per thread and round
 #pragma unroll
-      for (int i = 0; i < NP; ++i)
-        if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
-      __syncthreads();
+    for (int i = 0; i < NP; ++i) {
+      const int q_lo = kThreads * i;
+      if (q_lo < total) {
+        const int r_lo = q_lo / k, q_hi = min(q_lo + kThreads, total) - 1, r_hi = q_hi / k;
+        for (int r = r_lo; r <= r_hi; ++r) {
+          if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
+          __syncthreads();
+        }
+      }
     }
     const float4* g4 = reinterpret_cast<const float4*>(sm.gbuf[it & 1]);
     if (APPLY) {                                   // bounded wait for this chunk's theta_global
