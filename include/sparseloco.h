@@ -123,7 +123,9 @@ int sl_compress_batch(int R, const float* const* theta_local, const float* theta
  * Replicas are added in the order 0..R-1 starting from +0 and the sum is divided by R (always
  * R, however many replicas sent a position).  `update` [n_total] is fully overwritten;
  * positions nobody sent are +0.  A slot whose position is >= its chunk's length (other than the
- * 0xFFFF padding) is skipped and raises SL_FLAG_BAD_INDEX. */
+ * 0xFFFF padding) is skipped and raises SL_FLAG_BAD_INDEX.  Inside one replica's chunk message
+ * the positions are distinct (sl_compress writes them so); a message that names a position twice
+ * gets an unspecified sum at that position. */
 int sl_aggregate(int R, const uint16_t* const* idx, const uint8_t* const* codes,
                  const float* const* scales, const sl_layout* layout, int chunk, int k, int bits,
                  float* update, uint32_t* flags, void* stream);

@@ -101,7 +101,12 @@ __device__ __forceinline__ bool next_full_chunk(const Table<T>& tb, uint32_t& g,
 // TILED (arenas with matrices cut into 64 x 64 tiles): a chunk is 64 rows of 256 bytes `stride`
 // elements apart; theta_global then comes in by 16-byte cp.async copies of all threads instead
 // of one bulk copy, and the stores follow the same geometry.
-template <int T, bool APPLY, int NP, bool TILED>
+//
+// GROUPED (k a multiple of NP): a thread owns NP consecutive slots of ONE replica instead of NP
+// pairs 256 apart.  Its positions then arrive as one 2*NP-byte load and its codes as a few bytes,
+// and the accumulation takes R rounds in which the owners of replica r read their NP accumulator
+// cells, add, and write them back (positions inside one message are distinct, so the cells are).
+template <int T, bool APPLY, int NP, bool TILED, bool GROUPED>
 __global__ void __launch_bounds__(kThreads)
 aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   extern __shared__ __align__(16) unsigned char agg_smem_raw[];
@@ -120,7 +125,7 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   uint32_t cshift[NP];
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
-    const int q = tid + kThreads * i;
+    const int q = GROUPED ? tid * NP + i : tid + kThreads * i;
     rep[i] = -1;
     p_idx[i] = nullptr; p_code[i] = nullptr; p_scale[i] = nullptr; cshift[i] = 0;
     if (q < total) {
@@ -133,6 +138,9 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       p_scale[i] = a.m.scales[r];
     }
   }
+  // GROUPED: all NP pairs of a thread belong to replica rep[0] and start at slot j0 (a multiple of NP);
+  // only pair 0's pointers are used, the others are dead and cost no registers
+  const int my_r = rep[0];
   const uint32_t cmask = bits == 32 ? 0xFFFFFFFFu : (1u << bits) - 1u;
   const bool pow2 = (R & (R - 1)) == 0;
   const float Rf = (float)R, invR = 1.0f / Rf;
@@ -150,17 +158,49 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   // raw message entries of a chunk: position, code bits (or the float itself), scale
   uint32_t rp[NP], rc[NP];
   float rs[NP];
+  uint32_t gi[NP > 1 ? NP / 2 : 1];       // GROUPED: the positions, two per word
+  uint64_t gw = 0;                         // GROUPED: the bytes holding the NP codes
+  float gs = 0.0f;
   auto fetch = [&](uint32_t g) {
+    if constexpr (GROUPED) {
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      rp[i] = 0xFFFFu; rc[i] = 0; rs[i] = 0.0f;
-      if (rep[i] >= 0) {
-        rp[i] = __ldg(p_idx[i] + (uint64_t)g * (uint64_t)k);
-        if (bits == 32) {
-          rc[i] = __float_as_uint(__ldg(reinterpret_cast<const float*>(p_code[i] + (uint64_t)g * (uint64_t)a.stride)));
+      for (int i = 0; i < (NP > 1 ? NP / 2 : 1); ++i) gi[i] = 0xFFFFFFFFu;
+      gw = 0; gs = 0.0f;
+      if (my_r >= 0) {
+        const uint16_t* pi = p_idx[0] + (uint64_t)g * (uint64_t)k;
+        if constexpr (NP == 8) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(pi));
+          gi[0] = v.x; gi[1] = v.y; gi[2] = v.z; gi[3] = v.w;
+        } else if constexpr (NP == 4) {
+          const uint2 v = __ldg(reinterpret_cast<const uint2*>(pi));
+          gi[0] = v.x; gi[1] = v.y;
+        } else if constexpr (NP == 2) {
+          gi[0] = __ldg(reinterpret_cast<const uint32_t*>(pi));
         } else {
-          rc[i] = (uint32_t)__ldg(p_code[i] + (uint64_t)g * (uint64_t)a.stride);
-          rs[i] = __ldg(p_scale[i] + g);
+          gi[0] = 0xFFFF0000u | (uint32_t)__ldg(pi);
+        }
+        const uint8_t* pc = p_code[0] + (uint64_t)g * (uint64_t)a.stride;
+        if (bits == 32) {
+#pragma unroll
+          for (int i = 0; i < NP; ++i) rc[i] = __float_as_uint(__ldg(reinterpret_cast<const float*>(pc) + i));
+        } else {
+          const uint32_t nb = (cshift[0] + (uint32_t)NP * (uint32_t)bits + 7u) >> 3;   // 1..8 bytes
+          for (uint32_t b = 0; b < nb; ++b) gw |= (uint64_t)__ldg(pc + b) << (8u * b);
+          gs = __ldg(p_scale[0] + g);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < NP; ++i) {
+        rp[i] = 0xFFFFu; rc[i] = 0; rs[i] = 0.0f;
+        if (rep[i] >= 0) {
+          rp[i] = __ldg(p_idx[i] + (uint64_t)g * (uint64_t)k);
+          if (bits == 32) {
+            rc[i] = __float_as_uint(__ldg(reinterpret_cast<const float*>(p_code[i] + (uint64_t)g * (uint64_t)a.stride)));
+          } else {
+            rc[i] = (uint32_t)__ldg(p_code[i] + (uint64_t)g * (uint64_t)a.stride);
+            rs[i] = __ldg(p_scale[i] + g);
+          }
         }
       }
     }
@@ -199,8 +239,16 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       pos[i] = 0xFFFFu;
       val[i] = 0.0f;
       if (rep[i] >= 0) {
-        val[i] = bits == 32 ? __uint_as_float(rc[i]) : dequant((rc[i] >> cshift[i]) & cmask, rs[i], bits);
-        if (rp[i] != 0xFFFFu && rp[i] >= (uint32_t)kAC) bad = true; else pos[i] = rp[i];
+        uint32_t p;
+        if constexpr (GROUPED) {
+          p = (gi[i >> 1] >> (16 * (i & 1))) & 0xFFFFu;
+          val[i] = bits == 32 ? __uint_as_float(rc[i])
+                              : dequant((uint32_t)(gw >> (cshift[0] + (uint32_t)i * (uint32_t)bits)) & cmask, gs, bits);
+        } else {
+          p = rp[i];
+          val[i] = bits == 32 ? __uint_as_float(rc[i]) : dequant((rc[i] >> cshift[i]) & cmask, rs[i], bits);
+        }
+        if (p != 0xFFFFu && p >= (uint32_t)kAC) bad = true; else pos[i] = p;
       }
     }
     const uint64_t base_cur = base;
@@ -214,17 +262,32 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(acc)[tid + 256 * j] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
-    // pair i of all threads covers pairs 256 i .. 256 i + 255, i.e. the replicas r_lo..r_hi below (non-
-    // decreasing with i): one round per (i, replica) in that order applies every replica's entries
-    // after all entries of the replicas before it, with one predicated add per thread and round
+    if constexpr (GROUPED) {
+      // one round per replica: its owners read their cells, add, write back
+      for (int r = 0; r < R; ++r) {
+        if (my_r == r) {
+          float cur[NP];
 #pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int q_lo = kThreads * i;
-      if (q_lo < total) {
-        const int r_lo = q_lo / k, q_hi = min(q_lo + kThreads, total) - 1, r_hi = q_hi / k;
-        for (int r = r_lo; r <= r_hi; ++r) {
-          if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
-          __syncthreads();
+          for (int i = 0; i < NP; ++i) cur[i] = pos[i] != 0xFFFFu ? acc[pos[i]] : 0.0f;
+#pragma unroll
+          for (int i = 0; i < NP; ++i)
+            if (pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(cur[i], val[i]);
+        }
+        __syncthreads();
+      }
+    } else {
+      // pair i of all threads covers pairs 256 i .. 256 i + 255, i.e. the replicas r_lo..r_hi below (non-
+      // decreasing with i): one round per (i, replica) in that order applies every replica's entries
+      // after all entries of the replicas before it, with one predicated add per thread and round
+#pragma unroll
+      for (int i = 0; i < NP; ++i) {
+        const int q_lo = kThreads * i;
+        if (q_lo < total) {
+          const int r_lo = q_lo / k, q_hi = min(q_lo + kThreads, total) - 1, r_hi = q_hi / k;
+          for (int r = r_lo; r <= r_hi; ++r) {
+            if (rep[i] == r && pos[i] != 0xFFFFu) acc[pos[i]] = __fadd_rn(acc[pos[i]], val[i]);
+            __syncthreads();
+          }
         }
       }
     }
@@ -287,16 +350,24 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
     kernel<<<grid, kThreads, smem, st>>>(a);
     return cudaPeekAtLastError();
   };
+  const int np = pairs <= 1 ? 1 : pairs <= 2 ? 2 : pairs <= 4 ? 4 : 8;
+  const bool grouped = np > 1 && a.k % np == 0;     // (with one pair per thread the two mappings coincide)
   if (a.tb.side != 0) {
-    if (pairs <= 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, true>);
-    if (pairs <= 2) return launch(aggregate_c4096_kernel<T, APPLY, 2, true>);
-    if (pairs <= 4) return launch(aggregate_c4096_kernel<T, APPLY, 4, true>);
-    return launch(aggregate_c4096_kernel<T, APPLY, 8, true>);
+    if (np == 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, true, false>);
+    if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 2, true, true>)
+                                : launch(aggregate_c4096_kernel<T, APPLY, 2, true, false>);
+    if (np == 4) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 4, true, true>)
+                                : launch(aggregate_c4096_kernel<T, APPLY, 4, true, false>);
+    return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 8, true, true>)
+                   : launch(aggregate_c4096_kernel<T, APPLY, 8, true, false>);
   }
-  if (pairs <= 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, false>);
-  if (pairs <= 2) return launch(aggregate_c4096_kernel<T, APPLY, 2, false>);
-  if (pairs <= 4) return launch(aggregate_c4096_kernel<T, APPLY, 4, false>);
-  return launch(aggregate_c4096_kernel<T, APPLY, 8, false>);
+  if (np == 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, false, false>);
+  if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 2, false, true>)
+                              : launch(aggregate_c4096_kernel<T, APPLY, 2, false, false>);
+  if (np == 4) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 4, false, true>)
+                              : launch(aggregate_c4096_kernel<T, APPLY, 4, false, false>);
+  return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 8, false, true>)
+                 : launch(aggregate_c4096_kernel<T, APPLY, 8, false, false>);
 }
 
 __global__ void __launch_bounds__(256)
