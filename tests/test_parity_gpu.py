@@ -525,3 +525,26 @@ def test_peer_memory_replica_step_on_one_gpu():
         assert int(flags.item()) == 0
     finally:
         dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("k,bits,R", [
+    (128, 2, 16),    # 8 pairs per thread, a thread owns 8 slots of one replica
+    (128, 8, 16),    # ... whose codes span 8 bytes
+    (128, 32, 12),   # ... unquantised
+    (100, 2, 20),    # 8 pairs per thread, k not a multiple of 8: pairs 256 apart
+    (36, 4, 20),     # 4 pairs per thread, grouped
+    (6, 2, 64),      # 2 pairs per thread, grouped, codes start in mid-byte
+    (5, 2, 64),      # 2 pairs per thread, odd k
+    (7, 8, 40),
+])
+def test_aggregate_instances_for_many_pairs_per_chunk(k, bits, R):
+    sizes = [6 * 4096, 1024, 4096 + 2048, 4, 2 * 4096 + 4092, 4096]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), R, seed=1000 + k + bits + R)
+    for fused in (True, False):
+        gs, _, _ = run_and_compare(off, tg, tls, errs, 0.95, 4096, k, bits, 0.8,
+                                   what=f"aggregate k{k} b{bits} R{R} fused={fused}", fused=fused)
+    # the same instance without the fused outer update: the dense mean update on its own
+    upd = torch.full((int(off[-1]),), 7.0, dtype=torch.float32, device="cuda")
+    api.sl_aggregate(gs.idx, gs.codes, gs.scales, gs.layout, 4096, k, bits, upd, gs.flags)
+    assert_close(upd.cpu().numpy(), slo.aggregate(gs.messages_host(), off, 4096, k, bits), f"dense update k{k} b{bits} R{R}")
