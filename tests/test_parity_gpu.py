@@ -548,3 +548,54 @@ def test_aggregate_instances_for_many_pairs_per_chunk(k, bits, R):
     upd = torch.full((int(off[-1]),), 7.0, dtype=torch.float32, device="cuda")
     api.sl_aggregate(gs.idx, gs.codes, gs.scales, gs.layout, 4096, k, bits, upd, gs.flags)
     assert_close(upd.cpu().numpy(), slo.aggregate(gs.messages_host(), off, 4096, k, bits), f"dense update k{k} b{bits} R{R}")
+
+
+@pytest.mark.parametrize("cols", [None, "tiles"])
+def test_no_write_outside_the_callers_buffers(cols):
+    # every buffer handed to the library sits between two sentinel bands inside one allocation; after
+    # a whole outer step on a ragged arena (short chunks, a 3-element tensor, edge tiles) the bands
+    # must be untouched.  (compute-sanitizer is not available on the GPUs this runs on.)
+    sizes = [100 * 72, 4096 * 2 + 16, 4, 4096, 128 * 200, 8]     # multiples of 4: the tuned kernels take the full chunks
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    col_list = [72, 0, 0, 0, 200, 0] if cols else None
+    n, R, chunk, k, bits = int(off[-1]), 3, 4096, 64, 2
+    lay = api.Layout(off, col_list)
+    nc, st = api.sl_num_chunks(lay, chunk), api.sl_codes_stride(k, bits)
+    band = 1024                                  # bytes
+    need = [n * 4] * (1 + 2 * R) + [nc * k * 2] * R + [nc * st] * R + [nc * 4] * R
+    total = sum(band + (b + 255) // 256 * 256 for b in need) + band
+    pool = torch.full((total,), 0xA5, dtype=torch.uint8, device="cuda")
+    views, at = [], 0
+    for b in need:
+        at += band
+        views.append(pool[at:at + b])
+        at += (b + 255) // 256 * 256
+    f32v = lambda v: v.view(torch.float32)
+    tg_v, tl_v, err_v = f32v(views[0]), [f32v(v) for v in views[1:1 + R]], [f32v(v) for v in views[1 + R:1 + 2 * R]]
+    m = views[1 + 2 * R:]
+    idx_v = [v.view(torch.uint16) for v in m[:R]]
+    codes_v, sc_v = m[R:2 * R], [f32v(v) for v in m[2 * R:]]
+    tg, tls, errs = _case(n, R, seed=77)
+    tg_v.copy_(torch.from_numpy(tg))
+    for r in range(R):
+        tl_v[r].copy_(torch.from_numpy(tls[r]))
+        err_v[r].zero_()
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.sl_outer_step(tl_v, tg_v, err_v, lay, 0.95, chunk, k, bits, 0.8, idx_v, codes_v, sc_v, flags)
+    torch.cuda.synchronize()
+    # the result is the checker's ...
+    want = tg.copy()
+    h_err = [np.zeros(n, f32) for _ in range(R)]
+    msgs = oracle_compress_all(tls, want.copy(), h_err, off, 0.95, chunk, k, bits, cols=col_list)
+    upd = slo.aggregate([(i, c, s) for i, c, s, _ in msgs], off, chunk, k, bits, col_list)
+    slo.outer_apply(want, upd, 0.8)
+    assert_close(tg_v.cpu().numpy(), want, "guarded theta_global")
+    # ... and nothing outside the buffers changed
+    mask = torch.ones(total, dtype=torch.bool, device="cuda")
+    at = 0
+    for b in need:
+        at += band
+        mask[at:at + b] = False
+        at += (b + 255) // 256 * 256
+    assert bool((pool[mask] == 0xA5).all()), "a byte outside the caller's buffers was written"
+    assert int(flags.item()) == 0
