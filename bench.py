@@ -215,10 +215,39 @@ def time_oracle(wl_sample: synth.Workload, steps: int, warmup: int, seed: int, i
     return times, threads
 
 
+def run_reference_embed(args) -> None:
+    """--impl reference --embed: the float64 numpy checker of Eqs. 3-4 on a bounded sample of the rows."""
+    from oracle import embed as oe
+    wl = synth.workload(args.workload)
+    name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
+    k = args.k or d // 8
+    rows = min(V, 4000)
+    U = synth.gen_subspace_basis(d, k, args.seed)
+    T_S, T_perp = synth.gen_embedding_pair(rows, d, args.seed)
+    times = []
+    for s in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        oe.embed_reproject(T_S, T_perp, U)
+        if s >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    sec = float(np.mean(times))
+    desc = f"{rows} rows of a {V}x{d} table, k={k}, float64 numpy"
+    print(json.dumps({
+        "impl": "reference", "metric": "embed_reproject_rows_per_s", "value": rows / sec, "unit": "rows/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name} token embedding {V}x{d}, k={k}", "sample": desc},
+        "cpu_baseline": {"value": rows / sec, "unit": "rows/s", "cores": os.cpu_count(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": rows / sec, "unit": "rows/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
 def run_reference(args) -> None:
     rank, _, world = dist_env()
     if rank != 0:
         return
+    if args.embed:
+        return run_reference_embed(args)
     wl = synth.workload(args.workload)
     sample = cpu_sample_workload(wl)
     times, threads = time_oracle(sample, args.steps, args.warmup, args.seed)
