@@ -599,3 +599,38 @@ def test_no_write_outside_the_callers_buffers(cols):
         at += (b + 255) // 256 * 256
     assert bool((pool[mask] == 0xA5).all()), "a byte outside the caller's buffers was written"
     assert int(flags.item()) == 0
+
+
+@pytest.mark.parametrize("seed", list(range(24)))
+def test_random_configurations(seed):
+    # seeded random arenas (aligned or not, with short and tiny tensors, sometimes tiled), k, code
+    # width, R and beta: whichever kernels the dispatch picks, the step must match the checker
+    rng = np.random.default_rng(1234 + seed)
+    chunk = int(rng.choice([4096, 4096, 4096, 1024, 256, 100]))
+    tiled = chunk in (4096, 1024, 256) and rng.random() < 0.35
+    side = int(round(chunk ** 0.5))
+    align = 4 if rng.random() < 0.7 else 1
+    sizes, cols = [], []
+    for _ in range(int(rng.integers(1, 7))):
+        if tiled and rng.random() < 0.7:
+            r, c = int(rng.integers(1, 3 * side)), int(rng.integers(1, 3 * side))
+            c = max(align, c // align * align)
+            sizes.append(r * c)
+            cols.append(c)
+        else:
+            n = int(rng.integers(1, 3 * chunk + 50))
+            sizes.append(max(align, n // align * align))
+            cols.append(0)
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    k = int(rng.choice([1, 2, 5, 8, 16, 32, 64, 128]))
+    k = min(k, chunk)
+    bits = int(rng.choice([2, 4, 8, 32]))
+    R = int(rng.choice([1, 2, 3, 5, 8, 16]))
+    beta = float(rng.choice([0.0, 0.5, 0.95, 1.0]))
+    tg, tls, errs = _case(int(off[-1]), R, seed=5000 + seed)
+    errs = [(np.random.default_rng(seed * 31 + r).normal(0, 5e-4, int(off[-1]))).astype(f32) for r in range(R)]
+    nxt = lambda t, g: [(g + np.random.default_rng(seed * 1000 + t * 10 + r).normal(0, 1e-3, g.size)).astype(f32)
+                        for r in range(R)]
+    run_and_compare(off, tg, tls, errs, beta, chunk, k, bits, 0.8, rounds=2, next_locals=nxt,
+                    what=f"random #{seed}: chunk {chunk} k {k} b {bits} R {R} tiled {tiled} align {align}",
+                    fused=bool(seed % 2), cols=cols if tiled else None)
