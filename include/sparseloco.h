@@ -171,13 +171,16 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* layout, int chunk, i
  * The split made before training (same section: T_S <- TE U U^T, T_perp <- TE - T_S) is the
  * same call on T_S = TE and T_perp = 0.
  * T_S, T_perp: DEVICE, float32, V x d row-major, read and written.  U: DEVICE, float32, d x k
- * row-major (orthonormal columns; not checked), read only.  All three 16-byte aligned.
- * The two contractions run on the tensor cores in TF32 (operands cut to 10 mantissa bits,
- * float32 accumulation); the subtraction and the addition are float32, each rounded once, and
- * use the very value that is stored to T_S, so T_S + T_perp is conserved to float32 rounding.
- * Needs d % 4 == 0, k % 4 == 0, 4 <= k <= 256, V < 2^31 (else SL_ERR_UNSUPPORTED); V = 0 is a
- * no-op.  `flags` (DEVICE, may be NULL) receives SL_FLAG_TIMEOUT if an internal wait gave up,
- * in which case the tables' contents are unspecified.  Asynchronous on `stream`. */
+ * row-major (orthonormal columns; not checked), read only.
+ * Tuned path (d % 4 == 0, k % 4 == 0, 4 <= k <= 256, all three pointers 16-byte aligned): the two
+ * contractions run on the tensor cores in TF32 (operands cut to 10 mantissa bits, float32
+ * accumulation).  Any other shape with k <= 4096 (the paper's most aggressive settings reach
+ * k = 2) takes a plain float32 kernel (fused multiply-adds in index order), slower and exact to
+ * float32 rounding.  In both, the subtraction and the addition are float32, each rounded once,
+ * and use the very value that is stored to T_S, so T_S + T_perp is conserved to float32 rounding.
+ * V < 2^31 (else SL_ERR_UNSUPPORTED); V = 0 is a no-op.  `flags` (DEVICE, may be NULL) receives
+ * SL_FLAG_TIMEOUT if an internal wait of the tuned kernel gave up, in which case the tables'
+ * contents are unspecified.  Asynchronous on `stream`. */
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                        uint32_t* flags, void* stream);
 

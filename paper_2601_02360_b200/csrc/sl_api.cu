@@ -310,10 +310,10 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* L, int chunk, int k,
 
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                        uint32_t* flags, void* stream) {
-  if (!T_S || !T_perp || !U) return SL_ERR_INVALID_ARG;
-  if (!aligned(T_S, 16) || !aligned(T_perp, 16) || !aligned(U, 16) || (flags && !aligned(flags, 4)))
+  if (!T_S || !T_perp || !U || d < 1 || k < 1) return SL_ERR_INVALID_ARG;
+  if (!aligned(T_S, 4) || !aligned(T_perp, 4) || !aligned(U, 4) || (flags && !aligned(flags, 4)))
     return SL_ERR_ALIGNMENT;
-  if (d < 4 || d % 4 != 0 || k < 4 || k % 4 != 0 || k > 256 || V > 0x7FFFFFFFull) return SL_ERR_UNSUPPORTED;
+  if (V > 0x7FFFFFFFull || k > 4096) return SL_ERR_UNSUPPORTED;
   if (V == 0) return SL_OK;
   return launch_embed_reproject(T_S, T_perp, U, V, d, k, flags, (cudaStream_t)stream) == cudaSuccess
              ? SL_OK : SL_ERR_CUDA;

@@ -441,10 +441,60 @@ bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, ui
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Shapes the tensor-core kernel does not take (k or d not a multiple of 4, k above 256, unaligned
+// pointers): plain float32 fused multiply-adds, one CTA per kGenRows rows.  The coordinates
+// P = T_S U of those rows sit in shared memory; then every column of the rows is rebuilt from
+// them and Eqs. 3-4 are applied in place.  Slow (U is streamed from L2 for every CTA) but exact
+// to float32 rounding; needs kGenRows * k floats of shared memory (k <= 4096).
+constexpr int kGenRows = 8;
+constexpr int kGenThreads = 256;
+
+__global__ void __launch_bounds__(kGenThreads)
+embed_reproject_generic_kernel(float* __restrict__ T_S, float* __restrict__ T_perp, const float* __restrict__ U,
+                               uint64_t V, uint32_t d, uint32_t k) {
+  extern __shared__ float coord[];              // [kGenRows][k]
+  const uint64_t r0 = (uint64_t)blockIdx.x * kGenRows;
+  const uint32_t rows = (uint32_t)(V - r0 < (uint64_t)kGenRows ? V - r0 : (uint64_t)kGenRows);
+  // coordinates: thread -> (row, j); the row's elements are broadcast, U[i][j..] is read coalesced
+  for (uint32_t t = threadIdx.x; t < rows * k; t += kGenThreads) {
+    const uint32_t r = t / k, j = t - r * k;
+    const float* ts = T_S + (r0 + r) * d;
+    float acc = 0.0f;
+    for (uint32_t i = 0; i < d; ++i) acc = __fmaf_rn(ts[i], U[(uint64_t)i * k + j], acc);
+    coord[r * k + j] = acc;
+  }
+  __syncthreads();                              // every read of the old rows for the coordinates is done
+  for (uint32_t t = threadIdx.x; t < rows * d; t += kGenThreads) {
+    const uint32_t r = t / d, n = t - r * d;
+    const float* u = U + (uint64_t)n * k;
+    const float* c = coord + r * k;
+    float pi = 0.0f;
+    for (uint32_t j = 0; j < k; ++j) pi = __fmaf_rn(c[j], u[j], pi);
+    const uint64_t at = (r0 + r) * d + n;
+    T_perp[at] = __fadd_rn(T_perp[at], __fsub_rn(T_S[at], pi));
+    T_S[at] = pi;
+  }
+}
+
 }  // namespace
+
+bool embed_is_tuned(const float* T_S, const float* T_perp, const float* U, uint32_t d, uint32_t k) {
+  auto al16 = [](const void* p) { return ((uintptr_t)p & 15u) == 0; };
+  return d % 4 == 0 && k % 4 == 0 && k >= 4 && k <= 256 && al16(T_S) && al16(T_perp) && al16(U);
+}
 
 cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                                    uint32_t* flags, cudaStream_t st) {
+  if (!embed_is_tuned(T_S, T_perp, U, d, k)) {
+    const size_t smem = (size_t)kGenRows * k * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(embed_reproject_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    const uint64_t grid = (V + kGenRows - 1) / kGenRows;
+    if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    embed_reproject_generic_kernel<<<(unsigned)grid, kGenThreads, smem, st>>>(T_S, T_perp, U, V, d, k);
+    return cudaGetLastError();
+  }
   // a box row of the tables is 128 bytes of a much longer row whose neighbouring 128 bytes are wanted
   // next (the next 32-column part, the next K step): fetch 256 bytes into L2 at a time
   constexpr CUtensorMapL2promotion kTablePromo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;

@@ -116,11 +116,14 @@ def test_embed_reproject_argument_checks():
     call = lambda ts, tp, u, V, d, k: L.sl_embed_reproject(ts, tp, u, V, d, k, None, None)
     assert call(None, fake, fake, 8, 64, 8) == api.SL_ERR_INVALID_ARG
     assert call(fake, fake, None, 8, 64, 8) == api.SL_ERR_INVALID_ARG
-    assert call(fake + 4, fake, fake, 8, 64, 8) == api.SL_ERR_ALIGNMENT
-    assert call(fake, fake, fake + 8, 8, 64, 8) == api.SL_ERR_ALIGNMENT
-    for d, k in [(62, 8), (64, 6), (64, 0), (64, 260), (0, 4)]:
-        assert call(fake, fake, fake, 8, d, k) == api.SL_ERR_UNSUPPORTED
-    assert call(fake, fake, fake, 0, 64, 8) == api.SL_OK        # an empty table is a no-op
+    assert call(fake, fake, fake, 8, 64, 0) == api.SL_ERR_INVALID_ARG
+    assert call(fake, fake, fake, 8, 0, 4) == api.SL_ERR_INVALID_ARG
+    assert call(fake + 2, fake, fake, 8, 64, 8) == api.SL_ERR_ALIGNMENT
+    assert call(fake, fake, fake + 1, 8, 64, 8) == api.SL_ERR_ALIGNMENT
+    assert call(fake, fake, fake, 8, 64, 5000) == api.SL_ERR_UNSUPPORTED      # k above 4096
+    assert call(fake, fake, fake, 1 << 31, 64, 8) == api.SL_ERR_UNSUPPORTED   # V at or above 2^31
+    assert call(fake, fake, fake, 0, 64, 8) == api.SL_OK                      # an empty table is a no-op
+    assert call(fake, fake, fake, 0, 62, 6) == api.SL_OK
 
 
 def test_idx12_argument_checks():

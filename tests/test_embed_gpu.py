@@ -182,3 +182,40 @@ def test_neighbouring_memory_is_untouched():
     assert np.array_equal(hs[:32], T_S[:32]) and np.array_equal(hs[32 + V:], T_S[32 + V:])
     assert np.array_equal(hp[:32], T_perp[:32]) and np.array_equal(hp[32 + V:], T_perp[32 + V:])
     _check(T_S[32:32 + V], T_perp[32:32 + V], U, hs[32:32 + V], hp[32:32 + V])
+
+
+GEN_TOL = 2.0 ** -20      # float32 fused multiply-adds over d and k terms: far below (d + k) * 2^-24 of B in practice
+
+
+@pytest.mark.parametrize("V,d,k", [(50, 1536, 2), (33, 10, 3), (9, 7, 7), (100, 62, 6), (20, 64, 300), (17, 5, 1),
+                                   (300, 2048, 260)])
+def test_shapes_outside_the_tensor_core_path(V, d, k):
+    # the paper's smallest subspaces (k = 2 at d = 1536), odd d and k, k above 256: plain float32 kernel
+    if k <= d:
+        U = synth.gen_subspace_basis(d, k, seed=31)
+    else:     # more columns than rows cannot be orthonormal; the call does not check, any matrix will do
+        U = (np.random.default_rng(31).standard_normal((d, k)) / np.sqrt(k)).astype(np.float32)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=32)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, U)
+    ref_ts, ref_tp = oe.embed_reproject(T_S, T_perp, U)
+    B = oe.abs_bound(T_S, U)
+    assert np.all(np.abs(ts_gpu - ref_ts) <= GEN_TOL * B + 1e-30), float((np.abs(ts_gpu - ref_ts) / (B + 1e-30)).max())
+    assert np.array_equal(tp_gpu, (T_perp + (T_S - ts_gpu)).astype(np.float32))
+    assert np.all(np.abs(tp_gpu - ref_tp) <= GEN_TOL * B + 2.0 ** -22 * (np.abs(ref_tp) + np.abs(T_S) + np.abs(ref_ts)))
+
+
+def test_unaligned_tables_take_the_plain_kernel():
+    V, d, k = 40, 128, 32
+    U = synth.gen_subspace_basis(d, k, seed=33)
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=34)
+    buf = torch.zeros(V * d + 1, dtype=torch.float32, device="cuda")
+    ts = buf[1:]                                   # 4-byte aligned only
+    ts.copy_(torch.from_numpy(T_S).reshape(-1))
+    tp, u = torch.from_numpy(T_perp).cuda(), torch.from_numpy(U).cuda()
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.sl_embed_reproject(ts, tp, u, V, d, k, flags)
+    torch.cuda.synchronize()
+    ref_ts, _ = oe.embed_reproject(T_S, T_perp, U)
+    got = ts.cpu().numpy().reshape(V, d)
+    assert np.all(np.abs(got - ref_ts) <= GEN_TOL * oe.abs_bound(T_S, U) + 1e-30)
+    assert float(buf[0].item()) == 0.0 and int(flags.item()) == 0
