@@ -63,7 +63,7 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
 // Tuned kernel for full 4096-element chunks of a 16-byte aligned arena.  Persistent grid: CTA b
 // walks the full chunks among b, b+G, b+2G, ...  Software pipelined over chunks: while chunk i is
 // accumulated and written, the next chunk's theta_global is already on its way into shared memory
-// (one 16 KB TMA bulk copy, no multicast, double buffered, mbarrier completion) and its message
+// (one 16 KB TMA bulk copy per CTA, double buffered, mbarrier completion) and its message
 // entries are on their way into registers.  Per chunk:
 //  * the (replica, slot) pairs of the chunk are spread over the threads, NP per thread: pair
 //    q = tid + 256 i is slot q % k of replica q / k.  What does not depend on the chunk (replica,

@@ -220,7 +220,7 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 // handles the items w with w % kSel == q, so two selections are in flight while the producers
 // run ahead.
 //
-//  * Bulk data moves by TMA (cp.async.bulk + mbarrier complete_tx, no multicast).  theta_local of
+//  * Bulk data moves by TMA (cp.async.bulk + mbarrier complete_tx, every CTA fetching its own data).  theta_local of
 //    item w+2 is loaded by producer thread 0 into a 2-deep ring (a stage is dead after phase A).
 //    e lives in a 4-deep ring: loaded four items ahead by the selector that owns the stage,
 //    overwritten in place with e' by the producers, patched with the residual by the selector,

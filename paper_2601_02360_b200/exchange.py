@@ -15,8 +15,8 @@ parameters.
 buffer that all ranks of the node have mapped (symmetric memory over NVLink), and after one
 barrier `sl_aggregate_apply` is handed the PEERS' buffers as its message tables, so the
 averaging kernel pulls each chunk's messages over NVLink with plain loads while it works through
-the chunks - the transfer and the arithmetic overlap chunk by chunk, nothing is staged, and no
-load from a peer uses TMA multicast (the kernels read messages with ordinary read-only loads).
+the chunks - the transfer and the arithmetic overlap chunk by chunk, nothing is staged, and every
+load from a peer is an ordinary read-only load issued by the thread that needs the value.
 
 `outer_step_replica_pipelined` cuts the arena into groups of consecutive tensors and overlaps the
 gather of one group's message with the compression of the next group (two CUDA streams); the
