@@ -89,8 +89,11 @@ def test_exchange_with_12_bit_positions_on_one_gpu():
     import torch.distributed as dist
     from paper_2601_02360_b200 import exchange
     s = socket.socket(); s.bind(("127.0.0.1", 0)); port = s.getsockname()[1]; s.close()
-    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
-                            device_id=torch.device("cuda", 0))
+    try:
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                                device_id=torch.device("cuda", 0))
+    except Exception as exc:  # an environment without a usable NCCL: nothing of ours has run yet
+        pytest.skip(f"one-rank NCCL group unavailable: {exc}")
     try:
         wl = synth.sub_arena(synth.workload("180m"), [0, 1, 7, 8, 9]).replace(R=1)
         off = wl.offsets()
