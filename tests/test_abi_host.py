@@ -138,3 +138,20 @@ def test_idx12_argument_checks():
     assert L.sl_unpack_idx12(None, lay.ref(), 4096, 64, fake, None) == api.SL_ERR_INVALID_ARG
     assert L.sl_unpack_idx12(fake, lay.ref(), 8192, 64, fake, None) == api.SL_ERR_UNSUPPORTED   # 13-bit positions
     assert L.sl_unpack_idx12(fake, lay.ref(), 4096, 64, fake + 1, None) == api.SL_ERR_ALIGNMENT
+
+
+def test_header_is_valid_c_and_a_c_client_links(lib, tmp_path):
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    exe = str(tmp_path / "abi_c_client")
+    libdir = os.path.dirname(build.LIB_PATH)
+    cmd = ["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"),
+           os.path.join(ROOT, "tests", "support", "abi_c_client.c"), "-o", exe,
+           "-L", libdir, "-lsparseloco", f"-Wl,-rpath,{libdir}"]
+    built = subprocess.run(cmd, capture_output=True, text=True)
+    assert built.returncode == 0, built.stderr[-2000:]
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+    assert run.returncode == 0, (run.returncode, run.stdout, run.stderr[-1000:])
+    assert run.stdout.startswith("c client ok")
