@@ -1,1 +1,2 @@
-"""CPU checker of the SparseLoCo outer step: test infrastructure only."""
+"""CPU checkers of the SparseLoCo outer step (slo), of the 12-bit position format (idx12) and of the
+embedding re-projection (embed): test infrastructure only, never on the product path."""
