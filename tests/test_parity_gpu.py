@@ -545,6 +545,8 @@ def test_peer_memory_replica_step_on_one_gpu():
     (6, 2, 64),      # 2 pairs per thread, grouped, codes start in mid-byte
     (5, 2, 64),      # 2 pairs per thread, odd k
     (7, 8, 40),
+    (32, 2, 64),     # the most replicas a call takes: 64 rounds, 8 slots per thread
+    (16, 4, 64),
 ])
 def test_aggregate_instances_for_many_pairs_per_chunk(k, bits, R):
     sizes = [6 * 4096, 1024, 4096 + 2048, 4, 2 * 4096 + 4092, 4096]
