@@ -468,6 +468,7 @@ def run_embed(args) -> None:
     name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
     k = args.k or d // 8
     U = torch.from_numpy(synth.gen_subspace_basis(d, k, args.seed)).to(dev)
+    api.sl_round_tf32(U, U.numel())          # once, as the header asks: U never changes
     T_S_h, T_perp_h = synth.gen_embedding_pair(V, d, args.seed)
     T_S0 = torch.from_numpy(T_S_h).to(dev)
     T_S, T_perp = T_S0.clone(), torch.from_numpy(T_perp_h).to(dev)

@@ -173,8 +173,12 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* layout, int chunk, i
  * T_S, T_perp: DEVICE, float32, V x d row-major, read and written.  U: DEVICE, float32, d x k
  * row-major (orthonormal columns; not checked), read only.
  * Tuned path (d % 4 == 0, k % 4 == 0, 4 <= k <= 256, all three pointers 16-byte aligned): the two
- * contractions run on the tensor cores in TF32 (operands cut to 10 mantissa bits, float32
- * accumulation).  Any other shape with k <= 4096 (the paper's most aggressive settings reach
+ * contractions run on the tensor cores in TF32 with float32 accumulation.  The hardware cuts a
+ * float32 operand to TF32 (10 mantissa bits) instead of rounding it, which would shorten every
+ * product; the kernel therefore rounds the T_S tiles and the intermediate coordinates to the
+ * nearest TF32 value itself.  U is read as it is: round it once with sl_round_tf32 (it is a
+ * fixed matrix), otherwise the projection comes out about 7e-4 short in magnitude - a difference
+ * that stays in T_perp like any other residual.  Any other shape with k <= 4096 (the paper's most aggressive settings reach
  * k = 2) takes a plain float32 kernel (fused multiply-adds in index order), slower and exact to
  * float32 rounding.  In both, the subtraction and the addition are float32, each rounded once,
  * and use the very value that is stored to T_S, so T_S + T_perp is conserved to float32 rounding.
@@ -183,6 +187,10 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* layout, int chunk, i
  * contents are unspecified.  Asynchronous on `stream`. */
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                        uint32_t* flags, void* stream);
+
+/* x[i] <- the TF32 value nearest to x[i] (ties away from zero), kept as float32, for i < n; in place.
+ * For matrices that are fed to the tensor cores many times and never change (U above). */
+int sl_round_tf32(float* x, uint64_t n, void* stream);
 
 /* Static description of an SL_* return code. */
 const char* sl_strerror(int code);

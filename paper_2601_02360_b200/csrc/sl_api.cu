@@ -308,6 +308,12 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* L, int chunk, int k,
                              : unpack_impl<SL_MAX_TENSORS>(packed, L, chunk, k, idx, st);
 }
 
+int sl_round_tf32(float* x, uint64_t n, void* stream) {
+  if (!x && n) return SL_ERR_INVALID_ARG;
+  if (!aligned(x, 4)) return SL_ERR_ALIGNMENT;
+  return launch_round_tf32(x, n, (cudaStream_t)stream) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+}
+
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                        uint32_t* flags, void* stream) {
   if (!T_S || !T_perp || !U || d < 1 || k < 1) return SL_ERR_INVALID_ARG;

@@ -14,6 +14,11 @@
 //            buffered in tensor memory.  (An MMA of N = 64 costs as many cycles as one of
 //            N = 128, so the blocks are 128 wide; the epilogue takes them in parts of 32.)
 //
+// The tensor cores cut (do not round) a float32 operand to TF32, which would shorten the result by
+// about 1.5e-3 at every call; so the epilogue warps, idle during pass 1, round each T_S tile to the
+// nearest TF32 value in shared memory before the MMA warp may use it, and round P in tensor memory
+// between the passes.  U is used as given (the caller rounds it once: it never changes).
+//
 // All global traffic is bulk tensor copies (TMA): warp 0 loads the MMA operands; warp 6 loads,
 // for pass 2, the T_S / T_perp tiles of each 32-column part into swizzled shared-memory buffers;
 // warp 1 owns tensor memory and issues the MMAs; warps 2-5 (one thread per row) read O from
@@ -51,9 +56,10 @@ static_assert(kEBufs * kESize + kRing2InX * kSlot2 == kRing1 * kSlot1, "pass-2 b
 struct EmbedSmem {
   uint8_t x[kRing1 * kSlot1];                   // pass 1: operand ring; pass 2: tile buffers + ring slots
   uint8_t y[kRing2 - kRing2InX][kSlot2];
-  uint64_t full1[kRing1], empty1[kRing1], full2[kRing2], empty2[kRing2];
+  uint64_t full1[kRing1], ready1[kRing1], empty1[kRing1], full2[kRing2], empty2[kRing2];
   uint64_t o_full[2], o_empty[2], e_full[kEBufs], e_empty[kEBufs], e_done[kEBufs];
   uint64_t p_done, x_free;   // per sub-tile: pass 1 has read its ring / pass 2 has left the shared region
+  uint64_t p_ready;          // per sub-tile: the coordinates in tensor memory have been rounded to TF32
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
@@ -119,6 +125,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+      "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+      :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+         "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+         "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// float32 -> the nearest TF32 value (ties away from zero), as a float32 bit pattern
+__device__ __forceinline__ uint32_t round_tf32(uint32_t bits) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(__uint_as_float(bits)));
+  return r;
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
@@ -162,13 +185,14 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
 
   if (tid == 0) {
-    for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 1); mbar_init(&sm.empty1[s], 1); }
+    for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 1); mbar_init(&sm.ready1[s], 4); mbar_init(&sm.empty1[s], 1); }
     for (int s = 0; s < kRing2; ++s) { mbar_init(&sm.full2[s], 1); mbar_init(&sm.empty2[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
     for (int b = 0; b < kEBufs; ++b) {
       mbar_init(&sm.e_full[b], 1); mbar_init(&sm.e_empty[b], 1); mbar_init(&sm.e_done[b], 4);
     }
     mbar_init(&sm.p_done, 1);
+    mbar_init(&sm.p_ready, 4);
     mbar_init(&sm.x_free, 1);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -303,16 +327,16 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
   } else if (warp == 1) {
     if (lane == 0) {
       // ---- MMA issuer ----
-      uint32_t it1 = 0, it2 = 0, cg = 0;
+      uint32_t it1 = 0, it2 = 0, cg = 0, t = 0;
       bool ok = true;
       const uint32_t idesc1 = instr_desc(kRows, (int)kp, 1);
       const uint32_t idesc2 = instr_desc(kRows, kBlockN, 0);
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2);      // K-major tile, rows of 128 bytes
       const uint64_t desc_n = smem_desc(0, 4096, 512, 1);     // U rows as N-major operand
-      for (uint64_t g = g0; ok && g < g1; g += 4) {
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
         for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
           const uint32_t s = it1 % kRing1;
-          ok = mbar_wait(&sm.full1[s], (it1 / kRing1) & 1u, sm);
+          ok = mbar_wait(&sm.ready1[s], (it1 / kRing1) & 1u, sm);      // landed and rounded (see the epilogue warps)
           if (!ok) break;
           tc_fence_after();
           const uint32_t a0 = smem_u32(sm.x + s * kSlot1);
@@ -324,6 +348,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           mma_commit(&sm.empty1[s]);
         }
         if (ok) mma_commit(&sm.p_done);
+        ok = ok && mbar_wait(&sm.p_ready, t & 1u, sm);   // the epilogue warps have rounded P in place
         for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
           const uint32_t buf = cg & 1u;
           ok = wait_last(&sm.o_empty[buf], cg >> 1);
@@ -350,10 +375,52 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     const int q = warp & 3;
     const uint32_t row = (uint32_t)(32 * q + lane);
     const uint32_t sw = row & 7u;
-    uint32_t cg = 0, hcg = 0;
+    uint32_t cg = 0, hcg = 0, t = 0, it1 = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4) {
+    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
       const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+      // The tensor cores CUT a float32 operand to TF32, which would shorten every product; values that
+      // are already TF32 pass through unchanged.  So during pass 1 these warps round every T_S tile to the
+      // nearest TF32 value in place as soon as it has landed (element-wise: the swizzle is irrelevant) and
+      // only then hand it to the MMA warp; between the passes they do the same to the coordinates P in
+      // tensor memory.  (U is not touched: round it once with sl_round_tf32, it never changes.)
+      for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
+        const uint32_t s = it1 % kRing1;
+        ok = mbar_wait(&sm.full1[s], (it1 / kRing1) & 1u, sm);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t a0 = smem_u32(sm.x + s * kSlot1) + (uint32_t)(tid - 64) * 16;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float4 v = lds128(a0 + 2048 * i);
+          v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+          v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+          v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+          v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+          sts128(a0 + 2048 * i, v);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ready1[s]);
+      }
+      if (!ok) break;
+      ok = mbar_wait(&sm.p_done, t & 1u, sm);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      for (uint32_t cb = 0; cb < kp; cb += 32) {
+        uint32_t v[32];
+        const uint32_t ta = t_p + cb + ((uint32_t)(32 * q) << 16);
+        tmem_ld32(ta, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = round_tf32(v[i]);
+        tmem_st32(ta, v);
+      }
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.p_ready);
       for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
         const uint32_t buf = cg & 1u;
         const uint32_t left = (d - c * kBlockN + kPartN - 1) / kPartN;
@@ -441,6 +508,11 @@ bool make_map(CUtensorMap* m, const float* p, uint64_t inner, uint64_t outer, ui
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+__global__ void __launch_bounds__(256) round_tf32_kernel(float* __restrict__ x, uint64_t n) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
+    x[i] = __uint_as_float(round_tf32(__float_as_uint(x[i])));
+}
+
 // Shapes the tensor-core kernel does not take (k or d not a multiple of 4, k above 256, unaligned
 // pointers): plain float32 fused multiply-adds, one CTA per kGenRows rows.  The coordinates
 // P = T_S U of those rows sit in shared memory; then every column of the rows is rebuilt from
@@ -477,6 +549,13 @@ embed_reproject_generic_kernel(float* __restrict__ T_S, float* __restrict__ T_pe
 }
 
 }  // namespace
+
+cudaError_t launch_round_tf32(float* x, uint64_t n, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  const uint64_t blocks = (n + 255) / 256;
+  round_tf32_kernel<<<(unsigned)(blocks < 148u * 16u ? blocks : 148u * 16u), 256, 0, st>>>(x, n);
+  return cudaGetLastError();
+}
 
 bool embed_is_tuned(const float* T_S, const float* T_perp, const float* U, uint32_t d, uint32_t k) {
   auto al16 = [](const void* p) { return ((uintptr_t)p & 15u) == 0; };

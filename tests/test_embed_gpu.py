@@ -62,7 +62,11 @@ def test_parity_random(V, d, k):
     T_S, T_perp = synth.gen_embedding_pair(V, d, seed=2)
     ts_gpu, tp_gpu = _run(T_S, T_perp, U)
     err, ref = _check(T_S, T_perp, U, ts_gpu, tp_gpu)
-    # typical (not worst-case) accuracy: random signs make the error far smaller than the bound
+    # typical accuracy.  The tensor cores CUT a float32 operand to TF32 (they do not round).  The kernel
+    # rounds T_S and the coordinates itself; U is used as given (not rounded in this test), so each of
+    # its two uses loses between 0 and 2^-10 of its magnitude, about 0.75 * 2^-11 on average for these
+    # values: the result comes out about 7e-4 short.  The difference stays in T_perp (checked above:
+    # T_S + T_perp is conserved).
     assert np.sqrt((err ** 2).mean()) <= 2.0 ** -9 * np.sqrt((ref ** 2).mean())
 
 
@@ -219,3 +223,45 @@ def test_unaligned_tables_take_the_plain_kernel():
     got = ts.cpu().numpy().reshape(V, d)
     assert np.all(np.abs(got - ref_ts) <= GEN_TOL * oe.abs_bound(T_S, U) + 1e-30)
     assert float(buf[0].item()) == 0.0 and int(flags.item()) == 0
+
+
+def _tf32_rna(x):
+    """float32 -> nearest TF32 value (10 explicit mantissa bits), ties away from zero: the definition."""
+    b = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    b = ((b + 0x1000) & ~np.uint64(0x1FFF)).astype(np.uint32)        # add half of the cut part, clear it
+    return b.view(np.float32)
+
+
+def test_round_tf32_helper():
+    rng = np.random.default_rng(41)
+    x = np.concatenate([rng.standard_normal(5000).astype(np.float32) * np.float32(10.0) ** rng.integers(-20, 20, 5000),
+                        np.array([0.0, -0.0, 1.0, 1.0 + 2.0 ** -11, 1.0 + 2.0 ** -11 + 2.0 ** -23, 1.0 + 2.0 ** -10,
+                                  -(1.0 + 2.0 ** -11), 3.0e38, 1e-40, np.inf, -np.inf], dtype=np.float32)]).astype(np.float32)
+    t = torch.from_numpy(x.copy()).cuda()
+    api.sl_round_tf32(t, t.numel())
+    got = t.cpu().numpy()
+    want = _tf32_rna(x)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert np.all((got.view(np.uint32) & 0x1FFF) == 0)                 # representable in TF32
+    assert got[5002] == 1.0 and got[5003] == np.float32(1.0 + 2.0 ** -10)   # the tie goes away from zero
+    api.sl_round_tf32(t, t.numel())
+    assert np.array_equal(t.cpu().numpy().view(np.uint32), got.view(np.uint32))   # idempotent
+
+
+@pytest.mark.parametrize("V,d,k", [(2000, 2048, 256), (1000, 1024, 32)])
+def test_no_systematic_shortening_with_a_rounded_basis(V, d, k):
+    # with U rounded once (sl_round_tf32) every operand the tensor cores see is a TF32 value: what is
+    # left are rounding errors of random sign, far smaller than the 7e-4 that a cut basis costs
+    U = synth.gen_subspace_basis(d, k, seed=42)
+    u = torch.from_numpy(U).cuda()
+    api.sl_round_tf32(u, u.numel())
+    Ur = u.cpu().numpy()
+    assert np.array_equal(Ur.view(np.uint32), _tf32_rna(U).view(np.uint32))
+    T_S, T_perp = synth.gen_embedding_pair(V, d, seed=43)
+    ts_gpu, tp_gpu = _run(T_S, T_perp, Ur)
+    err, ref = _check(T_S, T_perp, Ur, ts_gpu, tp_gpu)
+    rel = np.sqrt((err ** 2).mean()) / np.sqrt((ref ** 2).mean())
+    assert rel <= 2.0 ** -11, rel
+    # no bias: the result is neither systematically shorter nor longer than the exact projection
+    ratio = float((ts_gpu.astype(np.float64) * ref).sum() / (ref * ref).sum())
+    assert abs(ratio - 1.0) <= 1e-4, ratio
