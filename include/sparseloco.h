@@ -188,6 +188,28 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* layout, int chunk, i
 int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,
                        uint32_t* flags, void* stream);
 
+/* Subspace compression of the activations that cross a pipeline-stage boundary (paper section 2.3).
+ * X: n_tok x d activations of a flattened batch (token t sits at position t mod L); ids: the
+ * tokens (int32, n_tok); T_perp: V x d, the fixed high-rank part of the embedding table; pos:
+ * L x d positional embedding; U: d x k orthonormal basis (round it once with sl_round_tf32).
+ *   sl_subspace_project:      Xt[t,:]   = (X[t,:] - T_perp[ids[t],:] - pos[t mod L,:]) U     n_tok x k
+ *                             with ids == NULL (activation gradients): Xt = X U
+ *   sl_subspace_reconstruct:  Xhat[t,:] = Xt[t,:] U^T + T_perp[ids[t],:] + pos[t mod L,:]    n_tok x d
+ *                             with ids == NULL: Xhat = Xt U^T
+ * All DEVICE, float32 row-major, inputs read only, the output fully overwritten.  Arithmetic: the
+ * differences / sums are float32, one rounding per operation in the order written; the
+ * contraction runs on the tensor cores in TF32 (its float32 operand - the difference, resp. Xt -
+ * rounded to the nearest TF32 value first) with float32 accumulation, for d % 4 == 0, k % 4 == 0,
+ * 4 <= k <= 256 and 16-byte aligned pointers; other shapes up to k = 4096 take plain float32
+ * kernels.  A token id outside [0, V) contributes no embedding and no position term and raises
+ * SL_FLAG_BAD_INDEX.  n_tok, V < 2^31.  Asynchronous on `stream`. */
+int sl_subspace_project(const float* X, const int32_t* ids, const float* T_perp, const float* pos, const float* U,
+                        uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k, float* Xt, uint32_t* flags,
+                        void* stream);
+int sl_subspace_reconstruct(const float* Xt, const int32_t* ids, const float* T_perp, const float* pos, const float* U,
+                            uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k, float* Xhat, uint32_t* flags,
+                            void* stream);
+
 /* x[i] <- the TF32 value nearest to x[i] (ties away from zero), kept as float32, for i < n; in place.
  * For matrices that are fed to the tensor cores many times and never change (U above). */
 int sl_round_tf32(float* x, uint64_t n, void* stream);

@@ -22,7 +22,7 @@ SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
 SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1280, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
-           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_round_tf32", "sl_idx12_stride",
+           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_round_tf32", "sl_subspace_project", "sl_subspace_reconstruct", "sl_idx12_stride",
            "sl_pack_idx12", "sl_unpack_idx12", "sl_strerror")
 
 
@@ -70,6 +70,11 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_outer_step.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.sl_embed_reproject.restype = i32
     L.sl_embed_reproject.argtypes = [vp, vp, vp, u64, ctypes.c_uint32, ctypes.c_uint32, vp, vp]
+    u32 = ctypes.c_uint32
+    L.sl_subspace_project.restype = i32
+    L.sl_subspace_project.argtypes = [vp, vp, vp, vp, vp, u64, u32, u64, u32, u32, vp, vp, vp]
+    L.sl_subspace_reconstruct.restype = i32
+    L.sl_subspace_reconstruct.argtypes = [vp, vp, vp, vp, vp, u64, u32, u64, u32, u32, vp, vp, vp]
     L.sl_round_tf32.restype = i32
     L.sl_round_tf32.argtypes = [vp, u64, vp]
     L.sl_idx12_stride.restype = u64
@@ -208,6 +213,18 @@ def sl_outer_step(theta_local: Sequence, theta_global, err: Sequence, layout, be
 def sl_embed_reproject(T_S, T_perp, U, V: int, d: int, k: int, flags=None, stream=None) -> None:
     _check(load().sl_embed_reproject(_ptr(T_S), _ptr(T_perp), _ptr(U), V, d, k, _ptr(flags), _stream(stream)),
            "sl_embed_reproject")
+
+
+def sl_subspace_project(X, ids, T_perp, pos, U, n_tok: int, L: int, V: int, d: int, k: int, Xt, flags=None,
+                        stream=None) -> None:
+    _check(load().sl_subspace_project(_ptr(X), _ptr(ids), _ptr(T_perp), _ptr(pos), _ptr(U), n_tok, L, V, d, k, _ptr(Xt),
+                                      _ptr(flags), _stream(stream)), "sl_subspace_project")
+
+
+def sl_subspace_reconstruct(Xt, ids, T_perp, pos, U, n_tok: int, L: int, V: int, d: int, k: int, Xhat, flags=None,
+                            stream=None) -> None:
+    _check(load().sl_subspace_reconstruct(_ptr(Xt), _ptr(ids), _ptr(T_perp), _ptr(pos), _ptr(U), n_tok, L, V, d, k,
+                                          _ptr(Xhat), _ptr(flags), _stream(stream)), "sl_subspace_reconstruct")
 
 
 def sl_round_tf32(x, n: int, stream=None) -> None:

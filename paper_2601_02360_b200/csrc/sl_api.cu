@@ -308,6 +308,37 @@ int sl_unpack_idx12(const uint8_t* packed, const sl_layout* L, int chunk, int k,
                              : unpack_impl<SL_MAX_TENSORS>(packed, L, chunk, k, idx, st);
 }
 
+namespace {
+int subspace_check(const float* a, const int32_t* ids, const float* T_perp, const float* pos, const float* U, uint64_t n_tok,
+                   uint32_t L, uint64_t V, uint32_t d, uint32_t k, const float* out, const uint32_t* flags) {
+  if (!a || !U || !out || d < 1 || k < 1) return SL_ERR_INVALID_ARG;
+  if (ids && (!T_perp || !pos || L < 1 || V < 1)) return SL_ERR_INVALID_ARG;
+  if (!aligned(a, 4) || !aligned(U, 4) || !aligned(out, 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
+  if (ids && (!aligned(ids, 4) || !aligned(T_perp, 4) || !aligned(pos, 4))) return SL_ERR_ALIGNMENT;
+  if (n_tok > 0x7FFFFFFFull || V > 0x7FFFFFFFull || k > 4096) return SL_ERR_UNSUPPORTED;
+  return SL_OK;
+}
+}  // namespace
+
+int sl_subspace_project(const float* X, const int32_t* ids, const float* T_perp, const float* pos, const float* U,
+                        uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k, float* Xt, uint32_t* flags,
+                        void* stream) {
+  const int rc = subspace_check(X, ids, T_perp, pos, U, n_tok, L, V, d, k, Xt, flags);
+  if (rc != SL_OK || n_tok == 0) return rc;
+  return launch_subspace_project(X, ids, T_perp, pos, U, n_tok, L, V, d, k, Xt, flags, (cudaStream_t)stream) == cudaSuccess
+             ? SL_OK : SL_ERR_CUDA;
+}
+
+int sl_subspace_reconstruct(const float* Xt, const int32_t* ids, const float* T_perp, const float* pos, const float* U,
+                            uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k, float* Xhat, uint32_t* flags,
+                            void* stream) {
+  const int rc = subspace_check(Xt, ids, T_perp, pos, U, n_tok, L, V, d, k, Xhat, flags);
+  if (rc != SL_OK || n_tok == 0) return rc;
+  return launch_subspace_reconstruct(Xt, ids, T_perp, pos, U, n_tok, L, V, d, k, Xhat, flags, (cudaStream_t)stream) ==
+                 cudaSuccess
+             ? SL_OK : SL_ERR_CUDA;
+}
+
 int sl_round_tf32(float* x, uint64_t n, void* stream) {
   if (!x && n) return SL_ERR_INVALID_ARG;
   if (!aligned(x, 4)) return SL_ERR_ALIGNMENT;

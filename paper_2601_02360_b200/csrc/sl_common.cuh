@@ -213,6 +213,12 @@ cudaError_t launch_pack_idx12(const uint16_t* idx, uint64_t n_chunks, int k, uin
                               cudaStream_t st);
 template <int T> cudaError_t launch_unpack_idx12(const Table<T>& tb, const uint8_t* packed, int chunk, int k,
                                                  uint16_t* idx, cudaStream_t st);
+cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const float* T_perp, const float* pos,
+                                    const float* U, uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k,
+                                    float* Xt, uint32_t* flags, cudaStream_t st);
+cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, const float* T_perp, const float* pos,
+                                        const float* U, uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k,
+                                        float* Xhat, uint32_t* flags, cudaStream_t st);
 cudaError_t launch_round_tf32(float* x, uint64_t n, cudaStream_t st);
 bool embed_is_tuned(const float* T_S, const float* T_perp, const float* U, uint32_t d, uint32_t k);
 cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, uint32_t d, uint32_t k,

@@ -1,0 +1,526 @@
+// Subspace compression of stage-boundary activations (paper §2.3):
+//     compress     Xt   = (X - T_perp[x] - Pos) U        n_tok x d  ->  n_tok x k  (what travels)
+//     reconstruct  Xhat = Xt U^T + T_perp[x] + Pos       n_tok x k  ->  n_tok x d
+//     gradients    Gt   = G U                            (compress without the embedding terms)
+// Token t of the flattened batch sits at position t mod L.  Both directions are one tcgen05
+// contraction (kind::tf32, accumulator in tensor memory) fused with the gather of the embedding
+// rows, built from the same pieces as the embedding re-projection kernel:
+//
+//   compress     K-loop over d in steps of 32 columns.  The X tile arrives by TMA (K-major,
+//                128-byte swizzle); four warps (one thread per token) then subtract the token's
+//                T_perp row and its Pos row - fetched with plain loads one step ahead - round to
+//                the nearest TF32 value (the tensor cores would cut instead) and hand the tile to
+//                the MMA warp; B = 32 rows of U, N-major.  The same warps write the accumulator
+//                out as Xt.
+//   reconstruct  the Xt tile (all k columns) arrives once per sub-tile, is rounded in place, and
+//                is the A operand of every 128-column block; B = 128 rows of U through a ring; the
+//                accumulator is double buffered; the epilogue adds the gathered rows and stores.
+//
+// Tokens are dealt in groups of 32 evenly over one CTA per SM, sub-tiles of up to 128 tokens.
+// Every wait is bounded (SL_FLAG_TIMEOUT); a token id outside [0, V) gathers nothing and raises
+// SL_FLAG_BAD_INDEX.  Other shapes (k or d not a multiple of 4, k above 256, unaligned pointers)
+// take plain float32 kernels.
+#include "sl_common.cuh"
+#include "sl_tc.cuh"
+
+namespace sl {
+namespace {
+
+using namespace tc;
+
+constexpr int kRows = 128;
+constexpr int kTileK = 32;
+constexpr int kBlockN = 128;
+constexpr int kRing = 4;
+constexpr int kSlotA = kRows * kTileK * 4;            // 16 KB
+constexpr int kSlotP = kSlotA + 256 * kTileK * 4;     // compress: X tile + 32 rows of U
+constexpr int kThreads = 192;                         // TMA warp, MMA warp, four row warps
+
+struct SubParams {
+  const float* T_perp;
+  const float* pos;
+  const int32_t* ids;       // NULL: no embedding terms (gradients)
+  float* out;
+  uint64_t n_tok, V;
+  uint32_t L, d, k, kp;
+  uint32_t* flags;
+};
+
+// the token a row thread serves in a sub-tile: its embedding row and position row (or none)
+struct RowInfo {
+  bool valid, gather;
+  const float* tp;
+  const float* ps;
+};
+__device__ __forceinline__ RowInfo row_info(const SubParams& p, uint64_t r0, uint32_t h, uint32_t row, bool& bad) {
+  RowInfo ri;
+  const uint64_t t = r0 + row;
+  ri.valid = row < h && t < p.n_tok;
+  ri.gather = false;
+  ri.tp = nullptr; ri.ps = nullptr;
+  if (ri.valid && p.ids) {
+    const int32_t id = p.ids[t];
+    if (id < 0 || (uint64_t)id >= p.V) bad = true;
+    else {
+      ri.gather = true;
+      ri.tp = p.T_perp + (uint64_t)id * p.d;
+      ri.ps = p.pos + (t % p.L) * (uint64_t)p.d;
+    }
+  }
+  return ri;
+}
+
+// ------------------------------------------------------------------------------------------ compress
+struct ProjSmem {
+  uint8_t ring[kRing * kSlotP];
+  uint64_t full[kRing], ready[kRing], empty[kRing], p_done, p_free;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+struct ProjMaps { CUtensorMap x128, x32, u_n; };
+
+__global__ void __launch_bounds__(kThreads, 1)
+subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_constant__ SubParams p) {
+  extern __shared__ uint8_t raw[];
+  ProjSmem& sm = *reinterpret_cast<ProjSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t k_tiles = (p.d + kTileK - 1) / kTileK;
+  const uint64_t G = (p.n_tok + 31) / 32;
+  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  if (tid == 0) {
+    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.ready[s], 4); mbar_init(&sm.empty[s], 1); }
+    mbar_init(&sm.p_done, 1);
+    mbar_init(&sm.p_free, 4);
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(256) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t t_p = sm.tmem_base;
+  bool bad = false;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+        const int r0 = (int)(g * 32);
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRing;
+          ok = mbar_wait(&sm.empty[s], ((it / kRing) & 1u) ^ 1u, sm.abort);
+          if (!ok) break;
+          uint8_t* slot = sm.ring + s * kSlotP;
+          mbar_expect_tx(&sm.full[s], h * 128 + p.kp * 128);
+          if (hg == 4) tma_load_2d(slot, &maps.x128, (int)(kt * kTileK), r0, &sm.full[s]);
+          else
+            for (uint32_t i = 0; i < hg; ++i)
+              tma_load_2d(slot + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full[s]);
+          for (uint32_t n = 0; n < p.kp / 32; ++n)
+            tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, t = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(kRows, (int)p.kp, 1);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2), desc_n = smem_desc(0, 4096, 512, 1);
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        if (t > 0) {                                 // the row warps have read the previous accumulator
+          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.abort);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRing;
+          ok = mbar_wait(&sm.ready[s], (it / kRing) & 1u, sm.abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(sm.ring + s * kSlotP);
+          const uint64_t da = desc_k | (uint64_t)((a0 >> 4) & 0x3FFF);
+          const uint64_t db = desc_n | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_ss(t_p, da + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+          mma_commit(&sm.empty[s]);
+        }
+        if (ok) mma_commit(&sm.p_done);
+      }
+    }
+  } else {
+    // ---- row warps: thread = token of the sub-tile; warp w reads tensor-memory lanes 32*(w%4).. ----
+    const uint32_t q = (uint32_t)(warp & 3);
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    const uint32_t sw = row & 7u;
+    uint32_t it = 0, t = 0;
+    bool ok = true;
+    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+      const uint64_t r0 = g * 32;
+      const RowInfo ri = row_info(p, r0, h, row, bad);
+      float4 nt[8], np_[8];      // the embedding and position values of the NEXT K step, fetched a step ahead
+      auto fetch = [&](uint32_t kt) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint32_t col = kt * kTileK + 4u * (uint32_t)ch;
+          const bool in = ri.gather && col < p.d;
+          nt[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          np_[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      };
+      fetch(0);
+      for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+        float4 ct[8], cp[8];
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) { ct[ch] = nt[ch]; cp[ch] = np_[ch]; }
+        if (kt + 1 < k_tiles) fetch(kt + 1);
+        const uint32_t s = it % kRing;
+        ok = mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t a0 = smem_u32(sm.ring + s * kSlotP) + row * 128;
+#pragma unroll
+        for (uint32_t ch = 0; ch < 8; ++ch) {
+          const uint32_t a = a0 + ((ch ^ sw) << 4);
+          float4 v = lds128(a);
+          v.x = __fsub_rn(__fsub_rn(v.x, ct[ch].x), cp[ch].x);
+          v.y = __fsub_rn(__fsub_rn(v.y, ct[ch].y), cp[ch].y);
+          v.z = __fsub_rn(__fsub_rn(v.z, ct[ch].z), cp[ch].z);
+          v.w = __fsub_rn(__fsub_rn(v.w, ct[ch].w), cp[ch].w);
+          v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+          v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+          v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+          v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+          sts128(a, v);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ready[s]);
+      }
+      if (!ok) break;
+      // the coordinates of this sub-tile's tokens: out of tensor memory, into Xt
+      ok = mbar_wait(&sm.p_done, t & 1u, sm.abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      for (uint32_t cb = 0; cb < p.kp; cb += 32) {
+        uint32_t v[32];
+        tmem_ld32(t_p + cb + ((32u * q) << 16), v);
+        tmem_ld_wait();
+        if (ri.valid) {
+          float* dst = p.out + (r0 + row) * (uint64_t)p.k + cb;
+#pragma unroll
+          for (int i = 0; i < 32; i += 4)
+            if (cb + (uint32_t)i < p.k)
+              *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.p_free);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_p), "r"(256) : "memory");
+  }
+  if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+  if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
+// --------------------------------------------------------------------------------------- reconstruct
+constexpr int kSlotB = kBlockN * kTileK * 4;          // 16 KB: 128 rows of U x 32 columns
+struct ReconSmem {
+  uint8_t a[8 * kSlotA];                              // the Xt tile: up to 8 boxes of 128 tokens x 32 columns
+  uint8_t ring[kRing][kSlotB];
+  uint64_t full[kRing], empty[kRing], o_full[2], o_empty[2], a_full, a_ready, a_free;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+struct ReconMaps { CUtensorMap xt128, xt32, u_k; };
+
+__global__ void __launch_bounds__(kThreads, 1)
+subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid_constant__ SubParams p) {
+  extern __shared__ uint8_t raw[];
+  ReconSmem& sm = *reinterpret_cast<ReconSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t k_tiles = p.kp / kTileK;
+  const uint32_t n_blocks = (p.d + kBlockN - 1) / kBlockN;
+  const uint64_t G = (p.n_tok + 31) / 32;
+  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  if (tid == 0) {
+    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
+    mbar_init(&sm.a_full, 1);
+    mbar_init(&sm.a_ready, 4);
+    mbar_init(&sm.a_free, 1);
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(256) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t t_o = sm.tmem_base;      // two accumulators of 128 columns
+  bool bad = false;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0, t = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+        const int r0 = (int)(g * 32);
+        if (t > 0) ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.abort);   // the last MMAs have read the old tile
+        if (!ok) break;
+        mbar_expect_tx(&sm.a_full, k_tiles * h * 128);
+        for (uint32_t kt = 0; kt < k_tiles; ++kt) {
+          if (hg == 4) tma_load_2d(sm.a + kt * kSlotA, &maps.xt128, (int)(kt * kTileK), r0, &sm.a_full);
+          else
+            for (uint32_t i = 0; i < hg; ++i)
+              tma_load_2d(sm.a + kt * kSlotA + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full);
+        }
+        for (uint32_t c = 0; ok && c < n_blocks; ++c)
+          for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
+            const uint32_t s = it % kRing;
+            ok = mbar_wait(&sm.empty[s], ((it / kRing) & 1u) ^ 1u, sm.abort);
+            if (!ok) break;
+            mbar_expect_tx(&sm.full[s], kSlotB);
+            tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(c * kBlockN), &sm.full[s]);
+          }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, cg = 0, t = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(kRows, kBlockN, 0);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2);
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        ok = mbar_wait(&sm.a_ready, t & 1u, sm.abort);          // landed and rounded
+        if (!ok) break;
+        tc_fence_after();
+        for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+          const uint32_t buf = cg & 1u, u = cg >> 1;
+          if (u) {
+            ok = mbar_wait(&sm.o_empty[buf], (u - 1) & 1u, sm.abort);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
+            const uint32_t s = it % kRing;
+            ok = mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t da = desc_k | (uint64_t)((smem_u32(sm.a + kt * kSlotA) >> 4) & 0x3FFF);
+            const uint64_t db = desc_k | (uint64_t)((smem_u32(sm.ring[s]) >> 4) & 0x3FFF);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mma_ss(t_o + buf * kBlockN, da + 2 * j, db + 2 * j, idesc, (kt | (uint32_t)j) != 0);
+            mma_commit(&sm.empty[s]);
+          }
+          if (!ok) break;
+          mma_commit(&sm.o_full[buf]);
+        }
+        if (ok) mma_commit(&sm.a_free);
+      }
+    }
+  } else {
+    const uint32_t q = (uint32_t)(warp & 3);
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    uint32_t cg = 0, t = 0;
+    bool ok = true;
+    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+      const uint64_t r0 = g * 32;
+      const RowInfo ri = row_info(p, r0, h, row, bad);
+      // round the Xt tile to the nearest TF32 value in place (element-wise: any thread, any chunk)
+      ok = mbar_wait(&sm.a_full, t & 1u, sm.abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      for (uint32_t i = (uint32_t)(tid - 64); i < k_tiles * 1024u; i += 128u) {
+        const uint32_t a = smem_u32(sm.a) + i * 16u;
+        float4 v = lds128(a);
+        v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+        v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+        v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+        v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+        sts128(a, v);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.a_ready);
+      for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+        const uint32_t buf = cg & 1u;
+        // this block's embedding and position values are requested before the accumulator is awaited
+        ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        for (uint32_t part = 0; part < 4; ++part) {
+          const uint32_t col0 = c * kBlockN + part * 32;
+          if (col0 >= p.d) break;
+          float4 tp[8], ps[8];
+#pragma unroll
+          for (int ch = 0; ch < 8; ++ch) {
+            const uint32_t col = col0 + 4u * (uint32_t)ch;
+            const bool in = ri.gather && col < p.d;
+            tp[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            ps[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+          uint32_t v[32];
+          tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
+          tmem_ld_wait();
+          if (ri.valid) {
+            float* dst = p.out + (r0 + row) * (uint64_t)p.d + col0;
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch)
+              if (col0 + 4u * (uint32_t)ch < p.d) {
+                float4 o;
+                o.x = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 0]), tp[ch].x), ps[ch].x);
+                o.y = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 1]), tp[ch].y), ps[ch].y);
+                o.z = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 2]), tp[ch].z), ps[ch].z);
+                o.w = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 3]), tp[ch].w), ps[ch].w);
+                __stcs(reinterpret_cast<float4*>(dst + 4 * ch), o);
+              }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.o_empty[buf]);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_o), "r"(256) : "memory");
+  }
+  if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+  if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
+// --------------------------------------------------------------------- plain float32 kernels (any shape)
+__global__ void __launch_bounds__(256) subspace_project_generic_kernel(const float* __restrict__ X, const float* __restrict__ U,
+                                                                       SubParams p) {
+  const uint64_t n = p.n_tok * (uint64_t)p.k;
+  bool bad = false;
+  for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t t = e / p.k;
+    const uint32_t j = (uint32_t)(e - t * p.k);
+    const float* x = X + t * p.d;
+    const float* tp = nullptr;
+    const float* ps = nullptr;
+    if (p.ids) {
+      const int32_t id = p.ids[t];
+      if (id < 0 || (uint64_t)id >= p.V) bad = true;
+      else { tp = p.T_perp + (uint64_t)id * p.d; ps = p.pos + (t % p.L) * (uint64_t)p.d; }
+    }
+    float acc = 0.0f;
+    for (uint32_t i = 0; i < p.d; ++i) {
+      float a = x[i];
+      if (tp) a = __fsub_rn(__fsub_rn(a, tp[i]), ps[i]);
+      acc = __fmaf_rn(a, U[(uint64_t)i * p.k + j], acc);
+    }
+    p.out[e] = acc;
+  }
+  if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+}
+
+__global__ void __launch_bounds__(256) subspace_reconstruct_generic_kernel(const float* __restrict__ Xt,
+                                                                           const float* __restrict__ U, SubParams p) {
+  const uint64_t n = p.n_tok * (uint64_t)p.d;
+  bool bad = false;
+  for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (uint64_t)gridDim.x * blockDim.x) {
+    const uint64_t t = e / p.d;
+    const uint32_t c = (uint32_t)(e - t * p.d);
+    const float* xt = Xt + t * p.k;
+    const float* u = U + (uint64_t)c * p.k;
+    float acc = 0.0f;
+    for (uint32_t j = 0; j < p.k; ++j) acc = __fmaf_rn(xt[j], u[j], acc);
+    if (p.ids) {
+      const int32_t id = p.ids[t];
+      if (id < 0 || (uint64_t)id >= p.V) bad = true;
+      else acc = __fadd_rn(__fadd_rn(acc, p.T_perp[(uint64_t)id * p.d + c]), p.pos[(t % p.L) * (uint64_t)p.d + c]);
+    }
+    p.out[e] = acc;
+  }
+  if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+}
+
+bool al16(const void* q) { return ((uintptr_t)q & 15u) == 0; }
+
+unsigned persistent_grid(uint64_t n_tok, cudaError_t* e) {
+  int dev = 0, sms = 0;
+  if ((*e = cudaGetDevice(&dev)) != cudaSuccess) return 0;
+  if ((*e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return 0;
+  const uint64_t tiles = (n_tok + kRows - 1) / kRows;
+  return (unsigned)(tiles < (uint64_t)sms ? tiles : (uint64_t)sms);
+}
+
+}  // namespace
+
+cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const float* T_perp, const float* pos,
+                                    const float* U, uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k,
+                                    float* Xt, uint32_t* flags, cudaStream_t st) {
+  SubParams p{T_perp, pos, ids, Xt, n_tok, V, L, d, k, (k + 31u) & ~31u, flags};
+  const bool tuned = d % 4 == 0 && k % 4 == 0 && k >= 4 && k <= 256 && al16(X) && al16(U) && al16(Xt) &&
+                     (!ids || (al16(T_perp) && al16(pos)));
+  if (!tuned) {
+    const uint64_t blocks = (n_tok * (uint64_t)k + 255) / 256;
+    subspace_project_generic_kernel<<<(unsigned)(blocks < 148u * 32u ? blocks : 148u * 32u), 256, 0, st>>>(X, U, p);
+    return cudaGetLastError();
+  }
+  ProjMaps m;
+  constexpr CUtensorMapL2promotion promo = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+  if (!make_map(&m.x128, X, d, n_tok, kRows, CU_TENSOR_MAP_SWIZZLE_128B, promo) ||
+      !make_map(&m.x32, X, d, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B, promo) ||
+      !make_map(&m.u_n, U, k, d, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+    return cudaErrorInvalidValue;
+  const int smem = (int)sizeof(ProjSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(subspace_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  const unsigned grid = persistent_grid(n_tok, &e);
+  if (e != cudaSuccess) return e;
+  subspace_project_kernel<<<grid, kThreads, smem, st>>>(m, p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, const float* T_perp, const float* pos,
+                                        const float* U, uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k,
+                                        float* Xhat, uint32_t* flags, cudaStream_t st) {
+  SubParams p{T_perp, pos, ids, Xhat, n_tok, V, L, d, k, (k + 31u) & ~31u, flags};
+  const bool tuned = d % 4 == 0 && k % 4 == 0 && k >= 4 && k <= 256 && al16(Xt) && al16(U) && al16(Xhat) &&
+                     (!ids || (al16(T_perp) && al16(pos)));
+  if (!tuned) {
+    const uint64_t blocks = (n_tok * (uint64_t)d + 255) / 256;
+    subspace_reconstruct_generic_kernel<<<(unsigned)(blocks < 148u * 32u ? blocks : 148u * 32u), 256, 0, st>>>(Xt, U, p);
+    return cudaGetLastError();
+  }
+  ReconMaps m;
+  if (!make_map(&m.xt128, Xt, k, n_tok, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.xt32, Xt, k, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B))
+    return cudaErrorInvalidValue;
+  const int smem = (int)sizeof(ReconSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(subspace_reconstruct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  const unsigned grid = persistent_grid(n_tok, &e);
+  if (e != cudaSuccess) return e;
+  subspace_reconstruct_kernel<<<grid, kThreads, smem, st>>>(m, p);
+  return cudaGetLastError();
+}
+
+}  // namespace sl

@@ -247,3 +247,14 @@ def gen_embedding_pair(V: int, d: int, seed: int = 0, std: float = 0.02) -> Tupl
     T_S = (rng.standard_normal((V, d), dtype=np.float32) * np.float32(std))
     T_perp = (rng.standard_normal((V, d), dtype=np.float32) * np.float32(std))
     return T_S, T_perp
+
+
+def gen_stage_boundary(n_tok: int, L: int, V: int, d: int, seed: int = 0, std: float = 1.0):
+    """Inputs of the activation compression of §2.3: (X n_tok x d, ids int32 n_tok, T_perp V x d,
+    pos L x d), all float32 N(0, .) i.i.d. (activations of unit scale, embeddings of scale 0.02)."""
+    rng = np.random.default_rng(_mix(0x5B9, n_tok, L, V, d, seed))
+    X = rng.standard_normal((n_tok, d), dtype=np.float32) * np.float32(std)
+    ids = rng.integers(0, V, size=n_tok).astype(np.int32)
+    T_perp = rng.standard_normal((V, d), dtype=np.float32) * np.float32(0.02)
+    pos = rng.standard_normal((L, d), dtype=np.float32) * np.float32(0.02)
+    return X, ids, T_perp, pos

@@ -10,7 +10,7 @@ int main(void) {
   typedef void (*fn)(void);
   const fn fns[] = {(fn)sl_num_chunks, (fn)sl_codes_stride, (fn)sl_compress, (fn)sl_compress_batch, (fn)sl_aggregate,
                     (fn)sl_outer_apply, (fn)sl_aggregate_apply, (fn)sl_outer_step, (fn)sl_idx12_stride,
-                    (fn)sl_pack_idx12, (fn)sl_unpack_idx12, (fn)sl_embed_reproject, (fn)sl_round_tf32,
+                    (fn)sl_pack_idx12, (fn)sl_unpack_idx12, (fn)sl_embed_reproject, (fn)sl_round_tf32, (fn)sl_subspace_project, (fn)sl_subspace_reconstruct,
                     (fn)sl_strerror};
   uint64_t offset[3] = {0, 4096 * 2 + 5, 4096 * 2 + 5 + 100};
   sl_layout lay;

@@ -1,0 +1,150 @@
+"""Parity of sl_subspace_project / sl_subspace_reconstruct (paper §2.3) with the float64 CPU checker.
+
+Tolerance (derived): the float32 operand of each contraction (the difference X - T_perp[x] - Pos,
+resp. Xt) is rounded to the nearest TF32 value, relative error <= 2^-11; U is used as given, and
+the tensor cores cut it to TF32, relative error < 2^-10 (none when the caller has rounded it);
+float32 accumulation adds far less.  With B the sum of the magnitudes of all products entering an
+output, the error is below (2^-11 + 2^-10 + ...) B < 2^-9 B; the differences / sums around the
+contraction are float32 operations and add a few units of 2^-24 of the magnitudes involved.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import subspace as osub
+from paper_2601_02360_b200 import api, synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2.0 ** -9
+
+
+def _dev(a):
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _project(X, ids, T_perp, pos, U, L):
+    n_tok, d = X.shape
+    k = U.shape[1]
+    out = torch.full((n_tok, k), 7.0, dtype=torch.float32, device="cuda")
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.sl_subspace_project(_dev(X), _dev(ids), _dev(T_perp), _dev(pos), _dev(U), n_tok, L,
+                            0 if T_perp is None else T_perp.shape[0], d, k, out, flags)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), int(flags.item())
+
+
+def _reconstruct(Xt, ids, T_perp, pos, U, L):
+    n_tok, k = Xt.shape
+    d = U.shape[0]
+    out = torch.full((n_tok, d), 7.0, dtype=torch.float32, device="cuda")
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.sl_subspace_reconstruct(_dev(Xt), _dev(ids), _dev(T_perp), _dev(pos), _dev(U), n_tok, L,
+                                0 if T_perp is None else T_perp.shape[0], d, k, out, flags)
+    torch.cuda.synchronize()
+    return out.cpu().numpy(), int(flags.item())
+
+
+def _scale_project(X, ids, T_perp, pos, U, L):
+    A = np.abs(X.astype(np.float64))
+    if ids is not None:
+        A = A + np.abs(T_perp.astype(np.float64))[ids] + np.abs(pos.astype(np.float64))[np.arange(len(X)) % L]
+    return A @ np.abs(U.astype(np.float64))
+
+
+@pytest.mark.parametrize("n_tok,L,V,d,k", [(1000, 128, 500, 512, 64), (4096, 1024, 2000, 2048, 256), (333, 50, 77, 132, 12),
+                                           (5, 2, 3, 8, 4), (129, 129, 10, 64, 64), (260, 64, 300, 1536, 192),
+                                           (2048, 512, 100, 1024, 8)])
+def test_parity_both_directions(n_tok, L, V, d, k):
+    U = synth.gen_subspace_basis(d, k, seed=1)
+    X, ids, T_perp, pos = synth.gen_stage_boundary(n_tok, L, V, d, seed=2)
+    xt, f = _project(X, ids, T_perp, pos, U, L)
+    assert f == 0
+    ref = osub.project(X, ids, T_perp, pos, U, L)
+    S = _scale_project(X, ids, T_perp, pos, U, L)
+    err = np.abs(xt - ref)
+    assert np.all(err <= TOL * S + 1e-30), float((err / (S + 1e-30)).max())
+    assert np.sqrt((err ** 2).mean()) <= 2.0 ** -9 * np.sqrt((ref ** 2).mean())
+    # reconstruction from the checker's coordinates (as float32)
+    Xt = ref.astype(np.float32)
+    xh, f = _reconstruct(Xt, ids, T_perp, pos, U, L)
+    assert f == 0
+    ref_h = osub.reconstruct(Xt, ids, T_perp, pos, U, L)
+    S_h = osub.abs_bound_reconstruct(Xt, U) + np.abs(T_perp.astype(np.float64))[ids] + np.abs(pos.astype(np.float64))[np.arange(n_tok) % L]
+    err_h = np.abs(xh - ref_h)
+    assert np.all(err_h <= TOL * S_h + 1e-30), float((err_h / (S_h + 1e-30)).max())
+
+
+def test_gradient_form_has_no_embedding_terms():
+    n_tok, d, k = 700, 1024, 128
+    U = synth.gen_subspace_basis(d, k, seed=3)
+    G, _, _, _ = synth.gen_stage_boundary(n_tok, 64, 10, d, seed=4)
+    gt, f = _project(G, None, None, None, U, 64)
+    ref = osub.project(G, None, None, None, U, 64)
+    S = np.abs(G.astype(np.float64)) @ np.abs(U.astype(np.float64))
+    assert f == 0 and np.all(np.abs(gt - ref) <= TOL * S + 1e-30)
+    gh, f = _reconstruct(ref.astype(np.float32), None, None, None, U, 64)
+    assert f == 0
+    assert np.all(np.abs(gh - ref.astype(np.float32).astype(np.float64) @ U.astype(np.float64).T)
+                  <= TOL * osub.abs_bound_reconstruct(ref, U) + 1e-30)
+
+
+@pytest.mark.parametrize("n_tok,L,V,d,k", [(300, 7, 20, 256, 8), (130, 16, 9, 512, 32), (128, 128, 5, 2048, 256)])
+def test_exact_when_tf32_is_exact(n_tok, L, V, d, k):
+    # identity columns and dyadic values with few bits: every operation is exact, so both directions
+    # must match the checker bit for bit (catches a mis-swizzled operand or a wrong gather row)
+    rng = np.random.default_rng(5)
+    cols = rng.permutation(d)[:k]
+    U = np.zeros((d, k), dtype=np.float32)
+    U[cols, np.arange(k)] = 1.0
+    q = lambda shape: (rng.integers(-32, 33, size=shape) / 16.0).astype(np.float32)
+    X, T_perp, pos = q((n_tok, d)), q((V, d)), q((L, d))
+    ids = rng.integers(0, V, size=n_tok).astype(np.int32)
+    xt, f = _project(X, ids, T_perp, pos, U, L)
+    assert f == 0 and np.array_equal(xt, osub.project(X, ids, T_perp, pos, U, L).astype(np.float32))
+    xh, f = _reconstruct(xt, ids, T_perp, pos, U, L)
+    assert f == 0 and np.array_equal(xh, osub.reconstruct(xt, ids, T_perp, pos, U, L).astype(np.float32))
+
+
+def test_round_trip_is_lossless_for_residuals_in_the_subspace():
+    n_tok, L, V, d, k = 1500, 256, 400, 1024, 128
+    u = _dev(synth.gen_subspace_basis(d, k, seed=6))
+    api.sl_round_tf32(u, u.numel())
+    U = u.cpu().numpy()
+    _, ids, T_perp, pos = synth.gen_stage_boundary(n_tok, L, V, d, seed=7)
+    C = np.random.default_rng(8).standard_normal((n_tok, k))
+    X = (C @ U.astype(np.float64).T + T_perp[ids] + pos[np.arange(n_tok) % L]).astype(np.float32)
+    xt, _ = _project(X, ids, T_perp, pos, U, L)
+    xh, _ = _reconstruct(xt, ids, T_perp, pos, U, L)
+    # U is orthonormal only up to the rounding of its entries, and both contractions are TF32
+    assert np.sqrt(((xh - X) ** 2).mean()) <= 2.0 ** -9 * np.sqrt((X ** 2).mean())
+
+
+def test_bad_token_id_is_flagged_and_gathers_nothing():
+    n_tok, L, V, d, k = 64, 8, 5, 64, 8
+    U = synth.gen_subspace_basis(d, k, seed=9)
+    X, ids, T_perp, pos = synth.gen_stage_boundary(n_tok, L, V, d, seed=10)
+    ids = ids.copy()
+    ids[3], ids[40] = V, -1
+    xt, f = _project(X, ids, T_perp, pos, U, L)
+    assert f == api.SL_FLAG_BAD_INDEX
+    good = np.ones(n_tok, bool)
+    good[[3, 40]] = False
+    ref = osub.project(X[good], ids[good], T_perp, pos[(np.arange(n_tok) % L)[good]], U, n_tok)   # per-row positions
+    assert np.all(np.abs(xt[good] - ref) <= TOL * _scale_project(X, np.clip(ids, 0, V - 1), T_perp, pos, U, L)[good] + 1e-30)
+    plain = X[[3, 40]].astype(np.float64) @ U.astype(np.float64)
+    assert np.all(np.abs(xt[[3, 40]] - plain) <= TOL * (np.abs(X[[3, 40]].astype(np.float64)) @ np.abs(U.astype(np.float64))))
+
+
+@pytest.mark.parametrize("n_tok,L,V,d,k", [(50, 10, 7, 1536, 2), (33, 5, 4, 10, 3), (20, 4, 6, 64, 300)])
+def test_shapes_outside_the_tensor_core_path(n_tok, L, V, d, k):
+    rng = np.random.default_rng(11)
+    U = synth.gen_subspace_basis(d, k, seed=11) if k <= d else (rng.standard_normal((d, k)) / np.sqrt(k)).astype(np.float32)
+    X, ids, T_perp, pos = synth.gen_stage_boundary(n_tok, L, V, d, seed=12)
+    xt, f = _project(X, ids, T_perp, pos, U, L)
+    ref = osub.project(X, ids, T_perp, pos, U, L)
+    assert f == 0 and np.all(np.abs(xt - ref) <= 2.0 ** -18 * _scale_project(X, ids, T_perp, pos, U, L) + 1e-30)
+    xh, f = _reconstruct(ref.astype(np.float32), ids, T_perp, pos, U, L)
+    ref_h = osub.reconstruct(ref.astype(np.float32), ids, T_perp, pos, U, L)
+    S_h = osub.abs_bound_reconstruct(ref, U) + np.abs(T_perp)[ids] + np.abs(pos)[np.arange(n_tok) % L]
+    assert f == 0 and np.all(np.abs(xh - ref_h) <= 2.0 ** -18 * S_h + 1e-30)
