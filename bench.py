@@ -457,6 +457,78 @@ def run_exchange(args) -> None:
     dist.destroy_process_group()
 
 
+def run_subspace(args) -> None:
+    """Stage-boundary activation compression (§2.3): sl_subspace_project and sl_subspace_reconstruct on
+    one micro-batch of the chosen model (batch 32 x sequence 2048 tokens of the paper's local batch
+    would be 64 K tokens; 16 K tokens here keep the buffers small), k = d/8.  One GPU, own JSON line."""
+    from paper_2601_02360_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    wl = synth.workload(args.workload)
+    name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
+    k = args.k or d // 8
+    L, n_tok = 2048, args.tokens
+    Xh, idsh, Tph, posh = synth.gen_stage_boundary(n_tok, L, V, d, args.seed)
+    X, ids, T_perp, pos = (torch.from_numpy(a).to(dev) for a in (Xh, idsh, Tph, posh))
+    U = torch.from_numpy(synth.gen_subspace_basis(d, k, args.seed)).to(dev)
+    api.sl_round_tf32(U, U.numel())
+    Xt = torch.empty(n_tok, k, dtype=torch.float32, device=dev)
+    Xhat = torch.empty(n_tok, d, dtype=torch.float32, device=dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)     # 256 MB > L2, written between steps
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(0)
+    t_p, t_r = [], []
+    for s in range(args.warmup + args.steps):
+        if s == args.warmup:
+            sampler.start()
+        flush.fill_(float(s))
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream)
+        api.sl_subspace_project(X, ids, T_perp, pos, U, n_tok, L, V, d, k, Xt, flags)
+        e[1].record(stream)
+        api.sl_subspace_reconstruct(Xt, ids, T_perp, pos, U, n_tok, L, V, d, k, Xhat, flags)
+        e[2].record(stream)
+        torch.cuda.synchronize()
+        if s >= args.warmup:
+            t_p.append(e[0].elapsed_time(e[1]))
+            t_r.append(e[1].elapsed_time(e[2]))
+    clocks = sampler.stop()
+    ms_p, ms_r = float(np.mean(t_p)), float(np.mean(t_r))
+    # compress reads X and one gathered T_perp row per token, writes Xt; Pos and U are L2-resident (counted once)
+    bytes_p = n_tok * d * 8 + n_tok * k * 4 + L * d * 4 + d * k * 4
+    bytes_r = n_tok * k * 4 + n_tok * d * 8 + L * d * 4 + d * k * 4
+    peak, peak_src = measured_peak_gbs()
+    ms = ms_p + ms_r
+    line = {
+        "metric": "subspace_roundtrip_tokens_per_s", "value": n_tok / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "tf32 contraction, f32 gather terms", "data": "synthetic",
+        "config": {"workload": f"{wl.name} stage boundary: {n_tok} tokens x d={d}, k={k}, L={L}, vocab {V}",
+                   "l2": "a 256 MB buffer is written between timed steps"},
+        "kernels_ms": {"sl_subspace_project": ms_p, "sl_subspace_reconstruct": ms_r},
+        "roofline": {"bound": "hbm", "kernel": "sl_subspace_reconstruct", "achieved": bytes_r / (ms_r * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": bytes_r / (ms_r * 1e-3) / 1e9 / peak, "traffic": None,
+                     "peak_source": peak_src, "algorithmic_bytes": bytes_r,
+                     "project": {"achieved": bytes_p / (ms_p * 1e-3) / 1e9, "frac": bytes_p / (ms_p * 1e-3) / 1e9 / peak,
+                                 "algorithmic_bytes": bytes_p},
+                     "tensor_tflops": 4 * n_tok * d * k / (ms * 1e-3) / 1e12},
+        "clocks": clocks, "device_flags": int(flags.item()), "gpu_launches": 2 * args.steps,
+    }
+    if not args.no_cpu:
+        from oracle import subspace as osub
+        rows = min(n_tok, 2048)
+        Uh = U.cpu().numpy()
+        t0 = time.perf_counter()
+        xt = osub.project(Xh[:rows], idsh[:rows], Tph, posh, Uh, L)
+        osub.reconstruct(xt, idsh[:rows], Tph, posh, Uh, L)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": rows / dt, "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"first {rows} tokens, float64 numpy, both directions"}
+    print(json.dumps(line))
+
+
 def run_embed(args) -> None:
     """The step right after the outer step for replicas that compress activations (§2.4, Eqs. 3-4):
     sl_embed_reproject on the token-embedding table of the chosen model (vocab x d, k = d/8, the
@@ -667,6 +739,10 @@ def main() -> None:
     ap.add_argument("--embed", action="store_true",
                     help="time sl_embed_reproject (token-embedding adaptation, Eqs. 3-4) on the model's "
                          "embedding table instead of the outer step; one GPU, its own JSON line")
+    ap.add_argument("--subspace", action="store_true",
+                    help="time sl_subspace_project + sl_subspace_reconstruct (activation compression of a "
+                         "pipeline-stage boundary) instead of the outer step; one GPU, its own JSON line")
+    ap.add_argument("--tokens", type=int, default=16384, help="with --subspace: tokens per micro-batch")
     ap.add_argument("--tiles", action="store_true",
                     help="cut matrices into square tiles of `chunk` elements instead of consecutive chunks")
     ap.add_argument("--variant", default="plain", choices=["plain", "ties_literal", "ties_dyadic"],
@@ -678,6 +754,8 @@ def main() -> None:
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.subspace:
+        run_subspace(args)
     elif args.embed:
         run_embed(args)
     elif args.exchange:
