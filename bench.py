@@ -495,7 +495,7 @@ def run_subspace(args) -> None:
             t_p.append(e[0].elapsed_time(e[1]))
             t_r.append(e[1].elapsed_time(e[2]))
     clocks = sampler.stop()
-    ms_p, ms_r = float(np.mean(t_p)), float(np.mean(t_r))
+    ms_p, ms_r = float(np.median(t_p)), float(np.median(t_r))     # short kernels: the median is robust to clock ramps
     # compress reads X and one gathered T_perp row per token, writes Xt; Pos and U are L2-resident (counted once)
     bytes_p = n_tok * d * 8 + n_tok * k * 4 + L * d * 4 + d * k * 4
     bytes_r = n_tok * k * 4 + n_tok * d * 8 + L * d * 4 + d * k * 4

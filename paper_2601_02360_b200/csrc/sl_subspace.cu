@@ -7,8 +7,8 @@
 // rows, built from the same pieces as the embedding re-projection kernel:
 //
 //   compress     K-loop over d in steps of 32 columns.  The X tile arrives by TMA (K-major,
-//                128-byte swizzle); four warps (one thread per token) then subtract the token's
-//                T_perp row and its Pos row - fetched with plain loads one step ahead - round to
+//                128-byte swizzle); eight warps (two threads per token) then subtract the token's
+//                T_perp row and its Pos row - fetched with plain loads two steps ahead - round to
 //                the nearest TF32 value (the tensor cores would cut instead) and hand the tile to
 //                the MMA warp; B = 32 rows of U, N-major.  The same warps write the accumulator
 //                out as Xt.
@@ -34,7 +34,8 @@ constexpr int kBlockN = 128;
 constexpr int kRing = 4;
 constexpr int kSlotA = kRows * kTileK * 4;            // 16 KB
 constexpr int kSlotP = kSlotA + 256 * kTileK * 4;     // compress: X tile + 32 rows of U
-constexpr int kThreads = 192;                         // TMA warp, MMA warp, four row warps
+constexpr int kRowWarps = 8;                          // two per 32-lane window of tensor memory
+constexpr int kThreads = 64 + 32 * kRowWarps;         // TMA warp, MMA warp, the row warps
 
 struct SubParams {
   const float* T_perp;
@@ -88,9 +89,9 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
   const uint64_t G = (p.n_tok + 31) / 32;
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
   if (tid == 0) {
-    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.ready[s], 4); mbar_init(&sm.empty[s], 1); }
+    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.ready[s], kRowWarps); mbar_init(&sm.empty[s], 1); }
     mbar_init(&sm.p_done, 1);
-    mbar_init(&sm.p_free, 4);
+    mbar_init(&sm.p_free, kRowWarps);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -154,8 +155,9 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
       }
     }
   } else {
-    // ---- row warps: thread = token of the sub-tile; warp w reads tensor-memory lanes 32*(w%4).. ----
-    const uint32_t q = (uint32_t)(warp & 3);
+    // ---- row warps: two threads per token of the sub-tile (each takes four of the eight 16-byte chunks
+    // of a tile row); warp w reads tensor-memory lanes 32*(w%4).. ----
+    const uint32_t q = (uint32_t)(warp & 3), half = (uint32_t)(warp - 2) >> 2;
     const uint32_t row = 32u * q + (uint32_t)lane;
     const uint32_t sw = row & 7u;
     uint32_t it = 0, t = 0;
@@ -164,52 +166,63 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
       const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
       const uint64_t r0 = g * 32;
       const RowInfo ri = row_info(p, r0, h, row, bad);
-      float4 nt[8], np_[8];      // the embedding and position values of the NEXT K step, fetched a step ahead
-      auto fetch = [&](uint32_t kt) {
+      // the embedding and position values of the next two K steps are in flight while one is used
+      float4 et[2][4], ep[2][4];
+      auto fetch = [&](uint32_t kt, float4 (&dt)[4], float4 (&dp)[4]) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint32_t col = kt * kTileK + 4u * (uint32_t)ch;
-          const bool in = ri.gather && col < p.d;
-          nt[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          np_[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = 0; c < 4; ++c) {
+          const uint32_t col = kt * kTileK + 16u * half + 4u * (uint32_t)c;
+          const bool in = ri.gather && kt < k_tiles && col < p.d;
+          dt[c] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          dp[c] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
       };
-      fetch(0);
-      for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
-        float4 ct[8], cp[8];
+      fetch(0, et[0], ep[0]);
+      fetch(1, et[1], ep[1]);
+      for (uint32_t kt = 0; ok && kt < k_tiles; kt += 2) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) { ct[ch] = nt[ch]; cp[ch] = np_[ch]; }
-        if (kt + 1 < k_tiles) fetch(kt + 1);
-        const uint32_t s = it % kRing;
-        ok = mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        const uint32_t a0 = smem_u32(sm.ring + s * kSlotP) + row * 128;
+        for (int par = 0; par < 2; ++par) {          // two K steps per trip so that the buffers keep static indices
+          const uint32_t kk = kt + (uint32_t)par;
+          if (kk < k_tiles) {
+            float4 ct[4], cp[4];
 #pragma unroll
-        for (uint32_t ch = 0; ch < 8; ++ch) {
-          const uint32_t a = a0 + ((ch ^ sw) << 4);
-          float4 v = lds128(a);
-          v.x = __fsub_rn(__fsub_rn(v.x, ct[ch].x), cp[ch].x);
-          v.y = __fsub_rn(__fsub_rn(v.y, ct[ch].y), cp[ch].y);
-          v.z = __fsub_rn(__fsub_rn(v.z, ct[ch].z), cp[ch].z);
-          v.w = __fsub_rn(__fsub_rn(v.w, ct[ch].w), cp[ch].w);
-          v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
-          v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
-          v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
-          v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
-          sts128(a, v);
+            for (int c = 0; c < 4; ++c) { ct[c] = et[par][c]; cp[c] = ep[par][c]; }
+            fetch(kk + 2, et[par], ep[par]);
+            const uint32_t s = it % kRing;
+            ok = ok && mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok) {
+              const uint32_t a0 = smem_u32(sm.ring + s * kSlotP) + row * 128;
+#pragma unroll
+              for (uint32_t c = 0; c < 4; ++c) {
+                const uint32_t a = a0 + (((4u * half + c) ^ sw) << 4);
+                float4 v = lds128(a);
+                v.x = __fsub_rn(__fsub_rn(v.x, ct[c].x), cp[c].x);
+                v.y = __fsub_rn(__fsub_rn(v.y, ct[c].y), cp[c].y);
+                v.z = __fsub_rn(__fsub_rn(v.z, ct[c].z), cp[c].z);
+                v.w = __fsub_rn(__fsub_rn(v.w, ct[c].w), cp[c].w);
+                v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+                v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+                v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+                v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+                sts128(a, v);
+              }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&sm.ready[s]);
+              ++it;
+            }
+          }
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.ready[s]);
       }
       if (!ok) break;
-      // the coordinates of this sub-tile's tokens: out of tensor memory, into Xt
+      // the coordinates of this sub-tile's tokens: out of tensor memory, into Xt (the two warps of a lane
+      // window take alternate blocks of 32 columns)
       ok = mbar_wait(&sm.p_done, t & 1u, sm.abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      for (uint32_t cb = 0; cb < p.kp; cb += 32) {
+      for (uint32_t cb = 32u * half; cb < p.kp; cb += 64) {
         uint32_t v[32];
         tmem_ld32(t_p + cb + ((32u * q) << 16), v);
         tmem_ld_wait();
@@ -239,16 +252,19 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
 
 // --------------------------------------------------------------------------------------- reconstruct
 constexpr int kSlotB = kBlockN * kTileK * 4;          // 16 KB: 128 rows of U x 32 columns
+constexpr int kRingB = 4;                             // slots of the U ring (a power of two: the roles index it with % and /)
 struct ReconSmem {
   uint8_t a[8 * kSlotA];                              // the Xt tile: up to 8 boxes of 128 tokens x 32 columns
-  uint8_t ring[kRing][kSlotB];
-  uint64_t full[kRing], empty[kRing], o_full[2], o_empty[2], a_full, a_ready, a_free;
+  uint8_t ring[kRingB][kSlotB];
+  uint64_t full[kRingB], empty[kRingB], o_full[2], o_empty[2], a_full, a_ready, a_free;
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
 struct ReconMaps { CUtensorMap xt128, xt32, u_k; };
 
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr int kReconThreads = 192;                    // TMA warp, MMA warp, four row warps
+
+__global__ void __launch_bounds__(kReconThreads, 1)
 subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid_constant__ SubParams p) {
   extern __shared__ uint8_t raw[];
   ReconSmem& sm = *reinterpret_cast<ReconSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
@@ -258,7 +274,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   const uint64_t G = (p.n_tok + 31) / 32;
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
   if (tid == 0) {
-    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
+    for (int s = 0; s < kRingB; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
     mbar_init(&sm.a_full, 1);
     mbar_init(&sm.a_ready, 4);
@@ -294,8 +310,8 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         }
         for (uint32_t c = 0; ok && c < n_blocks; ++c)
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
-            const uint32_t s = it % kRing;
-            ok = mbar_wait(&sm.empty[s], ((it / kRing) & 1u) ^ 1u, sm.abort);
+            const uint32_t s = it % kRingB;
+            ok = mbar_wait(&sm.empty[s], ((it / kRingB) & 1u) ^ 1u, sm.abort);
             if (!ok) break;
             mbar_expect_tx(&sm.full[s], kSlotB);
             tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(c * kBlockN), &sm.full[s]);
@@ -320,8 +336,8 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
             tc_fence_after();
           }
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
-            const uint32_t s = it % kRing;
-            ok = mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
+            const uint32_t s = it % kRingB;
+            ok = mbar_wait(&sm.full[s], (it / kRingB) & 1u, sm.abort);
             if (!ok) break;
             tc_fence_after();
             const uint64_t da = desc_k | (uint64_t)((smem_u32(sm.a + kt * kSlotA) >> 4) & 0x3FFF);
@@ -361,39 +377,48 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.a_ready);
+      // the embedding and position values of a 32-column part are requested one part ahead of their use
+      float4 tp[8], ps[8];
+      auto fetch = [&](uint32_t col0) {
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          const uint32_t col = col0 + 4u * (uint32_t)ch;
+          const bool in = ri.gather && col < p.d;
+          tp[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          ps[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      };
+      fetch(0);
       for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
         const uint32_t buf = cg & 1u;
-        // this block's embedding and position values are requested before the accumulator is awaited
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.abort);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
+#pragma unroll
         for (uint32_t part = 0; part < 4; ++part) {
           const uint32_t col0 = c * kBlockN + part * 32;
-          if (col0 >= p.d) break;
-          float4 tp[8], ps[8];
+          float4 ct[8], cs[8];
 #pragma unroll
-          for (int ch = 0; ch < 8; ++ch) {
-            const uint32_t col = col0 + 4u * (uint32_t)ch;
-            const bool in = ri.gather && col < p.d;
-            tp[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            ps[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-          uint32_t v[32];
-          tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
-          tmem_ld_wait();
-          if (ri.valid) {
-            float* dst = p.out + (r0 + row) * (uint64_t)p.d + col0;
+          for (int ch = 0; ch < 8; ++ch) { ct[ch] = tp[ch]; cs[ch] = ps[ch]; }
+          fetch(col0 + 32);
+          if (col0 < p.d) {
+            uint32_t v[32];
+            tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
+            tmem_ld_wait();
+            if (ri.valid) {
+              float* dst = p.out + (r0 + row) * (uint64_t)p.d + col0;
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch)
-              if (col0 + 4u * (uint32_t)ch < p.d) {
-                float4 o;
-                o.x = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 0]), tp[ch].x), ps[ch].x);
-                o.y = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 1]), tp[ch].y), ps[ch].y);
-                o.z = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 2]), tp[ch].z), ps[ch].z);
-                o.w = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 3]), tp[ch].w), ps[ch].w);
-                __stcs(reinterpret_cast<float4*>(dst + 4 * ch), o);
-              }
+              for (int ch = 0; ch < 8; ++ch)
+                if (col0 + 4u * (uint32_t)ch < p.d) {
+                  float4 o;
+                  o.x = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 0]), ct[ch].x), cs[ch].x);
+                  o.y = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 1]), ct[ch].y), cs[ch].y);
+                  o.z = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 2]), ct[ch].z), cs[ch].z);
+                  o.w = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 3]), ct[ch].w), cs[ch].w);
+                  __stcs(reinterpret_cast<float4*>(dst + 4 * ch), o);
+                }
+            }
           }
         }
         tc_fence_before();
@@ -519,7 +544,7 @@ cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, con
   if (e != cudaSuccess) return e;
   const unsigned grid = persistent_grid(n_tok, &e);
   if (e != cudaSuccess) return e;
-  subspace_reconstruct_kernel<<<grid, kThreads, smem, st>>>(m, p);
+  subspace_reconstruct_kernel<<<grid, kReconThreads, smem, st>>>(m, p);
   return cudaGetLastError();
 }
 
