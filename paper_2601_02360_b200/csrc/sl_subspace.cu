@@ -251,18 +251,35 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
 }
 
 // --------------------------------------------------------------------------------------- reconstruct
+// Per sub-tile of 128 tokens the Xt tile goes through a two-slot staging buffer into tensor memory
+// (rounded to TF32 on the way) and is the A operand of every 128-column block.  The embedding and
+// position rows of a 32-column part are gathered into a stage of shared memory by 16-byte
+// asynchronous copies, several parts ahead of their use (whole 128-byte segments per row, so every
+// line is fetched by one request); the epilogue adds them to the accumulator part in place and a
+// tensor-map store writes the finished part.  Warps: 0 operand TMA, 1 MMA, 2 part store,
+// 3..6 Xt staging -> tensor memory and the gathers, 7..10 epilogue.
 constexpr int kSlotB = kBlockN * kTileK * 4;          // 16 KB: 128 rows of U x 32 columns
 constexpr int kRingB = 4;                             // slots of the U ring (a power of two: the roles index it with % and /)
+constexpr int kStages = 4;                            // gather / output stages
+constexpr int kStageA = 2;                            // staging slots of the Xt tile
 struct ReconSmem {
-  uint8_t a[8 * kSlotA];                              // the Xt tile: up to 8 boxes of 128 tokens x 32 columns
   uint8_t ring[kRingB][kSlotB];
-  uint64_t full[kRingB], empty[kRingB], o_full[2], o_empty[2], a_full, a_ready, a_free;
+  uint8_t st_t[kStages][kSlotA];                      // gathered T_perp segments of a part, then the finished part
+  uint8_t st_p[kStages][kSlotA];                      // gathered position segments
+  uint8_t a[kStageA][kSlotA];
+  uint64_t full[kRingB], empty[kRingB], o_full[2], o_empty[2];
+  uint64_t a_full[kStageA], a_empty[kStageA], a_ready, a_free;
+  uint64_t g_full[kStages], g_done[kStages], g_empty[kStages];
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
-struct ReconMaps { CUtensorMap xt128, xt32, u_k; };
+struct ReconMaps { CUtensorMap xt128, xt32, u_k, o128, o32; };
 
-constexpr int kReconThreads = 192;                    // TMA warp, MMA warp, four row warps
+constexpr int kReconThreads = 352;
+
+__device__ __forceinline__ void cp_async_16z(uint32_t dst, const void* src, uint32_t bytes) {   // bytes 0: zero fill
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
 
 __global__ void __launch_bounds__(kReconThreads, 1)
 subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid_constant__ SubParams p) {
@@ -276,37 +293,42 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   if (tid == 0) {
     for (int s = 0; s < kRingB; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
-    mbar_init(&sm.a_full, 1);
+    for (int s = 0; s < kStageA; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 4); }
     mbar_init(&sm.a_ready, 4);
     mbar_init(&sm.a_free, 1);
+    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.g_full[s], 128); mbar_init(&sm.g_done[s], 4); mbar_init(&sm.g_empty[s], 1); }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(256) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t t_o = sm.tmem_base;      // two accumulators of 128 columns
+  const uint32_t t_a = sm.tmem_base;            // the Xt tile: 128 lanes x kp columns
+  const uint32_t t_o = sm.tmem_base + 256;      // two accumulators of 128 columns
   bool bad = false;
+  // 32-column parts of block c that lie inside the matrix
+  auto parts_of = [&](uint32_t c) { const uint32_t left = p.d - c * kBlockN; return left >= (uint32_t)kBlockN ? 4u : (left + 31u) / 32u; };
 
   if (warp == 0) {
     if (lane == 0) {
-      uint32_t it = 0, t = 0;
+      uint32_t it = 0, ia = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
         const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
         const int r0 = (int)(g * 32);
-        if (t > 0) ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.abort);   // the last MMAs have read the old tile
-        if (!ok) break;
-        mbar_expect_tx(&sm.a_full, k_tiles * h * 128);
-        for (uint32_t kt = 0; kt < k_tiles; ++kt) {
-          if (hg == 4) tma_load_2d(sm.a + kt * kSlotA, &maps.xt128, (int)(kt * kTileK), r0, &sm.a_full);
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++ia) {
+          const uint32_t s = ia % kStageA;
+          ok = mbar_wait(&sm.a_empty[s], ((ia / kStageA) & 1u) ^ 1u, sm.abort);
+          if (!ok) break;
+          mbar_expect_tx(&sm.a_full[s], h * 128);
+          if (hg == 4) tma_load_2d(sm.a[s], &maps.xt128, (int)(kt * kTileK), r0, &sm.a_full[s]);
           else
             for (uint32_t i = 0; i < hg; ++i)
-              tma_load_2d(sm.a + kt * kSlotA + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full);
+              tma_load_2d(sm.a[s] + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full[s]);
         }
         for (uint32_t c = 0; ok && c < n_blocks; ++c)
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
@@ -325,7 +347,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       const uint32_t idesc = instr_desc(kRows, kBlockN, 0);
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2);
       for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-        ok = mbar_wait(&sm.a_ready, t & 1u, sm.abort);          // landed and rounded
+        ok = mbar_wait(&sm.a_ready, t & 1u, sm.abort);          // the tile is in tensor memory, rounded
         if (!ok) break;
         tc_fence_after();
         for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
@@ -340,10 +362,10 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
             ok = mbar_wait(&sm.full[s], (it / kRingB) & 1u, sm.abort);
             if (!ok) break;
             tc_fence_after();
-            const uint64_t da = desc_k | (uint64_t)((smem_u32(sm.a + kt * kSlotA) >> 4) & 0x3FFF);
             const uint64_t db = desc_k | (uint64_t)((smem_u32(sm.ring[s]) >> 4) & 0x3FFF);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) mma_ss(t_o + buf * kBlockN, da + 2 * j, db + 2 * j, idesc, (kt | (uint32_t)j) != 0);
+            for (int j = 0; j < 4; ++j)
+              mma_ts(t_o + buf * kBlockN, t_a + kt * kTileK + 8 * j, db + 2 * j, idesc, (kt | (uint32_t)j) != 0);
             mma_commit(&sm.empty[s]);
           }
           if (!ok) break;
@@ -352,75 +374,153 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         if (ok) mma_commit(&sm.a_free);
       }
     }
-  } else {
+  } else if (warp == 2) {
+    // ---- part store: a finished part leaves by tensor-map store; its stage is free once the store has read it ----
+    if (lane == 0) {
+      uint32_t is = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
+        const int r0 = (int)(g * 32);
+        for (uint32_t c = 0; ok && c < n_blocks; ++c) {
+          const uint32_t np = parts_of(c);
+          for (uint32_t part = 0; part < np; ++part, ++is) {
+            const uint32_t s = is % kStages;
+            ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.abort);
+            if (!ok) break;
+            const int col0 = (int)(c * kBlockN + part * 32);
+            const uint32_t src = smem_u32(sm.st_t[s]);
+            if (hg == 4) tma_store_2d(&maps.o128, col0, r0, src);
+            else
+              for (uint32_t i = 0; i < hg; ++i) tma_store_2d(&maps.o32, col0, r0 + 32 * (int)i, src + i * 4096);
+            bulk_commit();
+            bulk_wait_read_all();
+            mbar_arrive(&sm.g_empty[s]);
+          }
+        }
+      }
+      bulk_wait_all();
+    }
+  } else if (warp < 7) {
+    // ---- staging warps: Xt tile -> tensor memory (thread = lane of its 32-lane window), then the gathers ----
     const uint32_t q = (uint32_t)(warp & 3);
     const uint32_t row = 32u * q + (uint32_t)lane;
-    uint32_t cg = 0, t = 0;
+    const uint32_t gt = (uint32_t)(tid - 96), gch = gt & 7u, grow = gt >> 3;   // gather: 8 threads per 128-byte segment
+    uint32_t ia = 0, ig = 0, t = 0;
     bool ok = true;
     for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
       const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
       const uint64_t r0 = g * 32;
-      const RowInfo ri = row_info(p, r0, h, row, bad);
-      // round the Xt tile to the nearest TF32 value in place (element-wise: any thread, any chunk)
-      ok = mbar_wait(&sm.a_full, t & 1u, sm.abort);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      for (uint32_t i = (uint32_t)(tid - 64); i < k_tiles * 1024u; i += 128u) {
-        const uint32_t a = smem_u32(sm.a) + i * 16u;
-        float4 v = lds128(a);
-        v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
-        v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
-        v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
-        v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
-        sts128(a, v);
+      // the eight rows this thread gathers for: row grow + 16 i
+      const float* tp[8];
+      const float* ps[8];
+      uint32_t mask = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const RowInfo ri = row_info(p, r0, h, grow + 16u * (uint32_t)i, bad);
+        tp[i] = ri.gather ? ri.tp + 4 * gch : p.T_perp;
+        ps[i] = ri.gather ? ri.ps + 4 * gch : p.pos;
+        mask |= ri.gather ? 1u << i : 0u;
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (t > 0) {                                   // the MMAs of the previous sub-tile have read the old tile
+        ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      for (uint32_t kt = 0; kt < k_tiles; ++kt, ++ia) {
+        const uint32_t s = ia % kStageA;
+        ok = mbar_wait(&sm.a_full[s], (ia / kStageA) & 1u, sm.abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint32_t v[32];
+        const uint32_t a0 = smem_u32(sm.a[s]) + row * 128;
+#pragma unroll
+        for (uint32_t ch = 0; ch < 8; ++ch) {
+          const float4 f = lds128(a0 + ((ch ^ (row & 7u)) << 4));
+          v[4 * ch + 0] = round_tf32(__float_as_uint(f.x));
+          v[4 * ch + 1] = round_tf32(__float_as_uint(f.y));
+          v[4 * ch + 2] = round_tf32(__float_as_uint(f.z));
+          v[4 * ch + 3] = round_tf32(__float_as_uint(f.w));
+        }
+        tmem_st32(t_a + kt * kTileK + ((32u * q) << 16), v);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.a_empty[s]);
+      }
+      if (!ok) break;
+      tmem_st_wait();
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.a_ready);
-      // the embedding and position values of a 32-column part are requested one part ahead of their use
-      float4 tp[8], ps[8];
-      auto fetch = [&](uint32_t col0) {
+      for (uint32_t c = 0; ok && c < n_blocks; ++c) {
+        const uint32_t np = parts_of(c);
+        for (uint32_t part = 0; part < np; ++part, ++ig) {
+          const uint32_t s = ig % kStages;
+          ok = mbar_wait(&sm.g_empty[s], ((ig / kStages) & 1u) ^ 1u, sm.abort);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (p.ids) {
+            const uint32_t col0 = c * kBlockN + part * 32;
+            const bool in_col = col0 + 4 * gch < p.d;
+            const uint32_t dt = smem_u32(sm.st_t[s]), dp = smem_u32(sm.st_p[s]);
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          const uint32_t col = col0 + 4u * (uint32_t)ch;
-          const bool in = ri.gather && col < p.d;
-          tp[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          ps[ch] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t r = grow + 16u * (uint32_t)i;
+              const uint32_t off = r * 128 + ((gch ^ (r & 7u)) << 4);
+              const bool in = in_col && ((mask >> i) & 1u);
+              cp_async_16z(dt + off, in ? (const void*)(tp[i] + col0) : (const void*)p.T_perp, in ? 16u : 0u);
+              cp_async_16z(dp + off, in ? (const void*)(ps[i] + col0) : (const void*)p.pos, in ? 16u : 0u);
+            }
+          }
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sm.g_full[s])) : "memory");
         }
-      };
-      fetch(0);
+      }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
+    // ---- epilogue warps: accumulator part + gathered rows, in place in the stage ----
+    const uint32_t q = (uint32_t)(warp & 3);
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    const uint32_t roff = row * 128, sw = row & 7u;
+    const bool add = p.ids != nullptr;
+    uint32_t cg = 0, ie = 0;
+    bool ok = true;
+    for (uint64_t g = g0; ok && g < g1; g += 4) {
       for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
         const uint32_t buf = cg & 1u;
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.abort);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t np = parts_of(c);
+        for (uint32_t part = 0; part < np; ++part, ++ie) {
+          const uint32_t s = ie % kStages;
+          uint32_t v[32];
+          tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
+          ok = mbar_wait(&sm.g_full[s], (ie / kStages) & 1u, sm.abort);
+          ok = __all_sync(0xffffffffu, ok);
+          tmem_ld_wait();
+          if (!ok) break;
+          const uint32_t bt = smem_u32(sm.st_t[s]) + roff, bp = smem_u32(sm.st_p[s]) + roff;
 #pragma unroll
-        for (uint32_t part = 0; part < 4; ++part) {
-          const uint32_t col0 = c * kBlockN + part * 32;
-          float4 ct[8], cs[8];
-#pragma unroll
-          for (int ch = 0; ch < 8; ++ch) { ct[ch] = tp[ch]; cs[ch] = ps[ch]; }
-          fetch(col0 + 32);
-          if (col0 < p.d) {
-            uint32_t v[32];
-            tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
-            tmem_ld_wait();
-            if (ri.valid) {
-              float* dst = p.out + (r0 + row) * (uint64_t)p.d + col0;
-#pragma unroll
-              for (int ch = 0; ch < 8; ++ch)
-                if (col0 + 4u * (uint32_t)ch < p.d) {
-                  float4 o;
-                  o.x = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 0]), ct[ch].x), cs[ch].x);
-                  o.y = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 1]), ct[ch].y), cs[ch].y);
-                  o.z = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 2]), ct[ch].z), cs[ch].z);
-                  o.w = __fadd_rn(__fadd_rn(__uint_as_float(v[4 * ch + 3]), ct[ch].w), cs[ch].w);
-                  __stcs(reinterpret_cast<float4*>(dst + 4 * ch), o);
-                }
+          for (uint32_t ch = 0; ch < 8; ++ch) {
+            const uint32_t o = (ch ^ sw) << 4;
+            float4 r = make_float4(__uint_as_float(v[4 * ch]), __uint_as_float(v[4 * ch + 1]), __uint_as_float(v[4 * ch + 2]),
+                                   __uint_as_float(v[4 * ch + 3]));
+            if (add) {
+              const float4 e = lds128(bt + o), f = lds128(bp + o);
+              r.x = __fadd_rn(__fadd_rn(r.x, e.x), f.x);
+              r.y = __fadd_rn(__fadd_rn(r.y, e.y), f.y);
+              r.z = __fadd_rn(__fadd_rn(r.z, e.z), f.z);
+              r.w = __fadd_rn(__fadd_rn(r.w, e.w), f.w);
             }
+            sts128(bt + o, r);
           }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.g_done[s]);
         }
+        if (!ok) break;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.o_empty[buf]);
@@ -431,7 +531,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_o), "r"(256) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sm.tmem_base), "r"(512) : "memory");
   }
   if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
   if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
@@ -537,7 +637,9 @@ cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, con
   ReconMaps m;
   if (!make_map(&m.xt128, Xt, k, n_tok, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !make_map(&m.xt32, Xt, k, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_map(&m.u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B))
+      !make_map(&m.u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.o128, Xhat, d, n_tok, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&m.o32, Xhat, d, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B))
     return cudaErrorInvalidValue;
   const int smem = (int)sizeof(ReconSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(subspace_reconstruct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
