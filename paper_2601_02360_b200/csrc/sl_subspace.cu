@@ -7,14 +7,15 @@
 // rows, built from the same pieces as the embedding re-projection kernel:
 //
 //   compress     K-loop over d in steps of 32 columns.  The X tile arrives by TMA (K-major,
-//                128-byte swizzle); eight warps (two threads per token) then subtract the token's
-//                T_perp row and its Pos row - fetched with plain loads two steps ahead - round to
-//                the nearest TF32 value (the tensor cores would cut instead) and hand the tile to
-//                the MMA warp; B = 32 rows of U, N-major.  The same warps write the accumulator
-//                out as Xt.
-//   reconstruct  the Xt tile (all k columns) arrives once per sub-tile, is rounded in place, and
-//                is the A operand of every 128-column block; B = 128 rows of U through a ring; the
-//                accumulator is double buffered; the epilogue adds the gathered rows and stores.
+//                128-byte swizzle); eight warps (eight threads per token row, so that a gathered
+//                128-byte segment is one request) then subtract the token's T_perp row and its Pos
+//                row - fetched with plain loads two steps ahead - round to the nearest TF32 value
+//                (the tensor cores would cut instead) and hand the tile to the MMA warp; B = 32
+//                rows of U, N-major.  The same warps write the accumulator out as Xt.
+//   reconstruct  the Xt tile (all k columns) is rounded and moved to tensor memory once per
+//                sub-tile and is the A operand of every 128-column block; B = 128 rows of U through
+//                a ring; the accumulator is double buffered; the gathered rows wait in stages of
+//                shared memory, the epilogue adds them and a tensor-map store writes the part.
 //
 // Tokens are dealt in groups of 32 evenly over one CTA per SM, sub-tiles of up to 128 tokens.
 // Every wait is bounded (SL_FLAG_TIMEOUT); a token id outside [0, V) gathers nothing and raises
@@ -155,26 +156,39 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
       }
     }
   } else {
-    // ---- row warps: two threads per token of the sub-tile (each takes four of the eight 16-byte chunks
-    // of a tile row); warp w reads tensor-memory lanes 32*(w%4).. ----
+    // ---- row warps.  Element-wise part: eight threads per token row, one 16-byte chunk each, so that a
+    // gathered 128-byte segment is one request; thread j serves chunk j % 8 of rows j / 8 + 32 i.
+    // Accumulator read-out: warp w reads tensor-memory lanes 32*(w%4).., the two warps of a window
+    // alternate over blocks of 32 columns. ----
     const uint32_t q = (uint32_t)(warp & 3), half = (uint32_t)(warp - 2) >> 2;
     const uint32_t row = 32u * q + (uint32_t)lane;
-    const uint32_t sw = row & 7u;
+    const uint32_t j = (uint32_t)(tid - 64), gch = j & 7u, grow = j >> 3;
+    const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);     // + 4096 i: the swizzle repeats every 8 rows
     uint32_t it = 0, t = 0;
     bool ok = true;
     for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
       const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
       const uint64_t r0 = g * 32;
-      const RowInfo ri = row_info(p, r0, h, row, bad);
+      const float* tp[4];
+      const float* ps[4];
+      uint32_t mask = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const RowInfo ri = row_info(p, r0, h, grow + 32u * (uint32_t)i, bad);
+        tp[i] = ri.gather ? ri.tp + 4 * gch : nullptr;
+        ps[i] = ri.gather ? ri.ps + 4 * gch : nullptr;
+        mask |= ri.gather ? 1u << i : 0u;
+      }
       // the embedding and position values of the next two K steps are in flight while one is used
       float4 et[2][4], ep[2][4];
       auto fetch = [&](uint32_t kt, float4 (&dt)[4], float4 (&dp)[4]) {
+        const uint32_t col = kt * kTileK + 4u * gch;
+        const bool in_col = kt < k_tiles && col < p.d;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t col = kt * kTileK + 16u * half + 4u * (uint32_t)c;
-          const bool in = ri.gather && kt < k_tiles && col < p.d;
-          dt[c] = in ? __ldg(reinterpret_cast<const float4*>(ri.tp + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          dp[c] = in ? __ldg(reinterpret_cast<const float4*>(ri.ps + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < 4; ++i) {
+          const bool in = in_col && ((mask >> i) & 1u);
+          dt[i] = in ? __ldg(reinterpret_cast<const float4*>(tp[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          dp[i] = in ? __ldg(reinterpret_cast<const float4*>(ps[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
       };
       fetch(0, et[0], ep[0]);
@@ -186,21 +200,21 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
           if (kk < k_tiles) {
             float4 ct[4], cp[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) { ct[c] = et[par][c]; cp[c] = ep[par][c]; }
+            for (int i = 0; i < 4; ++i) { ct[i] = et[par][i]; cp[i] = ep[par][i]; }
             fetch(kk + 2, et[par], ep[par]);
             const uint32_t s = it % kRing;
             ok = ok && mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
-              const uint32_t a0 = smem_u32(sm.ring + s * kSlotP) + row * 128;
+              const uint32_t a0 = smem_u32(sm.ring + s * kSlotP) + goff;
 #pragma unroll
-              for (uint32_t c = 0; c < 4; ++c) {
-                const uint32_t a = a0 + (((4u * half + c) ^ sw) << 4);
+              for (uint32_t i = 0; i < 4; ++i) {
+                const uint32_t a = a0 + 4096u * i;
                 float4 v = lds128(a);
-                v.x = __fsub_rn(__fsub_rn(v.x, ct[c].x), cp[c].x);
-                v.y = __fsub_rn(__fsub_rn(v.y, ct[c].y), cp[c].y);
-                v.z = __fsub_rn(__fsub_rn(v.z, ct[c].z), cp[c].z);
-                v.w = __fsub_rn(__fsub_rn(v.w, ct[c].w), cp[c].w);
+                v.x = __fsub_rn(__fsub_rn(v.x, ct[i].x), cp[i].x);
+                v.y = __fsub_rn(__fsub_rn(v.y, ct[i].y), cp[i].y);
+                v.z = __fsub_rn(__fsub_rn(v.z, ct[i].z), cp[i].z);
+                v.w = __fsub_rn(__fsub_rn(v.w, ct[i].w), cp[i].w);
                 v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
                 v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
                 v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
@@ -226,7 +240,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
         uint32_t v[32];
         tmem_ld32(t_p + cb + ((32u * q) << 16), v);
         tmem_ld_wait();
-        if (ri.valid) {
+        if (row < h && r0 + row < p.n_tok) {
           float* dst = p.out + (r0 + row) * (uint64_t)p.k + cb;
 #pragma unroll
           for (int i = 0; i < 32; i += 4)
