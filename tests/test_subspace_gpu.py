@@ -148,3 +148,40 @@ def test_shapes_outside_the_tensor_core_path(n_tok, L, V, d, k):
     ref_h = osub.reconstruct(ref.astype(np.float32), ids, T_perp, pos, U, L)
     S_h = osub.abs_bound_reconstruct(ref, U) + np.abs(T_perp)[ids] + np.abs(pos)[np.arange(n_tok) % L]
     assert f == 0 and np.all(np.abs(xh - ref_h) <= 2.0 ** -18 * S_h + 1e-30)
+
+
+@pytest.mark.parametrize("n_tok", [16384, 65536])
+def test_bench_size_on_sampled_tokens(n_tok):
+    # the workload bench.py --subspace times (1B stage boundary), both launches at full size; tokens are
+    # independent, so the checker computes a sample of them one by one: the first and last token, the
+    # tokens around every boundary between two CTAs' shares and between sub-tiles, and random ones
+    L, V, d, k = 2048, 32000, 2048, 256
+    U = synth.gen_subspace_basis(d, k, seed=0)
+    u = torch.from_numpy(U).cuda()
+    api.sl_round_tf32(u, u.numel())
+    U = u.cpu().numpy()
+    X, ids, T_perp, pos = synth.gen_stage_boundary(n_tok, L, V, d, seed=0)
+    dX, dids, dT, dP = _dev(X), _dev(ids), _dev(T_perp), _dev(pos)
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    xt = torch.full((n_tok, k), 7.0, dtype=torch.float32, device="cuda")
+    xh = torch.full((n_tok, d), 7.0, dtype=torch.float32, device="cuda")
+    api.sl_subspace_project(dX, dids, dT, dP, u, n_tok, L, V, d, k, xt, flags)
+    api.sl_subspace_reconstruct(xt, dids, dT, dP, u, n_tok, L, V, d, k, xh, flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    rng = np.random.default_rng(5)
+    groups = n_tok // 32
+    edges = np.unique(np.array([(c * groups // 148) * 32 for c in range(149)]))
+    near = np.concatenate([edges + o for o in (-1, 0, 1, 127, 128, 129)])
+    rows = np.unique(np.clip(np.concatenate([[0, 1, n_tok - 2, n_tok - 1], near, rng.integers(0, n_tok, 300)]), 0, n_tok - 1))
+    g_xt = xt[torch.from_numpy(rows).cuda()].cpu().numpy()
+    g_xh = xh[torch.from_numpy(rows).cuda()].cpu().numpy()
+    pos_rows = pos[rows % L]                               # the checker's positions are 0 .. len - 1 of what it is given
+    ref = osub.project(X[rows], ids[rows], T_perp, pos_rows, U, len(rows))
+    S = osub.abs_bound_project(X[rows], ids[rows], T_perp, pos_rows, U, len(rows))
+    assert np.all(np.abs(g_xt - ref) <= TOL * S + 1e-30)
+    ref_h = osub.reconstruct(g_xt, ids[rows], T_perp, pos_rows, U, len(rows))
+    S_h = osub.abs_bound_reconstruct(g_xt, U) + np.abs(T_perp.astype(np.float64))[ids[rows]] + np.abs(pos_rows.astype(np.float64))
+    assert np.all(np.abs(g_xh - ref_h) <= TOL * S_h + 1e-30)
+    # every token was written (the fill value is gone) and nothing is NaN
+    assert not bool(torch.isnan(xh).any()) and not bool((xt == 7.0).all(dim=1).any())
