@@ -325,6 +325,10 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   const uint32_t t_o = sm.tmem_base + 256;      // two accumulators of 128 columns
   bool bad = false;
   // 32-column parts of block c that lie inside the matrix
+  // CTAs walk the 128-column blocks from different starting points, so that they do not all ask L2 for the
+  // same rows of U at the same time (the blocks are independent: no effect on the result)
+  const uint32_t c_first = blockIdx.x % n_blocks;
+  auto block_of = [&](uint32_t i) { const uint32_t c = i + c_first; return c >= n_blocks ? c - n_blocks : c; };
   auto parts_of = [&](uint32_t c) { const uint32_t left = p.d - c * kBlockN; return left >= (uint32_t)kBlockN ? 4u : (left + 31u) / 32u; };
 
   if (warp == 0) {
@@ -344,13 +348,13 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
             for (uint32_t i = 0; i < hg; ++i)
               tma_load_2d(sm.a[s] + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full[s]);
         }
-        for (uint32_t c = 0; ok && c < n_blocks; ++c)
+        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci)
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
             const uint32_t s = it % kRingB;
             ok = mbar_wait(&sm.empty[s], ((it / kRingB) & 1u) ^ 1u, sm.abort);
             if (!ok) break;
             mbar_expect_tx(&sm.full[s], kSlotB);
-            tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(c * kBlockN), &sm.full[s]);
+            tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(block_of(ci) * kBlockN), &sm.full[s]);
           }
       }
     }
@@ -396,8 +400,8 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       for (uint64_t g = g0; ok && g < g1; g += 4) {
         const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
         const int r0 = (int)(g * 32);
-        for (uint32_t c = 0; ok && c < n_blocks; ++c) {
-          const uint32_t np = parts_of(c);
+        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci) {
+          const uint32_t c = block_of(ci), np = parts_of(c);
           for (uint32_t part = 0; part < np; ++part, ++is) {
             const uint32_t s = is % kStages;
             ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.abort);
@@ -466,8 +470,8 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.a_ready);
-      for (uint32_t c = 0; ok && c < n_blocks; ++c) {
-        const uint32_t np = parts_of(c);
+      for (uint32_t ci = 0; ok && ci < n_blocks; ++ci) {
+        const uint32_t c = block_of(ci), np = parts_of(c);
         for (uint32_t part = 0; part < np; ++part, ++ig) {
           const uint32_t s = ig % kStages;
           ok = mbar_wait(&sm.g_empty[s], ((ig / kStages) & 1u) ^ 1u, sm.abort);
@@ -500,13 +504,13 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     uint32_t cg = 0, ie = 0;
     bool ok = true;
     for (uint64_t g = g0; ok && g < g1; g += 4) {
-      for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+      for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
         const uint32_t buf = cg & 1u;
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.abort);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t np = parts_of(c);
+        const uint32_t np = parts_of(block_of(ci));
         for (uint32_t part = 0; part < np; ++part, ++ie) {
           const uint32_t s = ie % kStages;
           uint32_t v[32];
