@@ -107,11 +107,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
   const long long t0 = clock64();
   for (;;) {
     uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+    // try_wait suspends the thread until the phase completes or a hardware time limit passes
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
     if (ok) return true;
     if (abort || clock64() - t0 > kWaitClocks) { abort = 1; return false; }
-    __nanosleep(32);
   }
 }
 
