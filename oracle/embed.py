@@ -12,7 +12,7 @@ The projection of a row vector t onto S is  Pi_S(t) = t U U^T.
 Everything is the definition written out with numpy in float64: two matrix
 products and two element-wise updates, no blocking and no reordering.  Inputs
 may be float32 arrays; they are widened first and the results stay float64, so
-that a float32/TF32 implementation is judged against the exact value.
+that a float32/TF32 implementation is compared with the exact value.
 
 Pinned by tests/test_oracle_embed_pins.py: a hand-worked example, the closed
 form for U = columns of the identity, idempotence, TE conservation, the residual
