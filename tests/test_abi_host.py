@@ -140,6 +140,35 @@ def test_idx12_argument_checks():
     assert L.sl_unpack_idx12(fake, lay.ref(), 4096, 64, fake + 1, None) == api.SL_ERR_ALIGNMENT
 
 
+def test_subspace_argument_checks():
+    # all checks happen on the host before any launch, so fake addresses are enough
+    L = api.load()
+    fake = 0x10000
+    for fn in (L.sl_subspace_project, L.sl_subspace_reconstruct):
+        ok_args = [fake, fake, fake, fake, fake, 0, 64, 100, 256, 32, fake, None, None]     # n_tok = 0: nothing to do
+        assert fn(*ok_args) == api.SL_OK
+        def call(**kw):
+            a = list(ok_args)
+            a[5] = 128
+            for i, v in kw.items():
+                a[int(i[1:])] = v
+            return fn(*a)
+        assert call(_0=None) == api.SL_ERR_INVALID_ARG            # no input
+        assert call(_4=None) == api.SL_ERR_INVALID_ARG            # no basis
+        assert call(_10=None) == api.SL_ERR_INVALID_ARG           # no output
+        assert call(_8=0) == api.SL_ERR_INVALID_ARG               # d = 0
+        assert call(_9=0) == api.SL_ERR_INVALID_ARG               # k = 0
+        assert call(_2=None) == api.SL_ERR_INVALID_ARG            # token ids without an embedding table
+        assert call(_3=None) == api.SL_ERR_INVALID_ARG            # ... without positions
+        assert call(_6=0) == api.SL_ERR_INVALID_ARG               # ... with sequence length 0
+        assert call(_0=fake + 2) == api.SL_ERR_ALIGNMENT
+        assert call(_1=fake + 1) == api.SL_ERR_ALIGNMENT
+        assert call(_11=fake + 2) == api.SL_ERR_ALIGNMENT
+        assert call(_9=4100) == api.SL_ERR_UNSUPPORTED            # k above 4096
+        assert call(_5=1 << 31) == api.SL_ERR_UNSUPPORTED         # n_tok at or above 2^31
+        assert call(_7=1 << 31) == api.SL_ERR_UNSUPPORTED         # V at or above 2^31
+
+
 def test_header_is_valid_c_and_a_c_client_links(lib, tmp_path):
     import shutil
     import subprocess
