@@ -7,7 +7,7 @@
 // rows, built from the same pieces as the embedding re-projection kernel:
 //
 //   compress     K-loop over d in steps of 32 columns.  The X tile arrives by TMA (K-major,
-//                128-byte swizzle); eight warps (eight threads per token row, so that a gathered
+//                128-byte swizzle; three producer warps share a step's copies); eight warps (eight threads per token row, so that a gathered
 //                128-byte segment is one request) then subtract the token's T_perp row and its Pos
 //                row - fetched with plain loads two steps ahead - round to the nearest TF32 value
 //                (the tensor cores would cut instead) and hand the tile to the MMA warp; B = 32
@@ -36,7 +36,7 @@ constexpr int kRing = 4;
 constexpr int kSlotA = kRows * kTileK * 4;            // 16 KB
 constexpr int kSlotP = kSlotA + 256 * kTileK * 4;     // compress: X tile + 32 rows of U
 constexpr int kRowWarps = 8;                          // two per 32-lane window of tensor memory
-constexpr int kThreads = 64 + 32 * kRowWarps;         // TMA warp, MMA warp, the row warps
+constexpr int kThreads = 128 + 32 * kRowWarps;        // producer warps 0, 2, 3, MMA warp 1, the row warps
 
 struct SubParams {
   const float* T_perp;
@@ -90,7 +90,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
   const uint64_t G = (p.n_tok + 31) / 32;
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
   if (tid == 0) {
-    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.ready[s], kRowWarps); mbar_init(&sm.empty[s], 1); }
+    for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 3); mbar_init(&sm.ready[s], kRowWarps); mbar_init(&sm.empty[s], 1); }
     mbar_init(&sm.p_done, 1);
     mbar_init(&sm.p_free, kRowWarps);
     sm.abort = 0;
@@ -106,8 +106,14 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
   const uint32_t t_p = sm.tmem_base;
   bool bad = false;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 2 || warp == 3) {
+    // ---- three producer warps share the copies of a K step (issuing a tensor-map copy costs its thread
+    // about 0.05 us, and a step has up to nine): warp 0 the X tile and the first boxes of the U slice,
+    // warps 2 and 3 the other boxes; each announces its own bytes on the slot's barrier ----
     if (lane == 0) {
+      const uint32_t pi = warp == 0 ? 0u : (uint32_t)warp - 1u;          // 0, 1, 2
+      const uint32_t nb = p.kp / 32;                                      // boxes of 32 columns in a U slice
+      const uint32_t lo = pi == 0 ? 0u : (pi * nb + 1) / 3, hi = pi == 2 ? nb : ((pi + 1) * nb + 1) / 3;
       uint32_t it = 0;
       bool ok = true;
       for (uint64_t g = g0; ok && g < g1; g += 4) {
@@ -118,12 +124,14 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
           ok = mbar_wait(&sm.empty[s], ((it / kRing) & 1u) ^ 1u, sm.abort);
           if (!ok) break;
           uint8_t* slot = sm.ring + s * kSlotP;
-          mbar_expect_tx(&sm.full[s], h * 128 + p.kp * 128);
-          if (hg == 4) tma_load_2d(slot, &maps.x128, (int)(kt * kTileK), r0, &sm.full[s]);
-          else
-            for (uint32_t i = 0; i < hg; ++i)
-              tma_load_2d(slot + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full[s]);
-          for (uint32_t n = 0; n < p.kp / 32; ++n)
+          mbar_expect_tx(&sm.full[s], (pi == 0 ? h * 128 : 0u) + (hi - lo) * 4096);
+          if (pi == 0) {
+            if (hg == 4) tma_load_2d(slot, &maps.x128, (int)(kt * kTileK), r0, &sm.full[s]);
+            else
+              for (uint32_t i = 0; i < hg; ++i)
+                tma_load_2d(slot + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full[s]);
+          }
+          for (uint32_t n = lo; n < hi; ++n)
             tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
         }
       }
@@ -160,9 +168,9 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
     // gathered 128-byte segment is one request; thread j serves chunk j % 8 of rows j / 8 + 32 i.
     // Accumulator read-out: warp w reads tensor-memory lanes 32*(w%4).., the two warps of a window
     // alternate over blocks of 32 columns. ----
-    const uint32_t q = (uint32_t)(warp & 3), half = (uint32_t)(warp - 2) >> 2;
+    const uint32_t q = (uint32_t)(warp & 3), half = (uint32_t)(warp - 4) >> 2;
     const uint32_t row = 32u * q + (uint32_t)lane;
-    const uint32_t j = (uint32_t)(tid - 64), gch = j & 7u, grow = j >> 3;
+    const uint32_t j = (uint32_t)(tid - 128), gch = j & 7u, grow = j >> 3;
     const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);     // + 4096 i: the swizzle repeats every 8 rows
     uint32_t it = 0, t = 0;
     bool ok = true;
