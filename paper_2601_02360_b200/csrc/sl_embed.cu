@@ -49,7 +49,7 @@ constexpr int kESize = 2 * kEHalf;
 constexpr int kRing2 = 4;         // pass-2 ring: 128 rows of U x 32 columns per slot
 constexpr int kSlot2 = kBlockN * kTileK * 4;
 constexpr int kRing2InX = 2;      // its first slots lie behind the tile buffers, the others in `y`
-constexpr int kThreads = 256;
+constexpr int kThreads = 320;      // ten warps, see the kernel
 static_assert(kEBufs * kESize + kRing2InX * kSlot2 == kRing1 * kSlot1, "pass-2 buffers fill the pass-1 ring");
 
 struct EmbedSmem {
@@ -92,7 +92,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
 
   if (tid == 0) {
-    for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 1); mbar_init(&sm.ready1[s], 4); mbar_init(&sm.empty1[s], 1); }
+    for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 3); mbar_init(&sm.ready1[s], 4); mbar_init(&sm.empty1[s], 1); }
     for (int s = 0; s < kRing2; ++s) { mbar_init(&sm.full2[s], 1); mbar_init(&sm.empty2[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
     for (int b = 0; b < kEBufs; ++b) {
@@ -129,9 +129,31 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     }
   };
 
-  if (warp == 0) {
+  // pass 1: the boxes of a U slice are shared by three producer warps (issuing a tensor-map copy costs its
+  // thread about 0.05 us, and a K step has up to nine): warp 0 takes [0, u_split1), warp 8 [u_split1, u_split2),
+  // warp 9 the rest; each announces its own bytes on the slot's barrier
+  const uint32_t u_boxes = kp / 32, u_split1 = (u_boxes + 1) / 3, u_split2 = (2 * u_boxes + 1) / 3;
+  if (warp == 8 || warp == 9) {
     if (lane == 0) {
-      // ---- operand producer: T_S tiles and U for pass 1, U for pass 2 ----
+      const uint32_t lo = warp == 8 ? u_split1 : u_split2, hi = warp == 8 ? u_split2 : u_boxes;
+      uint32_t it1 = 0, t = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        if (t > 0) ok = mbar_wait(&sm.x_free, (t - 1) & 1u, sm);
+        for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
+          const uint32_t s = it1 % kRing1;
+          ok = mbar_wait(&sm.empty1[s], ((it1 / kRing1) & 1u) ^ 1u, sm);
+          if (!ok) break;
+          uint8_t* slot = sm.x + s * kSlot1;
+          mbar_expect_tx(&sm.full1[s], (hi - lo) * 4096);
+          for (uint32_t n = lo; n < hi; ++n)
+            tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
+        }
+      }
+    }
+  } else if (warp == 0) {
+    if (lane == 0) {
+      // ---- operand producer: T_S tiles and (its share of) U for pass 1, U for pass 2 ----
       uint32_t it1 = 0, it2 = 0, t = 0;
       bool ok = true;
       for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
@@ -147,14 +169,14 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           ok = mbar_wait(&sm.empty1[s], ((it1 / kRing1) & 1u) ^ 1u, sm);
           if (!ok) break;
           uint8_t* slot = sm.x + s * kSlot1;
-          mbar_expect_tx(&sm.full1[s], h * 128 + kp * 128);
+          mbar_expect_tx(&sm.full1[s], h * 128 + u_split1 * 4096);
           if (hg == 4) {
             tma_load_2d(slot, &maps.ts128, (int)(kt * kTileK), r0, &sm.full1[s]);
           } else {
             for (uint32_t i = 0; i < hg; ++i)
               tma_load_2d(slot + i * 4096, &maps.ts32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full1[s]);
           }
-          for (uint32_t n = 0; n < kp / 32; ++n)
+          for (uint32_t n = 0; n < u_split1; ++n)      // the other boxes of the slice come from warps 8 and 9
             tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
         }
         // ... and the pass-2 ring lies over the pass-1 ring: its last MMAs must have read it
