@@ -272,6 +272,184 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
   if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
+// ------------------------------------------------------- compress without embedding terms, two sub-tiles
+// Gt = G U for the activation gradients.  An SM takes in about 32 bytes per clock whatever the path, and of
+// the 48 KB a K step of the kernel above takes in, 32 KB are the slice of U.  With nothing to gather there
+// are registers and shared memory to spare, so two sub-tiles of 128 tokens advance through K together: they
+// share every U slice (64 KB per step for 256 tokens instead of 96 KB) and accumulate in the two halves of
+// tensor memory.  Used when every CTA has at least two sub-tiles anyway.
+constexpr int kRingD = 3;
+constexpr int kSlotD = 2 * kSlotA + 256 * kTileK * 4;   // two X tiles + 32 rows of U: 64 KB
+struct DualSmem {
+  uint8_t ring[kRingD * kSlotD];
+  uint64_t full[kRingD], ready[kRingD], empty[kRingD], p_done, p_free;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid_constant__ SubParams p) {
+  extern __shared__ uint8_t raw[];
+  DualSmem& sm = *reinterpret_cast<DualSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t k_tiles = (p.d + kTileK - 1) / kTileK;
+  const uint64_t G = (p.n_tok + 31) / 32;
+  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  // 32-token groups of the two sub-tiles of the tile that starts at group g
+  auto groups_a = [&](uint64_t g) { return (uint32_t)(g1 - g < 4 ? g1 - g : 4); };
+  auto groups_b = [&](uint64_t g) { return g + 4 >= g1 ? 0u : (uint32_t)(g1 - g - 4 < 4 ? g1 - g - 4 : 4); };
+  if (tid == 0) {
+    for (int s = 0; s < kRingD; ++s) { mbar_init(&sm.full[s], 3); mbar_init(&sm.ready[s], kRowWarps); mbar_init(&sm.empty[s], 1); }
+    mbar_init(&sm.p_done, 1);
+    mbar_init(&sm.p_free, kRowWarps);
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t t_p = sm.tmem_base;      // accumulator of sub-tile A; B is 256 columns further
+
+  if (warp == 0 || warp == 2 || warp == 3) {
+    // ---- three producer warps share the copies of a K step: warp 0 the two X tiles and the first boxes of
+    // the U slice, warps 2 and 3 the other boxes ----
+    if (lane == 0) {
+      const uint32_t pi = warp == 0 ? 0u : (uint32_t)warp - 1u;
+      const uint32_t nb = p.kp / 32;
+      const uint32_t lo = pi == 0 ? 0u : (pi * nb + 1) / 3, hi = pi == 2 ? nb : ((pi + 1) * nb + 1) / 3;
+      uint32_t it = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 8) {
+        const uint32_t ha = groups_a(g), hb = groups_b(g);
+        const int r0 = (int)(g * 32);
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRingD;
+          ok = mbar_wait(&sm.empty[s], ((it / kRingD) & 1u) ^ 1u, sm.abort);
+          if (!ok) break;
+          uint8_t* slot = sm.ring + s * kSlotD;
+          mbar_expect_tx(&sm.full[s], (pi == 0 ? (ha + hb) * 4096 : 0u) + (hi - lo) * 4096);
+          if (pi == 0) {
+            if (ha == 4) tma_load_2d(slot, &maps.x128, (int)(kt * kTileK), r0, &sm.full[s]);
+            else
+              for (uint32_t i = 0; i < ha; ++i)
+                tma_load_2d(slot + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full[s]);
+            if (hb == 4) tma_load_2d(slot + kSlotA, &maps.x128, (int)(kt * kTileK), r0 + kRows, &sm.full[s]);
+            else
+              for (uint32_t i = 0; i < hb; ++i)
+                tma_load_2d(slot + kSlotA + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + kRows + 32 * (int)i, &sm.full[s]);
+          }
+          for (uint32_t n = lo; n < hi; ++n)
+            tma_load_2d(slot + 2 * kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, t = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(kRows, (int)p.kp, 1);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2), desc_n = smem_desc(0, 4096, 512, 1);
+      for (uint64_t g = g0; ok && g < g1; g += 8, ++t) {
+        const bool two = groups_b(g) != 0;
+        if (t > 0) {                                 // the row warps have read the previous accumulators
+          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.abort);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRingD;
+          ok = mbar_wait(&sm.ready[s], (it / kRingD) & 1u, sm.abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(sm.ring + s * kSlotD);
+          const uint64_t da = desc_k | (uint64_t)((a0 >> 4) & 0x3FFF);
+          const uint64_t da2 = desc_k | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+          const uint64_t db = desc_n | (uint64_t)(((a0 + 2 * kSlotA) >> 4) & 0x3FFF);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_ss(t_p, da + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+          if (two) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mma_ss(t_p + 256, da2 + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+          }
+          mma_commit(&sm.empty[s]);
+        }
+        if (ok) mma_commit(&sm.p_done);
+      }
+    }
+  } else {
+    // ---- row warps: round the landed tiles to the nearest TF32 value in place (the tensor cores would cut),
+    // eight threads per row; then write the accumulators out ----
+    const uint32_t q = (uint32_t)(warp & 3), half = (uint32_t)(warp - 4) >> 2;
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    const uint32_t j = (uint32_t)(tid - 128), gch = j & 7u, grow = j >> 3;
+    const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);
+    uint32_t it = 0, t = 0;
+    bool ok = true;
+    for (uint64_t g = g0; ok && g < g1; g += 8, ++t) {
+      const uint32_t ha = groups_a(g), hb = groups_b(g);
+      const uint32_t chunks = hb ? 8u : 4u;          // 16-byte chunks per thread: rows grow + 32 i of A, then of B
+      for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+        const uint32_t s = it % kRingD;
+        ok = mbar_wait(&sm.full[s], (it / kRingD) & 1u, sm.abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t a0 = smem_u32(sm.ring + s * kSlotD) + goff;
+#pragma unroll
+        for (uint32_t i = 0; i < 8; ++i) {
+          if (i < chunks) {
+            const uint32_t a = a0 + 4096u * i;        // the B tile follows the A tile: i = 4 .. 7 are its rows
+            float4 v = lds128(a);
+            v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+            v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+            v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+            v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+            sts128(a, v);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ready[s]);
+      }
+      if (!ok) break;
+      ok = mbar_wait(&sm.p_done, t & 1u, sm.abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      for (uint32_t tile = 0; tile < (hb ? 2u : 1u); ++tile) {
+        const uint32_t h = (tile ? hb : ha) * 32;
+        const uint64_t r0 = g * 32 + (uint64_t)tile * kRows;
+        for (uint32_t cb = 32u * half; cb < p.kp; cb += 64) {
+          uint32_t v[32];
+          tmem_ld32(t_p + tile * 256 + cb + ((32u * q) << 16), v);
+          tmem_ld_wait();
+          if (row < h && r0 + row < p.n_tok) {
+            float* dst = p.out + (r0 + row) * (uint64_t)p.k + cb;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              if (cb + (uint32_t)i < p.k)
+                *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                  __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.p_free);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_p), "r"(512) : "memory");
+  }
+  if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
 // --------------------------------------------------------------------------------------- reconstruct
 // Per sub-tile of 128 tokens the Xt tile goes through a two-slot staging buffer into tensor memory
 // (rounded to TF32 on the way) and is the A operand of every 128-column block.  The embedding and
@@ -640,10 +818,19 @@ cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const fl
       !make_map(&m.x32, X, d, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B, promo) ||
       !make_map(&m.u_n, U, k, d, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
     return cudaErrorInvalidValue;
-  const int smem = (int)sizeof(ProjSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(subspace_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
   const unsigned grid = persistent_grid(n_tok, &e);
+  if (e != cudaSuccess) return e;
+  if (!ids && (n_tok + kRows - 1) / kRows >= 2ull * grid) {
+    // no embedding terms and at least two sub-tiles for every CTA: two sub-tiles share every U slice
+    const int smem = (int)sizeof(DualSmem) + 1024;
+    e = cudaFuncSetAttribute(subspace_project_dual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    subspace_project_dual_kernel<<<grid, kThreads, smem, st>>>(m, p);
+    return cudaGetLastError();
+  }
+  const int smem = (int)sizeof(ProjSmem) + 1024;
+  e = cudaFuncSetAttribute(subspace_project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   subspace_project_kernel<<<grid, kThreads, smem, st>>>(m, p);
   return cudaGetLastError();

@@ -185,3 +185,36 @@ def test_bench_size_on_sampled_tokens(n_tok):
     assert np.all(np.abs(g_xh - ref_h) <= TOL * S_h + 1e-30)
     # every token was written (the fill value is gone) and nothing is NaN
     assert not bool(torch.isnan(xh).any()) and not bool((xt == 7.0).all(dim=1).any())
+
+
+@pytest.mark.parametrize("n_tok,d,k", [(65536, 2048, 256), (40037, 1024, 192), (38000, 512, 64)])
+def test_gradient_form_at_sizes_where_two_sub_tiles_share_the_basis(n_tok, d, k):
+    # Gt = G U at sizes where every CTA has at least two sub-tiles (the launch that walks two sub-tiles
+    # through K together), checked on sampled tokens: ends, sub-tile and CTA boundaries, random ones;
+    # then back through the reconstruction without embedding terms
+    U = synth.gen_subspace_basis(d, k, seed=6)
+    u = torch.from_numpy(U).cuda()
+    api.sl_round_tf32(u, u.numel())
+    U = u.cpu().numpy()
+    rng = np.random.default_rng(7)
+    G = rng.standard_normal((n_tok, d), dtype=np.float32)
+    dG = _dev(G)
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    gt = torch.full((n_tok, k), 7.0, dtype=torch.float32, device="cuda")
+    gh = torch.full((n_tok, d), 7.0, dtype=torch.float32, device="cuda")
+    api.sl_subspace_project(dG, None, None, None, u, n_tok, 1, 0, d, k, gt, flags)
+    api.sl_subspace_reconstruct(gt, None, None, None, u, n_tok, 1, 0, d, k, gh, flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    groups = (n_tok + 31) // 32
+    edges = np.unique(np.array([(c * groups // 148) * 32 for c in range(149)]))
+    near = np.concatenate([edges + o for o in (-1, 0, 1, 127, 128, 129, 255, 256, 257)])
+    rows = np.unique(np.clip(np.concatenate([[0, 1, n_tok - 2, n_tok - 1], near, rng.integers(0, n_tok, 300)]), 0, n_tok - 1))
+    sel = torch.from_numpy(rows).cuda()
+    g_gt, g_gh = gt[sel].cpu().numpy(), gh[sel].cpu().numpy()
+    ref = osub.project(G[rows], None, None, None, U, 1)
+    S = osub.abs_bound_project(G[rows], None, None, None, U, 1)
+    assert np.all(np.abs(g_gt - ref) <= TOL * S + 1e-30)
+    ref_h = g_gt.astype(np.float64) @ U.astype(np.float64).T
+    assert np.all(np.abs(g_gh - ref_h) <= TOL * osub.abs_bound_reconstruct(g_gt, U) + 1e-30)
+    assert not bool((gt == 7.0).all(dim=1).any()) and not bool(torch.isnan(gt).any())
