@@ -497,6 +497,22 @@ def run_subspace(args) -> None:
             t_r.append(e[1].elapsed_time(e[2]))
     clocks = sampler.stop()
     ms_p, ms_r = float(np.median(t_p)), float(np.median(t_r))     # short kernels: the median is robust to clock ramps
+    # the same two launches for activation gradients (no embedding terms), outside the headline figures
+    t_gp, t_gr = [], []
+    for s in range(min(args.steps, 50) + 3):
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        flush.fill_(float(s))
+        flush.fill_(float(s) + 0.5)
+        e[0].record(stream)
+        api.sl_subspace_project(X, None, None, None, U, n_tok, L, 0, d, k, Xt, flags)
+        e[1].record(stream)
+        api.sl_subspace_reconstruct(Xt, None, None, None, U, n_tok, L, 0, d, k, Xhat, flags)
+        e[2].record(stream)
+        torch.cuda.synchronize()
+        if s >= 3:
+            t_gp.append(e[0].elapsed_time(e[1]))
+            t_gr.append(e[1].elapsed_time(e[2]))
     # compress reads X and one gathered T_perp row per token, writes Xt; Pos and U are L2-resident (counted once)
     bytes_p = n_tok * d * 8 + n_tok * k * 4 + L * d * 4 + d * k * 4
     bytes_r = n_tok * k * 4 + n_tok * d * 8 + L * d * 4 + d * k * 4
@@ -508,7 +524,9 @@ def run_subspace(args) -> None:
         "vs_baseline": None, "dtype": "tf32 contraction, f32 gather terms", "data": "synthetic",
         "config": {"workload": f"{wl.name} stage boundary: {n_tok} tokens x d={d}, k={k}, L={L}, vocab {V}",
                    "l2": "a 256 MB buffer is written between timed steps"},
-        "kernels_ms": {"sl_subspace_project": ms_p, "sl_subspace_reconstruct": ms_r},
+        "kernels_ms": {"sl_subspace_project": ms_p, "sl_subspace_reconstruct": ms_r,
+                       "gradient form (ids = NULL), project": float(np.median(t_gp)),
+                       "gradient form (ids = NULL), reconstruct": float(np.median(t_gr))},
         "roofline": {"bound": "hbm", "kernel": "sl_subspace_reconstruct", "achieved": bytes_r / (ms_r * 1e-3) / 1e9,
                      "peak": peak, "unit": "GB/s", "frac": bytes_r / (ms_r * 1e-3) / 1e9 / peak, "traffic": None,
                      "peak_source": peak_src, "algorithmic_bytes": bytes_r,

@@ -12,6 +12,8 @@
 //                row - fetched with plain loads two steps ahead - round to the nearest TF32 value
 //                (the tensor cores would cut instead) and hand the tile to the MMA warp; B = 32
 //                rows of U, N-major.  The same warps write the accumulator out as Xt.
+//                Without embedding terms and with at least two sub-tiles per CTA, two sub-tiles
+//                go through K together and share every U slice (see the dual kernel).
 //   reconstruct  the Xt tile (all k columns) is rounded and moved to tensor memory once per
 //                sub-tile and is the A operand of every 128-column block; B = 128 rows of U through
 //                a ring; the accumulator is double buffered; the gathered rows wait in stages of
