@@ -518,6 +518,7 @@ def run_subspace(args) -> None:
     bytes_r = n_tok * k * 4 + n_tok * d * 8 + L * d * 4 + d * k * 4
     peak, peak_src = measured_peak_gbs()
     ms = ms_p + ms_r
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
     line = {
         "metric": "subspace_roundtrip_tokens_per_s", "value": n_tok / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -532,7 +533,13 @@ def run_subspace(args) -> None:
                      "peak_source": peak_src, "algorithmic_bytes": bytes_r,
                      "project": {"achieved": bytes_p / (ms_p * 1e-3) / 1e9, "frac": bytes_p / (ms_p * 1e-3) / 1e9 / peak,
                                  "algorithmic_bytes": bytes_p},
-                     "tensor_tflops": 4 * n_tok * d * k / (ms * 1e-3) / 1e12},
+                     "tensor_tflops": 4 * n_tok * d * k / (ms * 1e-3) / 1e12,
+                     # what an SM takes in, per SM and second: every 128-token sub-tile streams all of U again
+                     # (the figure both launches run into is about 68 GB/s per SM, whatever the path)
+                     "sm_intake_gbs": {
+                         "project": (3 * n_tok * d * 4 + -(-n_tok // 128) * d * k * 4) / sms / (ms_p * 1e-3) / 1e9,
+                         "reconstruct": (2 * n_tok * d * 4 + n_tok * k * 4 + -(-n_tok // 128) * d * k * 4) / sms
+                                        / (ms_r * 1e-3) / 1e9}},
         "clocks": clocks, "device_flags": int(flags.item()), "gpu_launches": 2 * args.steps,
     }
     if not args.no_cpu:
