@@ -218,3 +218,37 @@ def test_gradient_form_at_sizes_where_two_sub_tiles_share_the_basis(n_tok, d, k)
     ref_h = g_gt.astype(np.float64) @ U.astype(np.float64).T
     assert np.all(np.abs(g_gh - ref_h) <= TOL * osub.abs_bound_reconstruct(g_gt, U) + 1e-30)
     assert not bool((gt == 7.0).all(dim=1).any()) and not bool(torch.isnan(gt).any())
+
+
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        d = int(rng.integers(1, 300)) * 4 if i % 4 else int(rng.integers(3, 700))      # every fourth: any d (plain kernels)
+        k = int(rng.integers(1, min(64, d // 4) + 1)) * 4 if i % 4 else int(rng.integers(1, min(d, 40) + 1))
+        out.append((int(rng.integers(1, 3000)), int(rng.integers(1, 300)), int(rng.integers(1, 2000)), d, min(k, d)))
+    return out
+
+
+@pytest.mark.parametrize("n_tok,L,V,d,k", _random_shapes(24, 11))
+def test_random_shapes_both_directions(n_tok, L, V, d, k):
+    # seeded random sizes: ragged token counts, sequence lengths that do not divide them, widths and subspace
+    # sizes off every tile boundary; three in four take the tensor-core kernels, the rest the plain ones
+    rng = np.random.default_rng(n_tok * 7 + d)
+    q, _ = np.linalg.qr(rng.standard_normal((d, k)))
+    U = np.ascontiguousarray(q[:, :k], dtype=np.float32)
+    X, ids, T_perp, pos = synth.gen_stage_boundary(n_tok, L, V, d, seed=n_tok)
+    xt, f = _project(X, ids, T_perp, pos, U, L)
+    assert f == 0
+    ref = osub.project(X, ids, T_perp, pos, U, L)
+    S = _scale_project(X, ids, T_perp, pos, U, L)
+    assert np.all(np.abs(xt - ref) <= TOL * S + 1e-30)
+    xh, f = _reconstruct(xt, ids, T_perp, pos, U, L)
+    assert f == 0
+    ref_h = osub.reconstruct(xt, ids, T_perp, pos, U, L)
+    S_h = osub.abs_bound_reconstruct(xt, U) + np.abs(T_perp.astype(np.float64))[ids] + np.abs(pos.astype(np.float64))[np.arange(n_tok) % L]
+    assert np.all(np.abs(xh - ref_h) <= TOL * S_h + 1e-30)
+    # and the gradient form on the same activations
+    gt, f = _project(X, None, None, None, U, L)
+    assert f == 0
+    assert np.all(np.abs(gt - osub.project(X, None, None, None, U, L)) <= TOL * (np.abs(X.astype(np.float64)) @ np.abs(U.astype(np.float64))) + 1e-30)
