@@ -174,6 +174,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
     const uint32_t row = 32u * q + (uint32_t)lane;
     const uint32_t j = (uint32_t)(tid - 128), gch = j & 7u, grow = j >> 3;
     const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);     // + 4096 i: the swizzle repeats every 8 rows
+    const bool wide = p.k % 8 == 0 && ((uintptr_t)p.out & 31u) == 0;   // every row piece of Xt starts on 32 bytes
     uint32_t it = 0, t = 0;
     bool ok = true;
     for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
@@ -252,11 +253,17 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
         tmem_ld_wait();
         if (row < h && r0 + row < p.n_tok) {
           float* dst = p.out + (r0 + row) * (uint64_t)p.k + cb;
+          if (wide) {                                // 32-byte stores: half as many write transactions
 #pragma unroll
-          for (int i = 0; i < 32; i += 4)
-            if (cb + (uint32_t)i < p.k)
-              *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                                                __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            for (int i = 0; i < 32; i += 8)
+              if (cb + (uint32_t)i < p.k) stg256(dst + i, v + i);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              if (cb + (uint32_t)i < p.k)
+                *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                  __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          }
         }
       }
       tc_fence_before();
@@ -389,6 +396,7 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
     const uint32_t row = 32u * q + (uint32_t)lane;
     const uint32_t j = (uint32_t)(tid - 128), gch = j & 7u, grow = j >> 3;
     const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);
+    const bool wide = p.k % 8 == 0 && ((uintptr_t)p.out & 31u) == 0;   // every row piece of Xt starts on 32 bytes
     uint32_t it = 0, t = 0;
     bool ok = true;
     for (uint64_t g = g0; ok && g < g1; g += 8, ++t) {
@@ -430,11 +438,17 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
           tmem_ld_wait();
           if (row < h && r0 + row < p.n_tok) {
             float* dst = p.out + (r0 + row) * (uint64_t)p.k + cb;
+            if (wide) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              if (cb + (uint32_t)i < p.k)
-                *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                                                  __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+              for (int i = 0; i < 32; i += 8)
+                if (cb + (uint32_t)i < p.k) stg256(dst + i, v + i);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                if (cb + (uint32_t)i < p.k)
+                  *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                    __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            }
           }
         }
       }

@@ -98,6 +98,11 @@ __device__ __forceinline__ float4 lds128(uint32_t a) {
 __device__ __forceinline__ void sts128(uint32_t a, float4 v) {
   asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
+// one 32-byte store (the address must be 32-byte aligned)
+__device__ __forceinline__ void stg256(float* p, const uint32_t* v) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]),
+               "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
 // number of uses so far of slot s of an n-slot ring after `it` round-robin uses in total
 __device__ __forceinline__ uint32_t ring_uses(uint32_t it, uint32_t s, uint32_t n) { return (it + n - 1 - s) / n; }
 
