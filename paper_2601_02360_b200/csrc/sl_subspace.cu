@@ -177,33 +177,40 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
     const bool wide = p.k % 8 == 0 && ((uintptr_t)p.out & 31u) == 0;   // every row piece of Xt starts on 32 bytes
     uint32_t it = 0, t = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
-      const uint64_t r0 = g * 32;
-      const float* tp[4];
-      const float* ps[4];
-      uint32_t mask = 0;
+    // the token rows this thread gathers for, and the embedding and position values of two K steps in flight
+    // while one is used; those of a sub-tile's first two steps are requested before the previous sub-tile's
+    // accumulator is written out, so that they are there when its K loop starts
+    const float* tp[4];
+    const float* ps[4];
+    uint32_t mask = 0;
+    float4 et[2][4], ep[2][4];
+    auto fetch = [&](uint32_t kt, float4 (&dt)[4], float4 (&dp)[4]) {
+      const uint32_t col = kt * kTileK + 4u * gch;
+      const bool in_col = kt < k_tiles && col < p.d;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const RowInfo ri = row_info(p, r0, h, grow + 32u * (uint32_t)i, bad);
+        const bool in = in_col && ((mask >> i) & 1u);
+        dt[i] = in ? __ldg(reinterpret_cast<const float4*>(tp[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        dp[i] = in ? __ldg(reinterpret_cast<const float4*>(ps[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    auto open_tile = [&](uint64_t g) {
+      const uint32_t h = (uint32_t)(g1 - g < 4 ? g1 - g : 4) * 32;
+      mask = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const RowInfo ri = row_info(p, g * 32, h, grow + 32u * (uint32_t)i, bad);
         tp[i] = ri.gather ? ri.tp + 4 * gch : nullptr;
         ps[i] = ri.gather ? ri.ps + 4 * gch : nullptr;
         mask |= ri.gather ? 1u << i : 0u;
       }
-      // the embedding and position values of the next two K steps are in flight while one is used
-      float4 et[2][4], ep[2][4];
-      auto fetch = [&](uint32_t kt, float4 (&dt)[4], float4 (&dp)[4]) {
-        const uint32_t col = kt * kTileK + 4u * gch;
-        const bool in_col = kt < k_tiles && col < p.d;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const bool in = in_col && ((mask >> i) & 1u);
-          dt[i] = in ? __ldg(reinterpret_cast<const float4*>(tp[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          dp[i] = in ? __ldg(reinterpret_cast<const float4*>(ps[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      };
       fetch(0, et[0], ep[0]);
       fetch(1, et[1], ep[1]);
+    };
+    if (g0 < g1) open_tile(g0);
+    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+      const uint64_t r0 = g * 32;
       for (uint32_t kt = 0; ok && kt < k_tiles; kt += 2) {
 #pragma unroll
         for (int par = 0; par < 2; ++par) {          // two K steps per trip so that the buffers keep static indices
@@ -241,6 +248,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
         }
       }
       if (!ok) break;
+      if (g + 4 < g1) open_tile(g + 4);
       // the coordinates of this sub-tile's tokens: out of tensor memory, into Xt (the two warps of a lane
       // window take alternate blocks of 32 columns)
       ok = mbar_wait(&sm.p_done, t & 1u, sm.abort);
