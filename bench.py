@@ -242,12 +242,43 @@ def run_reference_embed(args) -> None:
         "gpu_launches": 0}))
 
 
+def run_reference_subspace(args) -> None:
+    """--impl reference --subspace: the float64 numpy checker of section 2.3 on a bounded sample of the tokens."""
+    from oracle import subspace as osub
+    wl = synth.workload(args.workload)
+    name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
+    k = args.k or d // 8
+    L, rows = 2048, min(args.tokens, 2048)
+    U = synth.gen_subspace_basis(d, k, args.seed)
+    X, ids, T_perp, pos = synth.gen_stage_boundary(rows, L, V, d, args.seed)
+    times = []
+    for s in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        xt = osub.project(X, ids, T_perp, pos, U, L)
+        osub.reconstruct(xt, ids, T_perp, pos, U, L)
+        if s >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    sec = float(np.mean(times))
+    desc = f"{rows} tokens x d={d}, k={k}, float64 numpy, both directions"
+    print(json.dumps({
+        "impl": "reference", "metric": "subspace_roundtrip_tokens_per_s", "value": rows / sec, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{wl.name} stage boundary: {args.tokens} tokens x d={d}, k={k}, L={L}, vocab {V}",
+                   "sample": desc},
+        "cpu_baseline": {"value": rows / sec, "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": rows / sec, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
 def run_reference(args) -> None:
     rank, _, world = dist_env()
     if rank != 0:
         return
     if args.embed:
         return run_reference_embed(args)
+    if args.subspace:
+        return run_reference_subspace(args)
     wl = synth.workload(args.workload)
     sample = cpu_sample_workload(wl)
     times, threads = time_oracle(sample, args.steps, args.warmup, args.seed)
