@@ -25,8 +25,8 @@
  * Arena and chunks
  * ----------------
  *  Parameters live in a flat fp32 arena of `n_total` elements holding `n_tensors` tensors back
- *  to back (row-major).  Two chunk geometries (the paper says "64 x 64 (i.e., 4096 elements per
- *  chunk)", §3 "Training Configuration", Table 8, which can be read either way):
+ *  to back (row-major).  Two chunk geometries (the paper's chunk of 4096 elements is stated as a
+ *  64 by 64 block, §3 "Training Configuration", Table 8, which can be read either way):
  *   - consecutive (default): a chunk is a run of `chunk` consecutive elements of ONE tensor; the
  *     last chunk of a tensor may be short.  Position p of a chunk is its p-th element.
  *   - square tiles (sl_layout.cols[t] > 0): tensor t is a matrix of cols[t] columns cut into
@@ -100,6 +100,11 @@ uint64_t sl_num_chunks(const sl_layout* layout, int chunk);
 /* Bytes of `codes` ONE chunk owns: ceil(k*bits/8), or 4*k when bits == 32.  0 on bad arguments.
  * A replica's codes buffer is sl_num_chunks() * sl_codes_stride() bytes. */
 uint64_t sl_codes_stride(int k, int bits);
+
+/* Bytes of ONE replica's whole `codes` buffer for the arena: sl_num_chunks(layout, chunk) *
+ * sl_codes_stride(k, bits) (Eq. 2 line 3: the quantised values of the message).  0 on bad
+ * arguments (those of the two calls above, or k > chunk). */
+uint64_t sl_codes_bytes(const sl_layout* layout, int chunk, int k, int bits);
 
 /* Eq. 2 lines 1-4 for ONE replica: pseudo-gradient, error feedback, chunk-wise Top-k,
  * quantisation, residual.
@@ -213,6 +218,16 @@ int sl_subspace_reconstruct(const float* Xt, const int32_t* ids, const float* T_
 /* x[i] <- the TF32 value nearest to x[i] (ties away from zero), kept as float32, for i < n; in place.
  * For matrices that are fed to the tensor cores many times and never change (U above). */
 int sl_round_tf32(float* x, uint64_t n, void* stream);
+
+/* Debugging aid (the paper has no counterpart).  Every wait of a kernel of this library on one of
+ * its own on-chip copies is bounded: when the bound runs out the kernel stops issuing copies, lets
+ * the copies still in flight land, raises SL_FLAG_TIMEOUT in `*flags` and returns; the call's
+ * outputs are then unspecified and the device stays usable.  The default bound is about a second,
+ * which a healthy device never reaches.  This call replaces it, for every later call from any
+ * thread of the process, by `polls` non-blocking polls per wait (1 = give up unless the data is
+ * there already; negative = give up without looking), which lets a test drive that path; 0
+ * restores the default. */
+void sl_debug_set_wait_limit(int32_t polls);
 
 /* Static description of an SL_* return code. */
 const char* sl_strerror(int code);

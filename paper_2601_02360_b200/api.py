@@ -21,9 +21,9 @@ SL_OK, SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_CUDA = 0
 SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
 SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1280, 64
 
-EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_compress", "sl_compress_batch", "sl_aggregate",
+EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_codes_bytes", "sl_compress", "sl_compress_batch", "sl_aggregate",
            "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_round_tf32", "sl_subspace_project", "sl_subspace_reconstruct", "sl_idx12_stride",
-           "sl_pack_idx12", "sl_unpack_idx12", "sl_strerror")
+           "sl_pack_idx12", "sl_unpack_idx12", "sl_debug_set_wait_limit", "sl_strerror")
 
 
 class SlLayout(ctypes.Structure):
@@ -56,6 +56,8 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_num_chunks.argtypes = [lp, i32]
     L.sl_codes_stride.restype = u64
     L.sl_codes_stride.argtypes = [i32, i32]
+    L.sl_codes_bytes.restype = u64
+    L.sl_codes_bytes.argtypes = [lp, i32, i32, i32]
     L.sl_compress.restype = i32
     L.sl_compress.argtypes = [vp, vp, vp, lp, f32, i32, i32, i32, vp, vp, vp, vp, vp]
     L.sl_compress_batch.restype = i32
@@ -83,6 +85,8 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_pack_idx12.argtypes = [vp, u64, i32, vp, vp, vp]
     L.sl_unpack_idx12.restype = i32
     L.sl_unpack_idx12.argtypes = [vp, lp, i32, i32, vp, vp]
+    L.sl_debug_set_wait_limit.restype = None
+    L.sl_debug_set_wait_limit.argtypes = [ctypes.c_int32]
     L.sl_strerror.restype = ctypes.c_char_p
     L.sl_strerror.argtypes = [i32]
     if path is None:
@@ -156,6 +160,10 @@ def sl_num_chunks(layout, chunk: int) -> int:
 
 def sl_codes_stride(k: int, bits: int) -> int:
     return int(load().sl_codes_stride(k, bits))
+
+
+def sl_codes_bytes(layout, chunk: int, k: int, bits: int) -> int:
+    return int(load().sl_codes_bytes(_layout(layout).ref(), chunk, k, bits))
 
 
 def sl_compress(theta_local, theta_global, err, layout, beta: float, chunk: int, k: int, bits: int,
@@ -244,11 +252,14 @@ def sl_unpack_idx12(packed, layout, chunk: int, k: int, idx, stream=None) -> Non
            "sl_unpack_idx12")
 
 
+def sl_debug_set_wait_limit(polls: int) -> None:
+    load().sl_debug_set_wait_limit(polls)
+
+
 def alloc_messages(layout, chunk: int, k: int, bits: int, R: int, device="cuda"):
     """Device buffers for R replicas' messages: lists (idx, codes, scales)."""
     nc = sl_num_chunks(layout, chunk)
-    st = sl_codes_stride(k, bits)
     idx = [torch.empty(nc * k, dtype=torch.uint16, device=device) for _ in range(R)]
-    codes = [torch.empty(nc * st, dtype=torch.uint8, device=device) for _ in range(R)]
+    codes = [torch.empty(sl_codes_bytes(layout, chunk, k, bits), dtype=torch.uint8, device=device) for _ in range(R)]
     scales = [torch.empty(nc, dtype=torch.float32, device=device) for _ in range(R)]
     return idx, codes, scales

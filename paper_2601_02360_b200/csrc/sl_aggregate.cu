@@ -82,6 +82,7 @@ struct AggSmem {
   float acc[kAC];
   float gbuf[2][kAC];                // theta_global of the current / next chunk (APPLY only)
   uint64_t full[2];
+  volatile uint32_t abort_it;        // 0, or 1 + the iteration at which the bounded wait gave up
 };
 
 __device__ __forceinline__ uint32_t agg_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -101,6 +102,11 @@ __device__ __forceinline__ bool next_full_chunk(const Table<T>& tb, uint32_t& g,
 // TILED (arenas with matrices cut into 64 x 64 tiles): a chunk is 64 rows of 256 bytes `stride`
 // elements apart; theta_global then comes in by 16-byte cp.async copies of all threads instead
 // of one bulk copy, and the stores follow the same geometry.
+//
+// The wait for theta_global is bounded.  If it runs out, the iteration is marked in shared memory, the
+// threads that gave up skip their stores, every thread leaves the loop behind that iteration's closing
+// barrier (a mark of a later iteration, by a thread that has run ahead, is larger and is ignored), the
+// copies still in flight are allowed to land (bounded again), and SL_FLAG_TIMEOUT is raised.
 //
 // GROUPED (k a multiple of NP): a thread owns NP consecutive slots of ONE replica instead of NP
 // pairs 256 apart.  Its positions then arrive as one 2*NP-byte load and its codes as a few bytes,
@@ -145,9 +151,11 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const bool pow2 = (R & (R - 1)) == 0;
   const float Rf = (float)R, invR = 1.0f / Rf;
   const float nlr = -a.outer_lr;
-  bool bad = false, timed_out = false;
+  bool bad = false;
+  const uint32_t wait_limit = a.wait_polls == 0 ? kAggWaitLimit : a.wait_polls == 0xFFFFFFFFu ? 0u : a.wait_polls;
 
   if (APPLY && tid == 0) {
+    sm.abort_it = 0;
     for (int s = 0; s < 2; ++s)
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(agg_smem_u32(&sm.full[s])), "r"(TILED ? kThreads : 1) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -292,16 +300,22 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       }
     }
     const float4* g4 = reinterpret_cast<const float4*>(sm.gbuf[it & 1]);
+    bool have_theta = true;
     if (APPLY) {                                   // bounded wait for this chunk's theta_global
       const uint32_t bar = agg_smem_u32(&sm.full[it & 1]), parity = (it >> 1) & 1u;
       bool ok = false;
-      for (uint32_t spin = 0; spin < kAggWaitLimit && !ok; ++spin) {
+      for (uint32_t spin = 0; spin < wait_limit && !ok; ++spin) {
         uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (a.wait_polls)                          // a caller-set limit counts non-blocking polls ...
+          asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                       : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        else                                       // ... the default ones that suspend the thread for a while
+          asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                       : "=r"(done) : "r"(bar), "r"(parity) : "memory");
         ok = done != 0;
+        if (!ok && sm.abort_it) break;
       }
-      if (!ok) timed_out = true;
+      if (!ok) { sm.abort_it = it + 1; have_theta = false; }
     }
     float* out_cur = a.out + base_cur;
 #pragma unroll
@@ -321,20 +335,39 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
         u.x = __fmaf_rn(nlr, u.x, G.x); u.y = __fmaf_rn(nlr, u.y, G.y);
         u.z = __fmaf_rn(nlr, u.z, G.z); u.w = __fmaf_rn(nlr, u.w, G.w);
       }
-      __stcs(dst, u);
+      if (have_theta) __stcs(dst, u);
     }
     __syncthreads();                               // accumulator and theta buffer read by everyone before they are reused
+    if (APPLY) {
+      const uint32_t ab = sm.abort_it;
+      if (ab != 0 && ab <= it + 1) {               // gave up in this iteration: same decision in every thread
+        // copies in flight: this iteration's (it & 1) and, if there is a next chunk, its own ((it + 1) & 1)
+        if (TILED) {
+          asm volatile("cp.async.wait_all;" ::: "memory");
+        } else if (tid == 0) {
+          for (uint32_t j = it; j <= it + (valid ? 1u : 0u); ++j) {
+            const uint32_t bar = agg_smem_u32(&sm.full[j & 1]), parity = (j >> 1) & 1u;
+            for (uint32_t spin = 0; spin < kAggWaitLimit; ++spin) {
+              uint32_t done;
+              asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                           : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+              if (done) break;
+            }
+          }
+        }
+        if (tid == 0 && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
+        break;
+      }
+    }
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
-  if (timed_out && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 template <int T, bool APPLY>
 cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
-  int dev = 0, sms = 0;
   cudaError_t e;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  const int sms = sm_count(&e);
+  if (e != cudaSuccess) return e;
   const int pairs = (a.R * a.k + kThreads - 1) / kThreads;
   const size_t smem = APPLY ? sizeof(AggSmem) : sizeof(float) * kAC;
   // persistent grid: exactly as many CTAs as are resident at once, so that every CTA walks the
@@ -432,7 +465,10 @@ cudaError_t launch_outer_apply(float* theta, const float* update, uint64_t n, fl
   const int vec = (((uintptr_t)theta | (uintptr_t)update) & 15u) == 0;
   const uint64_t work = vec ? (n + 3) / 4 : n;
   uint64_t blocks = (work + 255) / 256;
-  const uint64_t cap = 148ull * 8ull;  // grid-stride over one full wave: 8 CTAs of 256 threads per SM
+  cudaError_t e;
+  const int sms = sm_count(&e);
+  if (e != cudaSuccess) return e;
+  const uint64_t cap = (uint64_t)sms * 8ull;  // grid-stride over one full wave: 8 CTAs of 256 threads per SM
   if (blocks > cap) blocks = cap;
   outer_apply_kernel<<<(unsigned)blocks, 256, 0, st>>>(theta, update, n, lr, vec);
   return cudaPeekAtLastError();

@@ -1,10 +1,17 @@
 // Host side of the C ABI declared in include/sparseloco.h: argument checks, the by-value
-// arena table, dispatch.  No allocation, no state, no synchronisation.
+// arena table (built on the caller's stack, about 28 KB for the largest arenas), dispatch.  No
+// allocation, no state, no synchronisation.
+#include <atomic>
 #include <cmath>
-#include <memory>
-#include <new>
 
 #include "sl_common.cuh"
+
+namespace sl {
+namespace {
+std::atomic<uint32_t> g_wait_polls{0};
+}
+uint32_t debug_wait_polls() { return g_wait_polls.load(std::memory_order_relaxed); }
+}  // namespace sl
 
 namespace {
 
@@ -99,8 +106,8 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
                   const sl_layout* L, float beta, int chunk, int k, int bits, uint16_t* const* idx,
                   uint8_t* const* codes, float* const* scales, uint32_t* flags, cudaStream_t st,
                   bool step, float outer_lr) {
-  std::unique_ptr<CompressArgs<T>> a(new (std::nothrow) CompressArgs<T>);
-  if (!a) return SL_ERR_CUDA;
+  CompressArgs<T> args;                 // by-value kernel parameters, built on the stack: no allocation
+  CompressArgs<T>* a = &args;
   bool m4;
   fill_table(a->tb, L, chunk, &m4);
   bool al16 = m4 && aligned(theta_global, 16);
@@ -121,10 +128,11 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
   a->bits = bits;
   a->R = R;
   a->stride = (uint32_t)codes_stride(k, bits);
+  a->wait_polls = debug_wait_polls();
   if (!step) return launch_compress<T>(*a, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 
-  std::unique_ptr<AggregateArgs<T>> g(new (std::nothrow) AggregateArgs<T>);
-  if (!g) return SL_ERR_CUDA;
+  AggregateArgs<T> gargs;
+  AggregateArgs<T>* g = &gargs;
   g->tb = a->tb;
   for (int r = 0; r < R; ++r) {
     g->m.idx[r] = idx[r];
@@ -139,6 +147,7 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
   g->bits = bits;
   g->R = R;
   g->stride = a->stride;
+  g->wait_polls = a->wait_polls;
   if (launch_compress<T>(*a, al16, st) != cudaSuccess) return SL_ERR_CUDA;
   return launch_aggregate<T>(*g, true, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 }
@@ -171,8 +180,8 @@ template <int T>
 int aggregate_impl(int R, const uint16_t* const* idx, const uint8_t* const* codes,
                    const float* const* scales, const sl_layout* L, int chunk, int k, int bits, float* out,
                    float outer_lr, bool apply, uint32_t* flags, cudaStream_t st) {
-  std::unique_ptr<AggregateArgs<T>> a(new (std::nothrow) AggregateArgs<T>);
-  if (!a) return SL_ERR_CUDA;
+  AggregateArgs<T> args;
+  AggregateArgs<T>* a = &args;
   bool m4;
   fill_table(a->tb, L, chunk, &m4);
   bool al16 = m4 && aligned(out, 16);
@@ -190,6 +199,7 @@ int aggregate_impl(int R, const uint16_t* const* idx, const uint8_t* const* code
   a->bits = bits;
   a->R = R;
   a->stride = (uint32_t)codes_stride(k, bits);
+  a->wait_polls = debug_wait_polls();
   return launch_aggregate<T>(*a, apply, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 }
 
@@ -216,11 +226,10 @@ int aggregate_checked(int R, const uint16_t* const* idx, const uint8_t* const* c
 
 template <int T>
 int unpack_impl(const uint8_t* packed, const sl_layout* L, int chunk, int k, uint16_t* idx, cudaStream_t st) {
-  std::unique_ptr<Table<T>> tb(new (std::nothrow) Table<T>);
-  if (!tb) return SL_ERR_CUDA;
+  Table<T> tb;
   bool m4;
-  fill_table(*tb, L, chunk, &m4);
-  return launch_unpack_idx12(*tb, packed, chunk, k, idx, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+  fill_table(tb, L, chunk, &m4);
+  return launch_unpack_idx12(tb, packed, chunk, k, idx, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 }
 
 }  // namespace
@@ -242,6 +251,11 @@ uint64_t sl_num_chunks(const sl_layout* L, int chunk) {
 uint64_t sl_codes_stride(int k, int bits) {
   if (k < 1 || !bits_ok(bits)) return 0;
   return codes_stride(k, bits);
+}
+
+uint64_t sl_codes_bytes(const sl_layout* L, int chunk, int k, int bits) {
+  if (k < 1 || k > chunk || !bits_ok(bits)) return 0;
+  return sl_num_chunks(L, chunk) * codes_stride(k, bits);
 }
 
 int sl_compress(const float* theta_local, const float* theta_global, float* err, const sl_layout* L,
@@ -354,6 +368,10 @@ int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, ui
   if (V == 0) return SL_OK;
   return launch_embed_reproject(T_S, T_perp, U, V, d, k, flags, (cudaStream_t)stream) == cudaSuccess
              ? SL_OK : SL_ERR_CUDA;
+}
+
+void sl_debug_set_wait_limit(int32_t polls) {
+  sl::g_wait_polls.store(polls < 0 ? 0xFFFFFFFFu : (uint32_t)polls, std::memory_order_relaxed);
 }
 
 const char* sl_strerror(int code) {

@@ -150,6 +150,8 @@ struct CompressArgs {
   float beta;
   int chunk, k, bits, R;
   uint32_t stride;  // bytes of codes per chunk
+  uint32_t wait_polls;  // polls a bounded wait makes before it gives up (0: the default, about a second;
+                        // 0xFFFFFFFF: none, every wait gives up at once)
 };
 
 template <int T>
@@ -161,6 +163,7 @@ struct AggregateArgs {
   float outer_lr;
   int chunk, k, bits, R;
   uint32_t stride;
+  uint32_t wait_polls;  // as in CompressArgs
 };
 
 // ---------------------------------------------------------------------------
@@ -196,6 +199,17 @@ __device__ __forceinline__ float dequant(uint32_t code, float s, int bits) {
   const uint32_t sign = (code >> (bits - 1)) & 1u;
   const float mag = __fmul_rn(s, (float)(2u * q + 1u) * (0.5f / (float)L));
   return __uint_as_float(__float_as_uint(mag) | (sign << 31));
+}
+
+// polls every bounded on-chip wait makes before it gives up, as set by sl_debug_set_wait_limit (0: default)
+uint32_t debug_wait_polls();
+
+// number of SMs of the current device (grid sizing); 0 with *e set when the query fails
+inline int sm_count(cudaError_t* e) {
+  int dev = 0, sms = 0;
+  if ((*e = cudaGetDevice(&dev)) != cudaSuccess) return 0;
+  if ((*e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return 0;
+  return sms;
 }
 
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }

@@ -255,13 +255,18 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 // selector q waits); 4+q = selector q has finished an item: message final, candidate list free
 // (selector q arrives, producers wait).  bar.arrive / bar.sync order the shared-memory accesses
 // around them (the producer/consumer idiom of the PTX manual), so no membar is used: it would
-// also wait for global stores in flight.  Every mbarrier wait is bounded; running out raises
-// SL_FLAG_TIMEOUT and the kernel carries on (no trap, no hang).
+// also wait for global stores in flight.  Every mbarrier wait is bounded.  A wait that runs out marks
+// its item in shared memory; the producers stop at that item (all at the same one: the mark is read
+// behind their barrier), release both selectors, which stop at their next hand-off, nothing more is
+// copied in, the threads that issued bulk copies wait (bounded again) until the ones in flight have
+// landed, and the kernel returns with SL_FLAG_TIMEOUT raised (no trap, no hang; the outputs of the
+// call are then unspecified).
 // ---------------------------------------------------------------------------
 constexpr int kC = 4096;
 constexpr int kSel = 2;               // selector warps
 constexpr int kTlStages = 2;
 constexpr int kEeStages = 4;
+static_assert(kEeStages == 2 * kSel && kTlStages == 2, "the give-up path counts copies per stage from these");
 constexpr int kCandMax = 512;
 constexpr int kCandReg = 6;           // candidates per lane held in registers: C <= 192 (k <= 64) ...
 constexpr int kCandRegBig = 11;       // ... or C <= 352 (k = 128); longer lists are walked in shared memory
@@ -279,10 +284,11 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// bounded wait on a phase; false = gave up (non-blocking test_wait with a short sleep between polls)
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// bounded wait on a phase; false = gave up, or another thread of the CTA already has (`abort` != 0);
+// non-blocking test_wait with a short sleep between polls
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit, const volatile uint32_t& abort) {
   const uint32_t addr = smem_u32(bar);
-  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -290,9 +296,26 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
     if (ok) return true;
+    if (abort) return false;
     __nanosleep(40);
   }
   return false;
+}
+// after a give-up: lets the last of `uses` bulk copies announced on `bar` land before the CTA's shared
+// memory goes away (always with the default bound, whatever limit the waits had)
+__device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t uses) {
+  if (uses == 0) return;
+  const uint32_t addr = smem_u32(bar), parity = (uses - 1) & 1u;
+  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return;
+    __nanosleep(40);
+  }
 }
 __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -336,6 +359,7 @@ struct alignas(16) FastSmem {
   float* p_scales[kPtrCache];
   uint64_t full_tl[kTlStages];
   uint64_t full_ee[kEeStages];
+  volatile uint32_t abort_item;       // 0, or 1 + the item at which a bounded wait gave up: every role stops there
 };
 static_assert(sizeof(FastSmem) <= 115712, "two CTAs per SM need 2 * (smem + 1 KB) <= 228 KB");
 
@@ -596,6 +620,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     sm.p_scales[tid] = a.p.scales[tid];
   }
   if (tid == 0) {
+    sm.abort_item = 0;
 #pragma unroll
     for (int q = 0; q < kSel; ++q) sm.count[q] = 0;
 #pragma unroll
@@ -606,7 +631,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     fence_async_smem();
   }
   __syncthreads();
-  bool timed_out = false;
+  const uint32_t wait_limit = a.wait_polls == 0 ? kWaitLimit : a.wait_polls == 0xFFFFFFFFu ? 0u : a.wait_polls;
 
   if (warp < kWarps) {
     // ======================= producers =======================================
@@ -632,11 +657,13 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         cp_async_16(reinterpret_cast<float4*>(sm.ee[st_ee]) + f, src_ee + off);
       }
     };
+    uint32_t tl_issued = 0;                       // thread 0: theta_local copies issued so far (the j-th goes to stage j % 2)
     for (int i = 0; i < kTlStages; ++i) {
       if (pf.valid) {
         if (TILED) {
           tile_load(pf, i, i);
         } else if (tid == 0) {
+          ++tl_issued;
           mbar_expect_tx(&sm.full_tl[i], kBytes);
           tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
         }
@@ -681,9 +708,9 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       const int st = w % kTlStages, se = w % kEeStages, q = w % kSel;
       if (TILED) {
         cp_async_wait_but_one();                  // this thread's copies for item w have landed (item w+1's may fly)
-      } else {
-        if (!mbar_wait(&sm.full_tl[st], (w / kTlStages) & 1u)) timed_out = true;
-        if (!mbar_wait(&sm.full_ee[se], (w / kEeStages) & 1u)) timed_out = true;
+      } else if (!mbar_wait(&sm.full_tl[st], (w / kTlStages) & 1u, wait_limit, sm.abort_item) ||
+                 !mbar_wait(&sm.full_ee[se], (w / kEeStages) & 1u, wait_limit, sm.abort_item)) {
+        sm.abort_item = w + 1;                    // phase A below then works on stale data: harmless, nothing of it leaves
       }
       const float4* tl4 = reinterpret_cast<const float4*>(sm.tl[st]);
       float4* ee4 = reinterpret_cast<float4*>(sm.ee[se]);
@@ -755,12 +782,16 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         if (TILED) tile_store(r_m2, base_m2, stride_m2, (w - kSel) % kEeStages);
       }
       named_sync(1, kThreads);
+      // a wait of this item gave up (every such mark was written before the barrier above; a mark of a
+      // later item, by a thread that has run ahead, is larger): all producers leave here
+      if (!TILED) { const uint32_t ab = sm.abort_item; if (ab != 0 && ab <= w + 1) break; }
       if (pf.valid) {
         // every producer has read theta_local(w) (TILED: and written back the stage of e(w-2)):
         // the stages take item w+2's
         if (TILED) {
           tile_load(pf, st, (w + kTlStages) % kEeStages);
         } else if (tid == 0) {
+          ++tl_issued;
           mbar_expect_tx(&sm.full_tl[st], kBytes);
           tma_load_1d(sm.tl[st], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[st]);
         }
@@ -803,6 +834,18 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       g_m1 = cur.g; r_m1 = cur.r; base_m1 = cur.base; stride_m1 = cur.stride;
       cur = nxt;
     }
+    if (!TILED && sm.abort_item != 0) {
+      // gave up at item w: the selectors wait for the candidate lists of items w and w+1, which will not
+      // come; release both (they find the mark and stop), then let this thread's copies in flight land
+      __syncwarp();
+      named_arrive(2 + (int)(w % kSel), kPairThreads);
+      named_arrive(2 + (int)((w + 1) % kSel), kPairThreads);
+      if (tid == 0) {
+        for (int i = 0; i < kTlStages; ++i) mbar_drain(&sm.full_tl[i], (tl_issued + kTlStages - 1 - i) / kTlStages);
+        if (a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
+      }
+      return;
+    }
     // the last kSel items' messages
     const uint32_t W = w;
     for (uint32_t wp = (W > (uint32_t)kSel ? W - kSel : 0); wp < W; ++wp) {
@@ -830,10 +873,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     cur.start(a.tb, blockIdx.x, G);
     cur.advance(a.tb, q, R, G);
     ItemCursor<T> pf = cur;                       // the item whose e is loaded next by this selector: w, w+2 at start, then w+4
+    uint32_t ee_issued = 0;                       // lane 0: e copies issued so far (the j-th goes to stage q + kSel * (j % 2))
     if (TILED) {
       pf.valid = false;                           // the producers move all the data
     } else if (lane == 0) {
       for (int i = q; i < kEeStages && pf.valid; i += kSel) {
+        ++ee_issued;
         mbar_expect_tx(&sm.full_ee[i], kBytes);
         tma_load_1d(sm.ee[i], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes, &sm.full_ee[i]);
         pf.advance(a.tb, kSel, R, G);
@@ -851,12 +896,14 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       const int se = w % kEeStages;
       float* ep = sm.ee[se];
       named_sync(2 + q, kPairThreads);            // candidate list q is ready
+      if (!TILED) { const uint32_t ab = sm.abort_item; if (ab != 0 && ab <= w + 1) break; }   // the producers gave up at or before this item
       // The store of this selector's previous item was issued a whole hand-off ago; once it has
       // read its stage, e of the item four ahead is loaded into it.
       if (!TILED && pending_stage >= 0) {
         if (lane == 0) {
           tma_store_wait_read_all();
           if (pf.valid) {
+            ++ee_issued;
             mbar_expect_tx(&sm.full_ee[pending_stage], kBytes);
             tma_load_1d(sm.ee[pending_stage], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes,
                         &sm.full_ee[pending_stage]);
@@ -933,9 +980,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       named_arrive(4 + q, kPairThreads);          // item w is finished: message final, candidate list free
       cur.advance(a.tb, kSel, R, G);
     }
-    if (!TILED && lane == 0) tma_store_wait_read_all();   // shared memory must outlive the bulk stores' reads
+    if (!TILED && lane == 0) {
+      tma_store_wait_read_all();                  // shared memory must outlive the bulk stores' reads ...
+      if (sm.abort_item != 0)                     // ... and, after a give-up, the copies still coming in
+        for (int i = 0; i < kEeStages / kSel; ++i) mbar_drain(&sm.full_ee[q + kSel * i], (ee_issued + 1 - i) / 2);
+    }
   }
-  if (timed_out && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 }  // namespace
@@ -958,9 +1008,8 @@ cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream
     if (e != cudaSuccess) return e;
   }
   if (compress_is_tuned(a, aligned16)) {
-    int dev = 0, sms = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int sms = sm_count(&e);
+    if (e != cudaSuccess) return e;
     // persistent grid: two CTAs per SM, each walking its share of the chunks
     const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * 2u);
     if (a.tb.side != 0) {

@@ -59,13 +59,14 @@ struct EmbedSmem {
   uint64_t o_full[2], o_empty[2], e_full[kEBufs], e_empty[kEBufs], e_done[kEBufs];
   uint64_t p_done, x_free;   // per sub-tile: pass 1 has read its ring / pass 2 has left the shared region
   uint64_t p_ready;          // per sub-tile: the coordinates in tensor memory have been rounded to TF32
+  uint64_t mma_idle;         // after a give-up only: the MMAs issued so far have retired
   uint32_t tmem_base;
-  volatile uint32_t abort;
+  WaitCtl ctl;
 };
 
 // bounded wait on one of this kernel's barriers (see tc::mbar_wait)
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, EmbedSmem& sm) {
-  return tc::mbar_wait(b, parity, sm.abort);
+  return tc::mbar_wait(b, parity, sm.ctl);
 }
 
 struct Maps {
@@ -79,7 +80,8 @@ __device__ __forceinline__ uint8_t* ring2_slot(EmbedSmem& sm, uint32_t s) {
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d, uint32_t kp, uint32_t* flags) {
+embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d, uint32_t kp, uint32_t* flags,
+                       uint32_t wait_polls) {
   extern __shared__ uint8_t raw[];
   EmbedSmem& sm = *reinterpret_cast<EmbedSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -101,7 +103,9 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     mbar_init(&sm.p_done, 1);
     mbar_init(&sm.p_ready, 4);
     mbar_init(&sm.x_free, 1);
-    sm.abort = 0;
+    mbar_init(&sm.mma_idle, 1);
+    sm.ctl.abort = 0;
+    sm.ctl.polls = wait_polls;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -117,18 +121,6 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
 
   // bounded wait for the last of `uses` uses of a barrier (nothing to wait for when it was never used)
   auto wait_last = [&](uint64_t* bar, uint32_t uses) { return uses == 0 || mbar_wait(bar, (uses - 1) & 1u, sm); };
-  // after an abort: give the copies this thread issued the time to land before the CTA exits
-  auto landed = [&](uint64_t* bar, uint32_t uses) {
-    const long long t0 = clock64();
-    while (uses) {
-      uint32_t done;
-      asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                   : "=r"(done) : "r"(smem_u32(bar)), "r"((uses - 1) & 1u) : "memory");
-      if (done || clock64() - t0 > kWaitClocks) break;
-      __nanosleep(64);
-    }
-  };
-
   // pass 1: the boxes of a U slice are shared by three producer warps (issuing a tensor-map copy costs its
   // thread about 0.05 us, and a K step has up to nine): warp 0 takes [0, u_split1), warp 8 [u_split1, u_split2),
   // warp 9 the rest; each announces its own bytes on the slot's barrier
@@ -150,6 +142,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
             tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
         }
       }
+      if (!ok)
+        for (uint32_t s = 0; s < (uint32_t)kRing1; ++s) landed(&sm.full1[s], ring_uses(it1, s, kRing1));
     }
   } else if (warp == 0) {
     if (lane == 0) {
@@ -298,6 +292,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           mma_commit(&sm.o_full[buf]);
         }
       }
+      if (!ok) mma_quiesce(&sm.mma_idle);
     }
   } else {
     // ---- epilogue: one thread per row; warp w may read tensor-memory lanes 32*(w%4).. only ----
@@ -403,7 +398,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tbase), "r"(512) : "memory");
   }
-  if (tid == 0 && sm.abort && flags) atomicOr(flags, (uint32_t)SL_FLAG_TIMEOUT);
+  if (tid == 0 && sm.ctl.abort && flags) atomicOr(flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 
@@ -452,7 +447,10 @@ embed_reproject_generic_kernel(float* __restrict__ T_S, float* __restrict__ T_pe
 cudaError_t launch_round_tf32(float* x, uint64_t n, cudaStream_t st) {
   if (n == 0) return cudaSuccess;
   const uint64_t blocks = (n + 255) / 256;
-  round_tf32_kernel<<<(unsigned)(blocks < 148u * 16u ? blocks : 148u * 16u), 256, 0, st>>>(x, n);
+  cudaError_t e;
+  const uint64_t cap = (uint64_t)sm_count(&e) * 16u;
+  if (e != cudaSuccess) return e;
+  round_tf32_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, st>>>(x, n);
   return cudaGetLastError();
 }
 
@@ -487,13 +485,12 @@ cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, ui
   const int smem = (int)sizeof(EmbedSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(embed_reproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  int dev = 0, sms = 0;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  const int sms = sm_count(&e);
+  if (e != cudaSuccess) return e;
   const uint32_t kp = (k + 31u) & ~31u;
   const uint64_t tiles = (V + kRows - 1) / kRows;          // never more CTAs than full sub-tiles
   const unsigned grid = (unsigned)(tiles < (uint64_t)sms ? tiles : (uint64_t)sms);
-  embed_reproject_kernel<<<grid, kThreads, smem, st>>>(m, V, d, kp, flags);
+  embed_reproject_kernel<<<grid, kThreads, smem, st>>>(m, V, d, kp, flags, debug_wait_polls());
   return cudaGetLastError();
 }
 

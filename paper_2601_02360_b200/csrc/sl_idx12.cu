@@ -55,9 +55,13 @@ __global__ void unpack_idx12_kernel(const __grid_constant__ Table<T> tb, const u
   }
 }
 
+// grid-stride launch: enough CTAs for the work, at most 32 per SM
 unsigned grid_for(uint64_t n, int block) {
   const uint64_t b = (n + block - 1) / block;
-  return (unsigned)(b < 1 ? 1 : (b > 148u * 32u ? 148u * 32u : b));
+  cudaError_t e;
+  const int sms = sm_count(&e);
+  const uint64_t cap = (uint64_t)(sms > 0 ? sms : 1) * 32u;
+  return (unsigned)(b < 1 ? 1 : (b > cap ? cap : b));
 }
 
 }  // namespace

@@ -48,6 +48,7 @@ struct SubParams {
   uint64_t n_tok, V;
   uint32_t L, d, k, kp;
   uint32_t* flags;
+  uint32_t wait_polls;      // caller-set limit of the bounded waits in polls (0: the default)
 };
 
 // the token a row thread serves in a sub-tile: its embedding row and position row (or none)
@@ -78,8 +79,9 @@ __device__ __forceinline__ RowInfo row_info(const SubParams& p, uint64_t r0, uin
 struct ProjSmem {
   uint8_t ring[kRing * kSlotP];
   uint64_t full[kRing], ready[kRing], empty[kRing], p_done, p_free;
+  uint64_t mma_idle;        // after a give-up only: the MMAs issued so far have retired
   uint32_t tmem_base;
-  volatile uint32_t abort;
+  WaitCtl ctl;
 };
 struct ProjMaps { CUtensorMap x128, x32, u_n; };
 
@@ -95,7 +97,9 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
     for (int s = 0; s < kRing; ++s) { mbar_init(&sm.full[s], 3); mbar_init(&sm.ready[s], kRowWarps); mbar_init(&sm.empty[s], 1); }
     mbar_init(&sm.p_done, 1);
     mbar_init(&sm.p_free, kRowWarps);
-    sm.abort = 0;
+    mbar_init(&sm.mma_idle, 1);
+    sm.ctl.abort = 0;
+    sm.ctl.polls = p.wait_polls;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -123,7 +127,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
         const int r0 = (int)(g * 32);
         for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
           const uint32_t s = it % kRing;
-          ok = mbar_wait(&sm.empty[s], ((it / kRing) & 1u) ^ 1u, sm.abort);
+          ok = mbar_wait(&sm.empty[s], ((it / kRing) & 1u) ^ 1u, sm.ctl);
           if (!ok) break;
           uint8_t* slot = sm.ring + s * kSlotP;
           mbar_expect_tx(&sm.full[s], (pi == 0 ? h * 128 : 0u) + (hi - lo) * 4096);
@@ -137,6 +141,8 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
             tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
         }
       }
+      if (!ok)                                       // gave up: let this thread's copies in flight land first
+        for (uint32_t s = 0; s < (uint32_t)kRing; ++s) landed(&sm.full[s], ring_uses(it, s, kRing));
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -146,13 +152,13 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2), desc_n = smem_desc(0, 4096, 512, 1);
       for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
         if (t > 0) {                                 // the row warps have read the previous accumulator
-          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.abort);
+          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.ctl);
           if (!ok) break;
           tc_fence_after();
         }
         for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
           const uint32_t s = it % kRing;
-          ok = mbar_wait(&sm.ready[s], (it / kRing) & 1u, sm.abort);
+          ok = mbar_wait(&sm.ready[s], (it / kRing) & 1u, sm.ctl);
           if (!ok) break;
           tc_fence_after();
           const uint32_t a0 = smem_u32(sm.ring + s * kSlotP);
@@ -164,6 +170,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
         }
         if (ok) mma_commit(&sm.p_done);
       }
+      if (!ok) mma_quiesce(&sm.mma_idle);
     }
   } else {
     // ---- row warps.  Element-wise part: eight threads per token row, one 16-byte chunk each, so that a
@@ -221,7 +228,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
             for (int i = 0; i < 4; ++i) { ct[i] = et[par][i]; cp[i] = ep[par][i]; }
             fetch(kk + 2, et[par], ep[par]);
             const uint32_t s = it % kRing;
-            ok = ok && mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.abort);
+            ok = ok && mbar_wait(&sm.full[s], (it / kRing) & 1u, sm.ctl);
             ok = __all_sync(0xffffffffu, ok);
             if (ok) {
               const uint32_t a0 = smem_u32(sm.ring + s * kSlotP) + goff;
@@ -251,7 +258,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
       if (g + 4 < g1) open_tile(g + 4);
       // the coordinates of this sub-tile's tokens: out of tensor memory, into Xt (the two warps of a lane
       // window take alternate blocks of 32 columns)
-      ok = mbar_wait(&sm.p_done, t & 1u, sm.abort);
+      ok = mbar_wait(&sm.p_done, t & 1u, sm.ctl);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -286,7 +293,7 @@ subspace_project_kernel(const __grid_constant__ ProjMaps maps, const __grid_cons
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_p), "r"(256) : "memory");
   }
   if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
-  if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+  if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 // ------------------------------------------------------- compress without embedding terms, two sub-tiles
@@ -300,8 +307,9 @@ constexpr int kSlotD = 2 * kSlotA + 256 * kTileK * 4;   // two X tiles + 32 rows
 struct DualSmem {
   uint8_t ring[kRingD * kSlotD];
   uint64_t full[kRingD], ready[kRingD], empty[kRingD], p_done, p_free;
+  uint64_t mma_idle;        // after a give-up only: the MMAs issued so far have retired
   uint32_t tmem_base;
-  volatile uint32_t abort;
+  WaitCtl ctl;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -319,7 +327,9 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
     for (int s = 0; s < kRingD; ++s) { mbar_init(&sm.full[s], 3); mbar_init(&sm.ready[s], kRowWarps); mbar_init(&sm.empty[s], 1); }
     mbar_init(&sm.p_done, 1);
     mbar_init(&sm.p_free, kRowWarps);
-    sm.abort = 0;
+    mbar_init(&sm.mma_idle, 1);
+    sm.ctl.abort = 0;
+    sm.ctl.polls = p.wait_polls;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -345,7 +355,7 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
         const int r0 = (int)(g * 32);
         for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
           const uint32_t s = it % kRingD;
-          ok = mbar_wait(&sm.empty[s], ((it / kRingD) & 1u) ^ 1u, sm.abort);
+          ok = mbar_wait(&sm.empty[s], ((it / kRingD) & 1u) ^ 1u, sm.ctl);
           if (!ok) break;
           uint8_t* slot = sm.ring + s * kSlotD;
           mbar_expect_tx(&sm.full[s], (pi == 0 ? (ha + hb) * 4096 : 0u) + (hi - lo) * 4096);
@@ -363,6 +373,8 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
             tma_load_2d(slot + 2 * kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
         }
       }
+      if (!ok)
+        for (uint32_t s = 0; s < (uint32_t)kRingD; ++s) landed(&sm.full[s], ring_uses(it, s, kRingD));
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -373,13 +385,13 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
       for (uint64_t g = g0; ok && g < g1; g += 8, ++t) {
         const bool two = groups_b(g) != 0;
         if (t > 0) {                                 // the row warps have read the previous accumulators
-          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.abort);
+          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.ctl);
           if (!ok) break;
           tc_fence_after();
         }
         for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
           const uint32_t s = it % kRingD;
-          ok = mbar_wait(&sm.ready[s], (it / kRingD) & 1u, sm.abort);
+          ok = mbar_wait(&sm.ready[s], (it / kRingD) & 1u, sm.ctl);
           if (!ok) break;
           tc_fence_after();
           const uint32_t a0 = smem_u32(sm.ring + s * kSlotD);
@@ -396,6 +408,7 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
         }
         if (ok) mma_commit(&sm.p_done);
       }
+      if (!ok) mma_quiesce(&sm.mma_idle);
     }
   } else {
     // ---- row warps: round the landed tiles to the nearest TF32 value in place (the tensor cores would cut),
@@ -412,7 +425,7 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
       const uint32_t chunks = hb ? 8u : 4u;          // 16-byte chunks per thread: rows grow + 32 i of A, then of B
       for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
         const uint32_t s = it % kRingD;
-        ok = mbar_wait(&sm.full[s], (it / kRingD) & 1u, sm.abort);
+        ok = mbar_wait(&sm.full[s], (it / kRingD) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         const uint32_t a0 = smem_u32(sm.ring + s * kSlotD) + goff;
@@ -433,7 +446,7 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
         if (lane == 0) mbar_arrive(&sm.ready[s]);
       }
       if (!ok) break;
-      ok = mbar_wait(&sm.p_done, t & 1u, sm.abort);
+      ok = mbar_wait(&sm.p_done, t & 1u, sm.ctl);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -471,7 +484,7 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_p), "r"(512) : "memory");
   }
-  if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+  if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 // --------------------------------------------------------------------------------------- reconstruct
@@ -494,8 +507,9 @@ struct ReconSmem {
   uint64_t full[kRingB], empty[kRingB], o_full[2], o_empty[2];
   uint64_t a_full[kStageA], a_empty[kStageA], a_ready, a_free;
   uint64_t g_full[kStages], g_done[kStages], g_empty[kStages];
+  uint64_t mma_idle;        // after a give-up only: the MMAs issued so far have retired
   uint32_t tmem_base;
-  volatile uint32_t abort;
+  WaitCtl ctl;
 };
 struct ReconMaps { CUtensorMap xt128, xt32, u_k, o128, o32; };
 
@@ -521,7 +535,9 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     mbar_init(&sm.a_ready, 4);
     mbar_init(&sm.a_free, 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(&sm.g_full[s], 128); mbar_init(&sm.g_done[s], 4); mbar_init(&sm.g_empty[s], 1); }
-    sm.abort = 0;
+    mbar_init(&sm.mma_idle, 1);
+    sm.ctl.abort = 0;
+    sm.ctl.polls = p.wait_polls;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -550,7 +566,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         const int r0 = (int)(g * 32);
         for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++ia) {
           const uint32_t s = ia % kStageA;
-          ok = mbar_wait(&sm.a_empty[s], ((ia / kStageA) & 1u) ^ 1u, sm.abort);
+          ok = mbar_wait(&sm.a_empty[s], ((ia / kStageA) & 1u) ^ 1u, sm.ctl);
           if (!ok) break;
           mbar_expect_tx(&sm.a_full[s], h * 128);
           if (hg == 4) tma_load_2d(sm.a[s], &maps.xt128, (int)(kt * kTileK), r0, &sm.a_full[s]);
@@ -561,11 +577,15 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         for (uint32_t ci = 0; ok && ci < n_blocks; ++ci)
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
             const uint32_t s = it % kRingB;
-            ok = mbar_wait(&sm.empty[s], ((it / kRingB) & 1u) ^ 1u, sm.abort);
+            ok = mbar_wait(&sm.empty[s], ((it / kRingB) & 1u) ^ 1u, sm.ctl);
             if (!ok) break;
             mbar_expect_tx(&sm.full[s], kSlotB);
             tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(block_of(ci) * kBlockN), &sm.full[s]);
           }
+      }
+      if (!ok) {
+        for (uint32_t s = 0; s < (uint32_t)kRingB; ++s) landed(&sm.full[s], ring_uses(it, s, kRingB));
+        for (uint32_t s = 0; s < (uint32_t)kStageA; ++s) landed(&sm.a_full[s], ring_uses(ia, s, kStageA));
       }
     }
   } else if (warp == 1) {
@@ -575,19 +595,19 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       const uint32_t idesc = instr_desc(kRows, kBlockN, 0);
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2);
       for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-        ok = mbar_wait(&sm.a_ready, t & 1u, sm.abort);          // the tile is in tensor memory, rounded
+        ok = mbar_wait(&sm.a_ready, t & 1u, sm.ctl);          // the tile is in tensor memory, rounded
         if (!ok) break;
         tc_fence_after();
         for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
           const uint32_t buf = cg & 1u, u = cg >> 1;
           if (u) {
-            ok = mbar_wait(&sm.o_empty[buf], (u - 1) & 1u, sm.abort);
+            ok = mbar_wait(&sm.o_empty[buf], (u - 1) & 1u, sm.ctl);
             if (!ok) break;
             tc_fence_after();
           }
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
             const uint32_t s = it % kRingB;
-            ok = mbar_wait(&sm.full[s], (it / kRingB) & 1u, sm.abort);
+            ok = mbar_wait(&sm.full[s], (it / kRingB) & 1u, sm.ctl);
             if (!ok) break;
             tc_fence_after();
             const uint64_t db = desc_k | (uint64_t)((smem_u32(sm.ring[s]) >> 4) & 0x3FFF);
@@ -601,6 +621,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         }
         if (ok) mma_commit(&sm.a_free);
       }
+      if (!ok) mma_quiesce(&sm.mma_idle);
     }
   } else if (warp == 2) {
     // ---- part store: a finished part leaves by tensor-map store; its stage is free once the store has read it ----
@@ -614,7 +635,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
           const uint32_t c = block_of(ci), np = parts_of(c);
           for (uint32_t part = 0; part < np; ++part, ++is) {
             const uint32_t s = is % kStages;
-            ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.abort);
+            ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.ctl);
             if (!ok) break;
             const int col0 = (int)(c * kBlockN + part * 32);
             const uint32_t src = smem_u32(sm.st_t[s]);
@@ -651,14 +672,14 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         mask |= ri.gather ? 1u << i : 0u;
       }
       if (t > 0) {                                   // the MMAs of the previous sub-tile have read the old tile
-        ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.abort);
+        ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
       }
       for (uint32_t kt = 0; kt < k_tiles; ++kt, ++ia) {
         const uint32_t s = ia % kStageA;
-        ok = mbar_wait(&sm.a_full[s], (ia / kStageA) & 1u, sm.abort);
+        ok = mbar_wait(&sm.a_full[s], (ia / kStageA) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         uint32_t v[32];
@@ -684,7 +705,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         const uint32_t c = block_of(ci), np = parts_of(c);
         for (uint32_t part = 0; part < np; ++part, ++ig) {
           const uint32_t s = ig % kStages;
-          ok = mbar_wait(&sm.g_empty[s], ((ig / kStages) & 1u) ^ 1u, sm.abort);
+          ok = mbar_wait(&sm.g_empty[s], ((ig / kStages) & 1u) ^ 1u, sm.ctl);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           if (p.ids) {
@@ -716,7 +737,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     for (uint64_t g = g0; ok && g < g1; g += 4) {
       for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
         const uint32_t buf = cg & 1u;
-        ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.abort);
+        ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -725,7 +746,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
           const uint32_t s = ie % kStages;
           uint32_t v[32];
           tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
-          ok = mbar_wait(&sm.g_full[s], (ie / kStages) & 1u, sm.abort);
+          ok = mbar_wait(&sm.g_full[s], (ie / kStages) & 1u, sm.ctl);
           ok = __all_sync(0xffffffffu, ok);
           tmem_ld_wait();
           if (!ok) break;
@@ -762,7 +783,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sm.tmem_base), "r"(512) : "memory");
   }
   if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
-  if (tid == 0 && sm.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+  if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
 // --------------------------------------------------------------------- plain float32 kernels (any shape)
@@ -816,9 +837,8 @@ __global__ void __launch_bounds__(256) subspace_reconstruct_generic_kernel(const
 bool al16(const void* q) { return ((uintptr_t)q & 15u) == 0; }
 
 unsigned persistent_grid(uint64_t n_tok, cudaError_t* e) {
-  int dev = 0, sms = 0;
-  if ((*e = cudaGetDevice(&dev)) != cudaSuccess) return 0;
-  if ((*e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return 0;
+  const int sms = sm_count(e);
+  if (*e != cudaSuccess) return 0;
   const uint64_t tiles = (n_tok + kRows - 1) / kRows;
   return (unsigned)(tiles < (uint64_t)sms ? tiles : (uint64_t)sms);
 }
@@ -828,12 +848,15 @@ unsigned persistent_grid(uint64_t n_tok, cudaError_t* e) {
 cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const float* T_perp, const float* pos,
                                     const float* U, uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k,
                                     float* Xt, uint32_t* flags, cudaStream_t st) {
-  SubParams p{T_perp, pos, ids, Xt, n_tok, V, L, d, k, (k + 31u) & ~31u, flags};
+  SubParams p{T_perp, pos, ids, Xt, n_tok, V, L, d, k, (k + 31u) & ~31u, flags, debug_wait_polls()};
   const bool tuned = d % 4 == 0 && k % 4 == 0 && k >= 4 && k <= 256 && al16(X) && al16(U) && al16(Xt) &&
                      (!ids || (al16(T_perp) && al16(pos)));
   if (!tuned) {
     const uint64_t blocks = (n_tok * (uint64_t)k + 255) / 256;
-    subspace_project_generic_kernel<<<(unsigned)(blocks < 148u * 32u ? blocks : 148u * 32u), 256, 0, st>>>(X, U, p);
+    cudaError_t e;
+    const uint64_t cap = (uint64_t)sm_count(&e) * 32u;
+    if (e != cudaSuccess) return e;
+    subspace_project_generic_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, st>>>(X, U, p);
     return cudaGetLastError();
   }
   ProjMaps m;
@@ -863,12 +886,15 @@ cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const fl
 cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, const float* T_perp, const float* pos,
                                         const float* U, uint64_t n_tok, uint32_t L, uint64_t V, uint32_t d, uint32_t k,
                                         float* Xhat, uint32_t* flags, cudaStream_t st) {
-  SubParams p{T_perp, pos, ids, Xhat, n_tok, V, L, d, k, (k + 31u) & ~31u, flags};
+  SubParams p{T_perp, pos, ids, Xhat, n_tok, V, L, d, k, (k + 31u) & ~31u, flags, debug_wait_polls()};
   const bool tuned = d % 4 == 0 && k % 4 == 0 && k >= 4 && k <= 256 && al16(Xt) && al16(U) && al16(Xhat) &&
                      (!ids || (al16(T_perp) && al16(pos)));
   if (!tuned) {
     const uint64_t blocks = (n_tok * (uint64_t)d + 255) / 256;
-    subspace_reconstruct_generic_kernel<<<(unsigned)(blocks < 148u * 32u ? blocks : 148u * 32u), 256, 0, st>>>(Xt, U, p);
+    cudaError_t e;
+    const uint64_t cap = (uint64_t)sm_count(&e) * 32u;
+    if (e != cudaSuccess) return e;
+    subspace_reconstruct_generic_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, st>>>(Xt, U, p);
     return cudaGetLastError();
   }
   ReconMaps m;

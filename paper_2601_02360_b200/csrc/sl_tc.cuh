@@ -106,9 +106,32 @@ __device__ __forceinline__ void stg256(float* p, const uint32_t* v) {
 // number of uses so far of slot s of an n-slot ring after `it` round-robin uses in total
 __device__ __forceinline__ uint32_t ring_uses(uint32_t it, uint32_t s, uint32_t n) { return (it + n - 1 - s) / n; }
 
-// bounded wait: false when the phase did not complete within kWaitClocks or another role gave up
-// (`abort` is the CTA's shared abort mark; it is set when a wait gives up)
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile uint32_t& abort) {
+// what the bounded waits of a CTA share: the abort mark (set when a wait gives up; every other wait
+// then gives up at once) and the caller-set limit in polls (0: the default bound of kWaitClocks;
+// 0xFFFFFFFF: no poll at all, every wait gives up at once)
+struct WaitCtl {
+  volatile uint32_t abort;
+  uint32_t polls;
+};
+
+__device__ __forceinline__ bool mbar_test(uint64_t* b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+// bounded wait: false when the phase did not complete within the bound or another role gave up
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, WaitCtl& c) {
+  if (c.polls) {                       // caller-set limit: that many non-blocking polls (0xFFFFFFFF: none at all)
+    const uint32_t n = c.polls == 0xFFFFFFFFu ? 0u : c.polls;
+    for (uint32_t i = 0; i < n; ++i) {
+      if (mbar_test(b, parity)) return true;
+      if (c.abort) break;
+    }
+    c.abort = 1;
+    return false;
+  }
   const long long t0 = clock64();
   for (;;) {
     uint32_t ok;
@@ -116,8 +139,23 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
                  : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
     if (ok) return true;
-    if (abort || clock64() - t0 > kWaitClocks) { abort = 1; return false; }
+    if (c.abort || clock64() - t0 > kWaitClocks) { c.abort = 1; return false; }
   }
+}
+
+// after an abort: gives the last of `uses` copies announced on `bar` by this thread the time to land
+// before the CTA exits (bounded by kWaitClocks whatever the caller-set limit; nothing when uses == 0)
+__device__ __forceinline__ void landed(uint64_t* bar, uint32_t uses) {
+  if (uses == 0) return;
+  const long long t0 = clock64();
+  while (!mbar_test(bar, (uses - 1) & 1u) && clock64() - t0 <= kWaitClocks) __nanosleep(64);
+}
+
+// after an abort, by the thread that issued the MMAs: waits (bounded) until every one of them has
+// retired, so that tensor memory can be given back; `bar` is a barrier of count 1 used for nothing else
+__device__ __forceinline__ void mma_quiesce(uint64_t* bar) {
+  mma_commit(bar);
+  landed(bar, 1);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -46,6 +46,10 @@ def test_sizes(lib):
     assert api.sl_codes_stride(63, 4) == 32
     assert api.sl_codes_stride(32, 32) == 128
     assert api.sl_codes_stride(64, 3) == 0
+    lay = api.Layout([0, 4096 * 2 + 5, 4096 * 2 + 105])
+    assert api.sl_codes_bytes(lay, 4096, 64, 2) == 4 * 16
+    assert api.sl_codes_bytes(lay, 4096, 32, 32) == 4 * 128
+    assert api.sl_codes_bytes(lay, 4096, 64, 3) == 0 and api.sl_codes_bytes(lay, 32, 64, 2) == 0
     assert api.strerror(api.SL_OK) == "ok" and "align" in api.strerror(api.SL_ERR_ALIGNMENT)
 
 
