@@ -60,6 +60,11 @@ def aggregate_apply_bytes(wl: synth.Workload) -> int:
     return wl.n_total * 8 + wl.R * message_bytes(wl)
 
 
+def step_bytes_api(wl: synth.Workload) -> int:
+    """Per-call count: N(16R + 8), every replica's compress reading theta_global itself, plus the messages."""
+    return wl.n_total * (16 * wl.R + 8) + 2 * wl.R * message_bytes(wl)
+
+
 def step_bytes_strict(wl: synth.Workload) -> int:
     """Least traffic of a whole step: N(12R + 8) + messages written once and read once."""
     return wl.n_total * (12 * wl.R + 8) + 2 * wl.R * message_bytes(wl)
@@ -664,6 +669,149 @@ def run_embed(args) -> None:
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------- the other rows, outside the headline
+def _median_row(ms_list, alg_bytes, peak, clocks, extra=None):
+    ms = float(np.median(ms_list))
+    row = {"ms": ms, "launches": len(ms_list), "algorithmic_bytes": int(alg_bytes),
+           "achieved_gbs": alg_bytes / (ms * 1e-3) / 1e9, "frac": alg_bytes / (ms * 1e-3) / 1e9 / peak, "clocks": clocks}
+    if extra:
+        row.update(extra)
+    return row
+
+
+def row_outer_step(wl: synth.Workload, seed: int, dev, peak: float, steps: int, tiles: bool = False) -> dict:
+    """One whole outer step (both launches) of another configuration: median of `steps` steps, theta_local
+    re-drawn between steps (untimed); frac = strict step bytes / time / peak, like step_hbm.frac_of_peak."""
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info(dev)
+    need = (2 * wl.R + 1) * wl.n_total * 4 + (3 << 30)
+    if free < need:
+        return {"skipped": f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free"}
+    st = DeviceState(wl, seed, dev, tiles=tiles)
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(dev.index or 0)
+    t_step, t_comp = [], []
+    for s in range(3 + steps):
+        st.redraw_locals(s)
+        if s == 3:
+            torch.cuda.synchronize()
+            sampler.start()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record(stream)
+        st.compress()
+        ev[1].record(stream)
+        st.aggregate_apply()
+        ev[2].record(stream)
+        torch.cuda.synchronize()
+        if s >= 3:
+            t_step.append(ev[0].elapsed_time(ev[2]))
+            t_comp.append(ev[0].elapsed_time(ev[1]))
+    clocks = sampler.stop()
+    flags = int(st.flags.item())
+    comp = float(np.median(t_comp))
+    row = _median_row(t_step, step_bytes_strict(wl), peak, clocks,
+                      {"R": wl.R, "k": wl.k, "bits": wl.bits, "geometry": "64x64 tiles" if tiles else "consecutive chunks",
+                       "params_per_s": wl.n_total / (float(np.median(t_step)) * 1e-3),
+                       "compress_ms": comp, "compress_frac": compress_bytes(wl) / (comp * 1e-3) / 1e9 / peak,
+                       "device_flags": flags})
+    del st
+    torch.cuda.empty_cache()
+    return row
+
+
+def row_embed(wl: synth.Workload, seed: int, dev, peak: float, launches: int, k: int) -> dict:
+    """sl_embed_reproject on the workload's embedding table (Eqs. 3-4); the launch is queued behind the copy
+    that restores T_S, so the host's launch work is outside the timed interval."""
+    from paper_2601_02360_b200 import api
+    name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
+    U = torch.from_numpy(synth.gen_subspace_basis(d, k, seed)).to(dev)
+    api.sl_round_tf32(U, U.numel())
+    T_S_h, T_perp_h = synth.gen_embedding_pair(V, d, seed)
+    T_S0 = torch.from_numpy(T_S_h).to(dev)
+    T_S, T_perp = T_S0.clone(), torch.from_numpy(T_perp_h).to(dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(dev.index or 0)
+    times = []
+    for s in range(5 + launches):
+        torch.cuda.synchronize()
+        if s == 5:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        T_S.copy_(T_S0)
+        e0.record(stream)
+        api.sl_embed_reproject(T_S, T_perp, U, V, d, k, flags)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if s >= 5:
+            times.append(e0.elapsed_time(e1))
+    return _median_row(times, 16 * V * d + 4 * d * k, peak, sampler.stop(),
+                       {"shape": f"{V}x{d}, k={k}", "device_flags": int(flags.item())})
+
+
+def row_subspace(wl: synth.Workload, seed: int, dev, peak: float, launches: int, n_tok: int, k: int) -> dict:
+    """sl_subspace_project / sl_subspace_reconstruct at a stage boundary (section 2.3), with the embedding
+    terms and in the gradient form (ids = NULL); a 256 MB buffer is written between launches (L2 flush)."""
+    from paper_2601_02360_b200 import api
+    name, V, d = next(t for t in wl.tensors if t[0].startswith("embed"))
+    L = 2048
+    Xh, idsh, Tph, posh = synth.gen_stage_boundary(n_tok, L, V, d, seed)
+    X, ids, T_perp, pos = (torch.from_numpy(a).to(dev) for a in (Xh, idsh, Tph, posh))
+    U = torch.from_numpy(synth.gen_subspace_basis(d, k, seed)).to(dev)
+    api.sl_round_tf32(U, U.numel())
+    Xt = torch.empty(n_tok, k, dtype=torch.float32, device=dev)
+    Xhat = torch.empty(n_tok, d, dtype=torch.float32, device=dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(64 << 20, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    out = {}
+    for form, args in (("with_embedding_terms", (ids, T_perp, pos, V)), ("gradient_form", (None, None, None, 0))):
+        sampler = ClockSampler(dev.index or 0)
+        t_p, t_r = [], []
+        for s in range(5 + launches):
+            torch.cuda.synchronize()
+            if s == 5:
+                sampler.start()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            flush.fill_(float(s))
+            e[0].record(stream)
+            api.sl_subspace_project(X, args[0], args[1], args[2], U, n_tok, L, args[3], d, k, Xt, flags)
+            e[1].record(stream)
+            flush.fill_(float(s) + 0.5)
+            e[2].record(stream)
+            api.sl_subspace_reconstruct(Xt, args[0], args[1], args[2], U, n_tok, L, args[3], d, k, Xhat, flags)
+            e[3].record(stream)
+            torch.cuda.synchronize()
+            if s >= 5:
+                t_p.append(e[0].elapsed_time(e[1]))
+                t_r.append(e[2].elapsed_time(e[3]))
+        clocks = sampler.stop()
+        gather = n_tok * d * 4 + L * d * 4 if args[0] is not None else 0      # one T_perp row per token, the position table once
+        bytes_p = n_tok * d * 4 + gather + n_tok * k * 4 + d * k * 4
+        bytes_r = n_tok * k * 4 + gather + n_tok * d * 4 + d * k * 4
+        out[form] = {"project": _median_row(t_p, bytes_p, peak, clocks), "reconstruct": _median_row(t_r, bytes_r, peak, clocks)}
+    out["shape"] = f"{n_tok} tokens x d={d}, k={k}, L={L}, vocab {V}"
+    out["device_flags"] = int(flags.item())
+    return out
+
+
+def measured_rows(args, wl: synth.Workload, dev, peak: float) -> dict:
+    """Everything else this library times, appended to the default line (outside its timed region)."""
+    n = args.row_launches
+    rows = {"note": "medians of CUDA-event times; frac = algorithmic bytes / time / peak"}
+    rows["tiles"] = row_outer_step(wl, args.seed, dev, peak, n, tiles=True)
+    rows["r2"] = row_outer_step(wl.replace(R=2), args.seed, dev, peak, n)
+    rows["r16_k128"] = row_outer_step(wl.replace(R=16, k=128), args.seed, dev, peak, n)
+    has_embed = any(t[0].startswith("embed") for t in wl.tensors)
+    if has_embed:
+        d = next(t for t in wl.tensors if t[0].startswith("embed"))[2]
+        rows["embed"] = row_embed(wl, args.seed, dev, peak, n, d // 8)
+        rows["embed_k128"] = row_embed(wl, args.seed, dev, peak, n, 128)
+        rows["subspace"] = row_subspace(wl, args.seed, dev, peak, n, 65536, d // 8)
+        rows["subspace_k128"] = row_subspace(wl, args.seed, dev, peak, n, 65536, 128)
+    return rows
+
+
 def run_ours(args) -> None:
     from paper_2601_02360_b200 import api
     rank, local, world = init_dist("nccl")
@@ -744,10 +892,17 @@ def run_ours(args) -> None:
                    "step": "sl_compress_batch + sl_aggregate_apply; theta_local re-drawn between steps (untimed)"},
         "roofline": {"kernel": "compress_c4096_kernel (sl_compress_batch)", "bound": "hbm",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "peak_source": peak_src, "algorithmic_bytes": compress_bytes(wl),
+                     "traffic": traffic,
+                     "traffic_source": ("ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the "
+                                        "51.4 M-parameter x 8-replica case (profiles/compress_c4096_1b_layer0.md), "
+                                        "scaled by N*R; a constant, not re-captured by this run") if traffic else None,
+                     "peak_source": peak_src, "algorithmic_bytes": compress_bytes(wl),
                      "launch_ms": comp_ms},
         "step_hbm": {"bytes_strict": step_bytes_strict(wl), "gbs_strict": strict, "frac_of_peak": strict / peak,
-                     "frac_of_8tbs_nominal": strict / 8000.0},
+                     "frac_of_8tbs_nominal": strict / 8000.0,
+                     # per-call count: every replica's compress re-reads theta_global, as on R separate machines
+                     "bytes_api": step_bytes_api(wl), "gbs_api": step_bytes_api(wl) / (step_ms * 1e-3) / 1e9,
+                     "frac_api": step_bytes_api(wl) / (step_ms * 1e-3) / 1e9 / peak},
         "kernels_ms": {"sl_compress_batch": comp_ms, "sl_aggregate_apply": agg_ms,
                        "aggregate_apply_gbs": aggregate_apply_bytes(wl) / (agg_ms * 1e-3) / 1e9},
         "clocks": clocks, "device_flags": flags,
@@ -766,6 +921,23 @@ def run_ours(args) -> None:
             "ms": cpu_ms,
             "sample": f"first {len(sample.tensors)} tensors of the workload ({n_s} params) x R={wl.R}, "
                       f"one outer step, replicas spread over {threads} host threads"}
+        # the same checker on ONE host thread, on a smaller sample (the first two tensors)
+        if len(wl.tensors) > 2:
+            s1 = synth.sub_arena(wl, [0, 1], wl.name + "_first2")
+            n1 = s1.n_total
+            from oracle import slo
+            tg1 = st.theta_global[:n1].cpu().numpy()
+            tl1 = [t[:n1].cpu().numpy() for t in st.theta_local]
+            e1 = [np.zeros(n1, np.float32) for _ in range(wl.R)]
+            t0 = time.perf_counter()
+            oracle_round(slo, tl1, tg1, e1, s1.offsets(), s1, 1)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline_1core"] = {"value": n1 / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "ms": dt * 1e3,
+                                          "sample": f"first 2 tensors ({n1} params) x R={wl.R}, one outer step, one host thread"}
+    plain_default = not (args.tiles or args.R or args.k or args.bits or args.first_tensors or args.variant != "plain")
+    if world == 1 and not args.no_rows and wl.name == "1b" and plain_default:
+        del st
+        line["rows"] = measured_rows(args, wl, dev, peak)
     print(json.dumps(line))
 
 
@@ -808,6 +980,9 @@ def main() -> None:
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-rows", action="store_true",
+                    help="leave out the `rows` object (tiles, R = 2, R = 16 / k = 128, embedding, activation subspace)")
+    ap.add_argument("--row-launches", type=int, default=50, help="timed launches per entry of `rows`")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
