@@ -733,10 +733,9 @@ def row_embed(wl: synth.Workload, seed: int, dev, peak: float, launches: int, k:
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(dev.index or 0)
     times = []
+    sampler.start()
     for s in range(5 + launches):
         torch.cuda.synchronize()
-        if s == 5:
-            sampler.start()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         T_S.copy_(T_S0)
         e0.record(stream)
@@ -768,10 +767,9 @@ def row_subspace(wl: synth.Workload, seed: int, dev, peak: float, launches: int,
     for form, args in (("with_embedding_terms", (ids, T_perp, pos, V)), ("gradient_form", (None, None, None, 0))):
         sampler = ClockSampler(dev.index or 0)
         t_p, t_r = [], []
+        sampler.start()
         for s in range(5 + launches):
             torch.cuda.synchronize()
-            if s == 5:
-                sampler.start()
             e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
             flush.fill_(float(s))
             e[0].record(stream)
@@ -805,10 +803,11 @@ def measured_rows(args, wl: synth.Workload, dev, peak: float) -> dict:
     has_embed = any(t[0].startswith("embed") for t in wl.tensors)
     if has_embed:
         d = next(t for t in wl.tensors if t[0].startswith("embed"))[2]
-        rows["embed"] = row_embed(wl, args.seed, dev, peak, n, d // 8)
-        rows["embed_k128"] = row_embed(wl, args.seed, dev, peak, n, 128)
-        rows["subspace"] = row_subspace(wl, args.seed, dev, peak, n, 65536, d // 8)
-        rows["subspace_k128"] = row_subspace(wl, args.seed, dev, peak, n, 65536, 128)
+        m = 4 * n                 # these launches take a quarter of a millisecond: more of them, so that the clock sampler sees some
+        rows["embed"] = row_embed(wl, args.seed, dev, peak, m, d // 8)
+        rows["embed_k128"] = row_embed(wl, args.seed, dev, peak, m, 128)
+        rows["subspace"] = row_subspace(wl, args.seed, dev, peak, m, 65536, d // 8)
+        rows["subspace_k128"] = row_subspace(wl, args.seed, dev, peak, m, 65536, 128)
     return rows
 
 

@@ -73,7 +73,9 @@ enum {
 enum {
   SL_FLAG_NONFINITE = 1u, /* some chunk's largest magnitude was Inf or NaN */
   SL_FLAG_BAD_INDEX = 2u, /* sl_aggregate*: a message slot named a position past its chunk; skipped */
-  SL_FLAG_TIMEOUT = 4u    /* a bounded wait on an on-chip copy ran out; the outputs are not to be trusted */
+  SL_FLAG_TIMEOUT = 4u,   /* a bounded wait on an on-chip copy ran out; the outputs are not to be trusted */
+  SL_FLAG_BOUNDS = 8u     /* debug build only (libsparseloco_debug.so, -DSL_DEBUG_BOUNDS): a kernel of Eq. 2 formed an
+                             index outside the buffer it was about to touch; the access was skipped */
 };
 
 #define SL_MAX_CHUNK 8192     /* elements; any chunk size in [1, SL_MAX_CHUNK] is accepted */
@@ -228,6 +230,13 @@ int sl_round_tf32(float* x, uint64_t n, void* stream);
  * there already; negative = give up without looking), which lets a test drive that path; 0
  * restores the default. */
 void sl_debug_set_wait_limit(int32_t polls);
+
+/* Debugging aid (the paper has no counterpart).  The debug build of the library range-checks every
+ * shared- and global-memory index of the Eq. 2 kernels (see SL_FLAG_BOUNDS).  This call launches one
+ * tiny kernel that puts an out-of-range index through that check: `*flags` (DEVICE) must come back with
+ * SL_FLAG_BOUNDS raised and `*probe` (DEVICE, one word) untouched, which shows that the checks are
+ * compiled in and skip the access.  The normal build returns SL_ERR_UNSUPPORTED and launches nothing. */
+int sl_debug_bounds_selftest(uint32_t* flags, uint32_t* probe, void* stream);
 
 /* Static description of an SL_* return code. */
 const char* sl_strerror(int code);

@@ -18,12 +18,12 @@ import torch
 from . import build as _build
 
 SL_OK, SL_ERR_INVALID_ARG, SL_ERR_ALIGNMENT, SL_ERR_UNSUPPORTED, SL_ERR_CUDA = 0, -1, -2, -3, -4
-SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT = 1, 2, 4
+SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT, SL_FLAG_BOUNDS = 1, 2, 4, 8
 SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1280, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_codes_bytes", "sl_compress", "sl_compress_batch", "sl_aggregate",
            "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_round_tf32", "sl_subspace_project", "sl_subspace_reconstruct", "sl_idx12_stride",
-           "sl_pack_idx12", "sl_unpack_idx12", "sl_debug_set_wait_limit", "sl_strerror")
+           "sl_pack_idx12", "sl_unpack_idx12", "sl_debug_set_wait_limit", "sl_debug_bounds_selftest", "sl_strerror")
 
 
 class SlLayout(ctypes.Structure):
@@ -87,6 +87,8 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_unpack_idx12.argtypes = [vp, lp, i32, i32, vp, vp]
     L.sl_debug_set_wait_limit.restype = None
     L.sl_debug_set_wait_limit.argtypes = [ctypes.c_int32]
+    L.sl_debug_bounds_selftest.restype = i32
+    L.sl_debug_bounds_selftest.argtypes = [vp, vp, vp]
     L.sl_strerror.restype = ctypes.c_char_p
     L.sl_strerror.argtypes = [i32]
     if path is None:
@@ -254,6 +256,11 @@ def sl_unpack_idx12(packed, layout, chunk: int, k: int, idx, stream=None) -> Non
 
 def sl_debug_set_wait_limit(polls: int) -> None:
     load().sl_debug_set_wait_limit(polls)
+
+
+def sl_debug_bounds_selftest(flags, probe, stream=None) -> int:
+    """Returns the status code (SL_ERR_UNSUPPORTED in the normal build) instead of raising."""
+    return int(load().sl_debug_bounds_selftest(_ptr(flags), _ptr(probe), _stream(stream)))
 
 
 def alloc_messages(layout, chunk: int, k: int, bits: int, R: int, device="cuda"):

@@ -23,8 +23,12 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const int tid = threadIdx.x;
   uint32_t g = blockIdx.x;
   if (TAILS) g = tail_chunk(a.tb, g, a.chunk);    // the g-th chunk that is not full
+  if (!SL_CHECK(a.flags, g < a.tb.n_chunks)) return;
   const ChunkRef c = locate(a.tb, g, a.chunk);
   const int len = c.len, k = a.k, bits = a.bits;
+  const uint64_t n_total = a.tb.offset[a.tb.n_tensors];
+  (void)n_total;
+  if (!SL_CHECK(a.flags, len >= 1 && len <= a.chunk)) return;
 
   for (int i = tid; i < len; i += kThreads) acc[i] = 0.0f;   // one accumulator per element of the chunk
   __syncthreads();
@@ -38,6 +42,7 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
       if (p == 0xFFFFu) continue;                 // padding slot
       const int i = c.elem(p);                    // position -> element number (they differ in edge tiles)
       if (i < 0) { bad = true; continue; }
+      if (!SL_CHECK(a.flags, i < len)) continue;
       float v;
       if (bits == 32) {
         v = reinterpret_cast<const float*>(codes)[j];
@@ -55,7 +60,7 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
   for (int i = tid; i < len; i += kThreads) {
     const float u = __fdiv_rn(acc[i], Rf);
     const uint64_t at = c.addr(i);
-    out[at] = APPLY ? __fmaf_rn(-a.outer_lr, u, out[at]) : u;
+    if (SL_CHECK(a.flags, at < n_total)) out[at] = APPLY ? __fmaf_rn(-a.outer_lr, u, out[at]) : u;
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
@@ -122,6 +127,8 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const int k = a.k, bits = a.bits, R = a.R;
   const int total = R * k;
   constexpr uint32_t kBytes = kAC * 4;
+  const uint64_t n_total = a.tb.offset[a.tb.n_tensors];
+  (void)n_total;
 
   // per-thread, chunk-independent description of its pairs
   const uint16_t* p_idx[NP];
@@ -170,6 +177,14 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   uint64_t gw = 0;                         // GROUPED: the bytes holding the NP codes
   float gs = 0.0f;
   auto fetch = [&](uint32_t g) {
+    if (!SL_CHECK(a.flags, g < a.tb.n_chunks)) {     // (debug build) no message is read for such a chunk
+#pragma unroll
+      for (int i = 0; i < NP; ++i) { rp[i] = 0xFFFFu; rc[i] = 0; rs[i] = 0.0f; }
+#pragma unroll
+      for (int i = 0; i < (NP > 1 ? NP / 2 : 1); ++i) gi[i] = 0xFFFFFFFFu;
+      gw = 0; gs = 0.0f;
+      return;
+    }
     if constexpr (GROUPED) {
 #pragma unroll
       for (int i = 0; i < (NP > 1 ? NP / 2 : 1); ++i) gi[i] = 0xFFFFFFFFu;
@@ -220,11 +235,12 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       for (int j = 0; j < 4; ++j) {
         const int f = tid + 256 * j;
         const float* src = a.out + base + (size_t)(f >> 4) * stride + (size_t)((f & 15) << 2);
+        if (SL_CHECK(a.flags, base + (size_t)(f >> 4) * stride + (size_t)((f & 15) << 2) + 4 <= n_total))
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
                      ::"r"(agg_smem_u32(reinterpret_cast<float4*>(sm.gbuf[buf]) + f)), "l"(src) : "memory");
       }
       asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-    } else if (tid == 0) {                         // one 16 KB bulk copy
+    } else if (tid == 0 && SL_CHECK(a.flags, base + kAC <= n_total)) {   // one 16 KB bulk copy
       asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBytes) : "memory");
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                    ::"r"(agg_smem_u32(sm.gbuf[buf])), "l"(a.out + base), "r"(kBytes), "r"(bar) : "memory");
@@ -321,8 +337,9 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int f = tid + 256 * j;                 // float4 f of the chunk: row f / 16 of a tile
-      float4* dst = reinterpret_cast<float4*>(TILED ? out_cur + (size_t)(f >> 4) * stride_cur + (size_t)((f & 15) << 2)
-                                                    : out_cur + (size_t)f * 4);
+      const size_t off = TILED ? (size_t)(f >> 4) * stride_cur + (size_t)((f & 15) << 2) : (size_t)f * 4;
+      float4* dst = reinterpret_cast<float4*>(out_cur + off);
+      if (!SL_CHECK(a.flags, base_cur + off + 4 <= n_total)) continue;
       const float4 s4 = reinterpret_cast<const float4*>(acc)[tid + 256 * j];
       float4 u;
       if (pow2) {

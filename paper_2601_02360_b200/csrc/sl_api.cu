@@ -11,6 +11,12 @@ namespace {
 std::atomic<uint32_t> g_wait_polls{0};
 }
 uint32_t debug_wait_polls() { return g_wait_polls.load(std::memory_order_relaxed); }
+#ifdef SL_DEBUG_BOUNDS
+__global__ void bounds_selftest_kernel(uint32_t* flags, uint32_t* probe) {
+  const uint32_t i = 1 + threadIdx.x;                       // the buffer has one word: index 1 is outside
+  if (SL_CHECK(flags, i < 1u)) probe[i] = 0xDEADBEEFu;      // must be skipped
+}
+#endif
 }  // namespace sl
 
 namespace {
@@ -368,6 +374,17 @@ int sl_embed_reproject(float* T_S, float* T_perp, const float* U, uint64_t V, ui
   if (V == 0) return SL_OK;
   return launch_embed_reproject(T_S, T_perp, U, V, d, k, flags, (cudaStream_t)stream) == cudaSuccess
              ? SL_OK : SL_ERR_CUDA;
+}
+
+int sl_debug_bounds_selftest(uint32_t* flags, uint32_t* probe, void* stream) {
+#ifdef SL_DEBUG_BOUNDS
+  if (!flags || !probe) return SL_ERR_INVALID_ARG;
+  sl::bounds_selftest_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(flags, probe);
+  return cudaPeekAtLastError() == cudaSuccess ? SL_OK : SL_ERR_CUDA;
+#else
+  (void)flags; (void)probe; (void)stream;
+  return SL_ERR_UNSUPPORTED;
+#endif
 }
 
 void sl_debug_set_wait_limit(int32_t polls) {

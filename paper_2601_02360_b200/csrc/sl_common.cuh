@@ -212,6 +212,23 @@ inline int sm_count(cudaError_t* e) {
   return sms;
 }
 
+// ---------------------------------------------------------------------------
+// Range checks of the debug build (-DSL_DEBUG_BOUNDS; the stand-in for a memory checker).  Every index
+// the Eq. 2 kernels form for shared or global memory goes through SL_CHECK(flags, condition): in the
+// debug build a false condition raises SL_FLAG_BOUNDS and the expression is false, so that the access
+// guarded by it is skipped (never a trap, never an assert); in the normal build the expression is the
+// constant true and the condition is not evaluated.
+// ---------------------------------------------------------------------------
+#ifdef SL_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_check(uint32_t* flags, bool in_range) {
+  if (!in_range && flags) atomicOr(flags, (uint32_t)SL_FLAG_BOUNDS);
+  return in_range;
+}
+#define SL_CHECK(flags, cond) (::sl::bounds_check((flags), (cond)))
+#else
+#define SL_CHECK(flags, cond) (true)
+#endif
+
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 

@@ -46,7 +46,8 @@ struct SelectScratch {
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void block_select_emit(float* ep, const ChunkRef& c, int k_eff, int bits, float s,
                                                   SelectScratch& sc, uint32_t* cw,
-                                                  uint16_t* __restrict__ oidx, uint8_t* __restrict__ ocodes) {
+                                                  uint16_t* __restrict__ oidx, uint8_t* __restrict__ ocodes,
+                                                  uint32_t* flags, uint32_t cwords) {
   const int len = c.len;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t prefix = 0, need = (uint32_t)k_eff;
@@ -59,7 +60,8 @@ __device__ __forceinline__ void block_select_emit(float* ep, const ChunkRef& c, 
     __syncthreads();
     for (int i = tid; i < len; i += kThreads) {
       const uint32_t key = key_of(ep[i]);
-      if ((key >> hs) == (prefix >> hs)) atomicAdd(&sc.hist[(key >> shift) & ((1u << width) - 1u)], 1u);
+      const uint32_t bin = (key >> shift) & ((1u << width) - 1u);
+      if ((key >> hs) == (prefix >> hs) && SL_CHECK(flags, bin < 256u)) atomicAdd(&sc.hist[bin], 1u);
     }
     __syncthreads();
     if (warp == 0) {
@@ -122,8 +124,8 @@ __device__ __forceinline__ void block_select_emit(float* ep, const ChunkRef& c, 
     const uint32_t eqm = __ballot_sync(kFull, eq);
     const bool keep = in && (key > kth || (eq && eq_base + __popc(eqm & lanemask_lt()) < need));
     const uint32_t km = __ballot_sync(kFull, keep);
-    if (keep) {
-      const uint32_t slot = out_base + __popc(km & lanemask_lt());
+    const uint32_t slot = out_base + __popc(km & lanemask_lt());
+    if (keep && SL_CHECK(flags, slot < (uint32_t)k_eff && (bits == 32 || ((slot * (uint32_t)bits) >> 5) < cwords))) {
       oidx[slot] = (uint16_t)c.pos(i);            // element number -> position (they differ in edge tiles)
       float sent;
       if (bits == 32) {
@@ -160,10 +162,14 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   const int r = (int)(blockIdx.x % (uint32_t)a.R);
   uint32_t g = blockIdx.x / (uint32_t)a.R;
   if (TAILS) g = tail_chunk(a.tb, g, a.chunk);    // the g-th chunk that is not full
+  if (!SL_CHECK(a.flags, g < a.tb.n_chunks)) return;
   const ChunkRef c = locate(a.tb, g, a.chunk);
   const int len = c.len;
   const int k = a.k, bits = a.bits;
   const int k_eff = k < len ? k : len;
+  const uint64_t n_total = a.tb.offset[a.tb.n_tensors];
+  (void)n_total;
+  if (!SL_CHECK(a.flags, len >= 1 && len <= a.chunk)) return;
 
   const float* __restrict__ tl = a.p.theta_local[r];
   const float* __restrict__ tg = a.theta_global;
@@ -173,6 +179,7 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   uint32_t tmax = 0;
   for (int i = tid; i < len; i += kThreads) {
     const uint64_t at = c.addr(i);
+    if (!SL_CHECK(a.flags, at < n_total)) continue;
     const float d = __fsub_rn(tg[at], tl[at]);
     const float e = __fmaf_rn(a.beta, er[at], d);
     ep[i] = e;
@@ -191,10 +198,13 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
 
   uint16_t* __restrict__ oidx = a.p.idx[r] + (uint64_t)g * (uint64_t)k;
   uint8_t* __restrict__ ocodes = a.p.codes[r] + (uint64_t)g * (uint64_t)a.stride;
-  block_select_emit(ep, c, k_eff, bits, s, sc, cw, oidx, ocodes);
+  block_select_emit(ep, c, k_eff, bits, s, sc, cw, oidx, ocodes, a.flags, cwords);
 
   // write-back
-  for (int i = tid; i < len; i += kThreads) er[c.addr(i)] = ep[i];
+  for (int i = tid; i < len; i += kThreads) {
+    const uint64_t at = c.addr(i);
+    if (SL_CHECK(a.flags, at < n_total)) er[at] = ep[i];
+  }
   for (int j = k_eff + tid; j < k; j += kThreads) oidx[j] = 0xFFFFu;
   if (bits != 32) {
     const uint8_t* cb = reinterpret_cast<const uint8_t*>(cw);
@@ -392,7 +402,7 @@ __device__ __forceinline__ uint32_t count_ge(const uint32_t (&ck)[NREG > 0 ? NRE
 template <int NREG>
 __device__ __forceinline__ void select_candidates(const uint32_t* cand_key, const uint16_t* cand_pos, uint32_t C,
                                                   uint32_t k, uint32_t T1, uint32_t smax, uint32_t* hist,
-                                                  uint32_t* bitmap, uint16_t* kept_pos, int lane) {
+                                                  uint32_t* bitmap, uint16_t* kept_pos, int lane, uint32_t* flags) {
   uint32_t ck[NREG > 0 ? NREG : 1];
   uint32_t cp[NREG > 0 ? NREG : 1];
   if (NREG > 0) {
@@ -476,7 +486,7 @@ __device__ __forceinline__ void select_candidates(const uint32_t* cand_key, cons
         const bool keep = ((uint32_t)lane + 32u * (uint32_t)i < C) &&
                           (ck[i] >= thr_ge || (ck[i] == thr_eq && cp[i] <= pos_le));
         const uint32_t bal = __ballot_sync(kFull, keep);
-        if (keep) {
+        if (keep && SL_CHECK(flags, cp[i] < (uint32_t)kC && base + __popc(bal & lanemask_lt()) < 128u)) {
           atomicOr(&bitmap[cp[i] >> 5], 1u << (cp[i] & 31u));
           kept_pos[base + __popc(bal & lanemask_lt())] = (uint16_t)cp[i];
         }
@@ -490,7 +500,7 @@ __device__ __forceinline__ void select_candidates(const uint32_t* cand_key, cons
       const uint32_t p_i = i < C ? (uint32_t)cand_pos[i] : 0u;
       const bool keep = i < C && (k_i >= thr_ge || (k_i == thr_eq && p_i <= pos_le));
       const uint32_t bal = __ballot_sync(kFull, keep);
-      if (keep) {
+      if (keep && SL_CHECK(flags, p_i < (uint32_t)kC && base + __popc(bal & lanemask_lt()) < 128u)) {
         atomicOr(&bitmap[p_i >> 5], 1u << (p_i & 31u));
         kept_pos[base + __popc(bal & lanemask_lt())] = (uint16_t)p_i;
       }
@@ -502,7 +512,7 @@ __device__ __forceinline__ void select_candidates(const uint32_t* cand_key, cons
 // Overflow path of the selector: exact radix select over the whole chunk by one warp; kept
 // positions go to the bitmap (one ballot = one bitmap word) and to kept_pos.
 __device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, uint32_t* hist, uint32_t* bitmap,
-                                                 uint16_t* kept_pos, int lane) {
+                                                 uint16_t* kept_pos, int lane, uint32_t* flags) {
   uint32_t prefix = 0, need = k;
 #pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
@@ -553,7 +563,8 @@ __device__ __forceinline__ void warp_select_full(const float* ep, uint32_t k, ui
     const bool keep = key > kth || (eq && eq_seen + __popc(eqm & lanemask_lt()) < need);
     const uint32_t km = __ballot_sync(kFull, keep);
     if (lane == 0) bitmap[w] = km;
-    if (keep) kept_pos[base + __popc(km & lanemask_lt())] = (uint16_t)(w * 32 + lane);
+    if (keep && SL_CHECK(flags, base + __popc(km & lanemask_lt()) < 128u))
+      kept_pos[base + __popc(km & lanemask_lt())] = (uint16_t)(w * 32 + lane);
     eq_seen += __popc(eqm);
     base += __popc(km);
   }
@@ -608,6 +619,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   const uint32_t G = gridDim.x;
   const int k = a.k, bits = a.bits, R = a.R;
   constexpr uint32_t kBytes = kC * 4;
+  const uint64_t n_total = a.tb.offset[a.tb.n_tensors];      // debug build: the range every arena offset must stay in
+  (void)n_total;
 
   for (int i = tid; i < kSel * (kC / 32); i += kFastThreads) (&sm.bitmap[0][0])[i] = 0;
   for (int i = tid; i < kSel * 256; i += kFastThreads) (&sm.hist[0][0])[i] = 0;
@@ -653,6 +666,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       for (int j = 0; j < 4; ++j) {
         const int f = t4 + 256 * j;
         const size_t off = (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2);
+        if (!SL_CHECK(a.flags, it.base + off + 4 <= n_total)) continue;
         cp_async_16(reinterpret_cast<float4*>(sm.tl[st_tl]) + f, src_tl + off);
         cp_async_16(reinterpret_cast<float4*>(sm.ee[st_ee]) + f, src_ee + off);
       }
@@ -662,7 +676,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       if (pf.valid) {
         if (TILED) {
           tile_load(pf, i, i);
-        } else if (tid == 0) {
+        } else if (tid == 0 && SL_CHECK(a.flags, pf.base + kC <= n_total)) {
           ++tl_issued;
           mbar_expect_tx(&sm.full_tl[i], kBytes);
           tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
@@ -682,7 +696,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       for (int j = 0; j < 4; ++j) {
         const int f = t4 + 256 * j;
         const size_t off = TILED ? (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2) : (size_t)f * 4;
-        G4[j] = __ldcs(reinterpret_cast<const float4*>(tg + off));
+        if (SL_CHECK(a.flags, it.base + off + 4 <= n_total)) G4[j] = __ldcs(reinterpret_cast<const float4*>(tg + off));
       }
     };
     if (cur.valid) load_theta(cur);
@@ -696,8 +710,9 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int f = tid + 256 * j;
-        __stcs(reinterpret_cast<float4*>(dst + (size_t)(f >> 4) * stride + (size_t)((f & 15) << 2)),
-               reinterpret_cast<const float4*>(sm.ee[st_ee])[f]);
+        const size_t off = (size_t)(f >> 4) * stride + (size_t)((f & 15) << 2);
+        if (SL_CHECK(a.flags, base + off + 4 <= n_total))
+          __stcs(reinterpret_cast<float4*>(dst + off), reinterpret_cast<const float4*>(sm.ee[st_ee])[f]);
       }
     };
     __syncwarp();
@@ -766,7 +781,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         __syncwarp();
         named_sync(4 + q, kPairThreads);          // selector q has finished item w-2
         // ---- E (item w-2): its message leaves shared memory (warp 0, three coalesced stores) ----
-        if (warp == 0) {
+        if (warp == 0 && SL_CHECK(a.flags, g_m2 < a.tb.n_chunks && r_m2 < R)) {
           const int sp = (w - kSel) % kEeStages;
           const bool pc = r_m2 < kPtrCache;
           uint16_t* oidx = (pc ? sm.p_idx[r_m2] : a.p.idx[r_m2]) + (uint64_t)g_m2 * (uint64_t)k;
@@ -790,7 +805,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
         // the stages take item w+2's
         if (TILED) {
           tile_load(pf, st, (w + kTlStages) % kEeStages);
-        } else if (tid == 0) {
+        } else if (tid == 0 && SL_CHECK(a.flags, pf.base + kC <= n_total)) {
           ++tl_issued;
           mbar_expect_tx(&sm.full_tl[st], kBytes);
           tma_load_1d(sm.tl[st], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[st]);
@@ -822,7 +837,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
               ckey[at] = key[e];
               cpos[at] = (uint16_t)(((e >> 2) << 10) + (t4 << 2) + (e & 3));
             }
-            atomicAdd(&hist[(key[e] - T1) >> sh], 1u);
+            if (SL_CHECK(a.flags, ((key[e] - T1) >> sh) < 256u)) atomicAdd(&hist[(key[e] - T1) >> sh], 1u);
             ++at;
           }
         }
@@ -854,7 +869,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       const int rp = last ? r_m1 : r_m2;
       __syncwarp();
       named_sync(4 + wp % kSel, kPairThreads);
-      if (warp == 0) {
+      if (warp == 0 && SL_CHECK(a.flags, gp < a.tb.n_chunks && rp < R)) {
         const int sp = wp % kEeStages;
         const bool pc = rp < kPtrCache;
         uint16_t* oidx = (pc ? sm.p_idx[rp] : a.p.idx[rp]) + (uint64_t)gp * (uint64_t)k;
@@ -878,9 +893,11 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       pf.valid = false;                           // the producers move all the data
     } else if (lane == 0) {
       for (int i = q; i < kEeStages && pf.valid; i += kSel) {
-        ++ee_issued;
-        mbar_expect_tx(&sm.full_ee[i], kBytes);
-        tma_load_1d(sm.ee[i], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes, &sm.full_ee[i]);
+        if (SL_CHECK(a.flags, pf.base + kC <= n_total)) {
+          ++ee_issued;
+          mbar_expect_tx(&sm.full_ee[i], kBytes);
+          tma_load_1d(sm.ee[i], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes, &sm.full_ee[i]);
+        }
         pf.advance(a.tb, kSel, R, G);
       }
     } else {
@@ -902,7 +919,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       if (!TILED && pending_stage >= 0) {
         if (lane == 0) {
           tma_store_wait_read_all();
-          if (pf.valid) {
+          if (pf.valid && SL_CHECK(a.flags, pf.base + kC <= n_total)) {
             ++ee_issued;
             mbar_expect_tx(&sm.full_ee[pending_stage], kBytes);
             tma_load_1d(sm.ee[pending_stage], (pf.r < kPtrCache ? sm.p_err[pf.r] : a.p.err[pf.r]) + pf.base, kBytes,
@@ -924,13 +941,13 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       uint16_t* midx = sm.msg_idx[se];
       uint32_t* mcodes = sm.msg_codes[se];
       // ---- C ----
-      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist[q], bitmap, kept_pos, lane);
+      if (C > (uint32_t)kCandMax) warp_select_full(ep, (uint32_t)k, sm.hist[q], bitmap, kept_pos, lane, a.flags);
       else if (C <= 32u * kCandReg)
-        select_candidates<kCandReg>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
+        select_candidates<kCandReg>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane, a.flags);
       else if (C <= 32u * kCandRegBig)
-        select_candidates<kCandRegBig>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
+        select_candidates<kCandRegBig>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane, a.flags);
       else
-        select_candidates<0>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane);
+        select_candidates<0>(sm.cand_key[q], sm.cand_pos[q], C, (uint32_t)k, T1, smax, sm.hist[q], bitmap, kept_pos, lane, a.flags);
       __syncwarp();
       if (lane == 0) sm.count[q] = 0;
       // ---- D ----
@@ -950,8 +967,10 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       __syncwarp();
       for (int t = lane; t < k; t += 32) {
         const uint32_t pos = kept_pos[t];
+        if (!SL_CHECK(a.flags, t < 128 && pos < (uint32_t)kC)) continue;
         const uint32_t wd = pos >> 5;
         const uint32_t slot = (uint32_t)prefix[wd] + __popc(bitmap[wd] & ((1u << (pos & 31u)) - 1u));
+        if (!SL_CHECK(a.flags, slot < (uint32_t)k && slot < 128u)) continue;
         const float v = ep[pos];
         midx[slot] = (uint16_t)pos;
         float sent;
@@ -973,7 +992,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       __syncwarp();
       reinterpret_cast<uint4*>(bitmap)[lane] = make_uint4(0, 0, 0, 0);
       // ---- E: the stage drains to the error buffer (TILED: the producers write it back) ----
-      if (!TILED && lane == 0)
+      if (!TILED && lane == 0 && SL_CHECK(a.flags, cur.base + kC <= n_total && cur.r < R))
         tma_store_1d((cur.r < kPtrCache ? sm.p_err[cur.r] : a.p.err[cur.r]) + cur.base, ep, kBytes);
       pending_stage = se;
       __syncwarp();
