@@ -55,6 +55,12 @@ def lib():
         L.slo_outer_apply.restype = i32
         L.slo_outer_apply.argtypes = [vp, vp, u64, f32]
         L.slo_quantise.restype = u32
+        L.slo_widen_bf16.argtypes = [vp, vp, u64]
+        L.slo_widen_bf16.restype = i32
+        L.slo_round_bf16.argtypes = [f32]
+        L.slo_round_bf16.restype = ctypes.c_uint16
+        L.slo_outer_apply_bf16.argtypes = [vp, vp, u64, f32]
+        L.slo_outer_apply_bf16.restype = i32
         L.slo_quantise.argtypes = [f32, f32, i32]
         L.slo_dequantise.restype = f32
         L.slo_dequantise.argtypes = [u32, f32, i32]
@@ -154,6 +160,41 @@ def outer_apply(theta_global: np.ndarray, update: np.ndarray, outer_lr: float) -
     rc = lib().slo_outer_apply(_p(theta_global), _p(update), theta_global.size, outer_lr)
     if rc != 0:
         raise ValueError("slo_outer_apply rejected its arguments")
+
+
+def widen_bf16(x: np.ndarray) -> np.ndarray:
+    """bfloat16 bit patterns (uint16) -> the float32 values they stand for (exact)."""
+    assert x.dtype == np.uint16 and x.flags.c_contiguous
+    out = np.empty(x.shape, dtype=np.float32)
+    assert lib().slo_widen_bf16(_p(x), _p(out), x.size) == 0
+    return out
+
+
+def round_bf16(v: float) -> int:
+    return int(lib().slo_round_bf16(v))
+
+
+def outer_apply_bf16(theta_global: np.ndarray, update: np.ndarray, outer_lr: float) -> None:
+    """theta_global: uint16 bfloat16 patterns, updated in place (float32 step, then one rounding to bfloat16)."""
+    assert theta_global.dtype == np.uint16 and update.dtype == np.float32
+    if lib().slo_outer_apply_bf16(_p(theta_global), _p(update), theta_global.size, outer_lr) != 0:
+        raise ValueError("slo_outer_apply_bf16 rejected its arguments")
+
+
+def outer_round_bf16(theta_locals, theta_global: np.ndarray, errs, offsets, beta: float, chunk: int, k: int,
+                     bits: int, outer_lr: float, cols=None):
+    """One whole outer step with the parameters stored as bfloat16 (uint16 patterns) and float32 error
+    buffers: the pseudo-gradient is formed in float32 from the widened parameters (Eq. 2 line 1), lines
+    2-5 are those of the float32 step, and theta_global is rounded to bfloat16 once, when it is stored."""
+    tg32 = widen_bf16(theta_global)
+    msgs, flags = [], 0
+    for tl, e in zip(theta_locals, errs):
+        i, c, s, f = compress(widen_bf16(tl), tg32, e, offsets, beta, chunk, k, bits, cols)
+        msgs.append((i, c, s))
+        flags |= f
+    upd = aggregate(msgs, offsets, chunk, k, bits, cols)
+    outer_apply_bf16(theta_global, upd, outer_lr)
+    return msgs, upd, flags
 
 
 def quantise(v: float, s: float, bits: int) -> int:

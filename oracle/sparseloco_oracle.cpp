@@ -24,6 +24,10 @@
 //        implementation of the chosen Q is pinned by its error bound, closed
 //        forms on dyadic inputs and bits = 32 (= the paper's setting).
 //   slo_aggregate, slo_outer_apply                     : pinned
+//   slo_widen_bf16, slo_outer_apply_bf16 (parameters stored as bfloat16, error buffer float32):
+//        the paper states no storage precision for Eq. 2, so the CHOICE of where the parameters
+//        are rounded is this build's reading ("parity unpinned" by the paper); the rounding
+//        itself and the step are pinned (tests/test_oracle_bf16_pins.py)
 #include <algorithm>
 #include <cmath>
 #include <cstdint>
@@ -287,6 +291,41 @@ int slo_aggregate(int R, const uint16_t* const* idx, const uint8_t* const* codes
 int slo_outer_apply(float* theta_global, const float* update, uint64_t n, float outer_lr) {
   if (!theta_global || !update) return SLO_ERR_INVALID_ARG;
   for (uint64_t i = 0; i < n; ++i) theta_global[i] = std::fmaf(-outer_lr, update[i], theta_global[i]);
+  return SLO_OK;
+}
+
+// Parameters stored as bfloat16 (the upper 16 bits of a binary32): widening is exact.
+int slo_widen_bf16(const uint16_t* in, float* out, uint64_t n) {
+  if (!in || !out) return SLO_ERR_INVALID_ARG;
+  for (uint64_t i = 0; i < n; ++i) {
+    const uint32_t b = (uint32_t)in[i] << 16;
+    std::memcpy(&out[i], &b, 4);
+  }
+  return SLO_OK;
+}
+
+// binary32 -> bfloat16, round to nearest, ties to even; a NaN stays a NaN (quiet bit set, sign and the
+// upper payload bits kept); values beyond the largest bfloat16 round to infinity like any IEEE rounding
+uint16_t slo_round_bf16(float v) {
+  uint32_t b;
+  std::memcpy(&b, &v, 4);
+  if ((b & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((b >> 16) | 0x0040u);
+  const uint32_t lower = b & 0xFFFFu, keep = b >> 16;
+  if (lower > 0x8000u || (lower == 0x8000u && (keep & 1u))) return (uint16_t)(keep + 1u);
+  return (uint16_t)keep;
+}
+
+// Eq. 2 line 5, second half, for bfloat16 parameters: the step is taken in binary32 exactly as
+// slo_outer_apply takes it (one fused rounding) on the widened parameter, and the result is then
+// rounded once more, to bfloat16, for storage.
+int slo_outer_apply_bf16(uint16_t* theta_global, const float* update, uint64_t n, float outer_lr) {
+  if (!theta_global || !update) return SLO_ERR_INVALID_ARG;
+  for (uint64_t i = 0; i < n; ++i) {
+    const uint32_t b = (uint32_t)theta_global[i] << 16;
+    float th;
+    std::memcpy(&th, &b, 4);
+    theta_global[i] = slo_round_bf16(std::fmaf(-outer_lr, update[i], th));
+  }
   return SLO_OK;
 }
 
