@@ -306,7 +306,7 @@ def run_reference(args) -> None:
 
 # --------------------------------------------------------------------------- the CUDA path, timed
 class DeviceState:
-    def __init__(self, wl: synth.Workload, seed: int, device, tiles: bool = False):
+    def __init__(self, wl: synth.Workload, seed: int, device, tiles: bool = False, bf16: bool = False):
         from paper_2601_02360_b200 import api
         self.api = api
         self.wl = wl
@@ -318,21 +318,36 @@ class DeviceState:
         self.layout = api.Layout(wl.offsets(), cols)
         self.n_chunks = api.sl_num_chunks(self.layout, wl.chunk)
         n = wl.n_total
+        self.bf16 = bf16          # parameters stored as bfloat16 (error buffers stay float32)
         self.theta_global = synth.gen_theta_global(wl, device, seed)
         self.rho = synth.row_scales(wl, seed)
-        self.theta_local = [torch.empty(n, dtype=torch.float32, device=device) for _ in range(wl.R)]
+        th_dtype = torch.bfloat16 if bf16 else torch.float32
+        if bf16:
+            self.theta_global = self.theta_global.to(torch.bfloat16)
+            self._tmp = torch.empty(n, dtype=torch.float32, device=device)     # a replica is drawn in float32, then rounded
+        self.theta_local = [torch.empty(n, dtype=th_dtype, device=device) for _ in range(wl.R)]
         self.err = [torch.zeros(n, dtype=torch.float32, device=device) for _ in range(wl.R)]
         self.idx, self.codes, self.scales = api.alloc_messages(self.layout, wl.chunk, wl.k, wl.bits,
                                                                wl.R, device)
         self.flags = torch.zeros(1, dtype=torch.int32, device=device)
 
     def redraw_locals(self, rnd: int) -> None:
+        if self.bf16:
+            tg32 = self.theta_global.float()
+            for r in range(self.wl.R):
+                synth.gen_theta_local(self.wl, tg32, rnd, r, self.seed, out=self._tmp, rho=self.rho)
+                self.theta_local[r].copy_(self._tmp)
+            return
         for r in range(self.wl.R):
             synth.gen_theta_local(self.wl, self.theta_global, rnd, r, self.seed,
                                   out=self.theta_local[r], rho=self.rho)
 
     def compress(self) -> None:
         w = self.wl
+        if self.bf16:
+            self.api.sl_compress_batch_bf16(self.theta_local, self.theta_global, self.err, self.layout, w.beta,
+                                            w.chunk, w.k, w.bits, self.idx, self.codes, self.scales, self.flags)
+            return
         self.api.sl_compress_batch(self.theta_local, self.theta_global, self.err, self.layout, w.beta,
                                    w.chunk, w.k, w.bits, self.idx, self.codes, self.scales, self.flags)
 
@@ -343,6 +358,10 @@ class DeviceState:
 
     def aggregate_apply(self) -> None:
         w = self.wl
+        if self.bf16:
+            self.api.sl_aggregate_apply_bf16(self.idx, self.codes, self.scales, self.layout, w.chunk, w.k, w.bits,
+                                             self.theta_global, w.outer_lr, self.flags)
+            return
         self.api.sl_aggregate_apply(self.idx, self.codes, self.scales, self.layout, w.chunk, w.k, w.bits,
                                     self.theta_global, w.outer_lr, self.flags)
 
@@ -679,7 +698,8 @@ def _median_row(ms_list, alg_bytes, peak, clocks, extra=None):
     return row
 
 
-def row_outer_step(wl: synth.Workload, seed: int, dev, peak: float, steps: int, tiles: bool = False) -> dict:
+def row_outer_step(wl: synth.Workload, seed: int, dev, peak: float, steps: int, tiles: bool = False,
+                   bf16: bool = False) -> dict:
     """One whole outer step (both launches) of another configuration: median of `steps` steps, theta_local
     re-drawn between steps (untimed); frac = strict step bytes / time / peak, like step_hbm.frac_of_peak."""
     torch.cuda.empty_cache()
@@ -687,7 +707,10 @@ def row_outer_step(wl: synth.Workload, seed: int, dev, peak: float, steps: int, 
     need = (2 * wl.R + 1) * wl.n_total * 4 + (3 << 30)
     if free < need:
         return {"skipped": f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free"}
-    st = DeviceState(wl, seed, dev, tiles=tiles)
+    st = DeviceState(wl, seed, dev, tiles=tiles, bf16=bf16)
+    # bfloat16 parameters: theta_local 2 + e 8 bytes per replica-parameter, theta_global 2 + 2
+    strict = step_bytes_strict(wl) - (wl.n_total * (2 * wl.R + 4) if bf16 else 0)
+    comp_b = compress_bytes(wl) - (wl.n_total * (2 * wl.R + 2) if bf16 else 0)
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(dev.index or 0)
     t_step, t_comp = [], []
@@ -709,10 +732,11 @@ def row_outer_step(wl: synth.Workload, seed: int, dev, peak: float, steps: int, 
     clocks = sampler.stop()
     flags = int(st.flags.item())
     comp = float(np.median(t_comp))
-    row = _median_row(t_step, step_bytes_strict(wl), peak, clocks,
+    row = _median_row(t_step, strict, peak, clocks,
                       {"R": wl.R, "k": wl.k, "bits": wl.bits, "geometry": "64x64 tiles" if tiles else "consecutive chunks",
+                       "parameters": "bfloat16, float32 error buffers" if bf16 else "float32",
                        "params_per_s": wl.n_total / (float(np.median(t_step)) * 1e-3),
-                       "compress_ms": comp, "compress_frac": compress_bytes(wl) / (comp * 1e-3) / 1e9 / peak,
+                       "compress_ms": comp, "compress_frac": comp_b / (comp * 1e-3) / 1e9 / peak,
                        "device_flags": flags})
     del st
     torch.cuda.empty_cache()
@@ -800,6 +824,7 @@ def measured_rows(args, wl: synth.Workload, dev, peak: float) -> dict:
     rows["tiles"] = row_outer_step(wl, args.seed, dev, peak, n, tiles=True)
     rows["r2"] = row_outer_step(wl.replace(R=2), args.seed, dev, peak, n)
     rows["r16_k128"] = row_outer_step(wl.replace(R=16, k=128), args.seed, dev, peak, n)
+    rows["bf16_params"] = row_outer_step(wl, args.seed, dev, peak, n, bf16=True)
     has_embed = any(t[0].startswith("embed") for t in wl.tensors)
     if has_embed:
         d = next(t for t in wl.tensors if t[0].startswith("embed"))[2]

@@ -155,6 +155,32 @@ int sl_outer_step(int R, const float* const* theta_local, float* theta_global, f
                   uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
                   void* stream);
 
+/* Eq. 2 with the parameters stored as bfloat16 (the upper 16 bits of a binary32, passed as uint16_t)
+ * and everything else as above: error buffers, scales and unquantised values stay float32.  The paper
+ * states no storage precision for this step (section 2.1); the reading taken here:
+ *   line 1   delta = theta_global - theta_local in float32 on the exactly widened values (one rounding);
+ *   lines 2-4 as in the float32 calls, so the error buffer keeps what the coarse parameters cannot;
+ *   line 5   theta_global = bf16( fma(-outer_lr, update, widen(theta_global)) ): the float32 step with one
+ *            rounding, then one more rounding for storage - to nearest, ties to even; a NaN stays a NaN
+ *            (quiet bit set), overflow goes to infinity.  An update below half a bfloat16 unit of a
+ *            parameter leaves that parameter unchanged.
+ * Messages (idx, codes, scales) are identical in format to the float32 calls', so sl_aggregate works on
+ * them unchanged.  The tuned kernels take consecutive chunks of 4096 with every tensor offset a multiple of
+ * 8 elements and 16-byte aligned arrays; everything else (tiles included) runs the generic kernels with
+ * identical results.  Arguments, flags and errors as in the float32 calls of the same names. */
+int sl_compress_batch_bf16(int R, const uint16_t* const* theta_local, const uint16_t* theta_global,
+                           float* const* err, const sl_layout* layout, float beta, int chunk, int k, int bits,
+                           uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
+                           void* stream);
+int sl_aggregate_apply_bf16(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                            const float* const* scales, const sl_layout* layout, int chunk, int k, int bits,
+                            uint16_t* theta_global, float outer_lr, uint32_t* flags, void* stream);
+int sl_outer_apply_bf16(uint16_t* theta_global, const float* update, uint64_t n, float outer_lr, void* stream);
+int sl_outer_step_bf16(int R, const uint16_t* const* theta_local, uint16_t* theta_global, float* const* err,
+                       const sl_layout* layout, float beta, int chunk, int k, int bits, float outer_lr,
+                       uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
+                       void* stream);
+
 /* 12-bit wire form of the positions (the message of Eq. 2 line 3 carries "indices and values"; a
  * position of a chunk of at most 4096 elements fits 12 bits, which takes a k = 64, 2-bit message
  * from 148 to 116 bytes per chunk).  Slot j of a chunk occupies bits [12 j, 12 j + 12) of the

@@ -22,7 +22,8 @@ SL_FLAG_NONFINITE, SL_FLAG_BAD_INDEX, SL_FLAG_TIMEOUT, SL_FLAG_BOUNDS = 1, 2, 4,
 SL_MAX_CHUNK, SL_MAX_TENSORS, SL_MAX_REPLICAS = 8192, 1280, 64
 
 EXPORTS = ("sl_num_chunks", "sl_codes_stride", "sl_codes_bytes", "sl_compress", "sl_compress_batch", "sl_aggregate",
-           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_embed_reproject", "sl_round_tf32", "sl_subspace_project", "sl_subspace_reconstruct", "sl_idx12_stride",
+           "sl_outer_apply", "sl_aggregate_apply", "sl_outer_step", "sl_compress_batch_bf16", "sl_aggregate_apply_bf16",
+           "sl_outer_apply_bf16", "sl_outer_step_bf16", "sl_embed_reproject", "sl_round_tf32", "sl_subspace_project", "sl_subspace_reconstruct", "sl_idx12_stride",
            "sl_pack_idx12", "sl_unpack_idx12", "sl_debug_set_wait_limit", "sl_debug_bounds_selftest", "sl_strerror")
 
 
@@ -70,6 +71,14 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     L.sl_aggregate_apply.argtypes = [i32, vp, vp, vp, lp, i32, i32, i32, vp, f32, vp, vp]
     L.sl_outer_step.restype = i32
     L.sl_outer_step.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
+    L.sl_compress_batch_bf16.restype = i32
+    L.sl_compress_batch_bf16.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, vp, vp, vp, vp, vp]
+    L.sl_aggregate_apply_bf16.restype = i32
+    L.sl_aggregate_apply_bf16.argtypes = [i32, vp, vp, vp, lp, i32, i32, i32, vp, f32, vp, vp]
+    L.sl_outer_apply_bf16.restype = i32
+    L.sl_outer_apply_bf16.argtypes = [vp, vp, u64, f32, vp]
+    L.sl_outer_step_bf16.restype = i32
+    L.sl_outer_step_bf16.argtypes = [i32, vp, vp, vp, lp, f32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.sl_embed_reproject.restype = i32
     L.sl_embed_reproject.argtypes = [vp, vp, vp, u64, ctypes.c_uint32, ctypes.c_uint32, vp, vp]
     u32 = ctypes.c_uint32
@@ -218,6 +227,43 @@ def sl_outer_step(theta_local: Sequence, theta_global, err: Sequence, layout, be
                                 _layout(layout).ref(), beta, chunk, k, bits, outer_lr, _ptr_table(idx),
                                 _ptr_table(codes), _ptr_table(scales), _ptr(flags), _stream(stream)),
            "sl_outer_step")
+
+
+def sl_compress_batch_bf16(theta_local: Sequence, theta_global, err: Sequence, layout, beta: float, chunk: int,
+                           k: int, bits: int, idx: Sequence, codes: Sequence, scales: Sequence, flags=None,
+                           stream=None) -> None:
+    """theta_local / theta_global: torch.bfloat16 (or uint16 pattern) tensors."""
+    R = len(theta_local)
+    assert len(err) == len(idx) == len(codes) == len(scales) == R
+    _check(load().sl_compress_batch_bf16(R, _ptr_table(theta_local), _ptr(theta_global), _ptr_table(err),
+                                         _layout(layout).ref(), beta, chunk, k, bits, _ptr_table(idx),
+                                         _ptr_table(codes), _ptr_table(scales), _ptr(flags), _stream(stream)),
+           "sl_compress_batch_bf16")
+
+
+def sl_aggregate_apply_bf16(idx: Sequence, codes: Sequence, scales: Sequence, layout, chunk: int, k: int,
+                            bits: int, theta_global, outer_lr: float, flags=None, stream=None) -> None:
+    R = len(idx)
+    assert len(codes) == len(scales) == R
+    _check(load().sl_aggregate_apply_bf16(R, _ptr_table(idx), _ptr_table(codes), _ptr_table(scales),
+                                          _layout(layout).ref(), chunk, k, bits, _ptr(theta_global), outer_lr,
+                                          _ptr(flags), _stream(stream)), "sl_aggregate_apply_bf16")
+
+
+def sl_outer_apply_bf16(theta_global, update, n: int, outer_lr: float, stream=None) -> None:
+    _check(load().sl_outer_apply_bf16(_ptr(theta_global), _ptr(update), n, outer_lr, _stream(stream)),
+           "sl_outer_apply_bf16")
+
+
+def sl_outer_step_bf16(theta_local: Sequence, theta_global, err: Sequence, layout, beta: float, chunk: int,
+                       k: int, bits: int, outer_lr: float, idx: Sequence, codes: Sequence, scales: Sequence,
+                       flags=None, stream=None) -> None:
+    R = len(theta_local)
+    assert len(err) == len(idx) == len(codes) == len(scales) == R
+    _check(load().sl_outer_step_bf16(R, _ptr_table(theta_local), _ptr(theta_global), _ptr_table(err),
+                                     _layout(layout).ref(), beta, chunk, k, bits, outer_lr, _ptr_table(idx),
+                                     _ptr_table(codes), _ptr_table(scales), _ptr(flags), _stream(stream)),
+           "sl_outer_step_bf16")
 
 
 def sl_embed_reproject(T_S, T_perp, U, V: int, d: int, k: int, flags=None, stream=None) -> None:

@@ -60,7 +60,13 @@ aggregate_generic_kernel(const __grid_constant__ AggregateArgs<T> a) {
   for (int i = tid; i < len; i += kThreads) {
     const float u = __fdiv_rn(acc[i], Rf);
     const uint64_t at = c.addr(i);
-    if (SL_CHECK(a.flags, at < n_total)) out[at] = APPLY ? __fmaf_rn(-a.outer_lr, u, out[at]) : u;
+    if (!SL_CHECK(a.flags, at < n_total)) continue;
+    if (APPLY && a.theta_bf16) {
+      uint16_t* o16 = reinterpret_cast<uint16_t*>(a.out);
+      o16[at] = (uint16_t)bf16_round(__fmaf_rn(-a.outer_lr, u, bf16_widen(o16[at])));
+    } else {
+      out[at] = APPLY ? __fmaf_rn(-a.outer_lr, u, out[at]) : u;
+    }
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
@@ -117,9 +123,12 @@ __device__ __forceinline__ bool next_full_chunk(const Table<T>& tb, uint32_t& g,
 // pairs 256 apart.  Its positions then arrive as one 2*NP-byte load and its codes as a few bytes,
 // and the accumulation takes R rounds in which the owners of replica r read their NP accumulator
 // cells, add, and write them back (positions inside one message are distinct, so the cells are).
-template <int T, bool APPLY, int NP, bool TILED, bool GROUPED>
+// BF (with APPLY, consecutive chunks): theta_global is a bfloat16 array; a chunk of it is 8 KB, widened as
+// it is read and rounded to nearest-even as it is stored.
+template <int T, bool APPLY, int NP, bool TILED, bool GROUPED, bool BF = false>
 __global__ void __launch_bounds__(kThreads)
 aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
+  static_assert(!BF || (APPLY && !TILED), "bfloat16 parameters: fused update on consecutive chunks only");
   extern __shared__ __align__(16) unsigned char agg_smem_raw[];
   AggSmem& sm = *reinterpret_cast<AggSmem*>(agg_smem_raw);
   float* acc = sm.acc;
@@ -241,9 +250,11 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
       }
       asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
     } else if (tid == 0 && SL_CHECK(a.flags, base + kAC <= n_total)) {   // one 16 KB bulk copy
-      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBytes) : "memory");
+      constexpr uint32_t kThBytes = BF ? kBytes / 2 : kBytes;
+      const void* src = BF ? (const void*)(reinterpret_cast<const uint16_t*>(a.out) + base) : (const void*)(a.out + base);
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kThBytes) : "memory");
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                   ::"r"(agg_smem_u32(sm.gbuf[buf])), "l"(a.out + base), "r"(kBytes), "r"(bar) : "memory");
+                   ::"r"(agg_smem_u32(sm.gbuf[buf])), "l"(src), "r"(kThBytes), "r"(bar) : "memory");
     }
   };
 
@@ -348,11 +359,17 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
         u.x = __fdiv_rn(s4.x, Rf); u.y = __fdiv_rn(s4.y, Rf); u.z = __fdiv_rn(s4.z, Rf); u.w = __fdiv_rn(s4.w, Rf);
       }
       if (APPLY) {
-        const float4 G = g4[tid + 256 * j];
+        float4 G;
+        if constexpr (BF) G = bf16x4_widen(reinterpret_cast<const uint2*>(sm.gbuf[it & 1])[tid + 256 * j]);
+        else G = g4[tid + 256 * j];
         u.x = __fmaf_rn(nlr, u.x, G.x); u.y = __fmaf_rn(nlr, u.y, G.y);
         u.z = __fmaf_rn(nlr, u.z, G.z); u.w = __fmaf_rn(nlr, u.w, G.w);
       }
-      if (have_theta) __stcs(dst, u);
+      if constexpr (BF) {
+        if (have_theta) __stcs(reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(a.out) + base_cur + off), bf16x4_round(u));
+      } else {
+        if (have_theta) __stcs(dst, u);
+      }
     }
     __syncthreads();                               // accumulator and theta buffer read by everyone before they are reused
     if (APPLY) {
@@ -411,6 +428,17 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
     return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 8, true, true>)
                    : launch(aggregate_c4096_kernel<T, APPLY, 8, true, false>);
   }
+  if constexpr (APPLY) {
+    if (a.theta_bf16) {
+      if (np == 1) return launch(aggregate_c4096_kernel<T, true, 1, false, false, true>);
+      if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, true, 2, false, true, true>)
+                                  : launch(aggregate_c4096_kernel<T, true, 2, false, false, true>);
+      if (np == 4) return grouped ? launch(aggregate_c4096_kernel<T, true, 4, false, true, true>)
+                                  : launch(aggregate_c4096_kernel<T, true, 4, false, false, true>);
+      return grouped ? launch(aggregate_c4096_kernel<T, true, 8, false, true, true>)
+                     : launch(aggregate_c4096_kernel<T, true, 8, false, false, true>);
+    }
+  }
   if (np == 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, false, false>);
   if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 2, false, true>)
                               : launch(aggregate_c4096_kernel<T, APPLY, 2, false, false>);
@@ -445,13 +473,26 @@ outer_apply_kernel(float* __restrict__ theta, const float* __restrict__ update, 
   }
 }
 
+__global__ void __launch_bounds__(256)
+outer_apply_bf16_kernel(uint16_t* __restrict__ theta, const float* __restrict__ update, uint64_t n, float lr) {
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  const float nlr = -lr;
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
+    theta[i] = (uint16_t)bf16_round(__fmaf_rn(nlr, update[i], bf16_widen(theta[i])));
+}
+
 }  // namespace
 
 template <int T>
 cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned16, cudaStream_t st) {
   if (a.tb.n_chunks == 0) return cudaSuccess;
   const size_t smem = (size_t)a.chunk * 4;
-  if (aligned16 && a.chunk == kAC && a.R * a.k <= kThreads * 8) {
+  bool tuned = aligned16 && a.chunk == kAC && a.R * a.k <= kThreads * 8;
+  if (tuned && apply && a.theta_bf16) {          // bfloat16 parameters: consecutive chunks starting on 16 bytes
+    tuned = a.tb.side == 0;
+    for (uint32_t t = 0; tuned && t <= a.tb.n_tensors; ++t) tuned = a.tb.offset[t] % 8 == 0;
+  }
+  if (tuned) {
     cudaError_t e0 = apply ? launch_aggregate_c4096<T, true>(a, st) : launch_aggregate_c4096<T, false>(a, st);
     if (e0 != cudaSuccess) return e0;
     const cudaError_t e = launch_aggregate_tails<T>(a, apply, st);
@@ -476,6 +517,16 @@ template cudaError_t launch_aggregate_tails<256>(const AggregateArgs<256>&, bool
 template cudaError_t launch_aggregate_tails<SL_MAX_TENSORS>(const AggregateArgs<SL_MAX_TENSORS>&, bool, cudaStream_t);
 template cudaError_t launch_aggregate<256>(const AggregateArgs<256>&, bool, bool, cudaStream_t);
 template cudaError_t launch_aggregate<SL_MAX_TENSORS>(const AggregateArgs<SL_MAX_TENSORS>&, bool, bool, cudaStream_t);
+
+cudaError_t launch_outer_apply_bf16(uint16_t* theta, const float* update, uint64_t n, float lr, cudaStream_t st) {
+  if (n == 0) return cudaSuccess;
+  cudaError_t e;
+  const uint64_t cap = (uint64_t)sm_count(&e) * 8ull;
+  if (e != cudaSuccess) return e;
+  const uint64_t blocks = (n + 255) / 256;
+  outer_apply_bf16_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, st>>>(theta, update, n, lr);
+  return cudaPeekAtLastError();
+}
 
 cudaError_t launch_outer_apply(float* theta, const float* update, uint64_t n, float lr, cudaStream_t st) {
   if (n == 0) return cudaSuccess;

@@ -111,7 +111,7 @@ template <int T>
 int compress_impl(int R, const float* const* theta_local, float* theta_global, float* const* err,
                   const sl_layout* L, float beta, int chunk, int k, int bits, uint16_t* const* idx,
                   uint8_t* const* codes, float* const* scales, uint32_t* flags, cudaStream_t st,
-                  bool step, float outer_lr) {
+                  bool step, float outer_lr, bool bf16) {
   CompressArgs<T> args;                 // by-value kernel parameters, built on the stack: no allocation
   CompressArgs<T>* a = &args;
   bool m4;
@@ -135,6 +135,7 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
   a->R = R;
   a->stride = (uint32_t)codes_stride(k, bits);
   a->wait_polls = debug_wait_polls();
+  a->theta_bf16 = bf16 ? 1 : 0;
   if (!step) return launch_compress<T>(*a, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 
   AggregateArgs<T> gargs;
@@ -154,6 +155,7 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
   g->R = R;
   g->stride = a->stride;
   g->wait_polls = a->wait_polls;
+  g->theta_bf16 = a->theta_bf16;
   if (launch_compress<T>(*a, al16, st) != cudaSuccess) return SL_ERR_CUDA;
   return launch_aggregate<T>(*g, true, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 }
@@ -161,31 +163,32 @@ int compress_impl(int R, const float* const* theta_local, float* theta_global, f
 int compress_checked(int R, const float* const* theta_local, float* theta_global,
                      float* const* err, const sl_layout* L, float beta, int chunk, int k, int bits,
                      uint16_t* const* idx, uint8_t* const* codes, float* const* scales,
-                     uint32_t* flags, void* stream, bool step = false, float outer_lr = 0.0f) {
+                     uint32_t* flags, void* stream, bool step = false, float outer_lr = 0.0f, bool bf16 = false) {
   if (R < 1 || R > SL_MAX_REPLICAS) return SL_ERR_INVALID_ARG;
   if (!theta_local || !theta_global || !err || !idx || !codes || !scales) return SL_ERR_INVALID_ARG;
   if (!std::isfinite(beta) || !std::isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
   const int rc = check_common(L, chunk, k, bits);
   if (rc != SL_OK) return rc;
-  if (!aligned(theta_global, 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
+  const uintptr_t th_al = bf16 ? 2 : 4;     // alignment of a parameter array: its element type's
+  if (!aligned(theta_global, th_al) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
   for (int r = 0; r < R; ++r) {
     if (!theta_local[r] || !err[r] || !idx[r] || !codes[r] || !scales[r]) return SL_ERR_INVALID_ARG;
-    if (!aligned(theta_local[r], 4) || !aligned(err[r], 4) || !aligned(scales[r], 4) ||
+    if (!aligned(theta_local[r], th_al) || !aligned(err[r], 4) || !aligned(scales[r], 4) ||
         !aligned(idx[r], 2) || (bits == 32 && !aligned(codes[r], 4)))
       return SL_ERR_ALIGNMENT;
   }
   cudaStream_t st = (cudaStream_t)stream;
   if (L->n_tensors <= 256)
     return compress_impl<256>(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx, codes,
-                              scales, flags, st, step, outer_lr);
+                              scales, flags, st, step, outer_lr, bf16);
   return compress_impl<SL_MAX_TENSORS>(R, theta_local, theta_global, err, L, beta, chunk, k, bits, idx,
-                                       codes, scales, flags, st, step, outer_lr);
+                                       codes, scales, flags, st, step, outer_lr, bf16);
 }
 
 template <int T>
 int aggregate_impl(int R, const uint16_t* const* idx, const uint8_t* const* codes,
                    const float* const* scales, const sl_layout* L, int chunk, int k, int bits, float* out,
-                   float outer_lr, bool apply, uint32_t* flags, cudaStream_t st) {
+                   float outer_lr, bool apply, uint32_t* flags, cudaStream_t st, bool bf16) {
   AggregateArgs<T> args;
   AggregateArgs<T>* a = &args;
   bool m4;
@@ -206,18 +209,19 @@ int aggregate_impl(int R, const uint16_t* const* idx, const uint8_t* const* code
   a->R = R;
   a->stride = (uint32_t)codes_stride(k, bits);
   a->wait_polls = debug_wait_polls();
+  a->theta_bf16 = bf16 ? 1 : 0;
   return launch_aggregate<T>(*a, apply, al16, st) == cudaSuccess ? SL_OK : SL_ERR_CUDA;
 }
 
 int aggregate_checked(int R, const uint16_t* const* idx, const uint8_t* const* codes,
                       const float* const* scales, const sl_layout* L, int chunk, int k, int bits,
-                      float* out, float outer_lr, bool apply, uint32_t* flags, void* stream) {
+                      float* out, float outer_lr, bool apply, uint32_t* flags, void* stream, bool bf16 = false) {
   if (R < 1 || R > SL_MAX_REPLICAS) return SL_ERR_INVALID_ARG;
   if (!idx || !codes || !scales || !out) return SL_ERR_INVALID_ARG;
   if (!std::isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
   const int rc = check_common(L, chunk, k, bits);
   if (rc != SL_OK) return rc;
-  if (!aligned(out, 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
+  if (!aligned(out, bf16 ? 2 : 4) || (flags && !aligned(flags, 4))) return SL_ERR_ALIGNMENT;
   for (int r = 0; r < R; ++r) {
     if (!idx[r] || !codes[r] || !scales[r]) return SL_ERR_INVALID_ARG;
     if (!aligned(idx[r], 2) || !aligned(scales[r], 4) || (bits == 32 && !aligned(codes[r], 4)))
@@ -225,9 +229,9 @@ int aggregate_checked(int R, const uint16_t* const* idx, const uint8_t* const* c
   }
   cudaStream_t st = (cudaStream_t)stream;
   if (L->n_tensors <= 256)
-    return aggregate_impl<256>(R, idx, codes, scales, L, chunk, k, bits, out, outer_lr, apply, flags, st);
+    return aggregate_impl<256>(R, idx, codes, scales, L, chunk, k, bits, out, outer_lr, apply, flags, st, bf16);
   return aggregate_impl<SL_MAX_TENSORS>(R, idx, codes, scales, L, chunk, k, bits, out, outer_lr, apply,
-                                        flags, st);
+                                        flags, st, bf16);
 }
 
 template <int T>
@@ -306,6 +310,39 @@ int sl_aggregate_apply(int R, const uint16_t* const* idx, const uint8_t* const* 
                        float* theta_global, float outer_lr, uint32_t* flags, void* stream) {
   return aggregate_checked(R, idx, codes, scales, L, chunk, k, bits, theta_global, outer_lr, true, flags,
                            stream);
+}
+
+int sl_compress_batch_bf16(int R, const uint16_t* const* theta_local, const uint16_t* theta_global,
+                           float* const* err, const sl_layout* L, float beta, int chunk, int k, int bits,
+                           uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
+                           void* stream) {
+  // the kernels take the parameter arrays through the float-typed slots of their argument block and
+  // reinterpret them when `theta_bf16` is set; nothing is dereferenced on the host
+  return compress_checked(R, reinterpret_cast<const float* const*>(theta_local),
+                          reinterpret_cast<float*>(const_cast<uint16_t*>(theta_global)), err, L, beta, chunk, k, bits,
+                          idx, codes, scales, flags, stream, false, 0.0f, true);
+}
+
+int sl_outer_step_bf16(int R, const uint16_t* const* theta_local, uint16_t* theta_global, float* const* err,
+                       const sl_layout* L, float beta, int chunk, int k, int bits, float outer_lr,
+                       uint16_t* const* idx, uint8_t* const* codes, float* const* scales, uint32_t* flags,
+                       void* stream) {
+  return compress_checked(R, reinterpret_cast<const float* const*>(theta_local), reinterpret_cast<float*>(theta_global),
+                          err, L, beta, chunk, k, bits, idx, codes, scales, flags, stream, true, outer_lr, true);
+}
+
+int sl_aggregate_apply_bf16(int R, const uint16_t* const* idx, const uint8_t* const* codes,
+                            const float* const* scales, const sl_layout* L, int chunk, int k, int bits,
+                            uint16_t* theta_global, float outer_lr, uint32_t* flags, void* stream) {
+  return aggregate_checked(R, idx, codes, scales, L, chunk, k, bits, reinterpret_cast<float*>(theta_global), outer_lr,
+                           true, flags, stream, true);
+}
+
+int sl_outer_apply_bf16(uint16_t* theta_global, const float* update, uint64_t n, float outer_lr, void* stream) {
+  if (!theta_global || !update || !std::isfinite(outer_lr)) return SL_ERR_INVALID_ARG;
+  if (!aligned(theta_global, 2) || !aligned(update, 4)) return SL_ERR_ALIGNMENT;
+  return launch_outer_apply_bf16(theta_global, update, n, outer_lr, (cudaStream_t)stream) == cudaSuccess
+             ? SL_OK : SL_ERR_CUDA;
 }
 
 uint64_t sl_idx12_stride(int k) { return k < 1 ? 0 : (12u * (uint64_t)k + 7u) / 8u; }

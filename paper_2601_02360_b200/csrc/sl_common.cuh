@@ -152,6 +152,7 @@ struct CompressArgs {
   uint32_t stride;  // bytes of codes per chunk
   uint32_t wait_polls;  // polls a bounded wait makes before it gives up (0: the default, about a second;
                         // 0xFFFFFFFF: none, every wait gives up at once)
+  int theta_bf16;       // 1: theta_local / theta_global point to bfloat16 arrays (error buffers stay float32)
 };
 
 template <int T>
@@ -164,6 +165,7 @@ struct AggregateArgs {
   int chunk, k, bits, R;
   uint32_t stride;
   uint32_t wait_polls;  // as in CompressArgs
+  int theta_bf16;       // 1 (aggregate + apply only): `out` is theta_global stored as bfloat16
 };
 
 // ---------------------------------------------------------------------------
@@ -172,6 +174,23 @@ struct AggregateArgs {
 // reconstruction at the level's midpoint s*(2q+1)/(2L).  Every product is one
 // explicitly rounded multiply so that nothing can be contracted.
 // ---------------------------------------------------------------------------
+// Parameters stored as bfloat16 (the upper half of a binary32).  Widening is exact; storing rounds to
+// nearest, ties to even; a NaN stays a NaN (quiet bit set, sign and upper payload kept).
+__device__ __forceinline__ float bf16_widen(uint32_t h) { return __uint_as_float(h << 16); }
+__device__ __forceinline__ uint32_t bf16_round(float v) {
+  const uint32_t b = __float_as_uint(v);
+  if ((b & 0x7FFFFFFFu) > 0x7F800000u) return (b >> 16) | 0x0040u;
+  return (b + 0x7FFFu + ((b >> 16) & 1u)) >> 16;      // adds just under half, and the last kept bit: half goes to even
+}
+// four consecutive bfloat16 values held in a uint2 <-> float4
+__device__ __forceinline__ float4 bf16x4_widen(uint2 v) {
+  return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                     __uint_as_float(v.y & 0xFFFF0000u));
+}
+__device__ __forceinline__ uint2 bf16x4_round(float4 v) {
+  return make_uint2(bf16_round(v.x) | (bf16_round(v.y) << 16), bf16_round(v.z) | (bf16_round(v.w) << 16));
+}
+
 __device__ __forceinline__ uint32_t key_of(float v) { return __float_as_uint(v) & 0x7FFFFFFFu; }
 
 // q = number of thresholds t_j = s*(j/L), j = 1..L-1, with |v| >= t_j.  The t_j are
@@ -240,6 +259,7 @@ template <int T> bool compress_is_tuned(const CompressArgs<T>& a, bool aligned16
 template <int T> cudaError_t launch_aggregate(const AggregateArgs<T>& a, bool apply, bool aligned16, cudaStream_t st);
 template <int T> cudaError_t launch_aggregate_tails(const AggregateArgs<T>& a, bool apply, cudaStream_t st);
 cudaError_t launch_outer_apply(float* theta, const float* update, uint64_t n, float lr, cudaStream_t st);
+cudaError_t launch_outer_apply_bf16(uint16_t* theta, const float* update, uint64_t n, float lr, cudaStream_t st);
 cudaError_t launch_pack_idx12(const uint16_t* idx, uint64_t n_chunks, int k, uint8_t* packed, uint32_t* flags,
                               cudaStream_t st);
 template <int T> cudaError_t launch_unpack_idx12(const Table<T>& tb, const uint8_t* packed, int chunk, int k,

@@ -180,7 +180,9 @@ compress_generic_kernel(const __grid_constant__ CompressArgs<T> a) {
   for (int i = tid; i < len; i += kThreads) {
     const uint64_t at = c.addr(i);
     if (!SL_CHECK(a.flags, at < n_total)) continue;
-    const float d = __fsub_rn(tg[at], tl[at]);
+    const float d = a.theta_bf16 ? __fsub_rn(bf16_widen(reinterpret_cast<const uint16_t*>(tg)[at]),
+                                             bf16_widen(reinterpret_cast<const uint16_t*>(tl)[at]))
+                                 : __fsub_rn(tg[at], tl[at]);
     const float e = __fmaf_rn(a.beta, er[at], d);
     ep[i] = e;
     tmax = max(tmax, key_of(e));
@@ -609,9 +611,12 @@ struct ItemCursor {
 // per-thread arrivals on one mbarrier were tried first: they serialise and cost more than the
 // copies).  In shared memory a tile is stored row after row, so everything between load and
 // store is the same.
-template <int T, bool TILED>
+// BF = true (consecutive chunks only): theta_local and theta_global are bfloat16 arrays; a theta_local
+// stage then holds 8 KB, and both are widened (exactly) as they are read.
+template <int T, bool TILED, bool BF>
 __global__ void __launch_bounds__(kFastThreads, 2)
 compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
+  static_assert(!(TILED && BF), "bfloat16 parameters take the tuned path for consecutive chunks only");
   extern __shared__ __align__(16) unsigned char smem_raw[];
   FastSmem& sm = *reinterpret_cast<FastSmem*>(smem_raw);
 
@@ -619,6 +624,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
   const uint32_t G = gridDim.x;
   const int k = a.k, bits = a.bits, R = a.R;
   constexpr uint32_t kBytes = kC * 4;
+  constexpr uint32_t kTlBytes = BF ? kC * 2 : kC * 4;        // bytes of theta_local per chunk
+  // theta_local of replica r, `elems` elements in
+  auto tl_src = [&](int r, uint64_t elems) -> const void* {
+    const float* p = r < kPtrCache ? sm.p_tl[r] : a.p.theta_local[r];
+    return BF ? (const void*)(reinterpret_cast<const uint16_t*>(p) + elems) : (const void*)(p + elems);
+  };
   const uint64_t n_total = a.tb.offset[a.tb.n_tensors];      // debug build: the range every arena offset must stay in
   (void)n_total;
 
@@ -678,8 +689,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
           tile_load(pf, i, i);
         } else if (tid == 0 && SL_CHECK(a.flags, pf.base + kC <= n_total)) {
           ++tl_issued;
-          mbar_expect_tx(&sm.full_tl[i], kBytes);
-          tma_load_1d(sm.tl[i], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[i]);
+          mbar_expect_tx(&sm.full_tl[i], kTlBytes);
+          tma_load_1d(sm.tl[i], tl_src(pf.r, pf.base), kTlBytes, &sm.full_tl[i]);
         }
         pf.advance(a.tb, 1, R, G);
       }
@@ -696,7 +707,12 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       for (int j = 0; j < 4; ++j) {
         const int f = t4 + 256 * j;
         const size_t off = TILED ? (size_t)(f >> 4) * it.stride + (size_t)((f & 15) << 2) : (size_t)f * 4;
-        if (SL_CHECK(a.flags, it.base + off + 4 <= n_total)) G4[j] = __ldcs(reinterpret_cast<const float4*>(tg + off));
+        if (SL_CHECK(a.flags, it.base + off + 4 <= n_total)) {
+          if constexpr (BF)
+            G4[j] = bf16x4_widen(__ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(a.theta_global) + it.base + off)));
+          else
+            G4[j] = __ldcs(reinterpret_cast<const float4*>(tg + off));
+        }
       }
     };
     if (cur.valid) load_theta(cur);
@@ -734,7 +750,9 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       uint32_t tmax = 0;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float4 L = tl4[t4 + 256 * j];
+        float4 L;
+        if constexpr (BF) L = bf16x4_widen(reinterpret_cast<const uint2*>(sm.tl[st])[t4 + 256 * j]);
+        else L = tl4[t4 + 256 * j];
         const float4 E = ee4[t4 + 256 * j];
         float4 v;
         v.x = __fmaf_rn(beta, E.x, __fsub_rn(G4[j].x, L.x));
@@ -807,8 +825,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
           tile_load(pf, st, (w + kTlStages) % kEeStages);
         } else if (tid == 0 && SL_CHECK(a.flags, pf.base + kC <= n_total)) {
           ++tl_issued;
-          mbar_expect_tx(&sm.full_tl[st], kBytes);
-          tma_load_1d(sm.tl[st], (pf.r < kPtrCache ? sm.p_tl[pf.r] : a.p.theta_local[pf.r]) + pf.base, kBytes, &sm.full_tl[st]);
+          mbar_expect_tx(&sm.full_tl[st], kTlBytes);
+          tma_load_1d(sm.tl[st], tl_src(pf.r, pf.base), kTlBytes, &sm.full_tl[st]);
         }
         pf.advance(a.tb, 1, R, G);
       }
@@ -1011,7 +1029,13 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
 
 template <int T>
 bool compress_is_tuned(const CompressArgs<T>& a, bool aligned16) {
-  // even k: the message's positions leave shared memory as 32-bit words
+  // even k: the message's positions leave shared memory as 32-bit words.  bfloat16 parameters: consecutive
+  // chunks only, and every tensor must start on 16 bytes of the 2-byte arrays too (offsets multiples of 8)
+  if (a.theta_bf16) {
+    if (a.tb.side != 0) return false;
+    for (uint32_t t = 0; t <= a.tb.n_tensors; ++t)
+      if (a.tb.offset[t] % 8 != 0) return false;
+  }
   return aligned16 && a.chunk == kC && a.k <= 128 && ((a.k * a.bits) % 32) == 0 && (a.k % 2) == 0;
 }
 
@@ -1031,17 +1055,16 @@ cudaError_t launch_compress(const CompressArgs<T>& a, bool aligned16, cudaStream
     if (e != cudaSuccess) return e;
     // persistent grid: two CTAs per SM, each walking its share of the chunks
     const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * 2u);
-    if (a.tb.side != 0) {
-      e = cudaFuncSetAttribute(compress_c4096_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)sizeof(FastSmem));
-      if (e != cudaSuccess) return e;
-      compress_c4096_kernel<T, true><<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
-    } else {
-      e = cudaFuncSetAttribute(compress_c4096_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)sizeof(FastSmem));
-      if (e != cudaSuccess) return e;
-      compress_c4096_kernel<T, false><<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
-    }
+    auto launch = [&](auto kernel) -> cudaError_t {
+      const cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FastSmem));
+      if (err != cudaSuccess) return err;
+      kernel<<<grid, kFastThreads, sizeof(FastSmem), st>>>(a);
+      return cudaSuccess;
+    };
+    if (a.tb.side != 0) e = launch(compress_c4096_kernel<T, true, false>);
+    else if (a.theta_bf16) e = launch(compress_c4096_kernel<T, false, true>);
+    else e = launch(compress_c4096_kernel<T, false, false>);
+    if (e != cudaSuccess) return e;
     if (a.tb.n_tails)
       compress_generic_kernel<T, true><<<a.tb.n_tails * (unsigned)a.R, kThreads, gsmem, st>>>(a);
     return cudaPeekAtLastError();

@@ -9,7 +9,8 @@ int main(void) {
   /* taking every entry point's address makes the linker resolve it */
   typedef void (*fn)(void);
   const fn fns[] = {(fn)sl_num_chunks, (fn)sl_codes_stride, (fn)sl_codes_bytes, (fn)sl_compress, (fn)sl_compress_batch, (fn)sl_aggregate,
-                    (fn)sl_outer_apply, (fn)sl_aggregate_apply, (fn)sl_outer_step, (fn)sl_idx12_stride,
+                    (fn)sl_outer_apply, (fn)sl_aggregate_apply, (fn)sl_outer_step, (fn)sl_compress_batch_bf16, (fn)sl_aggregate_apply_bf16, (fn)sl_outer_apply_bf16,
+                    (fn)sl_outer_step_bf16, (fn)sl_idx12_stride,
                     (fn)sl_pack_idx12, (fn)sl_unpack_idx12, (fn)sl_embed_reproject, (fn)sl_round_tf32, (fn)sl_subspace_project, (fn)sl_subspace_reconstruct,
                     (fn)sl_debug_set_wait_limit, (fn)sl_debug_bounds_selftest, (fn)sl_strerror};
   uint64_t offset[3] = {0, 4096 * 2 + 5, 4096 * 2 + 5 + 100};
