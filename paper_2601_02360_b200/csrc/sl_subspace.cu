@@ -487,6 +487,229 @@ subspace_project_dual_kernel(const __grid_constant__ ProjMaps maps, const __grid
   if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
+// ------------------------------------------------ compress with embedding terms, two sub-tiles per U slice
+// The same pairing for the projection WITH embedding terms: two sub-tiles of 128 tokens share every U slice
+// (128 KB instead of 160 KB taken in per K step and 256 tokens).  The gathered T_perp / position segments of
+// 256 token rows do not fit the registers of eight row warps, so this form has sixteen: thread j serves the
+// 16-byte chunk j % 8 of the rows j / 8 + 64 i (i = 0..3) of the 256-row pair - rows 0..127 are sub-tile A,
+// 128..255 sub-tile B - and keeps the values of the next K step in registers while it applies the current
+// ones.  Everything else (producers, MMA warp, ring, accumulators in the two halves of tensor memory) is the
+// kernel above.
+constexpr int kRowWarpsG = 16;
+constexpr int kThreadsG = 128 + 32 * kRowWarpsG;
+
+__global__ void __launch_bounds__(kThreadsG, 1)
+subspace_project_dual_gather_kernel(const __grid_constant__ ProjMaps maps, const __grid_constant__ SubParams p) {
+  extern __shared__ uint8_t raw[];
+  DualSmem& sm = *reinterpret_cast<DualSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t k_tiles = (p.d + kTileK - 1) / kTileK;
+  const uint64_t G = (p.n_tok + 31) / 32;
+  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  auto groups_a = [&](uint64_t g) { return (uint32_t)(g1 - g < 4 ? g1 - g : 4); };
+  auto groups_b = [&](uint64_t g) { return g + 4 >= g1 ? 0u : (uint32_t)(g1 - g - 4 < 4 ? g1 - g - 4 : 4); };
+  if (tid == 0) {
+    for (int s = 0; s < kRingD; ++s) { mbar_init(&sm.full[s], 3); mbar_init(&sm.ready[s], kRowWarpsG); mbar_init(&sm.empty[s], 1); }
+    mbar_init(&sm.p_done, 1);
+    mbar_init(&sm.p_free, kRowWarpsG);
+    mbar_init(&sm.mma_idle, 1);
+    sm.ctl.abort = 0;
+    sm.ctl.polls = p.wait_polls;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t t_p = sm.tmem_base;      // accumulator of sub-tile A; B is 256 columns further
+  bool bad = false;
+
+  if (warp == 0 || warp == 2 || warp == 3) {
+    if (lane == 0) {
+      const uint32_t pi = warp == 0 ? 0u : (uint32_t)warp - 1u;
+      const uint32_t nb = p.kp / 32;
+      const uint32_t lo = pi == 0 ? 0u : (pi * nb + 1) / 3, hi = pi == 2 ? nb : ((pi + 1) * nb + 1) / 3;
+      uint32_t it = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 8) {
+        const uint32_t ha = groups_a(g), hb = groups_b(g);
+        const int r0 = (int)(g * 32);
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRingD;
+          ok = mbar_wait(&sm.empty[s], ((it / kRingD) & 1u) ^ 1u, sm.ctl);
+          if (!ok) break;
+          uint8_t* slot = sm.ring + s * kSlotD;
+          mbar_expect_tx(&sm.full[s], (pi == 0 ? (ha + hb) * 4096 : 0u) + (hi - lo) * 4096);
+          if (pi == 0) {
+            if (ha == 4) tma_load_2d(slot, &maps.x128, (int)(kt * kTileK), r0, &sm.full[s]);
+            else
+              for (uint32_t i = 0; i < ha; ++i)
+                tma_load_2d(slot + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full[s]);
+            if (hb == 4) tma_load_2d(slot + kSlotA, &maps.x128, (int)(kt * kTileK), r0 + kRows, &sm.full[s]);
+            else
+              for (uint32_t i = 0; i < hb; ++i)
+                tma_load_2d(slot + kSlotA + i * 4096, &maps.x32, (int)(kt * kTileK), r0 + kRows + 32 * (int)i, &sm.full[s]);
+          }
+          for (uint32_t n = lo; n < hi; ++n)
+            tma_load_2d(slot + 2 * kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
+        }
+      }
+      if (!ok)
+        for (uint32_t s = 0; s < (uint32_t)kRingD; ++s) landed(&sm.full[s], ring_uses(it, s, kRingD));
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, t = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(kRows, (int)p.kp, 1);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2), desc_n = smem_desc(0, 4096, 512, 1);
+      for (uint64_t g = g0; ok && g < g1; g += 8, ++t) {
+        const bool two = groups_b(g) != 0;
+        if (t > 0) {
+          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.ctl);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRingD;
+          ok = mbar_wait(&sm.ready[s], (it / kRingD) & 1u, sm.ctl);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(sm.ring + s * kSlotD);
+          const uint64_t da = desc_k | (uint64_t)((a0 >> 4) & 0x3FFF);
+          const uint64_t da2 = desc_k | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+          const uint64_t db = desc_n | (uint64_t)(((a0 + 2 * kSlotA) >> 4) & 0x3FFF);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_ss(t_p, da + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+          if (two) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mma_ss(t_p + 256, da2 + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+          }
+          mma_commit(&sm.empty[s]);
+        }
+        if (ok) mma_commit(&sm.p_done);
+      }
+      if (!ok) mma_quiesce(&sm.mma_idle);
+    }
+  } else {
+    // ---- sixteen row warps ----
+    const uint32_t q = (uint32_t)(warp & 3), sub = (uint32_t)(warp - 4) >> 2;      // sub 0..3: tile sub & 1, column blocks sub >> 1
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    const uint32_t j = (uint32_t)(tid - 128), gch = j & 7u, grow = j >> 3;          // grow 0..63
+    const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);                  // + 8192 i: row grow + 64 i of the pair
+    const bool wide = p.k % 8 == 0 && ((uintptr_t)p.out & 31u) == 0;
+    uint32_t it = 0, t = 0;
+    bool ok = true;
+    const float* tp[4];
+    const float* ps[4];
+    uint32_t mask = 0;
+    float4 nt[4], np_[4];                           // the values of the K step after the current one
+    auto fetch = [&](uint32_t kt) {
+      const uint32_t col = kt * kTileK + 4u * gch;
+      const bool in_col = kt < k_tiles && col < p.d;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const bool in = in_col && ((mask >> i) & 1u);
+        nt[i] = in ? __ldg(reinterpret_cast<const float4*>(tp[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        np_[i] = in ? __ldg(reinterpret_cast<const float4*>(ps[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    auto open_tile = [&](uint64_t g) {
+      const uint32_t ha = groups_a(g) * 32, hb = groups_b(g) * 32;
+      mask = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t r = grow + 64u * (uint32_t)i;                                 // row of the pair
+        const RowInfo ri = r < (uint32_t)kRows ? row_info(p, g * 32, ha, r, bad) : row_info(p, g * 32 + kRows, hb, r - kRows, bad);
+        tp[i] = ri.gather ? ri.tp + 4 * gch : nullptr;
+        ps[i] = ri.gather ? ri.ps + 4 * gch : nullptr;
+        mask |= ri.gather ? 1u << i : 0u;
+      }
+      fetch(0);
+    };
+    if (g0 < g1) open_tile(g0);
+    for (uint64_t g = g0; ok && g < g1; g += 8, ++t) {
+      const uint32_t ha = groups_a(g), hb = groups_b(g);
+      for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+        float4 ct[4], cp[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { ct[i] = nt[i]; cp[i] = np_[i]; }
+        fetch(kt + 1);
+        const uint32_t s = it % kRingD;
+        ok = mbar_wait(&sm.full[s], (it / kRingD) & 1u, sm.ctl);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t a0 = smem_u32(sm.ring + s * kSlotD) + goff;
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) {
+          if (i < 2 || hb) {                        // rows 128.. exist only with a second sub-tile
+            const uint32_t a = a0 + 8192u * i;
+            float4 v = lds128(a);
+            v.x = __fsub_rn(__fsub_rn(v.x, ct[i].x), cp[i].x);
+            v.y = __fsub_rn(__fsub_rn(v.y, ct[i].y), cp[i].y);
+            v.z = __fsub_rn(__fsub_rn(v.z, ct[i].z), cp[i].z);
+            v.w = __fsub_rn(__fsub_rn(v.w, ct[i].w), cp[i].w);
+            v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+            v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+            v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+            v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+            sts128(a, v);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ready[s]);
+      }
+      if (!ok) break;
+      if (g + 8 < g1) open_tile(g + 8);
+      ok = mbar_wait(&sm.p_done, t & 1u, sm.ctl);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        const uint32_t tile = sub & 1u;
+        const uint32_t h = (tile ? hb : ha) * 32;
+        const uint64_t r0 = g * 32 + (uint64_t)tile * kRows;
+        if (h) {
+          for (uint32_t cb = 32u * (sub >> 1); cb < p.kp; cb += 64) {
+            uint32_t v[32];
+            tmem_ld32(t_p + tile * 256 + cb + ((32u * q) << 16), v);
+            tmem_ld_wait();
+            if (row < h && r0 + row < p.n_tok) {
+              float* dst = p.out + (r0 + row) * (uint64_t)p.k + cb;
+              if (wide) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 8)
+                  if (cb + (uint32_t)i < p.k) stg256(dst + i, v + i);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                  if (cb + (uint32_t)i < p.k)
+                    *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                      __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.p_free);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_p), "r"(512) : "memory");
+  }
+  if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+  if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
 // --------------------------------------------------------------------------------------- reconstruct
 // Per sub-tile of 128 tokens the Xt tile goes through a two-slot staging buffer into tensor memory
 // (rounded to TF32 on the way) and is the A operand of every 128-column block.  The embedding and
@@ -868,9 +1091,15 @@ cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const fl
   cudaError_t e;
   const unsigned grid = persistent_grid(n_tok, &e);
   if (e != cudaSuccess) return e;
-  if (!ids && (n_tok + kRows - 1) / kRows >= 2ull * grid) {
-    // no embedding terms and at least two sub-tiles for every CTA: two sub-tiles share every U slice
+  if ((n_tok + kRows - 1) / kRows >= 2ull * grid) {
+    // at least two sub-tiles for every CTA: two sub-tiles share every U slice
     const int smem = (int)sizeof(DualSmem) + 1024;
+    if (ids) {
+      e = cudaFuncSetAttribute(subspace_project_dual_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      if (e != cudaSuccess) return e;
+      subspace_project_dual_gather_kernel<<<grid, kThreadsG, smem, st>>>(m, p);
+      return cudaGetLastError();
+    }
     e = cudaFuncSetAttribute(subspace_project_dual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     subspace_project_dual_kernel<<<grid, kThreads, smem, st>>>(m, p);
