@@ -397,6 +397,121 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
 
+// Fused average + update for FEW entries per chunk (R * k <= 256, one per thread), consecutive chunks,
+// float32 parameters, outer_lr > 0.  An element no replica sent has the mean update +0, and
+// theta - outer_lr * (+0) is theta itself, bit for bit: for outer_lr > 0 the product is -0 and x + (-0) = x
+// for every x, both zeros included (and a position's sum starts from +0, so it is never -0).  So
+// theta_global is neither read nor rewritten as a whole: only the elements some replica sent are loaded,
+// updated and stored - about a fifth of the chunk's 32-byte sectors at R * k = 128 instead of all 16 KB
+// twice.  Thread q owns slot q % k of replica q / k.  Software pipeline over the CTA's chunks: the raw
+// entries of chunk i+2 are requested, the entries of chunk i+1 are decoded and the theta_global elements
+// they name are requested, and chunk i - whose elements arrived an iteration ago - is processed:
+//   every entry clears its accumulator cell; then one round per replica in the order 0..R-1 adds its
+//   values (positions inside a message are distinct, so a round has no conflicts; a bit map tells an
+//   entry whether an earlier replica already named its position); then the FIRST entry of every position
+//   divides the finished sum by R, applies the fused step to the element it loaded, and stores it.
+constexpr int kSparseMaxEntries = 256;
+
+struct SparseSmem {
+  float acc[kAC];
+  uint32_t seen[kAC / 32];
+};
+
+template <int T>
+__global__ void __launch_bounds__(kThreads)
+aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
+  __shared__ SparseSmem sm;
+  const int tid = threadIdx.x;
+  const int k = a.k, bits = a.bits, R = a.R;
+  const uint64_t n_total = a.tb.offset[a.tb.n_tensors];
+  (void)n_total;
+  const int my_r = tid < R * k ? tid / k : -1;
+  const int my_j = my_r >= 0 ? tid - my_r * k : 0;
+  const uint16_t* p_idx = my_r >= 0 ? a.m.idx[my_r] + my_j : nullptr;
+  const uint32_t bit0 = (uint32_t)my_j * (uint32_t)bits;
+  const uint8_t* p_code = my_r >= 0 ? (bits == 32 ? a.m.codes[my_r] + 4 * (size_t)my_j : a.m.codes[my_r] + (bit0 >> 3)) : nullptr;
+  const float* p_scale = my_r >= 0 ? a.m.scales[my_r] : nullptr;
+  const uint32_t cshift = bit0 & 7u, cmask = bits == 32 ? 0xFFFFFFFFu : (1u << bits) - 1u;
+  const bool pow2 = (R & (R - 1)) == 0;
+  const float Rf = (float)R, invR = 1.0f / Rf, nlr = -a.outer_lr;
+  bool bad = false;
+  if (tid < kAC / 32) sm.seen[tid] = 0;
+  __syncthreads();
+
+  struct Raw { uint32_t pos, code; float scale; };
+  auto fetch = [&](uint32_t g) {
+    Raw w{0xFFFFu, 0u, 0.0f};
+    if (my_r >= 0 && SL_CHECK(a.flags, g < a.tb.n_chunks)) {
+      w.pos = __ldg(p_idx + (uint64_t)g * (uint64_t)k);
+      if (bits == 32) {
+        w.code = __float_as_uint(__ldg(reinterpret_cast<const float*>(p_code + (uint64_t)g * (uint64_t)a.stride)));
+      } else {
+        w.code = (uint32_t)__ldg(p_code + (uint64_t)g * (uint64_t)a.stride);
+        w.scale = __ldg(p_scale + g);
+      }
+    }
+    return w;
+  };
+  // the chunks of this CTA, three in flight: A is processed, B is decoded, C is fetched
+  uint32_t gA = blockIdx.x, gB, gC, t_lo = 0, strideA = 64, strideB = 64, strideC = 64;
+  uint64_t baseA = 0, baseB = 0, baseC = 0;
+  bool vA = next_full_chunk(a.tb, gA, gridDim.x, t_lo, baseA, strideA);
+  gB = gA + gridDim.x;
+  bool vB = vA && next_full_chunk(a.tb, gB, gridDim.x, t_lo, baseB, strideB);
+  gC = gB + gridDim.x;
+  bool vC = vB && next_full_chunk(a.tb, gC, gridDim.x, t_lo, baseC, strideC);
+  (void)strideA; (void)strideB; (void)strideC;
+  // decoded entry of a chunk: position (0xFFFF: none), value, and the element of theta_global it names
+  auto decode = [&](const Raw& w, uint64_t base, uint32_t& pos, float& val, float& th) {
+    pos = 0xFFFFu; val = 0.0f; th = 0.0f;
+    if (my_r < 0 || w.pos == 0xFFFFu) return;
+    if (w.pos >= (uint32_t)kAC) { bad = true; return; }
+    if (!SL_CHECK(a.flags, base + w.pos < n_total)) return;
+    pos = w.pos;
+    val = bits == 32 ? __uint_as_float(w.code) : dequant((w.code >> cshift) & cmask, w.scale, bits);
+    th = __ldcg(a.out + base + pos);
+  };
+  Raw rawB{0xFFFFu, 0u, 0.0f}, rawC{0xFFFFu, 0u, 0.0f};
+  uint32_t posA = 0xFFFFu;
+  float valA = 0.0f, thA = 0.0f;
+  if (vA) { const Raw rawA = fetch(gA); decode(rawA, baseA, posA, valA, thA); }
+  if (vB) rawB = fetch(gB);
+  while (vA) {
+    if (vC) rawC = fetch(gC);
+    uint32_t posB = 0xFFFFu;
+    float valB = 0.0f, thB = 0.0f;
+    if (vB) decode(rawB, baseB, posB, valB, thB);
+    // ---- chunk A ----
+    const bool have = posA != 0xFFFFu;
+    const uint32_t word = posA >> 5, bit = 1u << (posA & 31u);
+    if (have) sm.acc[posA] = 0.0f;
+    __syncthreads();
+    bool first = false;
+    for (int r = 0; r < R; ++r) {
+      if (have && my_r == r) {
+        first = (atomicOr(&sm.seen[word], bit) & bit) == 0;
+        sm.acc[posA] = __fadd_rn(sm.acc[posA], valA);
+      }
+      __syncthreads();
+    }
+    if (have && first) {
+      const float sum = sm.acc[posA];
+      const float u = pow2 ? __fmul_rn(sum, invR) : __fdiv_rn(sum, Rf);
+      a.out[baseA + posA] = __fmaf_rn(nlr, u, thA);
+      atomicAnd(&sm.seen[word], ~bit);
+    }
+    __syncthreads();                               // cells and bits are free for the next chunk
+    // ---- shift the pipeline ----
+    posA = posB; valA = valB; thA = thB; baseA = baseB; vA = vB;
+    rawB = rawC; baseB = baseC; vB = vC;
+    if (vC) {
+      gC += gridDim.x;
+      vC = next_full_chunk(a.tb, gC, gridDim.x, t_lo, baseC, strideC);
+    }
+  }
+  if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+}
+
 template <int T, bool APPLY>
 cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
   cudaError_t e;
@@ -429,6 +544,15 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
                    : launch(aggregate_c4096_kernel<T, APPLY, 8, true, false>);
   }
   if constexpr (APPLY) {
+    if (!a.theta_bf16 && a.tb.side == 0 && a.outer_lr > 0.0f && a.R * a.k <= kSparseMaxEntries) {
+      int per_sm = 0;
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aggregate_sparse_kernel<T>, kThreads, 0);
+      if (e != cudaSuccess) return e;
+      if (per_sm < 1) per_sm = 1;
+      const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * (uint64_t)per_sm);
+      aggregate_sparse_kernel<T><<<grid, kThreads, 0, st>>>(a);
+      return cudaPeekAtLastError();
+    }
     if (a.theta_bf16) {
       if (np == 1) return launch(aggregate_c4096_kernel<T, true, 1, false, false, true>);
       if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, true, 2, false, true, true>)

@@ -645,3 +645,24 @@ def test_random_configurations(seed):
     run_and_compare(off, tg, tls, errs, beta, chunk, k, bits, 0.8, rounds=2, next_locals=nxt,
                     what=f"random #{seed}: chunk {chunk} k {k} b {bits} R {R} tiled {tiled} align {align}",
                     fused=bool(seed % 2), cols=cols if tiled else None)
+
+
+@pytest.mark.parametrize("lr", [0.8, 1.0, -0.5, 0.0])
+@pytest.mark.parametrize("R,k", [(2, 64), (1, 128), (4, 64), (2, 16), (5, 64)])
+def test_theta_global_update_touches_only_what_was_sent(R, k, lr):
+    # with few entries per chunk and a positive step the averaging kernel updates only the elements some
+    # replica sent; every other element must keep its bits - signed zeros included - exactly as the
+    # dense form theta - lr * 0 leaves them, and a negative or zero step takes the dense form
+    sizes = [40 * 4096, 2048, 3 * 4096]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), R, seed=R * 100 + k)
+    rng = np.random.default_rng(7)
+    z = rng.choice(tg.size, size=tg.size // 5, replace=False)
+    tg[z[: len(z) // 2]] = 0.0
+    tg[z[len(z) // 2:]] = -0.0
+    if R >= 2:                       # replica 1 mirrors replica 0 around theta_global on the first chunks: sums that cancel to +0
+        tls[1][:8 * 4096] = (2 * tg[:8 * 4096] - tls[0][:8 * 4096]).astype(f32)
+        errs[1][:8 * 4096] = -errs[0][:8 * 4096]
+    gs, tg_o, _ = run_and_compare(off, tg, tls, errs, 0.95, 4096, k, 2, lr, what=f"sparse update R{R} k{k} lr{lr}")
+    got = gs.theta_global.cpu().numpy()
+    assert np.array_equal(np.signbit(got), np.signbit(tg_o)), "a signed zero changed its sign"

@@ -37,7 +37,7 @@ def _arena(R, seed):
 
 @pytest.mark.parametrize("polls", [-1, 1])
 def test_compress_and_aggregate_give_up_cleanly(wait_limit, polls):
-    R, chunk, k, bits, beta, lr = 3, 4096, 64, 2, 0.95, 0.8
+    R, chunk, k, bits, beta, lr = 5, 4096, 64, 2, 0.95, 0.8      # R * k = 320: the averaging kernel that prefetches theta_global
     off, tg, tls, errs = _arena(R, 11)
     gs = GpuStep(off, R, chunk, k, bits)
     gs.upload(tg, tls, errs)
