@@ -39,6 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of compress_c4096_kernel on the captured small case
 # (51,384,320 parameters x 8 replicas, k = 64, 2-bit codes), per replica-parameter
 COMPRESS_DRAM_BYTES_PER_REPLICA_PARAM = 12.43
+MIN_ROW_SECONDS = 1.0          # a row of short launches runs at least this long, so that nvidia-smi (100 ms period) samples it
 KERNEL_LAUNCHES_PER_STEP = 4   # compress (full chunks, tails) + aggregate-apply (full chunks, tails)
 
 
@@ -758,7 +759,9 @@ def row_embed(wl: synth.Workload, seed: int, dev, peak: float, launches: int, k:
     sampler = ClockSampler(dev.index or 0)
     times = []
     sampler.start()
-    for s in range(5 + launches):
+    t_begin, s = time.perf_counter(), -1
+    while s + 1 < 5 + launches or time.perf_counter() - t_begin < MIN_ROW_SECONDS:   # long enough for the clock sampler
+        s += 1
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         T_S.copy_(T_S0)
@@ -792,7 +795,9 @@ def row_subspace(wl: synth.Workload, seed: int, dev, peak: float, launches: int,
         sampler = ClockSampler(dev.index or 0)
         t_p, t_r = [], []
         sampler.start()
-        for s in range(5 + launches):
+        t_begin, s = time.perf_counter(), -1
+        while s + 1 < 5 + launches or time.perf_counter() - t_begin < MIN_ROW_SECONDS:
+            s += 1
             torch.cuda.synchronize()
             e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
             flush.fill_(float(s))
