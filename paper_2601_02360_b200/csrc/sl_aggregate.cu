@@ -404,10 +404,12 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
 // theta - outer_lr * (+0) is theta itself, bit for bit: for outer_lr > 0 the product is -0 and x + (-0) = x
 // for every x, both zeros included (and a position's sum starts from +0, so it is never -0).  So
 // theta_global is neither read nor rewritten as a whole: only the elements some replica sent are loaded,
-// updated and stored - about a fifth of the chunk's 32-byte sectors at R * k = 128 instead of all 16 KB
-// twice.  Thread q owns slot q % k of replica q / k.  Software pipeline over the CTA's chunks: the raw
-// entries of chunk i+2 are requested, the entries of chunk i+1 are decoded and the theta_global elements
-// they name are requested, and chunk i - whose elements arrived an iteration ago - is processed:
+// updated and stored instead of all 16 KB twice.  Thread q owns slot q % k of replica q / k.  Software pipeline over the group's chunks, three in
+// flight (deeper ones were no faster: the launch is bound by DRAM, which moves 64 bytes for every element
+// read and as much for every element written back, about 16 KB per chunk at R * k = 128 - half of the dense
+// form, not a fifth): raw entries are requested two chunks ahead, one chunk ahead they are decoded and the
+// theta_global elements they name are requested, and the oldest chunk - whose elements arrived an
+// iteration ago - is processed:
 //   every entry clears its accumulator cell; then one round per replica in the order 0..R-1 adds its
 //   values (positions inside a message are distinct, so a round has no conflicts; a bit map tells an
 //   entry whether an earlier replica already named its position); then the FIRST entry of every position
@@ -419,11 +421,19 @@ struct SparseSmem {
   uint32_t seen[kAC / 32];
 };
 
-template <int T>
+// GROUPS: with R * k <= 256 / GROUPS entries per chunk the CTA's threads form GROUPS independent groups, each
+// walking its own chunks with its own accumulator, bit map and named barrier (the launch is bound by the
+// barriers of a chunk, so smaller groups on more chunks at once are faster).
+template <int T, int GROUPS>
 __global__ void __launch_bounds__(kThreads)
 aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
-  __shared__ SparseSmem sm;
-  const int tid = threadIdx.x;
+  extern __shared__ __align__(16) unsigned char sparse_smem_raw[];
+  constexpr int GT = kThreads / GROUPS;            // threads of a group (a multiple of 32)
+  const int gidx = (int)threadIdx.x / GT;
+  SparseSmem& sm = reinterpret_cast<SparseSmem*>(sparse_smem_raw)[gidx];
+  const int tid = (int)threadIdx.x - gidx * GT;    // index inside the group = the entry this thread owns
+  const uint32_t vcta = blockIdx.x * GROUPS + gidx, vgrid = gridDim.x * GROUPS;    // the group as a CTA of a larger grid
+  auto group_sync = [&]() { if (GROUPS == 1) __syncthreads(); else named_sync(1 + gidx, GT); };
   const int k = a.k, bits = a.bits, R = a.R;
   const uint64_t n_total = a.tb.offset[a.tb.n_tensors];
   (void)n_total;
@@ -437,8 +447,8 @@ aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
   const bool pow2 = (R & (R - 1)) == 0;
   const float Rf = (float)R, invR = 1.0f / Rf, nlr = -a.outer_lr;
   bool bad = false;
-  if (tid < kAC / 32) sm.seen[tid] = 0;
-  __syncthreads();
+  for (int i = tid; i < kAC / 32; i += GT) sm.seen[i] = 0;
+  group_sync();
 
   struct Raw { uint32_t pos, code; float scale; };
   auto fetch = [&](uint32_t g) {
@@ -454,62 +464,75 @@ aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
     }
     return w;
   };
-  // the chunks of this CTA, three in flight: A is processed, B is decoded, C is fetched
-  uint32_t gA = blockIdx.x, gB, gC, t_lo = 0, strideA = 64, strideB = 64, strideC = 64;
-  uint64_t baseA = 0, baseB = 0, baseC = 0;
-  bool vA = next_full_chunk(a.tb, gA, gridDim.x, t_lo, baseA, strideA);
-  gB = gA + gridDim.x;
-  bool vB = vA && next_full_chunk(a.tb, gB, gridDim.x, t_lo, baseB, strideB);
-  gC = gB + gridDim.x;
-  bool vC = vB && next_full_chunk(a.tb, gC, gridDim.x, t_lo, baseC, strideC);
-  (void)strideA; (void)strideB; (void)strideC;
   // decoded entry of a chunk: position (0xFFFF: none), value, and the element of theta_global it names
-  auto decode = [&](const Raw& w, uint64_t base, uint32_t& pos, float& val, float& th) {
-    pos = 0xFFFFu; val = 0.0f; th = 0.0f;
-    if (my_r < 0 || w.pos == 0xFFFFu) return;
-    if (w.pos >= (uint32_t)kAC) { bad = true; return; }
-    if (!SL_CHECK(a.flags, base + w.pos < n_total)) return;
-    pos = w.pos;
-    val = bits == 32 ? __uint_as_float(w.code) : dequant((w.code >> cshift) & cmask, w.scale, bits);
-    th = __ldcg(a.out + base + pos);
+  struct Dec { uint32_t pos; float val, th; };
+  auto decode = [&](const Raw& w, uint64_t base) {
+    Dec d{0xFFFFu, 0.0f, 0.0f};
+    if (my_r < 0 || w.pos == 0xFFFFu) return d;
+    if (w.pos >= (uint32_t)kAC) { bad = true; return d; }
+    if (!SL_CHECK(a.flags, base + w.pos < n_total)) return d;
+    d.pos = w.pos;
+    d.val = bits == 32 ? __uint_as_float(w.code) : dequant((w.code >> cshift) & cmask, w.scale, bits);
+    d.th = __ldcg(a.out + base + d.pos);
+    return d;
   };
-  Raw rawB{0xFFFFu, 0u, 0.0f}, rawC{0xFFFFu, 0u, 0.0f};
-  uint32_t posA = 0xFFFFu;
-  float valA = 0.0f, thA = 0.0f;
-  if (vA) { const Raw rawA = fetch(gA); decode(rawA, baseA, posA, valA, thA); }
-  if (vB) rawB = fetch(gB);
-  while (vA) {
-    if (vC) rawC = fetch(gC);
-    uint32_t posB = 0xFFFFu;
-    float valB = 0.0f, thB = 0.0f;
-    if (vB) decode(rawB, baseB, posB, valB, thB);
-    // ---- chunk A ----
+  // The group's chunks in flight, oldest first: stage 0 is processed in this iteration, stages 1..kDec hold
+  // decoded entries whose theta_global elements are on their way, the last kRaw stages raw entries on their way.
+  constexpr int kDec = 1, kRaw = 1, kStagesInFlight = 1 + kDec + kRaw;
+  uint64_t base_q[kStagesInFlight];
+  bool valid_q[kStagesInFlight];
+  Dec dec_q[1 + kDec];
+  Raw raw_q[kRaw];
+  uint32_t g_next = vcta, t_lo = 0, stride_unused = 64;
+  bool more = true;
+#pragma unroll
+  for (int i = 0; i < kStagesInFlight; ++i) {
+    base_q[i] = 0;
+    valid_q[i] = more && next_full_chunk(a.tb, g_next, vgrid, t_lo, base_q[i], stride_unused);
+    more = valid_q[i];
+    if (i <= kDec) {
+      dec_q[i] = Dec{0xFFFFu, 0.0f, 0.0f};
+      if (valid_q[i]) dec_q[i] = decode(fetch(g_next), base_q[i]);
+    } else {
+      raw_q[i - 1 - kDec] = Raw{0xFFFFu, 0u, 0.0f};
+      if (valid_q[i]) raw_q[i - 1 - kDec] = fetch(g_next);
+    }
+    if (valid_q[i]) g_next += vgrid;
+  }
+  while (valid_q[0]) {
+    // ---- the oldest chunk ----
+    const uint32_t posA = dec_q[0].pos;
     const bool have = posA != 0xFFFFu;
     const uint32_t word = posA >> 5, bit = 1u << (posA & 31u);
     if (have) sm.acc[posA] = 0.0f;
-    __syncthreads();
+    group_sync();
     bool first = false;
     for (int r = 0; r < R; ++r) {
       if (have && my_r == r) {
         first = (atomicOr(&sm.seen[word], bit) & bit) == 0;
-        sm.acc[posA] = __fadd_rn(sm.acc[posA], valA);
+        sm.acc[posA] = __fadd_rn(sm.acc[posA], dec_q[0].val);
       }
-      __syncthreads();
+      group_sync();
     }
     if (have && first) {
       const float sum = sm.acc[posA];
       const float u = pow2 ? __fmul_rn(sum, invR) : __fdiv_rn(sum, Rf);
-      a.out[baseA + posA] = __fmaf_rn(nlr, u, thA);
+      a.out[base_q[0] + posA] = __fmaf_rn(nlr, u, dec_q[0].th);
       atomicAnd(&sm.seen[word], ~bit);
     }
-    __syncthreads();                               // cells and bits are free for the next chunk
-    // ---- shift the pipeline ----
-    posA = posB; valA = valB; thA = thB; baseA = baseB; vA = vB;
-    rawB = rawC; baseB = baseC; vB = vC;
-    if (vC) {
-      gC += gridDim.x;
-      vC = next_full_chunk(a.tb, gC, gridDim.x, t_lo, baseC, strideC);
-    }
+    group_sync();                                  // cells and bits are free for the next chunk
+    // ---- shift: the oldest raw stage is decoded (its theta_global elements are requested), a new chunk is fetched ----
+#pragma unroll
+    for (int i = 0; i < kDec; ++i) dec_q[i] = dec_q[i + 1];
+#pragma unroll
+    for (int i = 0; i + 1 < kStagesInFlight; ++i) { base_q[i] = base_q[i + 1]; valid_q[i] = valid_q[i + 1]; }
+    dec_q[kDec] = Dec{0xFFFFu, 0.0f, 0.0f};
+    if (valid_q[kDec]) dec_q[kDec] = decode(raw_q[0], base_q[kDec]);
+#pragma unroll
+    for (int i = 0; i + 1 < kRaw; ++i) raw_q[i] = raw_q[i + 1];
+    valid_q[kStagesInFlight - 1] = more && next_full_chunk(a.tb, g_next, vgrid, t_lo, base_q[kStagesInFlight - 1], stride_unused);
+    more = valid_q[kStagesInFlight - 1];
+    if (more) { raw_q[kRaw - 1] = fetch(g_next); g_next += vgrid; }
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
@@ -547,13 +570,23 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
   }
   if constexpr (APPLY) {
     if (!a.theta_bf16 && a.tb.side == 0 && a.outer_lr > 0.0f && a.R * a.k <= kSparseMaxEntries) {
-      int per_sm = 0;
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aggregate_sparse_kernel<T>, kThreads, 0);
-      if (e != cudaSuccess) return e;
-      if (per_sm < 1) per_sm = 1;
-      const unsigned grid = (unsigned)std::min<uint64_t>((uint64_t)a.tb.n_chunks, (uint64_t)sms * (uint64_t)per_sm);
-      aggregate_sparse_kernel<T><<<grid, kThreads, 0, st>>>(a);
-      return cudaPeekAtLastError();
+      auto launch_sparse = [&](auto kernel, int groups) -> cudaError_t {
+        const size_t sm_bytes = sizeof(SparseSmem) * (size_t)groups;
+        cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_bytes);
+        if (err != cudaSuccess) return err;
+        int per_sm = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, sm_bytes);
+        if (err != cudaSuccess) return err;
+        if (per_sm < 1) per_sm = 1;
+        const uint64_t want = ((uint64_t)a.tb.n_chunks + groups - 1) / groups;
+        const unsigned grid = (unsigned)std::min<uint64_t>(want, (uint64_t)sms * (uint64_t)per_sm);
+        kernel<<<grid, kThreads, sm_bytes, st>>>(a);
+        return cudaPeekAtLastError();
+      };
+      const int entries = a.R * a.k;
+      if (entries <= 64) return launch_sparse(aggregate_sparse_kernel<T, 4>, 4);
+      if (entries <= 128) return launch_sparse(aggregate_sparse_kernel<T, 2>, 2);
+      return launch_sparse(aggregate_sparse_kernel<T, 1>, 1);
     }
     if (a.theta_bf16) {
       if (np == 1) return launch(aggregate_c4096_kernel<T, true, 1, false, false, true>);

@@ -648,7 +648,7 @@ def test_random_configurations(seed):
 
 
 @pytest.mark.parametrize("lr", [0.8, 1.0, -0.5, 0.0])
-@pytest.mark.parametrize("R,k", [(2, 64), (1, 128), (4, 64), (2, 16), (5, 64)])
+@pytest.mark.parametrize("R,k", [(2, 64), (1, 128), (4, 64), (2, 16), (5, 64), (2, 32), (3, 20), (1, 7)])
 def test_theta_global_update_touches_only_what_was_sent(R, k, lr):
     # with few entries per chunk and a positive step the averaging kernel updates only the elements some
     # replica sent; every other element must keep its bits - signed zeros included - exactly as the
