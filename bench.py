@@ -40,6 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (51,384,320 parameters x 8 replicas, k = 64, 2-bit codes), per replica-parameter
 COMPRESS_DRAM_BYTES_PER_REPLICA_PARAM = 12.43
 MIN_ROW_SECONDS = 1.0          # a row of short launches runs at least this long, so that nvidia-smi (100 ms period) samples it
+E2E_GROUPS = 24               # tensor groups of the host-buffer step (hoststep.outer_step_from_host)
 KERNEL_LAUNCHES_PER_STEP = 4   # compress (full chunks, tails) + aggregate-apply (full chunks, tails)
 
 
@@ -389,9 +390,11 @@ def host_memory_available() -> int:
 
 
 def run_e2e(st: DeviceState, steps: int, world: int):
-    """The same step with HOST inputs and outputs: every step copies the replicas' parameters
-    from pinned host memory to the device, runs the two calls, and reads the messages and the
-    new theta_global back.  Returns (ms per step, h2d bytes, d2h bytes, note)."""
+    """The same step with HOST inputs and outputs through the package's host-buffer call
+    (hoststep.outer_step_from_host): every step copies the replicas' parameters from pinned host memory to
+    the device, runs Eq. 2, and reads the messages and the new theta_global back, group of tensors by group
+    of tensors so that the copies in, the kernels and the copies out overlap.  Returns (ms per step, h2d
+    bytes, d2h bytes, note)."""
     wl = st.wl
     n = wl.n_total
     need = n * 4
@@ -406,6 +409,11 @@ def run_e2e(st: DeviceState, steps: int, world: int):
     torch.cuda.synchronize()
     h2d = wl.R * n * 4
     d2h = n * 4 + sum(t.numel() * t.element_size() for grp in host_msgs for t in grp)
+    from paper_2601_02360_b200 import hoststep
+    cols = None if st.layout.cols is None else st.layout.cols
+    groups = hoststep.plan_groups(wl.offsets(), wl.chunk, E2E_GROUPS, cols)
+    streams = hoststep.HostStepStreams(st.dev)
+    host_list = [host_tl[r % pool] for r in range(wl.R)]
     times = []
     for s in range(steps + 1):
         barrier(world)
@@ -413,19 +421,15 @@ def run_e2e(st: DeviceState, steps: int, world: int):
         e0 = torch.cuda.Event(enable_timing=True)
         e1 = torch.cuda.Event(enable_timing=True)
         e0.record()
-        for r in range(wl.R):
-            st.theta_local[r].copy_(host_tl[r % pool], non_blocking=True)
-        st.compress()
-        for grp_d, grp_h in zip((st.idx, st.codes, st.scales), host_msgs):
-            for d, h in zip(grp_d, grp_h):
-                h.copy_(d, non_blocking=True)
-        st.aggregate_apply()
-        host_tg.copy_(st.theta_global, non_blocking=True)
+        hoststep.outer_step_from_host(host_list, st.theta_local, st.theta_global, st.err, groups, wl.beta, wl.chunk,
+                                      wl.k, wl.bits, wl.outer_lr, st.idx, st.codes, st.scales, host_tg, host_msgs,
+                                      st.flags, streams)
         e1.record()
         torch.cuda.synchronize()
         if s > 0:   # the first pass warms the pinned pages and the copy engines
             times.append(e0.elapsed_time(e1))
-    note = f"pinned pool of {pool} distinct replica buffers" + ("" if pool == wl.R else f" reused for R={wl.R}")
+    note = (f"hoststep.outer_step_from_host over {len(groups)} tensor groups (copies in, kernels and copies out overlap); "
+            f"pinned pool of {pool} distinct replica buffers" + ("" if pool == wl.R else f" reused for R={wl.R}"))
     del host_tl, host_tg, host_msgs
     return float(np.mean(times)), h2d, d2h, note
 
