@@ -941,6 +941,15 @@ def run_ours(args) -> None:
         "clocks": clocks, "device_flags": flags,
         "gpu_launches": KERNEL_LAUNCHES_PER_STEP * args.steps,
     }
+    if wl.variant != "plain":
+        # how hard the tie-breaking is exercised: chunks of the first tensor whose k-th and (k+1)-th largest
+        # pseudo-gradient magnitudes are equal (a fresh draw, error buffers left out)
+        st.redraw_locals(10 ** 6)
+        n0 = (wl.sizes[0] // wl.chunk) * wl.chunk
+        dlt = (st.theta_global[:n0] - st.theta_local[0][:n0]).abs().view(-1, wl.chunk)
+        top = torch.topk(dlt, wl.k + 1, dim=1).values
+        line["config"]["tie_fraction"] = float((top[:, wl.k - 1] == top[:, wl.k]).float().mean())
+        del dlt, top
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu:
