@@ -863,7 +863,7 @@ def run_ours(args) -> None:
         wl = wl.replace(variant=args.variant)
     if args.first_tensors:
         wl = synth.sub_arena(wl, list(range(args.first_tensors)), f"{wl.name}[:{args.first_tensors}]")
-    st = DeviceState(wl, rank_seed(args.seed, rank), dev, tiles=args.tiles)
+    st = DeviceState(wl, rank_seed(args.seed, rank), dev, tiles=args.tiles, bf16=args.bf16)
     stream = torch.cuda.current_stream()
 
     sampler = ClockSampler(local)
@@ -906,11 +906,14 @@ def run_ours(args) -> None:
     step_ms = float(np.mean(t_step))
     comp_ms = float(np.mean(t_comp))
     agg_ms = float(np.mean(t_agg))
-    achieved = compress_bytes(wl) / (comp_ms * 1e-3) / 1e9
-    strict = step_bytes_strict(wl) / (step_ms * 1e-3) / 1e9
+    # bfloat16 parameters: theta_local 2 instead of 4 bytes per replica-parameter, theta_global 2 + 2 instead of 4 + 4
+    comp_bytes = compress_bytes(wl) - (wl.n_total * (2 * wl.R + 2) if args.bf16 else 0)
+    strict_bytes = step_bytes_strict(wl) - (wl.n_total * (2 * wl.R + 4) if args.bf16 else 0)
+    achieved = comp_bytes / (comp_ms * 1e-3) / 1e9
+    strict = strict_bytes / (step_ms * 1e-3) / 1e9
     # ncu DRAM bytes of the tuned compress launch on the small capture (profiles/), per
     # replica-parameter, scaled to this launch's units
-    traffic = COMPRESS_DRAM_BYTES_PER_REPLICA_PARAM * wl.n_total * wl.R if wl.chunk == 4096 else None
+    traffic = COMPRESS_DRAM_BYTES_PER_REPLICA_PARAM * wl.n_total * wl.R if wl.chunk == 4096 and not args.bf16 else None
     line = {
         "metric": METRIC, "value": job_value(wl.n_total, world, ms_per_step), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
@@ -920,6 +923,7 @@ def run_ours(args) -> None:
                    "chunks": wl.n_chunks(), "R": wl.R, "k": wl.k, "bits": wl.bits, "chunk": wl.chunk,
                    "beta": wl.beta, "outer_lr": wl.outer_lr, "variant": wl.variant,
                    "geometry": "64x64 tiles of each matrix" if args.tiles else "consecutive chunks",
+                   "parameters": "bfloat16, float32 error buffers" if args.bf16 else "float32",
                    "l2": "inputs (GBs per launch) far larger than the 126 MB L2; no flush needed",
                    "sharding": "none: every rank runs an independent parameter set" if world > 1 else "single GPU",
                    "step": "sl_compress_batch + sl_aggregate_apply; theta_local re-drawn between steps (untimed)"},
@@ -929,9 +933,9 @@ def run_ours(args) -> None:
                      "traffic_source": ("ncu dram__bytes_read.sum + dram__bytes_write.sum of this kernel on the "
                                         "51.4 M-parameter x 8-replica case (profiles/compress_c4096_1b_layer0.md), "
                                         "scaled by N*R; a constant, not re-captured by this run") if traffic else None,
-                     "peak_source": peak_src, "algorithmic_bytes": compress_bytes(wl),
+                     "peak_source": peak_src, "algorithmic_bytes": comp_bytes,
                      "launch_ms": comp_ms},
-        "step_hbm": {"bytes_strict": step_bytes_strict(wl), "gbs_strict": strict, "frac_of_peak": strict / peak,
+        "step_hbm": {"bytes_strict": strict_bytes, "gbs_strict": strict, "frac_of_peak": strict / peak,
                      "frac_of_8tbs_nominal": strict / 8000.0,
                      # per-call count: every replica's compress re-reads theta_global, as on R separate machines
                      "bytes_api": step_bytes_api(wl), "gbs_api": step_bytes_api(wl) / (step_ms * 1e-3) / 1e9,
@@ -976,7 +980,7 @@ def run_ours(args) -> None:
             dt = time.perf_counter() - t0
             line["cpu_baseline_1core"] = {"value": n1 / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "ms": dt * 1e3,
                                           "sample": f"first 2 tensors ({n1} params) x R={wl.R}, one outer step, one host thread"}
-    plain_default = not (args.tiles or args.R or args.k or args.bits or args.first_tensors or args.variant != "plain")
+    plain_default = not (args.bf16 or args.tiles or args.R or args.k or args.bits or args.first_tensors or args.variant != "plain")
     if world == 1 and not args.no_rows and wl.name == "1b" and plain_default:
         del st
         line["rows"] = measured_rows(args, wl, dev, peak)
@@ -1016,6 +1020,8 @@ def main() -> None:
     ap.add_argument("--tokens", type=int, default=16384, help="with --subspace: tokens per micro-batch")
     ap.add_argument("--tiles", action="store_true",
                     help="cut matrices into square tiles of `chunk` elements instead of consecutive chunks")
+    ap.add_argument("--bf16", action="store_true",
+                    help="parameters stored as bfloat16 (error buffers float32): the *_bf16 entry points")
     ap.add_argument("--variant", default="plain", choices=["plain", "ties_literal", "ties_dyadic"],
                     help="tie-heavy value laws of the density-sweep configuration")
     ap.add_argument("--seed", type=int, default=0)
