@@ -1009,6 +1009,251 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
+// ------------------------------------------------------------ reconstruct without embedding terms
+// Ghat = Gt U^T (activation gradients on their way back).  With nothing to gather, the launch above is bound
+// by the pace at which ONE thread can wait for a slot of U, issue its four MMAs and commit (a TF32 MMA covers
+// K = 8 only), and the shared memory of the position stages lies idle.  So this form has two MMA-issuing
+// warps, each with its own four-slot ring of U (the second ring in the idle stages), its own producer warp
+// and its own accumulator: warp m takes the 128-column blocks whose running number is m modulo 2 and writes
+// accumulator m, so the double buffer of the accumulators is also the split of the work.  The epilogue
+// takes the blocks in their order, as before.  Warps: 0 Xt tiles + ring 0, 1 MMA (even blocks), 2 part
+// store, 3..6 Xt staging -> tensor memory, 7..10 epilogue, 11 MMA (odd blocks), 12 ring 1.
+struct GradSmem {
+  uint8_t ring[2][kRingB][kSlotB];
+  uint8_t st[kStages][kSlotA];                        // finished parts on their way out
+  uint8_t a[kStageA][kSlotA];
+  uint64_t full[2][kRingB], empty[2][kRingB], o_full[2], o_empty[2];
+  uint64_t a_full[kStageA], a_empty[kStageA], a_ready, a_free;
+  uint64_t g_done[kStages], g_empty[kStages];
+  uint64_t mma_idle[2];
+  uint32_t tmem_base;
+  WaitCtl ctl;
+};
+constexpr int kGradThreads = 416;
+
+__global__ void __launch_bounds__(kGradThreads, 1)
+subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const __grid_constant__ SubParams p) {
+  extern __shared__ uint8_t raw[];
+  GradSmem& sm = *reinterpret_cast<GradSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t k_tiles = p.kp / kTileK;
+  const uint32_t n_blocks = (p.d + kBlockN - 1) / kBlockN;
+  const uint64_t G = (p.n_tok + 31) / 32;
+  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  if (tid == 0) {
+    for (int m = 0; m < 2; ++m)
+      for (int s = 0; s < kRingB; ++s) { mbar_init(&sm.full[m][s], 1); mbar_init(&sm.empty[m][s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); mbar_init(&sm.mma_idle[b], 1); }
+    for (int s = 0; s < kStageA; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 4); }
+    mbar_init(&sm.a_ready, 4);
+    mbar_init(&sm.a_free, 2);                         // both MMA warps are through with the tile
+    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.g_done[s], 4); mbar_init(&sm.g_empty[s], 1); }
+    sm.ctl.abort = 0;
+    sm.ctl.polls = p.wait_polls;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t t_a = sm.tmem_base;            // the Xt tile: 128 lanes x kp columns
+  const uint32_t t_o = sm.tmem_base + 256;      // two accumulators of 128 columns
+  const uint32_t c_first = blockIdx.x % n_blocks;
+  auto block_of = [&](uint32_t i) { const uint32_t c = i + c_first; return c >= n_blocks ? c - n_blocks : c; };
+  auto parts_of = [&](uint32_t c) { const uint32_t left = p.d - c * kBlockN; return left >= (uint32_t)kBlockN ? 4u : (left + 31u) / 32u; };
+
+  if (warp == 0 || warp == 12) {
+    // ---- producers: warp 0 the Xt tiles and the U slots of the even blocks, warp 12 those of the odd blocks ----
+    if (lane == 0) {
+      const uint32_t m = warp == 0 ? 0u : 1u;
+      uint32_t it = 0, ia = 0, cg = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+        const int r0 = (int)(g * 32);
+        if (m == 0) {
+          for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++ia) {
+            const uint32_t s = ia % kStageA;
+            ok = mbar_wait(&sm.a_empty[s], ((ia / kStageA) & 1u) ^ 1u, sm.ctl);
+            if (!ok) break;
+            mbar_expect_tx(&sm.a_full[s], h * 128);
+            if (hg == 4) tma_load_2d(sm.a[s], &maps.xt128, (int)(kt * kTileK), r0, &sm.a_full[s]);
+            else
+              for (uint32_t i = 0; i < hg; ++i)
+                tma_load_2d(sm.a[s] + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full[s]);
+          }
+        }
+        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
+          if ((cg & 1u) != m) continue;
+          for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
+            const uint32_t s = it % kRingB;
+            ok = mbar_wait(&sm.empty[m][s], ((it / kRingB) & 1u) ^ 1u, sm.ctl);
+            if (!ok) break;
+            mbar_expect_tx(&sm.full[m][s], kSlotB);
+            tma_load_2d(sm.ring[m][s], &maps.u_k, (int)(kt * kTileK), (int)(block_of(ci) * kBlockN), &sm.full[m][s]);
+          }
+        }
+      }
+      if (!ok) {
+        for (uint32_t s = 0; s < (uint32_t)kRingB; ++s) landed(&sm.full[m][s], ring_uses(it, s, kRingB));
+        if (m == 0)
+          for (uint32_t s = 0; s < (uint32_t)kStageA; ++s) landed(&sm.a_full[s], ring_uses(ia, s, kStageA));
+      }
+    }
+  } else if (warp == 1 || warp == 11) {
+    // ---- two MMA issuers: warp 1 the blocks with an even running number (accumulator 0), warp 11 the odd ones ----
+    if (lane == 0) {
+      const uint32_t m = warp == 1 ? 0u : 1u;
+      uint32_t it = 0, cg = 0, t = 0, mine = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(kRows, kBlockN, 0);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2);
+      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+        ok = mbar_wait(&sm.a_ready, t & 1u, sm.ctl);          // the tile is in tensor memory, rounded
+        if (!ok) break;
+        tc_fence_after();
+        for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+          if ((cg & 1u) != m) continue;
+          if (mine) {                                          // the epilogue has read this accumulator's previous block
+            ok = mbar_wait(&sm.o_empty[m], (mine - 1) & 1u, sm.ctl);
+            if (!ok) break;
+            tc_fence_after();
+          }
+          ++mine;
+          for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
+            const uint32_t s = it % kRingB;
+            ok = mbar_wait(&sm.full[m][s], (it / kRingB) & 1u, sm.ctl);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t db = desc_k | (uint64_t)((smem_u32(sm.ring[m][s]) >> 4) & 0x3FFF);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              mma_ts(t_o + m * kBlockN, t_a + kt * kTileK + 8 * j, db + 2 * j, idesc, (kt | (uint32_t)j) != 0);
+            mma_commit(&sm.empty[m][s]);
+          }
+          if (!ok) break;
+          mma_commit(&sm.o_full[m]);
+        }
+        if (ok) mma_commit(&sm.a_free);
+      }
+      if (!ok) mma_quiesce(&sm.mma_idle[m]);
+    }
+  } else if (warp == 2) {
+    // ---- part store ----
+    if (lane == 0) {
+      uint32_t is = 0;
+      bool ok = true;
+      for (uint64_t g = g0; ok && g < g1; g += 4) {
+        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
+        const int r0 = (int)(g * 32);
+        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci) {
+          const uint32_t c = block_of(ci), np = parts_of(c);
+          for (uint32_t part = 0; part < np; ++part, ++is) {
+            const uint32_t s = is % kStages;
+            ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.ctl);
+            if (!ok) break;
+            const int col0 = (int)(c * kBlockN + part * 32);
+            const uint32_t src = smem_u32(sm.st[s]);
+            if (hg == 4) tma_store_2d(&maps.o128, col0, r0, src);
+            else
+              for (uint32_t i = 0; i < hg; ++i) tma_store_2d(&maps.o32, col0, r0 + 32 * (int)i, src + i * 4096);
+            bulk_commit();
+            bulk_wait_read_all();
+            mbar_arrive(&sm.g_empty[s]);
+          }
+        }
+      }
+      bulk_wait_all();
+    }
+  } else if (warp < 7) {
+    // ---- staging warps: Xt tile -> tensor memory, rounded to TF32 (thread = lane of its 32-lane window) ----
+    const uint32_t q = (uint32_t)(warp & 3);
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    uint32_t ia = 0, t = 0;
+    bool ok = true;
+    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      if (t > 0) {                                   // both MMA warps have read the old tile
+        ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.ctl);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+      }
+      for (uint32_t kt = 0; kt < k_tiles; ++kt, ++ia) {
+        const uint32_t s = ia % kStageA;
+        ok = mbar_wait(&sm.a_full[s], (ia / kStageA) & 1u, sm.ctl);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint32_t v[32];
+        const uint32_t a0 = smem_u32(sm.a[s]) + row * 128;
+#pragma unroll
+        for (uint32_t ch = 0; ch < 8; ++ch) {
+          const float4 f = lds128(a0 + ((ch ^ (row & 7u)) << 4));
+          v[4 * ch + 0] = round_tf32(__float_as_uint(f.x));
+          v[4 * ch + 1] = round_tf32(__float_as_uint(f.y));
+          v[4 * ch + 2] = round_tf32(__float_as_uint(f.z));
+          v[4 * ch + 3] = round_tf32(__float_as_uint(f.w));
+        }
+        tmem_st32(t_a + kt * kTileK + ((32u * q) << 16), v);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.a_empty[s]);
+      }
+      if (!ok) break;
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.a_ready);
+    }
+  } else if (warp < 11) {
+    // ---- epilogue warps: accumulator part -> stage (swizzled like the store's box) ----
+    const uint32_t q = (uint32_t)(warp & 3);
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    const uint32_t roff = row * 128, sw = row & 7u;
+    uint32_t cg = 0, ie = 0;
+    bool ok = true;
+    for (uint64_t g = g0; ok && g < g1; g += 4) {
+      for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
+        const uint32_t buf = cg & 1u;
+        ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.ctl);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t np = parts_of(block_of(ci));
+        for (uint32_t part = 0; part < np; ++part, ++ie) {
+          const uint32_t s = ie % kStages;
+          uint32_t v[32];
+          tmem_ld32(t_o + buf * kBlockN + part * 32 + ((32u * q) << 16), v);
+          ok = mbar_wait(&sm.g_empty[s], ((ie / kStages) & 1u) ^ 1u, sm.ctl);   // the store has read the stage's last part
+          ok = __all_sync(0xffffffffu, ok);
+          tmem_ld_wait();
+          if (!ok) break;
+          const uint32_t bt = smem_u32(sm.st[s]) + roff;
+#pragma unroll
+          for (uint32_t ch = 0; ch < 8; ++ch)
+            sts128(bt + ((ch ^ sw) << 4), make_float4(__uint_as_float(v[4 * ch]), __uint_as_float(v[4 * ch + 1]),
+                                                      __uint_as_float(v[4 * ch + 2]), __uint_as_float(v[4 * ch + 3])));
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.g_done[s]);
+        }
+        if (!ok) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.o_empty[buf]);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sm.tmem_base), "r"(512) : "memory");
+  }
+  if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
 // --------------------------------------------------------------------- plain float32 kernels (any shape)
 __global__ void __launch_bounds__(256) subspace_project_generic_kernel(const float* __restrict__ X, const float* __restrict__ U,
                                                                        SubParams p) {
@@ -1133,10 +1378,18 @@ cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, con
       !make_map(&m.o128, Xhat, d, n_tok, kRows, CU_TENSOR_MAP_SWIZZLE_128B) ||
       !make_map(&m.o32, Xhat, d, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B))
     return cudaErrorInvalidValue;
-  const int smem = (int)sizeof(ReconSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(subspace_reconstruct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
   const unsigned grid = persistent_grid(n_tok, &e);
+  if (e != cudaSuccess) return e;
+  if (!ids) {                                        // no embedding terms: two MMA-issuing warps, two rings of U
+    const int gsmem = (int)sizeof(GradSmem) + 1024;
+    e = cudaFuncSetAttribute(subspace_reconstruct_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gsmem);
+    if (e != cudaSuccess) return e;
+    subspace_reconstruct_grad_kernel<<<grid, kGradThreads, gsmem, st>>>(m, p);
+    return cudaGetLastError();
+  }
+  const int smem = (int)sizeof(ReconSmem) + 1024;
+  e = cudaFuncSetAttribute(subspace_reconstruct_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   subspace_reconstruct_kernel<<<grid, kReconThreads, smem, st>>>(m, p);
   return cudaGetLastError();
