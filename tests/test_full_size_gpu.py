@@ -149,7 +149,7 @@ def test_tie_heavy_variants_of_the_sweep(variant, k, R):
     wl = sweep_sub_arena(synth.workload("1b").replace(k=k, R=R, variant=variant))
     st, _ = sampled_parity(wl, 2, False, 120, seed=5, min_short=30)
     if variant == "ties_dyadic":
-        # the stress is real only if the k-th and (k+1)-th magnitudes tie in most chunks (round 0 law:
+        # the stress is real only if the k-th and (k+1)-th magnitudes tie in most chunks (the law of outer round 0:
         # the pseudo-gradient of a fresh draw on the 2^-13 grid)
         st.redraw_locals(7)
         d = (st.theta_global[:2048 * 2048] - st.theta_local[0][:2048 * 2048]).abs().view(-1, 4096)

@@ -1,7 +1,8 @@
 """Pins of the checker's bfloat16 storage mode (parameters held as bfloat16, error buffers float32).
 
 The paper states no storage precision for Eq. 2 (section 2.1), so WHERE the parameters are rounded is
-this build's reading (the design doc lists it); what is pinned here is that the checker does exactly that
+a reading of this build (bfloat16 arrays for the parameters, the pseudo-gradient formed in float32 from the widened
+values, the float32 step rounded once more, to nearest-even, when it is stored); what is pinned here is that the checker does exactly that
 reading: exact widening, round-to-nearest-even on storage, the float32 step in between."""
 import json
 import os
