@@ -98,6 +98,22 @@ struct AggSmem {
 
 __device__ __forceinline__ uint32_t agg_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// the cold end of a give-up, kept out of line so that it does not weigh on the kernel's hot code: waits
+// (bounded) for the last two of the `issued` bulk copies of theta_global (the j-th went to buffer j & 1) and
+// raises the flag
+__device__ __noinline__ void agg_giveup_drain(uint64_t* full, uint32_t issued, uint32_t* flags) {
+  for (uint32_t j = issued >= 2 ? issued - 2 : 0; j < issued; ++j) {
+    const uint32_t bar = agg_smem_u32(&full[j & 1]), parity = (j >> 1) & 1u;
+    for (uint32_t spin = 0; spin < kAggWaitLimit; ++spin) {
+      uint32_t done;
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                   : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+      if (done) break;
+    }
+  }
+  if (flags) atomicOr(flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
 // first full chunk at or after g (stepping by `step`); t_lo caches the tensor of the last hit;
 // stride = elements between the chunk's rows of 64 (64 for a consecutive chunk)
 template <int T>
@@ -380,20 +396,8 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   }
   if (APPLY) {
     if (sm.abort_it != 0) {                        // gave up somewhere: the copies in flight may land first
-      if (TILED) {
-        asm volatile("cp.async.wait_all;" ::: "memory");
-      } else if (tid == 0) {
-        for (uint32_t j = issued >= 2 ? issued - 2 : 0; j < issued; ++j) {      // the j-th copy went to buffer j & 1
-          const uint32_t bar = agg_smem_u32(&sm.full[j & 1]), parity = (j >> 1) & 1u;
-          for (uint32_t spin = 0; spin < kAggWaitLimit; ++spin) {
-            uint32_t done;
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-            if (done) break;
-          }
-        }
-      }
-      if (tid == 0 && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
+      if (TILED) asm volatile("cp.async.wait_all;" ::: "memory");
+      if (tid == 0) agg_giveup_drain(sm.full, TILED ? 0u : issued, a.flags);
     }
   }
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);

@@ -331,6 +331,12 @@ __device__ __forceinline__ void mbar_drain(uint64_t* bar, uint32_t uses) {
     __nanosleep(40);
   }
 }
+// the cold end of a give-up, kept out of line so that it does not weigh on the kernels' hot code: waits for
+// the copies announced on `n` barriers `step` apart (uses[i] of them on barrier i) and raises the flag
+__device__ __noinline__ void giveup_drain(uint64_t* bars, int n, int step, uint32_t issued, int per, uint32_t* flags) {
+  for (int i = 0; i < n; ++i) mbar_drain(bars + i * step, (issued + per - 1 - i) / per);
+  if (flags) atomicOr(flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
 __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
@@ -888,10 +894,8 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
       }
       if (TILED) tile_store(rp, last ? base_m1 : base_m2, last ? stride_m1 : stride_m2, wp % kEeStages);
     }
-    if (!TILED && tid == 0 && sm.abort_item != 0) {   // gave up somewhere: let this thread's copies in flight land
-      for (int i = 0; i < kTlStages; ++i) mbar_drain(&sm.full_tl[i], (tl_issued + kTlStages - 1 - i) / kTlStages);
-      if (a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_TIMEOUT);
-    }
+    if (!TILED && tid == 0 && sm.abort_item != 0)     // gave up somewhere: let this thread's copies in flight land
+      giveup_drain(sm.full_tl, kTlStages, 1, tl_issued, kTlStages, a.flags);
   } else {
     // ======================= selectors =======================================
     const int q = warp - kWarps;
@@ -1020,7 +1024,7 @@ compress_c4096_kernel(const __grid_constant__ CompressArgs<T> a) {
     if (!TILED && lane == 0) {
       tma_store_wait_read_all();                  // shared memory must outlive the bulk stores' reads ...
       if (sm.abort_item != 0)                     // ... and, after a give-up, the copies still coming in
-        for (int i = 0; i < kEeStages / kSel; ++i) mbar_drain(&sm.full_ee[q + kSel * i], (ee_issued + 1 - i) / 2);
+        giveup_drain(&sm.full_ee[q], kEeStages / kSel, kSel, ee_issued, kEeStages / kSel, nullptr);
     }
   }
 }
