@@ -338,3 +338,7 @@ def test_random_shapes_both_directions(n_tok, L, V, d, k):
     gt, f = _project(X, None, None, None, U, L)
     assert f == 0
     assert np.all(np.abs(gt - osub.project(X, None, None, None, U, L)) <= TOL * (np.abs(X.astype(np.float64)) @ np.abs(U.astype(np.float64))) + 1e-30)
+    # ... and back without embedding terms (the launch with two MMA-issuing warps; d / 128 odd, even or one block)
+    gh, f = _reconstruct(gt, None, None, None, U, L)
+    assert f == 0
+    _check_reconstruct(gh, gt, None, None, None, U, L, f"gradient reconstruct {n_tok}x{d} k={k}")
