@@ -1144,7 +1144,7 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
   } else if (warp == 2) {
     // ---- part store ----
     if (lane == 0) {
-      uint32_t is = 0;
+      uint32_t is = 0, held = kStages;          // held: the stage whose store was issued last (kStages: none)
       bool ok = true;
       for (uint64_t g = g0; ok && g < g1; g += 4) {
         const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
@@ -1161,11 +1161,16 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
             else
               for (uint32_t i = 0; i < hg; ++i) tma_store_2d(&maps.o32, col0, r0 + 32 * (int)i, src + i * 4096);
             bulk_commit();
-            bulk_wait_read_all();
-            mbar_arrive(&sm.g_empty[s]);
+            // the store just issued is not waited for: the stage of the store BEFORE it is released once that
+            // one has read its source, so that the wait never sits between two stores
+            bulk_wait_read_but_one();
+            if (held != kStages) mbar_arrive(&sm.g_empty[held]);
+            held = s;
           }
         }
       }
+      bulk_wait_read_all();
+      if (held != kStages) mbar_arrive(&sm.g_empty[held]);
       bulk_wait_all();
     }
   } else if (warp < 7) {
