@@ -730,6 +730,7 @@ struct ReconSmem {
   uint64_t full[kRingB], empty[kRingB], o_full[2], o_empty[2];
   uint64_t a_full[kStageA], a_empty[kStageA], a_ready, a_free;
   uint64_t g_full[kStages], g_done[kStages], g_empty[kStages];
+  uint64_t t_free[kStages];                            // the epilogue has read the stage's T_perp segments
   uint64_t mma_idle;        // after a give-up only: the MMAs issued so far have retired
   uint32_t tmem_base;
   WaitCtl ctl;
@@ -757,7 +758,9 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     for (int s = 0; s < kStageA; ++s) { mbar_init(&sm.a_full[s], 1); mbar_init(&sm.a_empty[s], 4); }
     mbar_init(&sm.a_ready, 4);
     mbar_init(&sm.a_free, 1);
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.g_full[s], 128); mbar_init(&sm.g_done[s], 4); mbar_init(&sm.g_empty[s], 1); }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.g_full[s], 128); mbar_init(&sm.g_done[s], 4); mbar_init(&sm.g_empty[s], 1); mbar_init(&sm.t_free[s], 4);
+    }
     mbar_init(&sm.mma_idle, 1);
     sm.ctl.abort = 0;
     sm.ctl.polls = p.wait_polls;
@@ -861,7 +864,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
             ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.ctl);
             if (!ok) break;
             const int col0 = (int)(c * kBlockN + part * 32);
-            const uint32_t src = smem_u32(sm.st_t[s]);
+            const uint32_t src = smem_u32(sm.st_p[s]);        // the finished part sits in the position stage
             if (hg == 4) tma_store_2d(&maps.o128, col0, r0, src);
             else
               for (uint32_t i = 0; i < hg; ++i) tma_store_2d(&maps.o32, col0, r0 + 32 * (int)i, src + i * 4096);
@@ -928,19 +931,32 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
         const uint32_t c = block_of(ci), np = parts_of(c);
         for (uint32_t part = 0; part < np; ++part, ++ig) {
           const uint32_t s = ig % kStages;
-          ok = mbar_wait(&sm.g_empty[s], ((ig / kStages) & 1u) ^ 1u, sm.ctl);
+          const uint32_t col0 = c * kBlockN + part * 32;
+          const bool in_col = col0 + 4 * gch < p.d;
+          const uint32_t dt = smem_u32(sm.st_t[s]), dp = smem_u32(sm.st_p[s]);
+          // the T_perp half of the stage is free as soon as the epilogue has read it - the finished part waits
+          // for its store in the position half - so the gathers that come from DRAM start one store earlier
+          ok = mbar_wait(&sm.t_free[s], ((ig / kStages) & 1u) ^ 1u, sm.ctl);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           if (p.ids) {
-            const uint32_t col0 = c * kBlockN + part * 32;
-            const bool in_col = col0 + 4 * gch < p.d;
-            const uint32_t dt = smem_u32(sm.st_t[s]), dp = smem_u32(sm.st_p[s]);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               const uint32_t r = grow + 16u * (uint32_t)i;
               const uint32_t off = r * 128 + ((gch ^ (r & 7u)) << 4);
               const bool in = in_col && ((mask >> i) & 1u);
               cp_async_16z(dt + off, in ? (const void*)(tp[i] + col0) : (const void*)p.T_perp, in ? 16u : 0u);
+            }
+          }
+          ok = mbar_wait(&sm.g_empty[s], ((ig / kStages) & 1u) ^ 1u, sm.ctl);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (p.ids) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const uint32_t r = grow + 16u * (uint32_t)i;
+              const uint32_t off = r * 128 + ((gch ^ (r & 7u)) << 4);
+              const bool in = in_col && ((mask >> i) & 1u);
               cp_async_16z(dp + off, in ? (const void*)(ps[i] + col0) : (const void*)p.pos, in ? 16u : 0u);
             }
           }
@@ -986,11 +1002,11 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
               r.z = __fadd_rn(__fadd_rn(r.z, e.z), f.z);
               r.w = __fadd_rn(__fadd_rn(r.w, e.w), f.w);
             }
-            sts128(bt + o, r);
+            sts128(bp + o, r);                     // the finished part replaces the position segment it used
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.g_done[s]);
+          if (lane == 0) { mbar_arrive(&sm.t_free[s]); mbar_arrive(&sm.g_done[s]); }
         }
         if (!ok) break;
         tc_fence_before();
