@@ -403,8 +403,8 @@ aggregate_c4096_kernel(const __grid_constant__ AggregateArgs<T> a) {
   if (bad && a.flags) atomicOr(a.flags, (uint32_t)SL_FLAG_BAD_INDEX);
 }
 
-// Fused average + update for FEW entries per chunk (R * k <= 256, one per thread), consecutive chunks,
-// float32 parameters, outer_lr > 0.  An element no replica sent has the mean update +0, and
+// Fused average + update for FEW entries per chunk (R * k <= 256, one per thread), consecutive chunks or
+// 64 x 64 tiles, float32 parameters, outer_lr > 0.  An element no replica sent has the mean update +0, and
 // theta - outer_lr * (+0) is theta itself, bit for bit: for outer_lr > 0 the product is -0 and x + (-0) = x
 // for every x, both zeros included (and a position's sum starts from +0, so it is never -0).  So
 // theta_global is neither read nor rewritten as a whole: only the elements some replica sent are loaded,
@@ -469,34 +469,41 @@ aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
     return w;
   };
   // decoded entry of a chunk: position (0xFFFF: none), value, and the element of theta_global it names
-  struct Dec { uint32_t pos; float val, th; };
-  auto decode = [&](const Raw& w, uint64_t base) {
-    Dec d{0xFFFFu, 0.0f, 0.0f};
+  // (eoff: the element's offset from the chunk's first element - the position itself in a consecutive
+  // chunk, row p / 64 and column p % 64 of a tile whose rows are `stride` elements apart; the one formula
+  // serves both, since a consecutive chunk is reported with stride 64)
+  struct Dec { uint32_t pos; float val, th; uint64_t eoff; };
+  auto decode = [&](const Raw& w, uint64_t base, uint32_t stride) {
+    Dec d{0xFFFFu, 0.0f, 0.0f, 0};
     if (my_r < 0 || w.pos == 0xFFFFu) return d;
     if (w.pos >= (uint32_t)kAC) { bad = true; return d; }
-    if (!SL_CHECK(a.flags, base + w.pos < n_total)) return d;
+    const uint64_t eoff = (uint64_t)(w.pos >> 6) * stride + (w.pos & 63u);
+    if (!SL_CHECK(a.flags, base + eoff < n_total)) return d;
     d.pos = w.pos;
+    d.eoff = eoff;
     d.val = bits == 32 ? __uint_as_float(w.code) : dequant((w.code >> cshift) & cmask, w.scale, bits);
-    d.th = __ldcg(a.out + base + d.pos);
+    d.th = __ldcg(a.out + base + eoff);
     return d;
   };
   // The group's chunks in flight, oldest first: stage 0 is processed in this iteration, stages 1..kDec hold
   // decoded entries whose theta_global elements are on their way, the last kRaw stages raw entries on their way.
   constexpr int kDec = 1, kRaw = 1, kStagesInFlight = 1 + kDec + kRaw;
   uint64_t base_q[kStagesInFlight];
+  uint32_t stride_q[kStagesInFlight];
   bool valid_q[kStagesInFlight];
   Dec dec_q[1 + kDec];
   Raw raw_q[kRaw];
-  uint32_t g_next = vcta, t_lo = 0, stride_unused = 64;
+  uint32_t g_next = vcta, t_lo = 0;
   bool more = true;
 #pragma unroll
   for (int i = 0; i < kStagesInFlight; ++i) {
     base_q[i] = 0;
-    valid_q[i] = more && next_full_chunk(a.tb, g_next, vgrid, t_lo, base_q[i], stride_unused);
+    stride_q[i] = 64;
+    valid_q[i] = more && next_full_chunk(a.tb, g_next, vgrid, t_lo, base_q[i], stride_q[i]);
     more = valid_q[i];
     if (i <= kDec) {
-      dec_q[i] = Dec{0xFFFFu, 0.0f, 0.0f};
-      if (valid_q[i]) dec_q[i] = decode(fetch(g_next), base_q[i]);
+      dec_q[i] = Dec{0xFFFFu, 0.0f, 0.0f, 0};
+      if (valid_q[i]) dec_q[i] = decode(fetch(g_next), base_q[i], stride_q[i]);
     } else {
       raw_q[i - 1 - kDec] = Raw{0xFFFFu, 0u, 0.0f};
       if (valid_q[i]) raw_q[i - 1 - kDec] = fetch(g_next);
@@ -521,7 +528,7 @@ aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
     if (have && first) {
       const float sum = sm.acc[posA];
       const float u = pow2 ? __fmul_rn(sum, invR) : __fdiv_rn(sum, Rf);
-      a.out[base_q[0] + posA] = __fmaf_rn(nlr, u, dec_q[0].th);
+      a.out[base_q[0] + dec_q[0].eoff] = __fmaf_rn(nlr, u, dec_q[0].th);
       atomicAnd(&sm.seen[word], ~bit);
     }
     group_sync();                                  // cells and bits are free for the next chunk
@@ -529,12 +536,12 @@ aggregate_sparse_kernel(const __grid_constant__ AggregateArgs<T> a) {
 #pragma unroll
     for (int i = 0; i < kDec; ++i) dec_q[i] = dec_q[i + 1];
 #pragma unroll
-    for (int i = 0; i + 1 < kStagesInFlight; ++i) { base_q[i] = base_q[i + 1]; valid_q[i] = valid_q[i + 1]; }
-    dec_q[kDec] = Dec{0xFFFFu, 0.0f, 0.0f};
-    if (valid_q[kDec]) dec_q[kDec] = decode(raw_q[0], base_q[kDec]);
+    for (int i = 0; i + 1 < kStagesInFlight; ++i) { base_q[i] = base_q[i + 1]; stride_q[i] = stride_q[i + 1]; valid_q[i] = valid_q[i + 1]; }
+    dec_q[kDec] = Dec{0xFFFFu, 0.0f, 0.0f, 0};
+    if (valid_q[kDec]) dec_q[kDec] = decode(raw_q[0], base_q[kDec], stride_q[kDec]);
 #pragma unroll
     for (int i = 0; i + 1 < kRaw; ++i) raw_q[i] = raw_q[i + 1];
-    valid_q[kStagesInFlight - 1] = more && next_full_chunk(a.tb, g_next, vgrid, t_lo, base_q[kStagesInFlight - 1], stride_unused);
+    valid_q[kStagesInFlight - 1] = more && next_full_chunk(a.tb, g_next, vgrid, t_lo, base_q[kStagesInFlight - 1], stride_q[kStagesInFlight - 1]);
     more = valid_q[kStagesInFlight - 1];
     if (more) { raw_q[kRaw - 1] = fetch(g_next); g_next += vgrid; }
   }
@@ -563,17 +570,8 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
   };
   const int np = pairs <= 1 ? 1 : pairs <= 2 ? 2 : pairs <= 4 ? 4 : 8;
   const bool grouped = np > 1 && a.k % np == 0;     // (with one pair per thread the two mappings coincide)
-  if (a.tb.side != 0) {
-    if (np == 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, true, false>);
-    if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 2, true, true>)
-                                : launch(aggregate_c4096_kernel<T, APPLY, 2, true, false>);
-    if (np == 4) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 4, true, true>)
-                                : launch(aggregate_c4096_kernel<T, APPLY, 4, true, false>);
-    return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 8, true, true>)
-                   : launch(aggregate_c4096_kernel<T, APPLY, 8, true, false>);
-  }
   if constexpr (APPLY) {
-    if (!a.theta_bf16 && a.tb.side == 0 && a.outer_lr > 0.0f && a.R * a.k <= kSparseMaxEntries) {
+    if (!a.theta_bf16 && (a.tb.side == 0 || a.tb.side == 64) && a.outer_lr > 0.0f && a.R * a.k <= kSparseMaxEntries) {
       auto launch_sparse = [&](auto kernel, int groups) -> cudaError_t {
         const size_t sm_bytes = sizeof(SparseSmem) * (size_t)groups;
         cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm_bytes);
@@ -592,6 +590,17 @@ cudaError_t launch_aggregate_c4096(const AggregateArgs<T>& a, cudaStream_t st) {
       if (entries <= 128) return launch_sparse(aggregate_sparse_kernel<T, 2>, 2);
       return launch_sparse(aggregate_sparse_kernel<T, 1>, 1);
     }
+  }
+  if (a.tb.side != 0) {
+    if (np == 1) return launch(aggregate_c4096_kernel<T, APPLY, 1, true, false>);
+    if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 2, true, true>)
+                                : launch(aggregate_c4096_kernel<T, APPLY, 2, true, false>);
+    if (np == 4) return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 4, true, true>)
+                                : launch(aggregate_c4096_kernel<T, APPLY, 4, true, false>);
+    return grouped ? launch(aggregate_c4096_kernel<T, APPLY, 8, true, true>)
+                   : launch(aggregate_c4096_kernel<T, APPLY, 8, true, false>);
+  }
+  if constexpr (APPLY) {
     if (a.theta_bf16) {
       if (np == 1) return launch(aggregate_c4096_kernel<T, true, 1, false, false, true>);
       if (np == 2) return grouped ? launch(aggregate_c4096_kernel<T, true, 2, false, true, true>)

@@ -666,3 +666,17 @@ def test_theta_global_update_touches_only_what_was_sent(R, k, lr):
     gs, tg_o, _ = run_and_compare(off, tg, tls, errs, 0.95, 4096, k, 2, lr, what=f"sparse update R{R} k{k} lr{lr}")
     got = gs.theta_global.cpu().numpy()
     assert np.array_equal(np.signbit(got), np.signbit(tg_o)), "a signed zero changed its sign"
+
+
+@pytest.mark.parametrize("R,k", [(2, 64), (4, 16), (1, 32)])
+def test_theta_global_update_touches_only_what_was_sent_in_tiles(R, k):
+    # the same with matrices cut into 64 x 64 tiles (the position of an entry is a row and a column of its tile)
+    sizes = [320 * 192, 2048, 128 * 640, 4096 * 3]
+    cols = [192, 0, 640, 0]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.uint64)
+    tg, tls, errs = _case(int(off[-1]), R, seed=R * 10 + k)
+    tg[::7] = -0.0
+    gs, tg_o, _ = run_and_compare(off, tg, tls, errs, 0.95, 4096, k, 2, 0.8, rounds=2, cols=cols,
+                                  next_locals=lambda t, g: [(g + np.random.default_rng(t * 10 + r).normal(0, 1e-3, g.size)).astype(f32)
+                                                            for r in range(R)], what=f"sparse update in tiles R{R} k{k}")
+    assert np.array_equal(np.signbit(gs.theta_global.cpu().numpy()), np.signbit(tg_o))
