@@ -838,6 +838,8 @@ def measured_rows(args, wl: synth.Workload, dev, peak: float) -> dict:
     """Everything else this library times, appended to the default line (outside its timed region)."""
     n = args.row_launches
     rows = {"note": "medians of CUDA-event times; frac = algorithmic bytes / time / peak"}
+    rows["config_180m"] = row_outer_step(synth.workload("180m"), args.seed, dev, peak, n)     # benchmark configuration 2
+    rows["config_0p5b"] = row_outer_step(synth.workload("0p5b"), args.seed, dev, peak, n)     # benchmark configuration 3
     rows["tiles"] = row_outer_step(wl, args.seed, dev, peak, n, tiles=True)
     rows["r2"] = row_outer_step(wl.replace(R=2), args.seed, dev, peak, n)
     rows["r16_k128"] = row_outer_step(wl.replace(R=16, k=128), args.seed, dev, peak, n)
