@@ -19,7 +19,8 @@
 //                a ring; the accumulator is double buffered; the gathered rows wait in stages of
 //                shared memory, the epilogue adds them and a tensor-map store writes the part.
 //
-// Tokens are dealt in groups of 32 evenly over one CTA per SM, sub-tiles of up to 128 tokens.
+// One CTA per SM.  Compression deals the tokens in groups of 32 evenly over the CTAs, sub-tiles of up to 128
+// tokens; reconstruction deals the (sub-tile, 128-column block) pairs evenly, so a sub-tile may be shared.
 // Every wait is bounded (SL_FLAG_TIMEOUT); a token id outside [0, V) gathers nothing and raises
 // SL_FLAG_BAD_INDEX.  Other shapes (k or d not a multiple of 4, k above 256, unaligned pointers)
 // take plain float32 kernels.
@@ -74,6 +75,55 @@ __device__ __forceinline__ RowInfo row_info(const SubParams& p, uint64_t r0, uin
   }
   return ri;
 }
+
+// A CTA's share of a reconstruction.  The sub-tiles of 128 tokens are dealt whole, q to every CTA; the
+// remaining ones (fewer than there are CTAs) are cut by 128-column blocks, each among the same number of CTAs, so
+// the last piece of a CTA is a range of blocks of a sub-tile it shares.  (Every sub-tile streams all of U,
+// however few rows it has, and a piece costs its blocks plus the hand-over of the Xt tile: dealing whole
+// sub-tiles only would leave most CTAs waiting for those that got one more.)
+// The blocks of a piece are independent; CTA b walks them from the (b mod n)-th on, so that the CTAs do not
+// all ask L2 for the same rows of U at the same time (no effect on the result).
+struct Piece {
+  uint64_t r0;              // first token of the sub-tile
+  uint32_t hg, cb, n, rot;  // its groups of 32 tokens (1..4); first block and number of blocks; where the walk starts
+  __device__ __forceinline__ uint32_t block(uint32_t i) const {
+    const uint32_t c = i + rot;
+    return cb + (c >= n ? c - n : c);
+  }
+};
+struct Sched {
+  uint64_t G, n_sub;
+  uint32_t n_blocks, q, n_pieces, tail_cb, tail_n;
+  uint64_t tail_st;
+  __device__ __forceinline__ Sched(uint32_t n_blocks_, uint64_t G_) : G(G_), n_sub((G_ + 3) / 4), n_blocks(n_blocks_) {
+    const uint64_t grid = gridDim.x, b = blockIdx.x;
+    q = (uint32_t)(n_sub / grid);
+    const uint64_t rem = n_sub - (uint64_t)q * grid;
+    tail_cb = tail_n = 0;
+    tail_st = 0;
+    if (rem) {
+      const uint64_t sh = grid / rem;                 // CTAs that share one of the remaining sub-tiles
+      if (b < rem * sh) {
+        const uint32_t j = (uint32_t)(b % sh);
+        tail_st = (uint64_t)q * grid + b / sh;
+        tail_cb = (uint32_t)((uint64_t)j * n_blocks / sh);
+        tail_n = (uint32_t)((uint64_t)(j + 1) * n_blocks / sh) - tail_cb;
+      }
+    }
+    n_pieces = q + (tail_n ? 1u : 0u);
+  }
+  __device__ __forceinline__ Piece piece(uint32_t i) const {
+    Piece pc;
+    const bool whole = i < q;
+    const uint64_t st = whole ? (uint64_t)i * gridDim.x + blockIdx.x : tail_st;
+    pc.cb = whole ? 0u : tail_cb;
+    pc.n = whole ? n_blocks : tail_n;
+    pc.rot = blockIdx.x % pc.n;
+    pc.r0 = st * kRows;
+    pc.hg = (uint32_t)(G - 4 * st < 4 ? G - 4 * st : 4);
+    return pc;
+  }
+};
 
 // ------------------------------------------------------------------------------------------ compress
 struct ProjSmem {
@@ -751,7 +801,7 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   const uint32_t k_tiles = p.kp / kTileK;
   const uint32_t n_blocks = (p.d + kBlockN - 1) / kBlockN;
   const uint64_t G = (p.n_tok + 31) / 32;
-  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  const Sched sc(n_blocks, G);
   if (tid == 0) {
     for (int s = 0; s < kRingB; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
@@ -777,19 +827,16 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
   const uint32_t t_o = sm.tmem_base + 256;      // two accumulators of 128 columns
   bool bad = false;
   // 32-column parts of block c that lie inside the matrix
-  // CTAs walk the 128-column blocks from different starting points, so that they do not all ask L2 for the
-  // same rows of U at the same time (the blocks are independent: no effect on the result)
-  const uint32_t c_first = blockIdx.x % n_blocks;
-  auto block_of = [&](uint32_t i) { const uint32_t c = i + c_first; return c >= n_blocks ? c - n_blocks : c; };
   auto parts_of = [&](uint32_t c) { const uint32_t left = p.d - c * kBlockN; return left >= (uint32_t)kBlockN ? 4u : (left + 31u) / 32u; };
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0, ia = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
-        const int r0 = (int)(g * 32);
+      for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi) {
+        const Piece pc = sc.piece(pi);
+        const uint32_t hg = pc.hg, h = hg * 32;
+        const int r0 = (int)pc.r0;
         for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++ia) {
           const uint32_t s = ia % kStageA;
           ok = mbar_wait(&sm.a_empty[s], ((ia / kStageA) & 1u) ^ 1u, sm.ctl);
@@ -800,13 +847,13 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
             for (uint32_t i = 0; i < hg; ++i)
               tma_load_2d(sm.a[s] + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full[s]);
         }
-        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci)
+        for (uint32_t ci = 0; ok && ci < pc.n; ++ci)
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
             const uint32_t s = it % kRingB;
             ok = mbar_wait(&sm.empty[s], ((it / kRingB) & 1u) ^ 1u, sm.ctl);
             if (!ok) break;
             mbar_expect_tx(&sm.full[s], kSlotB);
-            tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(block_of(ci) * kBlockN), &sm.full[s]);
+            tma_load_2d(sm.ring[s], &maps.u_k, (int)(kt * kTileK), (int)(pc.block(ci) * kBlockN), &sm.full[s]);
           }
       }
       if (!ok) {
@@ -820,11 +867,12 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       bool ok = true;
       const uint32_t idesc = instr_desc(kRows, kBlockN, 0);
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2);
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi, ++t) {
+        const Piece pc = sc.piece(pi);
         ok = mbar_wait(&sm.a_ready, t & 1u, sm.ctl);          // the tile is in tensor memory, rounded
         if (!ok) break;
         tc_fence_after();
-        for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+        for (uint32_t c = 0; ok && c < pc.n; ++c, ++cg) {
           const uint32_t buf = cg & 1u, u = cg >> 1;
           if (u) {
             ok = mbar_wait(&sm.o_empty[buf], (u - 1) & 1u, sm.ctl);
@@ -854,11 +902,12 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     if (lane == 0) {
       uint32_t is = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
-        const int r0 = (int)(g * 32);
-        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci) {
-          const uint32_t c = block_of(ci), np = parts_of(c);
+      for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi) {
+        const Piece pc = sc.piece(pi);
+        const uint32_t hg = pc.hg;
+        const int r0 = (int)pc.r0;
+        for (uint32_t ci = 0; ok && ci < pc.n; ++ci) {
+          const uint32_t c = pc.block(ci), np = parts_of(c);
           for (uint32_t part = 0; part < np; ++part, ++is) {
             const uint32_t s = is % kStages;
             ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.ctl);
@@ -883,9 +932,10 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     const uint32_t gt = (uint32_t)(tid - 96), gch = gt & 7u, grow = gt >> 3;   // gather: 8 threads per 128-byte segment
     uint32_t ia = 0, ig = 0, t = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
-      const uint64_t r0 = g * 32;
+    for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi, ++t) {
+      const Piece pc = sc.piece(pi);
+      const uint32_t hg = pc.hg, h = hg * 32;
+      const uint64_t r0 = pc.r0;
       // the eight rows this thread gathers for: row grow + 16 i
       const float* tp[8];
       const float* ps[8];
@@ -927,8 +977,8 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.a_ready);
-      for (uint32_t ci = 0; ok && ci < n_blocks; ++ci) {
-        const uint32_t c = block_of(ci), np = parts_of(c);
+      for (uint32_t ci = 0; ok && ci < pc.n; ++ci) {
+        const uint32_t c = pc.block(ci), np = parts_of(c);
         for (uint32_t part = 0; part < np; ++part, ++ig) {
           const uint32_t s = ig % kStages;
           const uint32_t col0 = c * kBlockN + part * 32;
@@ -973,14 +1023,15 @@ subspace_reconstruct_kernel(const __grid_constant__ ReconMaps maps, const __grid
     const bool add = p.ids != nullptr;
     uint32_t cg = 0, ie = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4) {
-      for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
+    for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi) {
+      const Piece pc = sc.piece(pi);
+      for (uint32_t ci = 0; ok && ci < pc.n; ++ci, ++cg) {
         const uint32_t buf = cg & 1u;
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t np = parts_of(block_of(ci));
+        const uint32_t np = parts_of(pc.block(ci));
         for (uint32_t part = 0; part < np; ++part, ++ie) {
           const uint32_t s = ie % kStages;
           uint32_t v[32];
@@ -1055,7 +1106,7 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
   const uint32_t k_tiles = p.kp / kTileK;
   const uint32_t n_blocks = (p.d + kBlockN - 1) / kBlockN;
   const uint64_t G = (p.n_tok + 31) / 32;
-  const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  const Sched sc(n_blocks, G);
   if (tid == 0) {
     for (int m = 0; m < 2; ++m)
       for (int s = 0; s < kRingB; ++s) { mbar_init(&sm.full[m][s], 1); mbar_init(&sm.empty[m][s], 1); }
@@ -1077,8 +1128,6 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
   tc_fence_after();
   const uint32_t t_a = sm.tmem_base;            // the Xt tile: 128 lanes x kp columns
   const uint32_t t_o = sm.tmem_base + 256;      // two accumulators of 128 columns
-  const uint32_t c_first = blockIdx.x % n_blocks;
-  auto block_of = [&](uint32_t i) { const uint32_t c = i + c_first; return c >= n_blocks ? c - n_blocks : c; };
   auto parts_of = [&](uint32_t c) { const uint32_t left = p.d - c * kBlockN; return left >= (uint32_t)kBlockN ? 4u : (left + 31u) / 32u; };
 
   if (warp == 0 || warp == 12) {
@@ -1087,9 +1136,10 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
       const uint32_t m = warp == 0 ? 0u : 1u;
       uint32_t it = 0, ia = 0, cg = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
-        const int r0 = (int)(g * 32);
+      for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi) {
+        const Piece pc = sc.piece(pi);
+        const uint32_t hg = pc.hg, h = hg * 32;
+        const int r0 = (int)pc.r0;
         if (m == 0) {
           for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++ia) {
             const uint32_t s = ia % kStageA;
@@ -1102,14 +1152,14 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
                 tma_load_2d(sm.a[s] + i * 4096, &maps.xt32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.a_full[s]);
           }
         }
-        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
+        for (uint32_t ci = 0; ok && ci < pc.n; ++ci, ++cg) {
           if ((cg & 1u) != m) continue;
           for (uint32_t kt = 0; kt < k_tiles; ++kt, ++it) {
             const uint32_t s = it % kRingB;
             ok = mbar_wait(&sm.empty[m][s], ((it / kRingB) & 1u) ^ 1u, sm.ctl);
             if (!ok) break;
             mbar_expect_tx(&sm.full[m][s], kSlotB);
-            tma_load_2d(sm.ring[m][s], &maps.u_k, (int)(kt * kTileK), (int)(block_of(ci) * kBlockN), &sm.full[m][s]);
+            tma_load_2d(sm.ring[m][s], &maps.u_k, (int)(kt * kTileK), (int)(pc.block(ci) * kBlockN), &sm.full[m][s]);
           }
         }
       }
@@ -1127,11 +1177,12 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
       bool ok = true;
       const uint32_t idesc = instr_desc(kRows, kBlockN, 0);
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2);
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi, ++t) {
+        const Piece pc = sc.piece(pi);
         ok = mbar_wait(&sm.a_ready, t & 1u, sm.ctl);          // the tile is in tensor memory, rounded
         if (!ok) break;
         tc_fence_after();
-        for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+        for (uint32_t c = 0; ok && c < pc.n; ++c, ++cg) {
           if ((cg & 1u) != m) continue;
           if (mine) {                                          // the epilogue has read this accumulator's previous block
             ok = mbar_wait(&sm.o_empty[m], (mine - 1) & 1u, sm.ctl);
@@ -1162,11 +1213,12 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
     if (lane == 0) {
       uint32_t is = 0, held = kStages;          // held: the stage whose store was issued last (kStages: none)
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
-        const int r0 = (int)(g * 32);
-        for (uint32_t ci = 0; ok && ci < n_blocks; ++ci) {
-          const uint32_t c = block_of(ci), np = parts_of(c);
+      for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi) {
+        const Piece pc = sc.piece(pi);
+        const uint32_t hg = pc.hg;
+        const int r0 = (int)pc.r0;
+        for (uint32_t ci = 0; ok && ci < pc.n; ++ci) {
+          const uint32_t c = pc.block(ci), np = parts_of(c);
           for (uint32_t part = 0; part < np; ++part, ++is) {
             const uint32_t s = is % kStages;
             ok = mbar_wait(&sm.g_done[s], (is / kStages) & 1u, sm.ctl);
@@ -1195,7 +1247,8 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
     const uint32_t row = 32u * q + (uint32_t)lane;
     uint32_t ia = 0, t = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+    for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi, ++t) {
+      const Piece pc = sc.piece(pi);
       if (t > 0) {                                   // both MMA warps have read the old tile
         ok = mbar_wait(&sm.a_free, (t - 1) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
@@ -1234,14 +1287,15 @@ subspace_reconstruct_grad_kernel(const __grid_constant__ ReconMaps maps, const _
     const uint32_t roff = row * 128, sw = row & 7u;
     uint32_t cg = 0, ie = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4) {
-      for (uint32_t ci = 0; ok && ci < n_blocks; ++ci, ++cg) {
+    for (uint32_t pi = 0; ok && pi < sc.n_pieces; ++pi) {
+      const Piece pc = sc.piece(pi);
+      for (uint32_t ci = 0; ok && ci < pc.n; ++ci, ++cg) {
         const uint32_t buf = cg & 1u;
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm.ctl);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t np = parts_of(block_of(ci));
+        const uint32_t np = parts_of(pc.block(ci));
         for (uint32_t part = 0; part < np; ++part, ++ie) {
           const uint32_t s = ie % kStages;
           uint32_t v[32];
@@ -1400,8 +1454,10 @@ cudaError_t launch_subspace_reconstruct(const float* Xt, const int32_t* ids, con
       !make_map(&m.o32, Xhat, d, n_tok, 32, CU_TENSOR_MAP_SWIZZLE_128B))
     return cudaErrorInvalidValue;
   cudaError_t e;
-  const unsigned grid = persistent_grid(n_tok, &e);
+  const uint64_t sms = (uint64_t)sm_count(&e);
   if (e != cudaSuccess) return e;
+  const uint64_t units = ((n_tok + kRows - 1) / kRows) * ((d + kBlockN - 1) / kBlockN);   // (sub-tile, block) pairs
+  const unsigned grid = (unsigned)(units < sms ? units : sms);
   if (!ids) {                                        // no embedding terms: two MMA-issuing warps, two rings of U
     const int gsmem = (int)sizeof(GradSmem) + 1024;
     e = cudaFuncSetAttribute(subspace_reconstruct_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gsmem);
