@@ -192,6 +192,31 @@ def test_exact_on_every_cta_with_two_sub_tiles_each(d, k):
     assert f == 0 and np.array_equal(gh, (Xt.astype(np.float64) @ U.astype(np.float64).T).astype(np.float32))
 
 
+@pytest.mark.parametrize("extra_sub_tiles,extra_tokens,d,k", [
+    (1, 0, 1024, 64),       # one sub-tile left over: shared by more CTAs than it has blocks, most get nothing of it
+    (41, 17, 256, 64),      # 42 left over (the last ragged): three CTAs share each, two blocks do not split evenly
+    (74, 0, 320, 32),       # half as many left over as CTAs: two share each; d ends in a 64-column block
+    (-100, 5, 1024, 128),   # fewer sub-tiles than CTAs: nobody has a whole one
+])
+def test_reconstruction_exact_where_ctas_share_a_sub_tile(extra_sub_tiles, extra_tokens, d, k):
+    # The reconstruction deals whole sub-tiles of 128 tokens evenly and cuts the remaining ones by 128-column
+    # blocks among several CTAs.  Exact arithmetic (dyadic values, identity columns), so every entry must match
+    # the checker bit for bit in both forms: a block done twice shows nothing here, but a block left out (the
+    # output is filled with 7 beforehand) or gathered for the wrong rows does.
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    n_tok, L, V = (sms + extra_sub_tiles) * 128 + extra_tokens, 48, 200
+    rng = np.random.default_rng(1000 + extra_sub_tiles)
+    U = np.zeros((d, k), dtype=np.float32)
+    U[rng.permutation(d)[:k], np.arange(k)] = 1.0
+    q = lambda shape, m: (rng.integers(-m, m + 1, size=shape) / 4.0).astype(np.float32)
+    Xt, T_perp, pos = q((n_tok, k), 16), q((V, d), 8), q((L, d), 8)
+    ids = rng.integers(0, V, size=n_tok).astype(np.int32)
+    xh, f = _reconstruct(Xt, ids, T_perp, pos, U, L)
+    assert f == 0 and np.array_equal(xh, osub.reconstruct(Xt, ids, T_perp, pos, U, L).astype(np.float32))
+    gh, f = _reconstruct(Xt, None, None, None, U, L)
+    assert f == 0 and np.array_equal(gh, (Xt.astype(np.float64) @ U.astype(np.float64).T).astype(np.float32))
+
+
 def test_round_trip_is_lossless_for_residuals_in_the_subspace():
     n_tok, L, V, d, k = 1500, 256, 400, 1024, 128
     u = _dev(synth.gen_subspace_basis(d, k, seed=6))
