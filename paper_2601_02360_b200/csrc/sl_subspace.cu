@@ -760,6 +760,282 @@ subspace_project_dual_gather_kernel(const __grid_constant__ ProjMaps maps, const
   if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
 }
 
+// --------------------------- the same when the batch is a whole number of PAIRS of sequences of L tokens
+// (L a multiple of 32): sub-tile B is not the 128 tokens after sub-tile A but the same positions of the next
+// sequence, L tokens on, so that row r of B has the position row of row r of A and a thread fetches it once
+// for both (a quarter less to gather; 0.222 -> 0.213 ms at 64K tokens).  The work is dealt in units of 32
+// positions x 2 sequences, up to four units to a pass; a pass may cross from one pair of sequences to the
+// next, its tiles then come in as boxes of 32 rows.
+struct PairPass {
+  uint64_t c;               // where the pass starts in the CTA's range of units
+  uint32_t h;               // its units: groups of 32 tokens in A and in B
+};
+struct PairSched {
+  uint64_t lo, hi, L;
+  uint32_t per;             // units in a sequence
+  __device__ __forceinline__ PairSched(const SubParams& p) {
+    L = p.L;
+    per = p.L / 32;
+    const uint64_t n = (p.n_tok / (2 * (uint64_t)p.L)) * per;
+    lo = (uint64_t)blockIdx.x * n / gridDim.x;
+    hi = (uint64_t)(blockIdx.x + 1) * n / gridDim.x;
+  }
+  // the pass that starts at c (false: none); next = where the one after it starts
+  __device__ __forceinline__ bool at(uint64_t c, PairPass& ps, uint64_t& next) const {
+    if (c >= hi) return false;
+    const uint64_t left = hi - c;
+    ps.c = c;
+    ps.h = (uint32_t)(left < 4 ? left : 4);
+    next = c + ps.h;
+    return true;
+  }
+  // first token of group j of sub-tile A / B
+  __device__ __forceinline__ uint64_t ta(uint64_t c, uint32_t j) const {
+    const uint32_t u = (uint32_t)c + j, sp = u / per;              // (the host checks that the units fit 32 bits)
+    return (uint64_t)sp * 2 * L + (uint64_t)(u - sp * per) * 32;
+  }
+  __device__ __forceinline__ uint64_t tb(uint64_t c, uint32_t j) const { return ta(c, j) + L; }
+  // the four groups of a sub-tile are 128 consecutive tokens
+  __device__ __forceinline__ bool whole(const PairPass& ps) const { return ps.h == 4 && (uint32_t)ps.c % per + 3 < per; }
+};
+
+__global__ void __launch_bounds__(kThreadsG, 1)
+subspace_project_dual_samepos_kernel(const __grid_constant__ ProjMaps maps, const __grid_constant__ SubParams p) {
+  extern __shared__ uint8_t raw[];
+  DualSmem& sm = *reinterpret_cast<DualSmem*>(((uintptr_t)raw + 1023) & ~(uintptr_t)1023);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t k_tiles = (p.d + kTileK - 1) / kTileK;
+  const PairSched sc(p);
+  if (tid == 0) {
+    for (int s = 0; s < kRingD; ++s) { mbar_init(&sm.full[s], 3); mbar_init(&sm.ready[s], kRowWarpsG); mbar_init(&sm.empty[s], 1); }
+    mbar_init(&sm.p_done, 1);
+    mbar_init(&sm.p_free, kRowWarpsG);
+    mbar_init(&sm.mma_idle, 1);
+    sm.ctl.abort = 0;
+    sm.ctl.polls = p.wait_polls;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t t_p = sm.tmem_base;      // accumulator of sub-tile A; B is 256 columns further
+  bool bad = false;
+
+  if (warp == 0 || warp == 2 || warp == 3) {
+    if (lane == 0) {
+      const uint32_t pi = warp == 0 ? 0u : (uint32_t)warp - 1u;
+      const uint32_t nb = p.kp / 32;
+      const uint32_t lo = pi == 0 ? 0u : (pi * nb + 1) / 3, hi = pi == 2 ? nb : ((pi + 1) * nb + 1) / 3;
+      uint32_t it = 0;
+      bool ok = true;
+      PairPass ps;
+      for (uint64_t c = sc.lo, cn; ok && sc.at(c, ps, cn); c = cn) {
+        const uint32_t ha = ps.h, hb = ps.h;
+        const bool wa = sc.whole(ps), wb = wa;
+        int ra[4], rb[4];
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) { ra[i] = (int)sc.ta(ps.c, i); rb[i] = (int)sc.tb(ps.c, i); }
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRingD;
+          ok = mbar_wait(&sm.empty[s], ((it / kRingD) & 1u) ^ 1u, sm.ctl);
+          if (!ok) break;
+          uint8_t* slot = sm.ring + s * kSlotD;
+          mbar_expect_tx(&sm.full[s], (pi == 0 ? (ha + hb) * 4096 : 0u) + (hi - lo) * 4096);
+          if (pi == 0) {
+            if (wa) tma_load_2d(slot, &maps.x128, (int)(kt * kTileK), ra[0], &sm.full[s]);
+            else {
+#pragma unroll
+              for (uint32_t i = 0; i < 4; ++i)
+                if (i < ha) tma_load_2d(slot + i * 4096, &maps.x32, (int)(kt * kTileK), ra[i], &sm.full[s]);
+            }
+            if (wb) tma_load_2d(slot + kSlotA, &maps.x128, (int)(kt * kTileK), rb[0], &sm.full[s]);
+            else {
+#pragma unroll
+              for (uint32_t i = 0; i < 4; ++i)
+                if (i < hb) tma_load_2d(slot + kSlotA + i * 4096, &maps.x32, (int)(kt * kTileK), rb[i], &sm.full[s]);
+            }
+          }
+          for (uint32_t n = lo; n < hi; ++n)
+            tma_load_2d(slot + 2 * kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full[s]);
+        }
+      }
+      if (!ok)
+        for (uint32_t s = 0; s < (uint32_t)kRingD; ++s) landed(&sm.full[s], ring_uses(it, s, kRingD));
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      uint32_t it = 0, t = 0;
+      bool ok = true;
+      const uint32_t idesc = instr_desc(kRows, (int)p.kp, 1);
+      const uint64_t desc_k = smem_desc(0, 16, 1024, 2), desc_n = smem_desc(0, 4096, 512, 1);
+      PairPass ps;
+      for (uint64_t c = sc.lo, cn; ok && sc.at(c, ps, cn); c = cn, ++t) {
+        if (t > 0) {
+          ok = mbar_wait(&sm.p_free, (t - 1) & 1u, sm.ctl);
+          if (!ok) break;
+          tc_fence_after();
+        }
+        for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+          const uint32_t s = it % kRingD;
+          ok = mbar_wait(&sm.ready[s], (it / kRingD) & 1u, sm.ctl);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(sm.ring + s * kSlotD);
+          const uint64_t da = desc_k | (uint64_t)((a0 >> 4) & 0x3FFF);
+          const uint64_t da2 = desc_k | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+          const uint64_t db = desc_n | (uint64_t)(((a0 + 2 * kSlotA) >> 4) & 0x3FFF);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_ss(t_p, da + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mma_ss(t_p + 256, da2 + 2 * j, db + 64 * j, idesc, (kt | (uint32_t)j) != 0);
+          mma_commit(&sm.empty[s]);
+        }
+        if (ok) mma_commit(&sm.p_done);
+      }
+      if (!ok) mma_quiesce(&sm.mma_idle);
+    }
+  } else {
+    // ---- sixteen row warps ----
+    const uint32_t q = (uint32_t)(warp & 3), sub = (uint32_t)(warp - 4) >> 2;      // sub 0..3: tile sub & 1, column blocks sub >> 1
+    const uint32_t row = 32u * q + (uint32_t)lane;
+    const uint32_t j = (uint32_t)(tid - 128), gch = j & 7u, grow = j >> 3;          // grow 0..63
+    const uint32_t goff = grow * 128 + ((gch ^ (grow & 7u)) << 4);                  // + 8192 i: row grow + 64 i of the pair
+    const bool wide = p.k % 8 == 0 && ((uintptr_t)p.out & 31u) == 0;
+    uint32_t it = 0, t = 0;
+    bool ok = true;
+    const float* tp[4];
+    const float* ps[2];
+    uint32_t mask = 0;
+    constexpr int kPosRows = 2;                     // rows i and i + 2 of a thread share their position row
+    float4 nt[4], np_[kPosRows];                    // the values of the K step after the current one
+    auto fetch = [&](uint32_t kt) {
+      const uint32_t col = kt * kTileK + 4u * gch;
+      const bool in_col = kt < k_tiles && col < p.d;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const bool in = in_col && ((mask >> i) & 1u);
+        nt[i] = in ? __ldg(reinterpret_cast<const float4*>(tp[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < kPosRows) {
+          const bool inp = in_col && ((mask >> (4 + i)) & 1u);
+          np_[i] = inp ? __ldg(reinterpret_cast<const float4*>(ps[i] + kt * kTileK)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    };
+    // mask bit i: row i has terms.  The position row of rows i and i + 2 is fetched once, under bit 4 + i,
+    // when either of them has terms (a token id out of range leaves only its own row without)
+    auto open_tile = [&](const PairPass& pp) {
+      mask = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t r = (grow + 64u * (uint32_t)i) & 127u, gj = r >> 5;             // row of its sub-tile, its group
+        const bool in_b = i >= 2;
+        const RowInfo ri = row_info(p, in_b ? sc.tb(pp.c, gj) : sc.ta(pp.c, gj), pp.h > gj ? 32u : 0u, r & 31u, bad);
+        tp[i] = ri.gather ? ri.tp + 4 * gch : nullptr;
+        mask |= ri.gather ? 1u << i : 0u;
+        if (ri.gather) { ps[i & 1] = ri.ps + 4 * gch; mask |= 16u << (i & 1); }
+      }
+      fetch(0);
+    };
+    // only where the pass starts is carried through the loop; what it covers is worked out again where needed
+    uint64_t c = sc.lo;
+    {
+      PairPass first;
+      uint64_t cn;
+      if (sc.at(c, first, cn)) open_tile(first);
+    }
+    for (; ok && c < sc.hi; ++t) {
+      PairPass cur;
+      uint64_t cn;
+      sc.at(c, cur, cn);
+      for (uint32_t kt = 0; ok && kt < k_tiles; ++kt, ++it) {
+        float4 ct[4], cp[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          ct[i] = nt[i];
+          cp[i] = (mask >> i) & 1u ? np_[i & 1] : make_float4(0.f, 0.f, 0.f, 0.f);       // (none for a row without terms)
+        }
+        fetch(kt + 1);
+        const uint32_t s = it % kRingD;
+        ok = mbar_wait(&sm.full[s], (it / kRingD) & 1u, sm.ctl);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint32_t a0 = smem_u32(sm.ring + s * kSlotD) + goff;
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) {
+          {
+            const uint32_t a = a0 + 8192u * i;
+            float4 v = lds128(a);
+            v.x = __fsub_rn(__fsub_rn(v.x, ct[i].x), cp[i].x);
+            v.y = __fsub_rn(__fsub_rn(v.y, ct[i].y), cp[i].y);
+            v.z = __fsub_rn(__fsub_rn(v.z, ct[i].z), cp[i].z);
+            v.w = __fsub_rn(__fsub_rn(v.w, ct[i].w), cp[i].w);
+            v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+            v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+            v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+            v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+            sts128(a, v);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.ready[s]);
+      }
+      if (!ok) break;
+      {
+        PairPass nxt;
+        uint64_t cnn;
+        if (sc.at(cn, nxt, cnn)) open_tile(nxt);
+      }
+      ok = mbar_wait(&sm.p_done, t & 1u, sm.ctl);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      {
+        const uint32_t tile = sub & 1u;
+        const uint32_t h = cur.h * 32;
+        const uint64_t tok = (tile ? sc.tb(cur.c, q) : sc.ta(cur.c, q)) + (uint64_t)lane;   // row = 32 q + lane: group q of the sub-tile
+        if (h) {
+          for (uint32_t cb = 32u * (sub >> 1); cb < p.kp; cb += 64) {
+            uint32_t v[32];
+            tmem_ld32(t_p + tile * 256 + cb + ((32u * q) << 16), v);
+            tmem_ld_wait();
+            if (row < h && tok < p.n_tok) {
+              float* dst = p.out + tok * (uint64_t)p.k + cb;
+              if (wide) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 8)
+                  if (cb + (uint32_t)i < p.k) stg256(dst + i, v + i);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                  if (cb + (uint32_t)i < p.k)
+                    *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
+                                                                      __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.p_free);
+      c = cn;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(t_p), "r"(512) : "memory");
+  }
+  if (bad && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_BAD_INDEX);
+  if (tid == 0 && sm.ctl.abort && p.flags) atomicOr(p.flags, (uint32_t)SL_FLAG_TIMEOUT);
+}
+
 // --------------------------------------------------------------------------------------- reconstruct
 // Per sub-tile of 128 tokens the Xt tile goes through a two-slot staging buffer into tensor memory
 // (rounded to TF32 on the way) and is the A operand of every 128-column block.  The embedding and
@@ -1415,9 +1691,12 @@ cudaError_t launch_subspace_project(const float* X, const int32_t* ids, const fl
     // at least two sub-tiles for every CTA: two sub-tiles share every U slice
     const int smem = (int)sizeof(DualSmem) + 1024;
     if (ids) {
-      e = cudaFuncSetAttribute(subspace_project_dual_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+      // a whole number of pairs of sequences: the two sub-tiles of a pass are the same positions of two sequences
+      const bool same_pos = L >= 32 && L % 32 == 0 && n_tok % (2ull * L) == 0 && n_tok / 32 < 0xFFFFFFF0ull;
+      auto kern = same_pos ? subspace_project_dual_samepos_kernel : subspace_project_dual_gather_kernel;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       if (e != cudaSuccess) return e;
-      subspace_project_dual_gather_kernel<<<grid, kThreadsG, smem, st>>>(m, p);
+      kern<<<grid, kThreadsG, smem, st>>>(m, p);
       return cudaGetLastError();
     }
     e = cudaFuncSetAttribute(subspace_project_dual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);

@@ -247,6 +247,39 @@ def test_bad_token_id_is_flagged_and_gathers_nothing():
     assert np.all(np.abs(xt[[3, 40]] - plain) <= TOL * (np.abs(X[[3, 40]].astype(np.float64)) @ np.abs(U.astype(np.float64))))
 
 
+@pytest.mark.parametrize("L,extra_pairs,d,k", [
+    (128, 2, 256, 64),      # four units of 32 positions in a sequence: passes cross from one pair of sequences to the next
+    (96, 60, 256, 32),      # three units in a sequence: no pass is 128 consecutive tokens
+    (2048, 0, 256, 64),     # the benchmark's sequence length: 64 units in a sequence, passes of 128 consecutive tokens
+])
+def test_projection_exact_where_a_pass_pairs_two_sequences(L, extra_pairs, d, k):
+    # A batch that is a whole number of pairs of sequences, with two sub-tiles or more for every CTA: the
+    # projection with embedding terms pairs the same positions of two sequences and fetches a position row once
+    # for both.  Exact arithmetic (dyadic values, identity columns): bit for bit against the checker.  Then two
+    # token ids out of range, one in each sequence of a pair at the SAME position: each leaves only its own row
+    # without terms, the row that shares its position row keeps them.
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    pairs = -(-sms * 256 // (2 * L)) + extra_pairs
+    n_tok, V = pairs * 2 * L, 300
+    rng = np.random.default_rng(L + d)
+    U = np.zeros((d, k), dtype=np.float32)
+    U[rng.permutation(d)[:k], np.arange(k)] = 1.0
+    q = lambda shape, m: (rng.integers(-m, m + 1, size=shape) / 4.0).astype(np.float32)
+    X, T_perp, pos = q((n_tok, d), 8), q((V, d), 8), q((L, d), 8)
+    ids = rng.integers(0, V, size=n_tok).astype(np.int32)
+    want = osub.project(X, ids, T_perp, pos, U, L)
+    xt, f = _project(X, ids, T_perp, pos, U, L)
+    assert f == 0 and np.array_equal(xt, want.astype(np.float32))
+    bad_a, bad_b = 2 * L * 3 + 17, 2 * L * 5 + L + 40 % L              # first sequence of pair 3, second of pair 5
+    ids2 = ids.copy()
+    ids2[bad_a], ids2[bad_b] = V + 7, -2
+    xt2, f = _project(X, ids2, T_perp, pos, U, L)
+    assert f == api.SL_FLAG_BAD_INDEX
+    want2 = want.copy()
+    want2[[bad_a, bad_b]] = X[[bad_a, bad_b]].astype(np.float64) @ U.astype(np.float64)     # no terms for those rows
+    assert np.array_equal(xt2, want2.astype(np.float32))
+
+
 @pytest.mark.parametrize("n_tok,L,V,d,k", [(50, 10, 7, 1536, 2), (33, 5, 4, 10, 3), (20, 4, 6, 64, 300)])
 def test_shapes_outside_the_tensor_core_path(n_tok, L, V, d, k):
     rng = np.random.default_rng(11)

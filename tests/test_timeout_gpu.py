@@ -97,6 +97,7 @@ def test_tensor_core_kernels_give_up_cleanly(wait_limit, polls):
         api.sl_embed_reproject(d_ts, d_tp, d_u, V, d, k, flags)
         api.sl_subspace_project(d_x, d_ids, d_tp2, d_pos, d_u, n_tok, L, V, d, k, d_xt, flags)
         api.sl_subspace_project(d_x, None, None, None, d_u, n_tok, L, 0, d, k, d_xt, flags)     # the two-sub-tile form
+        api.sl_subspace_project(d_x, d_ids, d_tp2, d_pos, d_u, n_tok // (2 * L) * 2 * L, L, V, d, k, d_xt, flags)   # pairs of sequences
         api.sl_subspace_reconstruct(d_xt, d_ids, d_tp2, d_pos, d_u, n_tok, L, V, d, k, d_xh, flags)
         api.sl_subspace_reconstruct(d_xt, None, None, None, d_u, n_tok, L, 0, d, k, d_xh, flags)    # two MMA warps, two rings
         torch.cuda.synchronize()
