@@ -79,6 +79,10 @@ __device__ __forceinline__ uint8_t* ring2_slot(EmbedSmem& sm, uint32_t s) {
   return s < (uint32_t)kRing2InX ? sm.x + kEBufs * kESize + s * kSlot2 : sm.y[s - kRing2InX];
 }
 
+// PAIR (k <= 128, more than one sub-tile per CTA): two sub-tiles A and B go through pass 1 together and share
+// every slice of U - a slot holds their two T_S tiles and at most 16 KB of U, their coordinates lie side by
+// side in tensor memory (columns [0, 128) and [128, 256)) - then pass 2 runs for A and for B.
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d, uint32_t kp, uint32_t* flags,
                        uint32_t wait_polls) {
@@ -92,6 +96,10 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
   // this CTA's rows: groups [g0, g1) of 32 rows
   const uint64_t G = (V + 31) / 32;
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  constexpr uint64_t kStep = PAIR ? 8 : 4;                  // groups of 32 rows per turn of the loops below
+  constexpr uint32_t kUoff = PAIR ? 2 * kSlotA : kSlotA;    // where the slice of U lies in a pass-1 slot
+  auto groups_a = [&](uint64_t g) { return (uint32_t)(g1 - g < 4 ? g1 - g : 4); };
+  auto groups_b = [&](uint64_t g) { return !PAIR || g + 4 >= g1 ? 0u : (uint32_t)(g1 - g - 4 < 4 ? g1 - g - 4 : 4); };
 
   if (tid == 0) {
     for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 3); mbar_init(&sm.ready1[s], 4); mbar_init(&sm.empty1[s], 1); }
@@ -130,7 +138,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       const uint32_t lo = warp == 8 ? u_split1 : u_split2, hi = warp == 8 ? u_split2 : u_boxes;
       uint32_t it1 = 0, t = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      for (uint64_t g = g0; ok && g < g1; g += kStep, ++t) {
         if (t > 0) ok = mbar_wait(&sm.x_free, (t - 1) & 1u, sm);
         for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
           const uint32_t s = it1 % kRing1;
@@ -139,7 +147,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           uint8_t* slot = sm.x + s * kSlot1;
           mbar_expect_tx(&sm.full1[s], (hi - lo) * 4096);
           for (uint32_t n = lo; n < hi; ++n)
-            tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
+            tma_load_2d(slot + kUoff + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
         }
       }
       if (!ok)
@@ -150,8 +158,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       // ---- operand producer: T_S tiles and (its share of) U for pass 1, U for pass 2 ----
       uint32_t it1 = 0, it2 = 0, t = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+      for (uint64_t g = g0; ok && g < g1; g += kStep, ++t) {
+        const uint32_t hg = groups_a(g), hb = groups_b(g), h = (hg + hb) * 32;
         const int r0 = (int)(g * 32);
         // the pass-1 ring lies over the pass-2 buffers of the previous sub-tile: wait until its last tile
         // store has left shared memory (by then its MMAs have long read their ring slots).  Waits that
@@ -170,18 +178,26 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
             for (uint32_t i = 0; i < hg; ++i)
               tma_load_2d(slot + i * 4096, &maps.ts32, (int)(kt * kTileK), r0 + 32 * (int)i, &sm.full1[s]);
           }
+          if (PAIR) {
+            if (hb == 4) {
+              tma_load_2d(slot + kSlotA, &maps.ts128, (int)(kt * kTileK), r0 + kRows, &sm.full1[s]);
+            } else {
+              for (uint32_t i = 0; i < hb; ++i)
+                tma_load_2d(slot + kSlotA + i * 4096, &maps.ts32, (int)(kt * kTileK), r0 + kRows + 32 * (int)i, &sm.full1[s]);
+            }
+          }
           for (uint32_t n = 0; n < u_split1; ++n)      // the other boxes of the slice come from warps 8 and 9
-            tma_load_2d(slot + kSlotA + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
+            tma_load_2d(slot + kUoff + n * 4096, &maps.u_n, (int)(n * 32), (int)(kt * kTileK), &sm.full1[s]);
         }
         // ... and the pass-2 ring lies over the pass-1 ring: its last MMAs must have read it
         ok = ok && mbar_wait(&sm.p_done, t & 1u, sm);
-        for (uint32_t c = 0; ok && c < n_blocks; ++c)
+        for (uint32_t c = 0; ok && c < n_blocks * (hb ? 2u : 1u); ++c)     // (PAIR: the blocks of A, then those of B)
           for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it2) {
             const uint32_t s = it2 % kRing2;
             ok = mbar_wait(&sm.empty2[s], ((it2 / kRing2) & 1u) ^ 1u, sm);
             if (!ok) break;
             mbar_expect_tx(&sm.full2[s], kSlot2);
-            tma_load_2d(ring2_slot(sm, s), &maps.u_k, (int)(kt * kTileK), (int)(c * kBlockN), &sm.full2[s]);
+            tma_load_2d(ring2_slot(sm, s), &maps.u_k, (int)(kt * kTileK), (int)((c >= n_blocks ? c - n_blocks : c) * kBlockN), &sm.full2[s]);
           }
       }
       if (!ok) {
@@ -194,11 +210,12 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       // ---- tile producer: the T_S / T_perp tiles of each 32-column part of pass 2 ----
       uint32_t hcg = 0, t = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
-        const int r0 = (int)(g * 32);
+      for (uint64_t g = g0; ok && g < g1; g += kStep, ++t) {
         // the tile buffers lie over the pass-1 ring: wait until this sub-tile's pass 1 has read it
         ok = mbar_wait(&sm.p_done, t & 1u, sm);
+       for (uint32_t sub = 0; ok && sub < (groups_b(g) ? 2u : 1u); ++sub) {
+        const uint32_t hg = sub ? groups_b(g) : groups_a(g), h = hg * 32;
+        const int r0 = (int)(g * 32) + (int)sub * kRows;
         for (uint32_t hb = 0; ok && hb < n_parts; ++hb, ++hcg) {
           const uint32_t b = hcg % kEBufs;
           ok = wait_last(&sm.e_empty[b], hcg / kEBufs);
@@ -217,6 +234,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
             }
           }
         }
+       }
       }
       if (!ok)
         for (uint32_t b = 0; b < (uint32_t)kEBufs; ++b) landed(&sm.e_full[b], ring_uses(hcg, b, kEBufs));
@@ -226,9 +244,10 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       // ---- tile store: writes each finished part back and frees its buffer ----
       uint32_t hcg = 0;
       bool ok = true;
-      for (uint64_t g = g0; ok && g < g1; g += 4) {
-        const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4);
-        const int r0 = (int)(g * 32);
+      for (uint64_t g = g0; ok && g < g1; g += kStep) {
+       for (uint32_t sub = 0; ok && sub < (groups_b(g) ? 2u : 1u); ++sub) {
+        const uint32_t hg = sub ? groups_b(g) : groups_a(g);
+        const int r0 = (int)(g * 32) + (int)sub * kRows;
         for (uint32_t hb = 0; ok && hb < n_parts; ++hb, ++hcg) {
           const uint32_t b = hcg % kEBufs;
           ok = mbar_wait(&sm.e_done[b], (hcg / kEBufs) & 1u, sm);
@@ -243,6 +262,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           bulk_wait_read_all();          // the copies have read the buffer: the tile producer may refill it
           mbar_arrive(&sm.e_empty[b]);
         }
+       }
         if (ok) mbar_arrive(&sm.x_free);  // the next sub-tile's operand ring may overwrite the buffers
       }
       bulk_wait_all();
@@ -256,7 +276,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       const uint32_t idesc2 = instr_desc(kRows, kBlockN, 0);
       const uint64_t desc_k = smem_desc(0, 16, 1024, 2);      // K-major tile, rows of 128 bytes
       const uint64_t desc_n = smem_desc(0, 4096, 512, 1);     // U rows as N-major operand
-      for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
+      for (uint64_t g = g0; ok && g < g1; g += kStep, ++t) {
+        const bool two = groups_b(g) != 0;
         for (uint32_t kt = 0; ok && kt < k_tiles1; ++kt, ++it1) {
           const uint32_t s = it1 % kRing1;
           ok = mbar_wait(&sm.ready1[s], (it1 / kRing1) & 1u, sm);      // landed and rounded (see the epilogue warps)
@@ -264,15 +285,21 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           tc_fence_after();
           const uint32_t a0 = smem_u32(sm.x + s * kSlot1);
           const uint64_t da = desc_k | (uint64_t)((a0 >> 4) & 0x3FFF);
-          const uint64_t db = desc_n | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+          const uint64_t db = desc_n | (uint64_t)(((a0 + kUoff) >> 4) & 0x3FFF);
 #pragma unroll
           for (int j = 0; j < 4; ++j)   // K = 8 per instruction: 32 bytes along a swizzled row of A, 8 rows of U
             mma_ss(t_p, da + 2 * j, db + 64 * j, idesc1, (kt | (uint32_t)j) != 0);
+          if (PAIR && two) {
+            const uint64_t da2 = desc_k | (uint64_t)(((a0 + kSlotA) >> 4) & 0x3FFF);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) mma_ss(t_p + 128, da2 + 2 * j, db + 64 * j, idesc1, (kt | (uint32_t)j) != 0);
+          }
           mma_commit(&sm.empty1[s]);
         }
         if (ok) mma_commit(&sm.p_done);
         ok = ok && mbar_wait(&sm.p_ready, t & 1u, sm);   // the epilogue warps have rounded P in place
-        for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+        for (uint32_t c = 0; ok && c < n_blocks * (two ? 2u : 1u); ++c, ++cg) {
+          const uint32_t t_pa = t_p + (c >= n_blocks ? 128u : 0u);          // the coordinates of A, then of B
           const uint32_t buf = cg & 1u;
           ok = wait_last(&sm.o_empty[buf], cg >> 1);
           if (!ok) break;
@@ -285,7 +312,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
             const uint64_t db = desc_k | (uint64_t)((smem_u32(ring2_slot(sm, s)) >> 4) & 0x3FFF);
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              mma_ts(t_o + buf * kBlockN, t_p + kt * kTileK + 8 * j, db + 2 * j, idesc2, (kt | (uint32_t)j) != 0);
+              mma_ts(t_o + buf * kBlockN, t_pa + kt * kTileK + 8 * j, db + 2 * j, idesc2, (kt | (uint32_t)j) != 0);
             mma_commit(&sm.empty2[s]);
           }
           if (!ok) break;
@@ -301,8 +328,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
     const uint32_t sw = row & 7u;
     uint32_t cg = 0, hcg = 0, t = 0, it1 = 0;
     bool ok = true;
-    for (uint64_t g = g0; ok && g < g1; g += 4, ++t) {
-      const uint32_t hg = (uint32_t)(g1 - g < 4 ? g1 - g : 4), h = hg * 32;
+    for (uint64_t g = g0; ok && g < g1; g += kStep, ++t) {
+      const uint32_t hgb = groups_b(g);
       // The tensor cores CUT a float32 operand to TF32, which would shorten every product; values that
       // are already TF32 pass through unchanged.  So during pass 1 these warps round every T_S tile to the
       // nearest TF32 value in place as soon as it has landed (element-wise: the swizzle is irrelevant) and
@@ -323,6 +350,17 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
           sts128(a0 + 2048 * i, v);
         }
+        if (PAIR && hgb) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float4 v = lds128(a0 + kSlotA + 2048 * i);
+            v.x = __uint_as_float(round_tf32(__float_as_uint(v.x)));
+            v.y = __uint_as_float(round_tf32(__float_as_uint(v.y)));
+            v.z = __uint_as_float(round_tf32(__float_as_uint(v.z)));
+            v.w = __uint_as_float(round_tf32(__float_as_uint(v.w)));
+            sts128(a0 + kSlotA + 2048 * i, v);
+          }
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.ready1[s]);
@@ -332,20 +370,23 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      for (uint32_t cb = 0; cb < kp; cb += 32) {
-        uint32_t v[32];
-        const uint32_t ta = t_p + cb + ((uint32_t)(32 * q) << 16);
-        tmem_ld32(ta, v);
-        tmem_ld_wait();
+      for (uint32_t half = 0; half < (hgb ? 2u : 1u); ++half)
+        for (uint32_t cb = 0; cb < kp; cb += 32) {
+          uint32_t v[32];
+          const uint32_t ta = t_p + 128 * half + cb + ((uint32_t)(32 * q) << 16);
+          tmem_ld32(ta, v);
+          tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = round_tf32(v[i]);
-        tmem_st32(ta, v);
-      }
+          for (int i = 0; i < 32; ++i) v[i] = round_tf32(v[i]);
+          tmem_st32(ta, v);
+        }
       tmem_st_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.p_ready);
-      for (uint32_t c = 0; ok && c < n_blocks; ++c, ++cg) {
+      for (uint32_t cc = 0; ok && cc < n_blocks * (hgb ? 2u : 1u); ++cc, ++cg) {
+        const uint32_t c = cc >= n_blocks ? cc - n_blocks : cc;               // the blocks of A, then those of B
+        const uint32_t h = (cc >= n_blocks ? hgb : groups_a(g)) * 32;
         const uint32_t buf = cg & 1u;
         const uint32_t left = (d - c * kBlockN + kPartN - 1) / kPartN;
         const uint32_t np = left < 4 ? left : 4;      // parts of this block that exist
@@ -483,14 +524,18 @@ cudaError_t launch_embed_reproject(float* T_S, float* T_perp, const float* U, ui
       !make_map(&m.u_k, U, k, d, kBlockN, CU_TENSOR_MAP_SWIZZLE_128B))
     return cudaErrorInvalidValue;
   const int smem = (int)sizeof(EmbedSmem) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(embed_reproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-  if (e != cudaSuccess) return e;
+  cudaError_t e;
   const int sms = sm_count(&e);
   if (e != cudaSuccess) return e;
   const uint32_t kp = (k + 31u) & ~31u;
   const uint64_t tiles = (V + kRows - 1) / kRows;          // never more CTAs than full sub-tiles
   const unsigned grid = (unsigned)(tiles < (uint64_t)sms ? tiles : (uint64_t)sms);
-  embed_reproject_kernel<<<grid, kThreads, smem, st>>>(m, V, d, kp, flags, debug_wait_polls());
+  // more than four groups of 32 rows for every CTA and room for two coordinate tiles: two sub-tiles share pass 1
+  const bool pair = kp <= 128 && (V + 31) / 32 > 4ull * grid;
+  auto kern = pair ? embed_reproject_kernel<true> : embed_reproject_kernel<false>;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kThreads, smem, st>>>(m, V, d, kp, flags, debug_wait_polls());
   return cudaGetLastError();
 }
 

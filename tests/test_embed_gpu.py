@@ -152,7 +152,8 @@ def _hadamard(n):
     return H
 
 
-@pytest.mark.parametrize("d,k,kind", [(1024, 128, "hadamard"), (2048, 256, "identity"), (256, 64, "hadamard")])
+@pytest.mark.parametrize("d,k,kind", [(1024, 128, "hadamard"), (2048, 256, "identity"), (256, 64, "hadamard"),
+                                      (640, 100, "identity")])
 def test_exact_on_every_cta_with_two_sub_tiles_each(d, k, kind):
     # enough rows for at least two sub-tiles on every CTA (148 x 256 and a ragged rest), dyadic entries
     # and a basis of identity or +-1/sqrt(d) Hadamard columns (d a power of 4): every product, every sum
