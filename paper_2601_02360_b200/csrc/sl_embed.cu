@@ -56,7 +56,7 @@ struct EmbedSmem {
   uint8_t x[kRing1 * kSlot1];                   // pass 1: operand ring; pass 2: tile buffers + ring slots
   uint8_t y[kRing2 - kRing2InX][kSlot2];
   uint64_t full1[kRing1], ready1[kRing1], empty1[kRing1], full2[kRing2], empty2[kRing2];
-  uint64_t o_full[2], o_empty[2], e_full[kEBufs], e_empty[kEBufs], e_done[kEBufs];
+  uint64_t o_full[2], o_empty[2], e_full[kEBufs + 1], e_empty[kEBufs + 1], e_done[kEBufs + 1];
   uint64_t p_done, x_free;   // per sub-tile: pass 1 has read its ring / pass 2 has left the shared region
   uint64_t p_ready;          // per sub-tile: the coordinates in tensor memory have been rounded to TF32
   uint64_t mma_idle;         // after a give-up only: the MMAs issued so far have retired
@@ -75,10 +75,6 @@ struct Maps {
   CUtensorMap u_k;                        // U, box 128 rows (d) x 32 floats (k)
 };
 
-__device__ __forceinline__ uint8_t* ring2_slot(EmbedSmem& sm, uint32_t s) {
-  return s < (uint32_t)kRing2InX ? sm.x + kEBufs * kESize + s * kSlot2 : sm.y[s - kRing2InX];
-}
-
 // PAIR (k <= 128, more than one sub-tile per CTA): two sub-tiles A and B go through pass 1 together and share
 // every slice of U - a slot holds their two T_S tiles and at most 16 KB of U, their coordinates lie side by
 // side in tensor memory (columns [0, 128) and [128, 256)) - then pass 2 runs for A and for B.
@@ -96,6 +92,14 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
   // this CTA's rows: groups [g0, g1) of 32 rows
   const uint64_t G = (V + 31) / 32;
   const uint64_t g0 = (uint64_t)blockIdx.x * G / gridDim.x, g1 = (uint64_t)(blockIdx.x + 1) * G / gridDim.x;
+  // PAIR: the U blocks of pass 2 are half as large (k <= 128), two ring slots are enough and the shared region
+  // holds a sixth tile buffer instead of the other two
+  constexpr int kEB = PAIR ? kEBufs + 1 : kEBufs, kR2 = PAIR ? 2 : kRing2, kR2X = PAIR ? 0 : kRing2InX;
+  static_assert(kEB * kESize + kR2X * kSlot2 == kRing1 * kSlot1, "pass-2 buffers fill the pass-1 ring");
+  auto r2slot = [&](uint32_t s2) -> uint8_t* {
+    if constexpr (kR2X == 0) return sm.y[s2];
+    else return s2 < (uint32_t)kR2X ? sm.x + kEB * kESize + s2 * kSlot2 : sm.y[s2 - kR2X];
+  };
   constexpr uint64_t kStep = PAIR ? 8 : 4;                  // groups of 32 rows per turn of the loops below
   constexpr uint32_t kUoff = PAIR ? 2 * kSlotA : kSlotA;    // where the slice of U lies in a pass-1 slot
   auto groups_a = [&](uint64_t g) { return (uint32_t)(g1 - g < 4 ? g1 - g : 4); };
@@ -103,9 +107,9 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
 
   if (tid == 0) {
     for (int s = 0; s < kRing1; ++s) { mbar_init(&sm.full1[s], 3); mbar_init(&sm.ready1[s], 4); mbar_init(&sm.empty1[s], 1); }
-    for (int s = 0; s < kRing2; ++s) { mbar_init(&sm.full2[s], 1); mbar_init(&sm.empty2[s], 1); }
+    for (int s = 0; s < kR2; ++s) { mbar_init(&sm.full2[s], 1); mbar_init(&sm.empty2[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&sm.o_full[b], 1); mbar_init(&sm.o_empty[b], 4); }
-    for (int b = 0; b < kEBufs; ++b) {
+    for (int b = 0; b < kEB; ++b) {
       mbar_init(&sm.e_full[b], 1); mbar_init(&sm.e_empty[b], 1); mbar_init(&sm.e_done[b], 4);
     }
     mbar_init(&sm.p_done, 1);
@@ -193,16 +197,16 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
         ok = ok && mbar_wait(&sm.p_done, t & 1u, sm);
         for (uint32_t c = 0; ok && c < n_blocks * (hb ? 2u : 1u); ++c)     // (PAIR: the blocks of A, then those of B)
           for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it2) {
-            const uint32_t s = it2 % kRing2;
-            ok = mbar_wait(&sm.empty2[s], ((it2 / kRing2) & 1u) ^ 1u, sm);
+            const uint32_t s = it2 % kR2;
+            ok = mbar_wait(&sm.empty2[s], ((it2 / kR2) & 1u) ^ 1u, sm);
             if (!ok) break;
             mbar_expect_tx(&sm.full2[s], kSlot2);
-            tma_load_2d(ring2_slot(sm, s), &maps.u_k, (int)(kt * kTileK), (int)((c >= n_blocks ? c - n_blocks : c) * kBlockN), &sm.full2[s]);
+            tma_load_2d(r2slot(s), &maps.u_k, (int)(kt * kTileK), (int)((c >= n_blocks ? c - n_blocks : c) * kBlockN), &sm.full2[s]);
           }
       }
       if (!ok) {
         for (uint32_t s = 0; s < (uint32_t)kRing1; ++s) landed(&sm.full1[s], ring_uses(it1, s, kRing1));
-        for (uint32_t s = 0; s < (uint32_t)kRing2; ++s) landed(&sm.full2[s], ring_uses(it2, s, kRing2));
+        for (uint32_t s = 0; s < (uint32_t)kR2; ++s) landed(&sm.full2[s], ring_uses(it2, s, kR2));
       }
     }
   } else if (warp == 6) {
@@ -217,8 +221,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
         const uint32_t hg = sub ? groups_b(g) : groups_a(g), h = hg * 32;
         const int r0 = (int)(g * 32) + (int)sub * kRows;
         for (uint32_t hb = 0; ok && hb < n_parts; ++hb, ++hcg) {
-          const uint32_t b = hcg % kEBufs;
-          ok = wait_last(&sm.e_empty[b], hcg / kEBufs);
+          const uint32_t b = hcg % kEB;
+          ok = wait_last(&sm.e_empty[b], hcg / kEB);
           if (!ok) break;
           const int x = (int)(hb * kPartN);
           uint8_t* ets = sm.x + b * kESize;
@@ -237,7 +241,7 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
        }
       }
       if (!ok)
-        for (uint32_t b = 0; b < (uint32_t)kEBufs; ++b) landed(&sm.e_full[b], ring_uses(hcg, b, kEBufs));
+        for (uint32_t b = 0; b < (uint32_t)kEB; ++b) landed(&sm.e_full[b], ring_uses(hcg, b, kEB));
     }
   } else if (warp == 7) {
     if (lane == 0) {
@@ -249,8 +253,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
         const uint32_t hg = sub ? groups_b(g) : groups_a(g);
         const int r0 = (int)(g * 32) + (int)sub * kRows;
         for (uint32_t hb = 0; ok && hb < n_parts; ++hb, ++hcg) {
-          const uint32_t b = hcg % kEBufs;
-          ok = mbar_wait(&sm.e_done[b], (hcg / kEBufs) & 1u, sm);
+          const uint32_t b = hcg % kEB;
+          ok = mbar_wait(&sm.e_done[b], (hcg / kEB) & 1u, sm);
           if (!ok) break;
           const int x = (int)(hb * kPartN);
           const uint32_t e = smem_u32(sm.x + b * kESize);
@@ -305,11 +309,11 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
           if (!ok) break;
           tc_fence_after();
           for (uint32_t kt = 0; kt < k_tiles2; ++kt, ++it2) {
-            const uint32_t s = it2 % kRing2;
-            ok = mbar_wait(&sm.full2[s], (it2 / kRing2) & 1u, sm);
+            const uint32_t s = it2 % kR2;
+            ok = mbar_wait(&sm.full2[s], (it2 / kR2) & 1u, sm);
             if (!ok) break;
             tc_fence_after();
-            const uint64_t db = desc_k | (uint64_t)((smem_u32(ring2_slot(sm, s)) >> 4) & 0x3FFF);
+            const uint64_t db = desc_k | (uint64_t)((smem_u32(r2slot(s)) >> 4) & 0x3FFF);
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               mma_ts(t_o + buf * kBlockN, t_pa + kt * kTileK + 8 * j, db + 2 * j, idesc2, (kt | (uint32_t)j) != 0);
@@ -392,8 +396,8 @@ embed_reproject_kernel(const __grid_constant__ Maps maps, uint64_t V, uint32_t d
         const uint32_t np = left < 4 ? left : 4;      // parts of this block that exist
         ok = mbar_wait(&sm.o_full[buf], (cg >> 1) & 1u, sm);
         for (uint32_t part = 0; part < np; ++part, ++hcg) {
-          const uint32_t b = hcg % kEBufs;
-          ok = ok && mbar_wait(&sm.e_full[b], (hcg / kEBufs) & 1u, sm);
+          const uint32_t b = hcg % kEB;
+          ok = ok && mbar_wait(&sm.e_full[b], (hcg / kEB) & 1u, sm);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
